@@ -1,0 +1,348 @@
+"""Pins for the float64 oracle: closed forms, invariants, finite differences,
+library routines and brute force -- none of them a re-typing of the oracle's own
+formula.  A dropped term, a wrong sign or a transposed operand fails at least
+one test here."""
+import math
+import os
+
+import numpy as np
+import pytest
+import scipy.linalg
+import scipy.stats
+
+from oracle import kurtail_oracle as ko
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _golden_values():
+    out = {}
+    with open(os.path.join(GOLD, "kurtosis_closed_forms.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            name, val = line.split()[:2]
+            out[name] = float(val)
+    return out
+
+
+GV = _golden_values()
+
+
+# ---------------- kurtosis (Eq. 3) ----------------
+def test_gaussian_rows_give_three():
+    rng = np.random.default_rng(0)
+    n = 4096
+    Y = rng.standard_normal((512, n))
+    k = ko.kurtosis_rows(Y)
+    # E[k] = 3 (n-1)/(n+1), sd ~ sqrt(24/n)
+    assert abs(k.mean() - GV["normal"] * (n - 1) / (n + 1)) < 4 * math.sqrt(24 / n / 512)
+    assert np.all(np.abs(k - 3) < 6 * math.sqrt(24 / n))
+
+
+def test_uniform_and_laplace_samples():
+    rng = np.random.default_rng(1)
+    n = 200000
+    ku = ko.kurtosis_rows(rng.uniform(-2, 5, (4, n)))
+    kl = ko.kurtosis_rows(rng.laplace(0.3, 1.7, (4, n)))
+    assert np.allclose(ku, GV["uniform"], atol=0.02)
+    assert np.allclose(kl, GV["laplace"], atol=0.35)
+    assert ko.KAPPA_UNIFORM == GV["uniform"]
+
+
+def test_exact_closed_forms():
+    a = 3.7
+    two_point = np.array([[a, -a] * 64])
+    assert ko.kurtosis_rows(two_point)[0] == pytest.approx(GV["two_point"], abs=1e-14)
+    ints = np.arange(256, dtype=np.float64)[None, :]
+    assert ko.kurtosis_rows(ints)[0] == pytest.approx(GV["integers_0_255"], rel=1e-13)
+    assert GV["integers_0_255"] == pytest.approx(3 - 1.2 * (256 ** 2 + 1) / (256 ** 2 - 1), rel=1e-15)
+    onehot = np.zeros((1, 256)); onehot[0, 17] = -5.0
+    assert ko.kurtosis_rows(onehot)[0] == pytest.approx(GV["one_hot_256"], rel=1e-13)
+
+
+def test_matches_scipy_library_routines():
+    rng = np.random.default_rng(2)
+    Y = rng.standard_t(3, (64, 300)) + rng.normal(0, 3, (64, 1))
+    k = ko.kurtosis_rows(Y)
+    assert np.allclose(k, scipy.stats.kurtosis(Y, axis=1, fisher=False, bias=True), rtol=1e-12)
+    mu, m2, m3, m4 = ko.row_moments(Y)
+    assert np.allclose(mu, Y.mean(axis=1))
+    for order, m in ((2, m2), (3, m3), (4, m4)):
+        assert np.allclose(m, scipy.stats.moment(Y, order, axis=1), rtol=1e-12, atol=1e-12)
+
+
+def test_kurtosis_invariances_and_bound():
+    rng = np.random.default_rng(3)
+    Y = rng.standard_t(4, (32, 128))
+    k = ko.kurtosis_rows(Y)
+    assert np.all(k >= 1.0)
+    assert np.allclose(ko.kurtosis_rows(7.5 * Y - 11.0), k, rtol=1e-10)
+    assert np.allclose(ko.kurtosis_rows(Y[:, rng.permutation(128)]), k, rtol=1e-12)
+    assert np.allclose(ko.kurtosis_rows(-Y), k, rtol=1e-12)
+
+
+def test_degenerate_rows_are_skipped():
+    Y = np.ones((3, 16)); Y[1] = 0.0; Y[2] = np.arange(16)
+    deg = ko.degenerate_rows(Y)
+    assert list(deg) == [True, True, False]
+    k2 = ko.kurtosis_rows(Y)[2]
+    assert ko.kurtosis_loss(Y, np.eye(16)) == pytest.approx(abs(k2 - 1.8) / 3)
+    _, dR = ko.loss_grad(Y, np.eye(16))
+    assert np.all(np.isfinite(dR))
+
+
+# ---------------- loss ----------------
+def test_loss_identity_rotation_is_raw_kurtosis():
+    rng = np.random.default_rng(4)
+    X = rng.standard_t(3, (40, 64))
+    direct = np.mean(np.abs(scipy.stats.kurtosis(X, axis=1, fisher=False) - 9 / 5))
+    assert ko.kurtosis_loss(X, np.eye(64)) == pytest.approx(direct, rel=1e-12)
+
+
+def test_loss_brute_force_tiny():
+    rng = np.random.default_rng(5)
+    X = rng.normal(size=(5, 4)); R = scipy.stats.ortho_group.rvs(4, random_state=1)
+    total = 0.0
+    for t in range(5):
+        y = [sum(X[t, i] * R[i, j] for i in range(4)) for j in range(4)]
+        mu = sum(y) / 4
+        m2 = sum((v - mu) ** 2 for v in y) / 4
+        m4 = sum((v - mu) ** 4 for v in y) / 4
+        total += abs(m4 / m2 ** 2 - 1.8)
+    assert ko.kurtosis_loss(X, R) == pytest.approx(total / 5, rel=1e-12)
+
+
+def test_orthogonal_rotation_preserves_row_norms_and_mean_identity():
+    rng = np.random.default_rng(6)
+    X = rng.standard_t(3, (16, 32))
+    R = scipy.stats.ortho_group.rvs(32, random_state=2)
+    Y = ko.rotate(X, R)
+    assert np.allclose((Y ** 2).sum(1), (X ** 2).sum(1), rtol=1e-12)
+    mu, m2, _, _ = ko.row_moments(Y)
+    assert np.allclose(m2 + mu ** 2, (X ** 2).sum(1) / 32, rtol=1e-12)
+    assert np.allclose(mu, X @ R.sum(axis=1) / 32, rtol=1e-10, atol=1e-12)
+
+
+def test_hadamard_flattens_one_hot_outlier():
+    d = 64
+    H = ko.hadamard(d)
+    assert np.allclose(H.T @ H, np.eye(d), atol=1e-14)
+    assert np.allclose(np.abs(H), 1 / math.sqrt(d))
+    assert np.array_equal(np.sign(H), scipy.linalg.hadamard(d))
+    X = np.zeros((2, d)); X[0, 5] = 9.0; X[1, 0] = 9.0
+    Y = ko.rotate(X, H)
+    assert np.allclose(np.abs(Y[0]), 9.0 / math.sqrt(d))        # max shrinks by sqrt(d)
+    assert ko.kurtosis_rows(Y)[0] == pytest.approx(1.0, abs=1e-12)  # +-a row
+    assert ko.degenerate_rows(Y)[1]                                 # channel 0 -> constant row
+    # the raw one-hot row has the largest kurtosis an n-vector can have
+    assert ko.kurtosis_rows(X)[0] == pytest.approx((d * d - 3 * d + 3) / (d - 1))
+
+
+# ---------------- gradient ----------------
+def _rows_away_from_kink(X, R, margin=1e-3):
+    k = ko.kurtosis_rows(ko.rotate(X, R))
+    return np.all(np.abs(k - 1.8) > margin)
+
+
+@pytest.mark.parametrize("N,d,seed", [(8, 4, 0), (16, 8, 1), (32, 16, 2)])
+def test_gradient_matches_central_differences(N, d, seed):
+    rng = np.random.default_rng(seed)
+    X = rng.standard_t(3, (N, d)) + 0.3       # non-zero mean and skew: exercises the m3 term
+    R = scipy.stats.ortho_group.rvs(d, random_state=seed) + 0.01 * rng.normal(size=(d, d))
+    assert _rows_away_from_kink(X, R)
+    _, dR = ko.loss_grad(X, R)
+    h = 1e-6
+    fd = np.zeros_like(dR)
+    for i in range(d):
+        for j in range(d):
+            Rp = R.copy(); Rp[i, j] += h
+            Rm = R.copy(); Rm[i, j] -= h
+            fd[i, j] = (ko.kurtosis_loss(X, Rp) - ko.kurtosis_loss(X, Rm)) / (2 * h)
+    assert np.linalg.norm(dR - fd) / np.linalg.norm(fd) < 1e-6
+
+
+def test_gradient_with_low_kurtosis_rows_has_negative_sign():
+    # balanced rows of +-1 plus small noise have kappa < 1.8: sign flips
+    rng = np.random.default_rng(7)
+    base = np.array([1.0, -1.0] * 4)
+    X = np.stack([rng.permutation(base) for _ in range(6)]) + 0.05 * rng.normal(size=(6, 8))
+    R = np.eye(8)
+    assert np.all(ko.kurtosis_rows(X) < 1.8)
+    _, dR = ko.loss_grad(X, R)
+    h = 1e-6
+    Rp = R.copy(); Rp[2, 3] += h
+    Rm = R.copy(); Rm[2, 3] -= h
+    fd = (ko.kurtosis_loss(X, Rp) - ko.kurtosis_loss(X, Rm)) / (2 * h)
+    assert dR[2, 3] == pytest.approx(fd, rel=1e-5)
+
+
+def test_dY_is_orthogonal_to_ones_and_to_Y():
+    rng = np.random.default_rng(8)
+    Y = rng.standard_t(3, (20, 48)) + 0.7
+    G = ko.loss_dY(Y)
+    assert np.allclose(G.sum(axis=1), 0, atol=1e-14)       # kappa is shift invariant
+    assert np.allclose((G * Y).sum(axis=1), 0, atol=1e-13)  # kappa is scale invariant
+    # hence <R, dR> = tr(Y^T G) = 0 for any R
+    X = rng.normal(size=(20, 48)); R = scipy.stats.ortho_group.rvs(48, random_state=3)
+    _, dR = ko.loss_grad(X, R)
+    assert abs((R * dR).sum()) < 1e-12 * np.abs(R * dR).sum() + 1e-15
+
+
+# ---------------- Cayley step ----------------
+def test_skew_direction_is_skew_and_tangent():
+    rng = np.random.default_rng(9)
+    R = scipy.stats.ortho_group.rvs(12, random_state=4)
+    dR = rng.normal(size=(12, 12))
+    W = ko.skew_direction(R, dR)
+    assert np.array_equal(W, -W.T)
+    # W R equals the projection of dR onto the tangent space {R S : S skew}
+    S = 0.5 * (R.T @ dR - dR.T @ R)
+    assert np.allclose(W @ R, R @ S, atol=1e-12)
+
+
+def test_cayley_exact_is_orthogonal_and_matches_scipy():
+    rng = np.random.default_rng(10)
+    d = 16
+    R = scipy.stats.ortho_group.rvs(d, random_state=5)
+    W = ko.skew_direction(R, rng.normal(size=(d, d)))
+    a = 0.3
+    Rn = ko.cayley_exact(R, W, a)
+    assert ko.orthogonality_error(Rn) < 1e-13
+    assert np.sign(np.linalg.det(Rn)) == np.sign(np.linalg.det(R))
+    ref = scipy.linalg.inv(np.eye(d) + a / 2 * W) @ (np.eye(d) - a / 2 * W) @ R
+    assert np.allclose(Rn, ref, atol=1e-12)
+    assert np.allclose(ko.cayley_exact(R, np.zeros((d, d)), a), R)
+    # first order: R+ = R - a W R + O(a^2)
+    small = 1e-5
+    assert np.allclose(ko.cayley_exact(R, W, small), R - small * W @ R, atol=10 * small ** 2 * np.linalg.norm(W) ** 2)
+
+
+def test_cayley_closed_form_rotation_angle_d2():
+    th, w, a = 0.4, 1.3, 0.25
+    R = np.array([[math.cos(th), -math.sin(th)], [math.sin(th), math.cos(th)]])
+    W = w * np.array([[0.0, -1.0], [1.0, 0.0]])
+    Rn = ko.cayley_exact(R, W, a)
+    th_new = math.atan2(Rn[1, 0], Rn[0, 0])
+    assert th_new - th == pytest.approx(-2 * math.atan(a * w / 2), abs=1e-13)
+
+
+@pytest.mark.parametrize("iters", [0, 1, 2, 3, 4])
+def test_stepwise_converges_to_exact_geometrically(iters):
+    rng = np.random.default_rng(11)
+    d = 10
+    R = scipy.stats.ortho_group.rvs(d, random_state=6)
+    W = ko.skew_direction(R, rng.normal(size=(d, d)))
+    a = 0.6 / np.linalg.norm(W, 2)             # ||a W / 2||_2 = 0.3
+    err = np.linalg.norm(ko.cayley_stepwise(R, W, a, iters) - ko.cayley_exact(R, W, a), 2)
+    rho = 0.3
+    assert err <= 2.5 * rho ** (iters + 1) * 1.0 + 1e-14
+    if iters:
+        prev = np.linalg.norm(ko.cayley_stepwise(R, W, a, iters - 1) - ko.cayley_exact(R, W, a), 2)
+        assert err <= rho * prev * 1.0001
+
+
+def test_step_size_rule_and_descent():
+    rng = np.random.default_rng(12)
+    W = rng.normal(size=(6, 6)); W = W - W.T
+    nrm = np.linalg.norm(W)
+    assert ko.step_size(W, 1e-3) == 1e-3
+    assert ko.step_size(W, 1e3) == pytest.approx(1.0 / (nrm + 1e-8))
+    X = rng.standard_t(3, (64, 8)); X[:, 2] *= 30
+    R = scipy.stats.ortho_group.rvs(8, random_state=7)
+    L0, dR = ko.loss_grad(X, R)
+    Rn, alpha, _ = ko.orth_step(R, dR, 1e-3)
+    assert ko.kurtosis_loss(X, Rn) < L0
+
+
+def test_polish_is_quadratic_and_fit_stays_orthogonal():
+    rng = np.random.default_rng(13)
+    R = scipy.stats.ortho_group.rvs(12, random_state=8) + 1e-3 * rng.normal(size=(12, 12))
+    e0 = ko.orthogonality_error(R)
+    e1 = ko.orthogonality_error(ko.polish(R))
+    assert e1 < 3 * 12 * e0 ** 2
+    X = rng.standard_t(3, (128, 12)); X[:, 5] *= 40
+    R0 = np.eye(12)
+    Rf, losses = ko.fit(X, R0, 100, 5e-3)
+    assert ko.orthogonality_error(Rf) < 1e-9
+    assert losses[-1] < losses[0]
+
+
+def test_cayley_adam_invariants():
+    rng = np.random.default_rng(14)
+    d = 8
+    R = scipy.stats.ortho_group.rvs(d, random_state=9)
+    st = dict(M=np.zeros((d, d)), v=0.0, k=0)
+    for _ in range(5):
+        Rprev = R
+        R = ko.cayley_adam_step(R, rng.normal(size=(d, d)), st, 1e-2)
+        assert ko.orthogonality_error(R) < 1e-6
+        assert abs((st["M"] * Rprev).sum()) < 1e-12  # momentum is tangent at the old point: <W R, R> = 0
+
+
+# ---------------- quantizer ----------------
+def _golden_quant_cases():
+    rows, codes = [], []
+    with open(os.path.join(GOLD, "quant4_cases.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            a, b = line.split(";")
+            rows.append([float(v) for v in a.split()])
+            codes.append([int(float(v)) for v in b.split()])
+    return np.array(rows, dtype=np.float32), np.array(codes, dtype=np.int8)
+
+
+def test_quant4_golden_codes_and_ties():
+    Y, want = _golden_quant_cases()
+    codes, s = ko.quant4_codes(Y)
+    assert np.array_equal(s, np.ones(len(Y), dtype=np.float32))
+    assert np.array_equal(codes, want)
+
+
+def test_quant4_exact_multiples_have_zero_error():
+    rng = np.random.default_rng(15)
+    q = rng.integers(-7, 8, size=(32, 64)); q[:, 0] = 7
+    s = rng.uniform(0.01, 3.0, size=(32, 1)).astype(np.float32)
+    Y = (q.astype(np.float32) * np.float32(0.125) * 8).astype(np.float32) * np.float32(1.0)
+    Y = (q * 0.25).astype(np.float32)     # s = 7*0.25/7 = 0.25 exactly
+    codes, sc = ko.quant4_codes(Y)
+    assert np.array_equal(codes, q)
+    assert np.all(sc == np.float32(0.25))
+    assert ko.quant4_error(Y) == 0.0
+
+
+def test_quant4_range_max_and_zero_row():
+    rng = np.random.default_rng(16)
+    Y = rng.standard_t(3, (64, 128)).astype(np.float32)
+    Y[5] = 0
+    codes, s = ko.quant4_codes(Y)
+    assert codes.min() >= -7 and codes.max() <= 7
+    am = np.abs(Y).argmax(axis=1)
+    assert np.all(np.abs(codes[np.arange(64), am])[np.arange(64) != 5] == 7)
+    assert s[5] == 0 and np.all(codes[5] == 0)
+    # reconstruction error is at most half a step everywhere
+    err = np.abs(Y - codes.astype(np.float32) * s[:, None])
+    assert np.all(err <= 0.5 * s[:, None] * (1 + 1e-5))
+
+
+def test_quant4_uniform_rows_give_step_squared_over_twelve():
+    rng = np.random.default_rng(17)
+    Y = rng.uniform(-1, 1, (256, 4096)).astype(np.float32)
+    s = 1.0 / 7
+    # rounding error is uniform on (-s/2, s/2) except in the clipped half-bins at the ends
+    assert ko.quant4_error(Y) == pytest.approx(s * s / 12, rel=0.02)
+
+
+def test_quant4_error_rotated_uses_the_product():
+    rng = np.random.default_rng(18)
+    X = rng.standard_t(3, (32, 16)); X[:, 3] *= 50
+    H = ko.hadamard(16)
+    assert ko.quant4_error_rotated(X, np.eye(16)) == pytest.approx(ko.quant4_error(X.astype(np.float32)))
+    # a one-hot row becomes +-a/sqrt(d) everywhere: every entry sits on the +-7 level
+    E1 = np.zeros((4, 16)); E1[np.arange(4), [1, 5, 9, 14]] = [3.0, -2.0, 8.0, 0.5]
+    assert ko.quant4_error_rotated(E1, H) < 1e-12
+    # a transposed operand would change this: column scaling vs row scaling
+    A = rng.normal(size=(16, 16))
+    assert ko.quant4_error_rotated(X, A) == pytest.approx(ko.quant4_error((X @ A).astype(np.float32)))
+    assert ko.quant4_error_rotated(X, A) != pytest.approx(ko.quant4_error((X @ A.T).astype(np.float32)))
