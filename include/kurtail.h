@@ -1,0 +1,196 @@
+/*
+ * kurtail.h -- C ABI of libkurtail, a B200 (sm_100a) implementation of KurTail
+ * rotation learning (arXiv 2503.01483): find an orthogonal R (d x d) that
+ * minimises the kurtosis loss of the rotated calibration activations Y = X R.
+ *
+ * General conventions
+ * -------------------
+ * Pointers.  Every matrix pointer is a DEVICE pointer unless the parameter is
+ *   documented "host".  Matrices are row-major.  The caller owns X, R, dR, the
+ *   code/scale outputs and the workspace; the library never frees or
+ *   reallocates them, and allocates no device memory after kt_create().
+ * Shapes.  N = number of tokens (rows of X), any N >= 1 (ragged tails are
+ *   handled).  d = channels, a multiple of 128.  X.ld >= d in elements; the
+ *   base of X must be 16-byte aligned and X.ld * sizeof(element) a multiple of
+ *   16 (the tiles are fetched by TMA).  R and dR are dense d x d float32,
+ *   16-byte aligned.
+ * Precision.  X is used as bfloat16 (float32 X is rounded once on entry), R is
+ *   kept in float32 and rounded to bfloat16 for the token GEMMs; all products
+ *   accumulate in float32 on the tensor cores.
+ * Stream.  All work is issued on the stream given to kt_create().  Calls that
+ *   return a host scalar synchronise that stream; the others are stream
+ *   ordered and return after enqueueing.
+ * Errors.  Every call returns a kt_status; nothing throws, aborts or prints.
+ *   Argument errors are detected before any work is enqueued and leave all
+ *   outputs untouched.  Device-side waits are bounded; if one runs out the
+ *   kernel records it and the next synchronising call returns KT_ERR_TIMEOUT.
+ *   There is no CPU or library fallback: a device that is not sm_100 gives
+ *   KT_ERR_ARCH.
+ */
+#ifndef KURTAIL_H_
+#define KURTAIL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct kt_ctx kt_ctx;
+
+typedef enum {
+  KT_OK = 0,
+  KT_ERR_INVALID_ARG = 1, /* null pointer, negative count, unknown enum     */
+  KT_ERR_SHAPE = 2,       /* d not a multiple of 128, N < 1, ld < cols      */
+  KT_ERR_ALIGN = 3,       /* base or leading dimension not 16-byte aligned  */
+  KT_ERR_WORKSPACE = 4,   /* workspace missing or smaller than required     */
+  KT_ERR_ARCH = 5,        /* current device is not compute capability 10.x  */
+  KT_ERR_CUDA = 6,        /* a CUDA runtime/driver call failed              */
+  KT_ERR_NONFINITE = 7,   /* the loss came out NaN/Inf (outputs are written)*/
+  KT_ERR_TIMEOUT = 8      /* a bounded device-side wait ran out             */
+} kt_status;
+
+typedef enum { KT_BF16 = 0, KT_F32 = 1 } kt_dtype;
+
+/* A row-major matrix: rows x cols elements of `dtype`, leading dimension `ld`
+ * elements. */
+typedef struct {
+  const void* data;
+  int32_t dtype; /* kt_dtype */
+  int32_t reserved;
+  int64_t rows, cols, ld;
+} kt_mat;
+
+/* Tunables.  kt_default_config() fills the defaults given in brackets. */
+typedef struct {
+  float kappa_target;   /* [1.8] kurtosis of the uniform distribution, the target
+                           of the loss (Section 2, loss equation)              */
+  int32_t cayley_iters; /* [2]   fixed-point iterations s of the Cayley step    */
+  float q;              /* [0.5] contraction bound: alpha <= 2q / ||W||_F       */
+  float eps;            /* [1e-8] added to ||W||_F in that bound                */
+  float polish_thresh;  /* [1e-6] the Newton-Schulz polish runs when
+                           max|R^T R - I| exceeds this; < 0: every step;
+                           +inf: never                                          */
+  int32_t retract_terms;/* [2]   bf16 split terms (1..3) of the iterate in the
+                           retraction products; more = closer to float32       */
+  int32_t guard_every;  /* [1]   in kt_fit: run the orthogonality guard every
+                           this many steps (and always after the last one)     */
+  int32_t reserved[5];
+} kt_config;
+
+/* Filled by kt_fit / kt_fit_layers (host memory). */
+typedef struct {
+  int32_t steps_done;
+  int32_t degenerate_rows; /* rows skipped in the last evaluated loss          */
+  double loss_first;       /* loss at R before the first step                   */
+  double loss_last;        /* loss at R before the last step                    */
+  double orth_err;         /* max|R^T R - I| seen by the last guard, before its
+                              polish                                            */
+  float alpha_last;        /* step size used by the last step                   */
+  float w_norm_last;       /* ||W||_F of the last step                          */
+  double* loss_history;    /* optional host array of `steps` entries, or NULL   */
+} kt_fit_report;
+
+/* --- life cycle ---------------------------------------------------------- */
+
+/* Fills *cfg with the defaults. */
+void kt_default_config(kt_config* cfg);
+
+/* Creates a context on the CURRENT device.  `cfg` may be NULL (defaults).
+ * `cuda_stream` is a cudaStream_t (NULL = the legacy default stream).  Allocates
+ * a few KiB of device and pinned host memory for scalars; released by
+ * kt_destroy().  KT_ERR_ARCH on a device that is not sm_100. */
+kt_status kt_create(kt_ctx** ctx, const kt_config* cfg, void* cuda_stream);
+void kt_destroy(kt_ctx* ctx);
+const char* kt_status_string(kt_status s);
+
+/* Bytes of scratch the calls below need for an N x d problem whose X has
+ * element type `x_dtype`.  Host-only; never touches the device. */
+kt_status kt_workspace_bytes(const kt_ctx* ctx, int64_t N, int64_t d, int32_t x_dtype, size_t* bytes);
+
+/* Hands the context a caller-allocated device buffer (256-byte aligned).  The
+ * buffer must stay valid until replaced or the context is destroyed.  Calls
+ * check that it is large enough for their N and d (KT_ERR_WORKSPACE if not). */
+kt_status kt_set_workspace(kt_ctx* ctx, void* dev_ptr, size_t bytes);
+
+/* --- rotation initialisers (Section 3: Hadamard rotations) ---------------- */
+
+/* Writes R (d x d float32).  kind 0: identity.  kind 1: normalised Sylvester
+ * Hadamard H[i][j] = (-1)^popcount(i & j) / sqrt(d); d must be a power of two
+ * (KT_ERR_SHAPE otherwise).  Stream ordered. */
+kt_status kt_init_rotation(kt_ctx* ctx, float* R, int64_t d, int32_t kind);
+
+/* --- the loss (Section 2, Eq. 3 and the loss equation) -------------------- */
+
+/* *loss (host) = (1/N) sum_t |kappa(Y_t) - kappa_target|, Y = X R, kappa the
+ * ratio of the fourth central moment to the squared second central moment of
+ * the d entries of row t.  Rows without spread (m2 <= 1e-6 * mean square) add
+ * zero.  Y is never written to memory.  Synchronises. */
+kt_status kt_kurtosis_loss(kt_ctx* ctx, kt_mat X, const float* R, double* loss);
+
+/* Same loss, plus dR (d x d float32, device) = dL/dR = X^T (dL/dY), the
+ * Euclidean gradient (Section 3, "Learning the Rotations": R is the weight of a
+ * linear layer trained with this loss).  `loss` (host) may be NULL, in which
+ * case the call is stream ordered and does not synchronise. */
+kt_status kt_loss_grad(kt_ctx* ctx, kt_mat X, const float* R, float* dR, double* loss);
+
+/* Test hook: per-row moments of Y = X R, moments[t] = {mean, m2, m3, m4}
+ * (N x 4 float32, device).  Stream ordered. */
+kt_status kt_row_moments(kt_ctx* ctx, kt_mat X, const float* R, float* moments);
+
+/* Test hook: Y = X R as float32 (N x d dense, device).  Stream ordered. */
+kt_status kt_rotate(kt_ctx* ctx, kt_mat X, const float* R, float* Y);
+
+/* --- the step on the orthogonal group (Section 3, "Optimization in the
+ *     Orthogonal Space": Cayley SGD) -------------------------------------- */
+
+/* R <- retraction of R along -dR:  W = (dR R^T - R dR^T)/2,
+ * alpha = min(lr, 2q/(||W||_F + eps)), Y0 = R - alpha W R,
+ * Yi = R - alpha/2 W (R + Y(i-1)) for i = 1..cayley_iters, R <- Y(last), then
+ * the orthogonality guard (see kt_config.polish_thresh).  Built from d x d
+ * tensor-core products only.  R is updated in place; dR is read only.  Uses
+ * the workspace (sized for any N >= 1 and this d).  Stream ordered. */
+kt_status kt_orth_step(kt_ctx* ctx, float* R, const float* dR, int64_t d, float lr);
+
+/* *err (host) = max|R^T R - I|.  Uses the workspace.  Synchronises. */
+kt_status kt_orth_error(kt_ctx* ctx, const float* R, int64_t d, double* err);
+
+/* `steps` x (kt_loss_grad; kt_orth_step) on the context's stream with no host
+ * synchronisation in between; bit-identical to composing those calls when
+ * guard_every == 1.  R in/out.  `report` (host) may be NULL.  Synchronises at
+ * the end.  On an error R holds the last completed step. */
+kt_status kt_fit(kt_ctx* ctx, kt_mat X, float* R, int32_t steps, float lr, kt_fit_report* report);
+
+/* Layer-wise driver (Section 3, "Training Cost": activations are stored per
+ * layer, then one rotation is optimised at a time).  X_layers[l] and
+ * R_layers[l] for l in [first_layer, L) are fitted one after another on the
+ * stream; all layer buffers stay resident in device memory.  All layers must
+ * share N, d and dtype.  per_layer (host, L entries) may be NULL. */
+kt_status kt_fit_layers(kt_ctx* ctx, const kt_mat* X_layers, float* const* R_layers, int32_t L,
+                        int32_t first_layer, int32_t steps, float lr, kt_fit_report* per_layer);
+
+/* kt_fit with HOST buffers: copies X_host (N x d, pinned or pageable host
+ * memory) into X_dev_staging (device, N*ld elements), R_host (d x d float32)
+ * into R_dev, fits, and copies R back to R_host.  The copies run on the
+ * context's stream. */
+kt_status kt_fit_host(kt_ctx* ctx, kt_mat X_host, void* X_dev_staging, float* R_host, float* R_dev,
+                      int32_t steps, float lr, kt_fit_report* report);
+
+/* --- 4-bit fake quantisation (Section 2, "Uniform Quantization for k-bit
+ *     Precision", symmetric case with k = 4, and Eq. 1) -------------------- */
+
+/* *mse (host) = mean over all N*d entries of (Y - Q(Y))^2 with Y = X R and, per
+ * token, s = max|Y_t| / 7, Q(y) = clamp(round_half_even(y / s), -7, 7) * s.
+ * Y is recomputed instead of stored.  Synchronises. */
+kt_status kt_quant4_error(kt_ctx* ctx, kt_mat X, const float* R, double* mse);
+
+/* Test hook: quantise a given float32 Y (N x d dense, device): codes (N x d
+ * int8, device) and scales (N float32, device).  Float32 IEEE divide and
+ * round-half-even decide the codes.  No workspace needed.  Stream ordered. */
+kt_status kt_quant4_codes(kt_ctx* ctx, const float* Y, int64_t N, int64_t d, int8_t* codes, float* scales);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KURTAIL_H_ */

@@ -1,0 +1,400 @@
+// Memory-bound kernels around the GEMMs: casts and bf16 splits, transposes, the
+// per-row moment merge and loss reduction, the skew/step-size/axpy pieces of the
+// Cayley step, the orthogonality guard, the 4-bit quantizer and the rotation
+// initialisers.  Every reduction is fixed-order (no floating-point atomics), so
+// repeated runs are bit-identical.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+
+namespace kt {
+
+// Device-resident scalars shared by the kernels of one context.
+struct Scalars {
+  double loss;              // last loss
+  double qmse;              // last quantisation MSE
+  float alpha;              // step size of the current Cayley step
+  float wnorm;              // ||W||_F of the current step
+  unsigned int max_e_bits;  // max|R^T R - I| as float bits
+  unsigned int gate;        // 1 = the polish runs
+  unsigned int err_word;    // != 0: a bounded wait ran out (code of the waiting role)
+  unsigned int deg_rows;    // rows skipped by the last loss
+  unsigned int pad[2];
+};
+
+constexpr float kDegenerateRel = 1e-6f;
+
+// ------------------------------------------------------------ block reduce
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+  return v;
+}
+// Sum over a 256-thread block in a fixed order; result valid in thread `lin` 0.
+__device__ __forceinline__ double block_sum_256(double v, double* sh /*8*/, int lin) {
+  v = warp_sum(v);
+  if ((lin & 31) == 0) sh[lin >> 5] = v;
+  __syncthreads();
+  double r = 0.0;
+  if (lin == 0) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) r += sh[i];
+  }
+  __syncthreads();
+  return r;
+}
+
+__device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bfloat16& lo) {
+  hi = __float2bfloat16_rn(x);
+  lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+
+// ------------------------------------------------------ casts and transposes
+// src float32 rows x cols -> bf16 hi (and lo = bf16(src - hi) when lo != null).
+// TRANSPOSE: out[c][r], else out[r][c]; ldo = leading dimension of the outputs.
+// grid (cols/32, rows/32), block (32, 8); rows and cols multiples of 32.
+template <bool TRANSPOSE>
+__global__ void k_split_bf16(const float* __restrict__ src, long long ld, __nv_bfloat16* __restrict__ hi,
+                             __nv_bfloat16* __restrict__ lo, long long ldo) {
+  __shared__ float tile[32][33];
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  if (!TRANSPOSE) {
+    for (int r = ty; r < 32; r += 8) {
+      const float x = src[static_cast<long long>(r0 + r) * ld + c0 + tx];
+      __nv_bfloat16 h, l;
+      split_bf16(x, h, l);
+      const long long o = static_cast<long long>(r0 + r) * ldo + c0 + tx;
+      hi[o] = h;
+      if (lo) lo[o] = l;
+    }
+  } else {
+    for (int r = ty; r < 32; r += 8) tile[r][tx] = src[static_cast<long long>(r0 + r) * ld + c0 + tx];
+    __syncthreads();
+    for (int c = ty; c < 32; c += 8) {
+      const float x = tile[tx][c];
+      __nv_bfloat16 h, l;
+      split_bf16(x, h, l);
+      const long long o = static_cast<long long>(c0 + c) * ldo + r0 + tx;
+      hi[o] = h;
+      if (lo) lo[o] = l;
+    }
+  }
+}
+
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+// X (N x d, leading dimension ld, T = float or bf16) -> Xt (d x ldt bf16, the
+// transpose, columns in [N, 64*ceil(N/64)) zero) and, when xb != null, a dense
+// bf16 copy Xb (N x d).  grid (d/64, ceil(N/64)), block (32, 8).
+template <typename T>
+__global__ void k_prepare_x(const T* __restrict__ X, long long ld, int N, int d, __nv_bfloat16* __restrict__ xt,
+                            long long ldt, __nv_bfloat16* __restrict__ xb) {
+  __shared__ __nv_bfloat16 tile[64][66];
+  const int c0 = blockIdx.x * 64, r0 = blockIdx.y * 64;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  for (int r = ty; r < 64; r += 8) {
+    const int row = r0 + r;
+    __nv_bfloat16 v0 = __float2bfloat16_rn(0.f), v1 = v0;
+    if (row < N) {
+      const T* s = X + static_cast<long long>(row) * ld + c0 + 2 * tx;
+      v0 = __float2bfloat16_rn(to_f32(s[0]));
+      v1 = __float2bfloat16_rn(to_f32(s[1]));
+      if (xb) {
+        __nv_bfloat162 pr;
+        pr.x = v0;
+        pr.y = v1;
+        *reinterpret_cast<__nv_bfloat162*>(xb + static_cast<long long>(row) * d + c0 + 2 * tx) = pr;
+      }
+    }
+    tile[r][2 * tx] = v0;
+    tile[r][2 * tx + 1] = v1;
+  }
+  __syncthreads();
+  for (int c = ty; c < 64; c += 8) {
+    __nv_bfloat162 pr;
+    pr.x = tile[2 * tx][c];
+    pr.y = tile[2 * tx + 1][c];
+    *reinterpret_cast<__nv_bfloat162*>(xt + static_cast<long long>(c0 + c) * ldt + r0 + 2 * tx) = pr;
+  }
+}
+
+// float32 X (N x d, ld) -> dense bf16 Xb (N x d).  grid ceil(N*d/2/256), block 256.
+__global__ void k_cast_x(const float* __restrict__ X, long long ld, long long N, int d,
+                         __nv_bfloat16* __restrict__ xb) {
+  const long long i2 = (static_cast<long long>(blockIdx.x) * 256 + threadIdx.x) * 2;
+  if (i2 >= N * d) return;
+  const long long row = i2 / d;
+  const int col = static_cast<int>(i2 % d);
+  const float* s = X + row * ld + col;
+  __nv_bfloat162 pr;
+  pr.x = __float2bfloat16_rn(s[0]);
+  pr.y = __float2bfloat16_rn(s[1]);
+  *reinterpret_cast<__nv_bfloat162*>(xb + i2) = pr;
+}
+
+// ------------------------------------------------ moments merge and the loss
+// Merges the per-column-tile records {mean_p, S2_p, S3_p, S4_p} (each over bn
+// columns, central about mean_p) of every row into the row's mean and central
+// moments m2, m3, m4 over all d columns (Eq. 3), then kappa = m4/m2^2, the row's
+// loss term |kappa - kappa_t| and the coefficients of dL/dY for the backward:
+//   G = a c^3 - ab c - am3,  a = sgn(kappa-kappa_t) 4/(N d m2^2), ab = a m4/m2, am3 = a m3.
+// A row with m2 <= 1e-6 * (m2 + mean^2), or all zero, contributes nothing.
+// grid ceil(N/256), block 256.
+__global__ void k_moments_finalize(const float4* __restrict__ partial, int P, int N, int d, int bn, float kappa_t,
+                                   float4* __restrict__ moments, float4* __restrict__ coef,
+                                   double* __restrict__ block_loss, unsigned int* __restrict__ block_deg) {
+  __shared__ double sh[8];
+  const int row = blockIdx.x * 256 + threadIdx.x;
+  double term = 0.0, deg = 0.0;
+  if (row < N) {
+    double mu = 0.0;
+    for (int p = 0; p < P; ++p) mu += static_cast<double>(partial[static_cast<long long>(p) * N + row].x);
+    mu /= P;
+    double M2 = 0.0, M3 = 0.0, M4 = 0.0;
+    const double n = bn;
+    for (int p = 0; p < P; ++p) {
+      const float4 r = partial[static_cast<long long>(p) * N + row];
+      const double dl = static_cast<double>(r.x) - mu, dl2 = dl * dl;
+      M2 += r.y + n * dl2;
+      M3 += r.z + 3.0 * dl * r.y + n * dl2 * dl;
+      M4 += r.w + 4.0 * dl * r.z + 6.0 * dl2 * r.y + n * dl2 * dl2;
+    }
+    const double m2 = M2 / d, m3 = M3 / d, m4 = M4 / d;
+    const double ms = m2 + mu * mu;
+    const bool degenerate = (ms == 0.0) || (m2 <= static_cast<double>(kDegenerateRel) * ms);
+    float4 cf = make_float4(static_cast<float>(mu), 0.f, 0.f, 0.f);
+    if (!degenerate) {
+      const double kappa = m4 / (m2 * m2);
+      const double diff = kappa - static_cast<double>(kappa_t);
+      term = fabs(diff);
+      const double sgn = (diff > 0.0) ? 1.0 : ((diff < 0.0) ? -1.0 : 0.0);
+      const double a = sgn * 4.0 / (static_cast<double>(N) * d * m2 * m2);
+      cf.y = static_cast<float>(a);
+      cf.z = static_cast<float>(a * m4 / m2);
+      cf.w = static_cast<float>(a * m3);
+    } else {
+      deg = 1.0;
+    }
+    if (moments)
+      moments[row] = make_float4(static_cast<float>(mu), static_cast<float>(m2), static_cast<float>(m3),
+                                 static_cast<float>(m4));
+    if (coef) coef[row] = cf;
+  }
+  const double bl = block_sum_256(term, sh, threadIdx.x);
+  const double bd = block_sum_256(deg, sh, threadIdx.x);
+  if (threadIdx.x == 0) {
+    block_loss[blockIdx.x] = bl;
+    block_deg[blockIdx.x] = static_cast<unsigned int>(bd);
+  }
+}
+
+// One block: *dst = scale * sum(vals[0..n)) (also to *dst2 when not null);
+// *count_dst = sum(counts) when counts != null.
+__global__ void k_final_sum(const double* __restrict__ vals, int n, double scale, double* __restrict__ dst,
+                            double* __restrict__ dst2, const unsigned int* __restrict__ counts,
+                            unsigned int* __restrict__ count_dst) {
+  __shared__ double sh[8];
+  double s = 0.0, c = 0.0;
+  for (int i = threadIdx.x; i < n; i += 256) {
+    s += vals[i];
+    if (counts) c += counts[i];
+  }
+  s = block_sum_256(s, sh, threadIdx.x);
+  c = block_sum_256(c, sh, threadIdx.x);
+  if (threadIdx.x == 0) {
+    *dst = s * scale;
+    if (dst2) *dst2 = s * scale;
+    if (count_dst) *count_dst = static_cast<unsigned int>(c);
+  }
+}
+
+// Sum of float32 values into per-block doubles (fixed order). block 256.
+__global__ void k_block_sums_f32(const float* __restrict__ v, long long n, double* __restrict__ block_out) {
+  __shared__ double sh[8];
+  double s = 0.0;
+  for (long long i = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x; i < n;
+       i += static_cast<long long>(gridDim.x) * 256)
+    s += v[i];
+  s = block_sum_256(s, sh, threadIdx.x);
+  if (threadIdx.x == 0) block_out[blockIdx.x] = s;
+}
+
+// ------------------------------------------------------------- Cayley pieces
+// W = (A - A^T)/2 for a d x d float32 A, written as bf16 (the rounding is odd,
+// so the bf16 W is exactly skew), plus per-block sums of W^2 (of the float32 W).
+// grid (d/32, d/32), block (32, 8).
+__global__ void k_skew(const float* __restrict__ A, int d, __nv_bfloat16* __restrict__ w_hi,
+                       double* __restrict__ block_norm2) {
+  __shared__ float tT[32][33];
+  __shared__ double sh[8];
+  const int bj = blockIdx.x, bi = blockIdx.y;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  // tile (bj, bi) of A, to be read transposed
+  for (int r = ty; r < 32; r += 8) tT[r][tx] = A[static_cast<long long>(bj * 32 + r) * d + bi * 32 + tx];
+  __syncthreads();
+  double acc = 0.0;
+  for (int r = ty; r < 32; r += 8) {
+    const long long o = static_cast<long long>(bi * 32 + r) * d + bj * 32 + tx;
+    const float w = 0.5f * (A[o] - tT[tx][r]);
+    w_hi[o] = __float2bfloat16_rn(w);
+    acc += static_cast<double>(w) * w;
+  }
+  const int lin = ty * 32 + tx;
+  acc = block_sum_256(acc, sh, lin);
+  if (lin == 0) block_norm2[blockIdx.y * gridDim.x + blockIdx.x] = acc;
+}
+
+// One block: ||W||_F and alpha = min(lr, 2q/(||W||_F + eps)); also clears the
+// guard's running maximum for this step.
+__global__ void k_step_size(const double* __restrict__ block_norm2, int n, float lr, float q, float eps,
+                            Scalars* __restrict__ sc) {
+  __shared__ double sh[8];
+  double s = 0.0;
+  for (int i = threadIdx.x; i < n; i += 256) s += block_norm2[i];
+  s = block_sum_256(s, sh, threadIdx.x);
+  if (threadIdx.x == 0) {
+    const double nrm = sqrt(s);
+    const double cap = 2.0 * static_cast<double>(q) / (nrm + static_cast<double>(eps));
+    const double a = (static_cast<double>(lr) < cap) ? static_cast<double>(lr) : cap;
+    sc->alpha = static_cast<float>(a);
+    sc->wnorm = static_cast<float>(nrm);
+  }
+}
+
+// Y = R - (alpha * cmul) P;  if dst: dst = Y;  Z = zr R + Y, written as bf16
+// hi/lo, transposed (zt_*) and/or as is (z_*).  All matrices d x d, dense.
+// grid (d/32, d/32), block (32, 8).  dst may alias R.
+__global__ void k_axpy_split(const float* R, const float* __restrict__ P, const Scalars* __restrict__ sc,
+                             float cmul, float zr, int d, float* dst, __nv_bfloat16* __restrict__ zt_hi,
+                             __nv_bfloat16* __restrict__ zt_lo, __nv_bfloat16* __restrict__ z_hi,
+                             __nv_bfloat16* __restrict__ z_lo) {
+  __shared__ float tile[32][33];
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  const float beta = sc->alpha * cmul;
+  for (int r = ty; r < 32; r += 8) {
+    const long long o = static_cast<long long>(r0 + r) * d + c0 + tx;
+    const float rv = R[o];
+    const float y = fmaf(-beta, P[o], rv);
+    const float z = fmaf(zr, rv, y);
+    if (dst) dst[o] = y;
+    tile[r][tx] = z;
+    if (z_hi) {
+      __nv_bfloat16 h, l;
+      split_bf16(z, h, l);
+      z_hi[o] = h;
+      if (z_lo) z_lo[o] = l;
+    }
+  }
+  if (zt_hi) {
+    __syncthreads();
+    for (int c = ty; c < 32; c += 8) {
+      const float z = tile[tx][c];
+      __nv_bfloat16 h, l;
+      split_bf16(z, h, l);
+      const long long o = static_cast<long long>(c0 + c) * d + r0 + tx;
+      zt_hi[o] = h;
+      if (zt_lo) zt_lo[o] = l;
+    }
+  }
+}
+
+// E = S - I (S = R^T R, d x d float32): max|E| into sc->max_e_bits (atomic max on
+// the bit pattern of a non-negative float: exact, order independent) and E as
+// bf16 when e_hi != null.  grid d*d/4/256, block 256; d*d a multiple of 1024.
+__global__ void k_guard(const float* __restrict__ S, int d, __nv_bfloat16* __restrict__ e_hi,
+                        Scalars* __restrict__ sc) {
+  const long long i4 = (static_cast<long long>(blockIdx.x) * 256 + threadIdx.x) * 4;
+  const float4 s = *reinterpret_cast<const float4*>(S + i4);
+  const int row = static_cast<int>(i4 / d), col = static_cast<int>(i4 % d);
+  float e[4] = {s.x, s.y, s.z, s.w};
+  float mx = 0.f;
+  bool bad = false;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    if (col + j == row) e[j] -= 1.0f;
+    bad |= (e[j] != e[j]);
+    mx = fmaxf(mx, fabsf(e[j]));
+  }
+  if (bad) mx = __uint_as_float(0x7f800000u);  // a NaN in R^T R reads as +inf
+  if (e_hi) {
+    __nv_bfloat162 a, b;
+    a.x = __float2bfloat16_rn(e[0]);
+    a.y = __float2bfloat16_rn(e[1]);
+    b.x = __float2bfloat16_rn(e[2]);
+    b.y = __float2bfloat16_rn(e[3]);
+    *reinterpret_cast<__nv_bfloat162*>(e_hi + i4) = a;
+    *reinterpret_cast<__nv_bfloat162*>(e_hi + i4 + 2) = b;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if ((threadIdx.x & 31) == 0 && mx > 0.f) atomicMax(&sc->max_e_bits, __float_as_uint(mx));
+}
+
+// gate = (max|E| > thresh).
+__global__ void k_guard_decide(Scalars* sc, float thresh) {
+  const float mx = __uint_as_float(sc->max_e_bits);
+  sc->gate = (mx > thresh) ? 1u : 0u;
+}
+
+// R <- R - Q/2 when the gate is open.  grid d*d/4/256, block 256.
+__global__ void k_polish_apply(float* __restrict__ R, const float* __restrict__ Q, const Scalars* __restrict__ sc) {
+  if (sc->gate == 0u) return;
+  const long long i4 = (static_cast<long long>(blockIdx.x) * 256 + threadIdx.x) * 4;
+  float4 r = *reinterpret_cast<float4*>(R + i4);
+  const float4 qv = *reinterpret_cast<const float4*>(Q + i4);
+  r.x = fmaf(-0.5f, qv.x, r.x);
+  r.y = fmaf(-0.5f, qv.y, r.y);
+  r.z = fmaf(-0.5f, qv.z, r.z);
+  r.w = fmaf(-0.5f, qv.w, r.w);
+  *reinterpret_cast<float4*>(R + i4) = r;
+}
+
+// ------------------------------------------------------------------ quantizer
+// One block per row of a dense float32 Y (N x d): s = max|Y_t| / 7 (IEEE divide),
+// code = clamp(rint(Y / s), -7, 7) (IEEE divide, ties to even); s == 0 -> zeros.
+__global__ void k_quant4_codes(const float* __restrict__ Y, int d, int8_t* __restrict__ codes,
+                               float* __restrict__ scales) {
+  __shared__ float sh[8];
+  const long long base = static_cast<long long>(blockIdx.x) * d;
+  float mx = 0.f;
+  for (int j = threadIdx.x; j < d; j += 256) mx = fmaxf(mx, fabsf(Y[base + j]));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = mx;
+  __syncthreads();
+  mx = sh[0];
+#pragma unroll
+  for (int i = 1; i < 8; ++i) mx = fmaxf(mx, sh[i]);
+  const float s = __fdiv_rn(mx, 7.0f);
+  if (threadIdx.x == 0) scales[blockIdx.x] = s;
+  for (int j = threadIdx.x; j < d; j += 256) {
+    float qv = 0.f;
+    if (s > 0.f) {
+      qv = rintf(__fdiv_rn(Y[base + j], s));
+      qv = fminf(fmaxf(qv, -7.0f), 7.0f);
+    }
+    codes[base + j] = static_cast<int8_t>(qv);
+  }
+}
+
+// ---------------------------------------------------------------- initialisers
+// kind 0: identity; kind 1: Sylvester Hadamard (-1)^popcount(i&j) * scale.
+__global__ void k_init_rotation(float* __restrict__ R, int d, int kind, float scale) {
+  const long long idx = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
+  if (idx >= static_cast<long long>(d) * d) return;
+  const int i = static_cast<int>(idx / d), j = static_cast<int>(idx % d);
+  float v;
+  if (kind == 0) {
+    v = (i == j) ? 1.0f : 0.0f;
+  } else {
+    v = (__popc(i & j) & 1) ? -scale : scale;
+  }
+  R[idx] = v;
+}
+
+}  // namespace kt

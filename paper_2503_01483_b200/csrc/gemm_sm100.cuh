@@ -1,0 +1,343 @@
+// Persistent, warp-specialised tcgen05 GEMM with fused epilogues.
+//
+//   D[m][n] = sum over terms q, sum over k of  A_q[m][k] * B_q[n][k]
+//
+// A_q is M x K and B_q is N x K, both bf16 with k contiguous ("K-major"); the
+// accumulator is float32 in tensor memory.  One CTA per SM walks the output
+// tiles (128 x BN); warp 0 feeds shared memory with TMA, warp 1 issues the MMAs,
+// warps 2..5 drain the accumulator.  Two accumulators alternate, so the epilogue
+// of one tile overlaps the MMAs of the next.  What the epilogue does with a
+// finished tile is selected by `EPI`:
+//
+//   kStoreF32  write D as float32
+//   kMoments   per row: mean and central power sums of the tile's BN columns
+//              (Eq. 3 of the paper, one partial record per column tile)
+//   kGrad      G = a c^3 - ab c - am3, c = D - mu  (derivative of the loss
+//              through Eq. 3), written transposed as bf16
+//   kAbsMax    per-row max |D| (first pass of the symmetric quantizer)
+//   kQuantErr  per-row sum of (D - Q(D))^2 for the 4-bit symmetric quantizer
+#pragma once
+#include <cuda.h>
+
+#include "sm100_prims.cuh"
+
+namespace kt {
+
+constexpr int kBM = 128;           // rows per tile = tensor-memory lanes
+constexpr int kBK = 64;            // k elements per pipeline stage (one 128-byte swizzle row)
+constexpr int kGemmThreads = 192;  // 6 warps
+constexpr int kMaxTerms = 3;
+
+enum Epi : int { kStoreF32 = 0, kMoments = 1, kGrad = 2, kAbsMax = 3, kQuantErr = 4 };
+
+struct GemmParams {
+  CUtensorMap tmA[kMaxTerms];
+  CUtensorMap tmB[kMaxTerms];
+  int terms;
+  int M, N, K;
+  int m_tiles, n_tiles;
+  // epilogue operands (which are used depends on EPI)
+  float* out;                 // kStoreF32: M x N, leading dimension ldo
+  long long ldo;
+  float4* partial;            // kMoments: [n_tiles][M] records {mean, S2, S3, S4}
+  const float4* coef;         // kGrad: per row {mu, a, ab, am3}
+  __nv_bfloat16* gt;          // kGrad: G transposed, [N][ldg]
+  long long ldg;
+  unsigned int* rowmax;       // kAbsMax (out) / kQuantErr (in): per-row max|D| as float bits
+  float* qerr;                // kQuantErr: [n_tiles][M] partial squared errors
+  const unsigned int* gate;   // when not null and *gate == 0 the kernel does nothing
+  unsigned int* err_word;     // receives the code of a wait that ran out
+};
+
+template <int BN>
+struct GemmSmem {
+  static constexpr int kStages = (BN == 256) ? 4 : 6;
+  static constexpr int kABytes = kBM * kBK * 2;
+  static constexpr int kBBytes = BN * kBK * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kBarBytes = 256;
+  static constexpr int kTotal = 1024 /*alignment slack*/ + kStages * kStageBytes + kBarBytes;
+};
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_constant__ GemmParams p) {
+  using S = GemmSmem<BN>;
+  constexpr int kStages = S::kStages;
+  constexpr uint32_t kTmemCols = 2 * BN;  // two accumulators: 256 or 512 columns
+  constexpr uint32_t kIdesc = umma_idesc_bf16_f32(kBM, BN);
+
+  if (p.gate != nullptr && *p.gate == 0u) return;  // uniform over the grid
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t smem_a = smem_base;
+  const uint32_t smem_b = smem_base + kStages * S::kABytes;
+  const uint32_t bar_base = smem_base + kStages * S::kStageBytes;
+  // barrier slots (8 bytes each): full[kStages], empty[kStages], acc_full[2], acc_empty[2]
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
+  auto acc_full_bar = [&](int b) { return bar_base + 8u * (2 * kStages + b); };
+  auto acc_empty_bar = [&](int b) { return bar_base + 8u * (2 * kStages + 2 + b); };
+  uint8_t* generic_base = smem_raw + (smem_base - smem_u32(smem_raw));
+  volatile uint32_t* tmem_slot =
+      reinterpret_cast<volatile uint32_t*>(generic_base + kStages * S::kStageBytes + 192);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int total_tiles = p.m_tiles * p.n_tiles;
+  const int k_blocks = (p.K + kBK - 1) / kBK;
+  const int iters = k_blocks * p.terms;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int q = 0; q < p.terms; ++q) {
+      prefetch_tensormap(&p.tmA[q]);
+      prefetch_tensormap(&p.tmB[q]);
+    }
+  }
+  if (warp == 1) {
+    if (lane == 0) {
+      for (int s = 0; s < kStages; ++s) {
+        mbar_init(full_bar(s), 1);
+        mbar_init(empty_bar(s), 1);
+      }
+      for (int b = 0; b < 2; ++b) {
+        mbar_init(acc_full_bar(b), 1);
+        mbar_init(acc_empty_bar(b), 4);
+      }
+      fence_barrier_init();
+    }
+    __syncwarp();
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      uint32_t issued_mask = 0;  // stages that have had a load issued
+      uint32_t last_parity = 0;  // parity of the last load issued, per stage
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int m0 = (tile / p.n_tiles) * kBM;
+        const int n0 = (tile % p.n_tiles) * BN;
+        for (int it = 0; it < iters; ++it) {
+          const int kb = it / p.terms;
+          const int q = it - kb * p.terms;
+          if (!mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, 1u)) {
+            ok = false;
+            break;
+          }
+          mbar_arrive_expect_tx(full_bar(stage), S::kStageBytes);
+          tma_load_2d(smem_a + stage * S::kABytes, &p.tmA[q], kb * kBK, m0, full_bar(stage));
+          tma_load_2d(smem_b + stage * S::kBBytes, &p.tmB[q], kb * kBK, n0, full_bar(stage));
+          issued_mask |= 1u << stage;
+          last_parity = (last_parity & ~(1u << stage)) | (phase << stage);
+          if (++stage == kStages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+      }
+      if (!ok) {
+        // leave no copy in flight behind: wait (bounded) for every load issued
+        for (int s = 0; s < kStages; ++s) {
+          if (!(issued_mask & (1u << s))) continue;
+          const uint64_t t0 = global_timer_ns();
+          while (!mbar_try_wait(full_bar(s), (last_parity >> s) & 1u)) {
+            if (global_timer_ns() - t0 > 1000000ull) break;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // -------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int lt = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++lt) {
+        const int buf = lt & 1;
+        const uint32_t acc_phase = (lt >> 1) & 1;
+        if (!mbar_wait_bounded(acc_empty_bar(buf), acc_phase ^ 1u, abort_flag, 2u)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * BN);
+        for (int it = 0; it < iters; ++it) {
+          if (!mbar_wait_bounded(full_bar(stage), phase, abort_flag, 3u)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after_sync();
+          const uint64_t a_desc = umma_desc_kmajor_sw128(smem_a + stage * S::kABytes, 1024);
+          const uint64_t b_desc = umma_desc_kmajor_sw128(smem_b + stage * S::kBBytes, 1024);
+#pragma unroll
+          for (int kk = 0; kk < kBK / 16; ++kk) {
+            // 16 k-elements = 32 bytes further along the swizzled row: +2 in address>>4 units
+            tc_mma_bf16(d_tmem, a_desc + 2u * kk, b_desc + 2u * kk, kIdesc, (it > 0 || kk > 0) ? 1u : 0u);
+          }
+          tc_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
+          if (++stage == kStages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+        if (ok) tc_commit(acc_full_bar(buf));  // accumulator complete
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue
+    const int lane_group = warp & 3;  // a warp may touch only tensor-memory lanes 32*(warp%4)..+31
+    int lt = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++lt) {
+      const int m_tile = tile / p.n_tiles;
+      const int n_tile = tile % p.n_tiles;
+      const int row = m_tile * kBM + lane_group * 32 + lane;
+      const int n0 = n_tile * BN;
+      const int buf = lt & 1;
+      const uint32_t acc_phase = (lt >> 1) & 1;
+      // the tensor-memory loads below are warp-collective: the whole warp goes on or the whole warp leaves
+      const bool got = mbar_wait_bounded(acc_full_bar(buf), acc_phase, abort_flag, 4u);
+      if (!__all_sync(0xffffffffu, got)) {
+        ok = false;
+        break;
+      }
+      tc_fence_after_sync();
+      const uint32_t t_addr =
+          tmem_base + (static_cast<uint32_t>(lane_group * 32) << 16) + static_cast<uint32_t>(buf * BN);
+      const bool row_ok = row < p.M;
+      uint32_t v[32];
+
+      if constexpr (EPI == kStoreF32) {
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          tmem_ld_32x32(t_addr + c0, v);
+          tc_wait_ld();
+          if (row_ok) {
+            float4* dst = reinterpret_cast<float4*>(p.out + static_cast<long long>(row) * p.ldo + n0 + c0);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                   __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+            }
+          }
+        }
+      } else if constexpr (EPI == kMoments) {
+        // pass 1: mean of the BN columns; pass 2: central power sums about it
+        float s1 = 0.f;
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          tmem_ld_32x32(t_addr + c0, v);
+          tc_wait_ld();
+          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            a0 += __uint_as_float(v[j]);
+            a1 += __uint_as_float(v[j + 1]);
+            a2 += __uint_as_float(v[j + 2]);
+            a3 += __uint_as_float(v[j + 3]);
+          }
+          s1 += (a0 + a1) + (a2 + a3);
+        }
+        const float mean = s1 * (1.0f / BN);
+        float s2 = 0.f, s3 = 0.f, s4 = 0.f;
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          tmem_ld_32x32(t_addr + c0, v);
+          tc_wait_ld();
+          float b2 = 0.f, b3 = 0.f, b4 = 0.f;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const float c = __uint_as_float(v[j]) - mean;
+            const float c2 = c * c;
+            b2 += c2;
+            b3 = fmaf(c2, c, b3);
+            b4 = fmaf(c2, c2, b4);
+          }
+          s2 += b2;
+          s3 += b3;
+          s4 += b4;
+        }
+        if (row_ok) p.partial[static_cast<long long>(n_tile) * p.M + row] = make_float4(mean, s2, s3, s4);
+      } else if constexpr (EPI == kGrad) {
+        float4 cf = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (row_ok) cf = p.coef[row];
+        __nv_bfloat16* gcol = p.gt + static_cast<long long>(n0) * p.ldg + row;
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          tmem_ld_32x32(t_addr + c0, v);
+          tc_wait_ld();
+          if (row_ok) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const float c = __uint_as_float(v[j]) - cf.x;
+              // a c^3 - ab c - am3
+              const float g = fmaf(c, fmaf(cf.y * c, c, -cf.z), -cf.w);
+              gcol[static_cast<long long>(c0 + j) * p.ldg] = __float2bfloat16_rn(g);
+            }
+          }
+        }
+      } else if constexpr (EPI == kAbsMax) {
+        float mx = 0.f;
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          tmem_ld_32x32(t_addr + c0, v);
+          tc_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, fabsf(__uint_as_float(v[j])));
+        }
+        // non-negative floats order like their bit patterns; a max is exact, so arrival order does not matter
+        if (row_ok) atomicMax(p.rowmax + row, __float_as_uint(mx));
+      } else if constexpr (EPI == kQuantErr) {
+        float amax = 0.f;
+        if (row_ok) amax = __uint_as_float(p.rowmax[row]);
+        const float s = __fdiv_rn(amax, 7.0f);
+        float e2 = 0.f;
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          tmem_ld_32x32(t_addr + c0, v);
+          tc_wait_ld();
+          if (s > 0.f) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const float y = __uint_as_float(v[j]);
+              float qv = rintf(__fdiv_rn(y, s));
+              qv = fminf(fmaxf(qv, -7.0f), 7.0f);
+              const float e = __fsub_rn(y, __fmul_rn(qv, s));
+              e2 = fmaf(e, e, e2);
+            }
+          }
+        }
+        if (row_ok) p.qerr[static_cast<long long>(n_tile) * p.M + row] = e2;
+      }
+
+      // hand the accumulator back to the MMA warp
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty_bar(buf));
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+  if (threadIdx.x == 0 && *abort_flag != 0 && p.err_word != nullptr) atomicMax(p.err_word, *abort_flag);
+}
+
+}  // namespace kt
