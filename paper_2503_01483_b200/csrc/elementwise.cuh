@@ -224,11 +224,11 @@ __global__ void k_block_sums_f32(const float* __restrict__ v, long long n, doubl
 }
 
 // ------------------------------------------------------------- Cayley pieces
-// W = (A - A^T)/2 for a d x d float32 A, written as bf16 (the rounding is odd,
-// so the bf16 W is exactly skew), plus per-block sums of W^2 (of the float32 W).
+// W = (A - A^T)/2 for a d x d float32 A, written as bf16 hi (and lo when asked;
+// the rounding is odd, so each bf16 part is exactly skew), plus per-block sums of W^2 (of the float32 W).
 // grid (d/32, d/32), block (32, 8).
 __global__ void k_skew(const float* __restrict__ A, int d, __nv_bfloat16* __restrict__ w_hi,
-                       double* __restrict__ block_norm2) {
+                       __nv_bfloat16* __restrict__ w_lo, double* __restrict__ block_norm2) {
   __shared__ float tT[32][33];
   __shared__ double sh[8];
   const int bj = blockIdx.x, bi = blockIdx.y;
@@ -240,7 +240,10 @@ __global__ void k_skew(const float* __restrict__ A, int d, __nv_bfloat16* __rest
   for (int r = ty; r < 32; r += 8) {
     const long long o = static_cast<long long>(bi * 32 + r) * d + bj * 32 + tx;
     const float w = 0.5f * (A[o] - tT[tx][r]);
-    w_hi[o] = __float2bfloat16_rn(w);
+    __nv_bfloat16 h, l;
+    split_bf16(w, h, l);
+    w_hi[o] = h;
+    if (w_lo) w_lo[o] = l;
     acc += static_cast<double>(w) * w;
   }
   const int lin = ty * 32 + tx;

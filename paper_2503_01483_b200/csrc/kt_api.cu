@@ -1,0 +1,774 @@
+// Host side of libkurtail: argument checks, workspace carving, tensor-map
+// construction and the sequencing of kernels on one stream.  See
+// include/kurtail.h for the contract of every entry point.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <new>
+
+#include "../../include/kurtail.h"
+#include "elementwise.cuh"
+#include "gemm_sm100.cuh"
+
+namespace kt {
+
+constexpr int kHistMax = 4096;  // loss-history slots kept on the device between host read-backs
+
+struct DeviceBlock {
+  Scalars sc;
+  double hist[kHistMax];
+};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Where everything lives inside the caller's workspace for an (N, d) problem.
+struct WsLayout {
+  size_t rt_hi, rt_lo;  // R^T as bf16 hi/lo  [d][d]
+  size_t r_hi, r_lo;    // R   as bf16 hi/lo  [d][d]
+  size_t z_hi, z_lo;    // transposed iterate of the retraction; also dR hi (before) and E hi (after)
+  size_t w_hi, w_lo;    // skew direction W as bf16
+  size_t fbuf;          // d x d float32: A, then P, then R^T R, then R E
+  size_t dr;            // d x d float32: gradient inside kt_fit
+  size_t xb;            // dense bf16 copy of a float32 X  [N][d]
+  size_t xt, gt;        // X^T and G^T as bf16  [d][ldt]
+  size_t partial;       // [P][N] float4 partial moment records
+  size_t coef, moments; // [N] float4 each
+  size_t block_loss, block_deg, norm_blocks;
+  size_t rowmax, qerr;  // quantizer: [N] uint, [P][N] float
+  size_t total;
+  long long ldt;
+  int P, bn, loss_blocks, norm_n;
+};
+
+static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype) {
+  WsLayout L;
+  memset(&L, 0, sizeof(L));
+  L.bn = (d % 256 == 0) ? 256 : 128;
+  L.P = static_cast<int>(d / L.bn);
+  L.ldt = static_cast<long long>(align_up(static_cast<size_t>(N), 64));
+  L.loss_blocks = static_cast<int>((N + 255) / 256);
+  L.norm_n = static_cast<int>((d / 32) * (d / 32));
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes, 256);
+    return o;
+  };
+  const size_t dd = static_cast<size_t>(d) * d;
+  L.rt_hi = take(dd * 2);
+  L.rt_lo = take(dd * 2);
+  L.r_hi = take(dd * 2);
+  L.r_lo = take(dd * 2);
+  L.z_hi = take(dd * 2);
+  L.z_lo = take(dd * 2);
+  L.w_hi = take(dd * 2);
+  L.w_lo = take(dd * 2);
+  L.fbuf = take(dd * 4);
+  L.dr = take(dd * 4);
+  L.xb = take(x_dtype == KT_F32 ? static_cast<size_t>(N) * d * 2 : 0);
+  L.xt = take(static_cast<size_t>(d) * L.ldt * 2);
+  L.gt = take(static_cast<size_t>(d) * L.ldt * 2);
+  L.partial = take(static_cast<size_t>(L.P) * N * 16);
+  L.coef = take(static_cast<size_t>(N) * 16);
+  L.moments = take(static_cast<size_t>(N) * 16);
+  L.block_loss = take(static_cast<size_t>(L.loss_blocks) * 8);
+  L.block_deg = take(static_cast<size_t>(L.loss_blocks) * 4);
+  L.norm_blocks = take(static_cast<size_t>(L.norm_n > 1024 ? L.norm_n : 1024) * 8);
+  L.rowmax = take(static_cast<size_t>(N) * 4);
+  L.qerr = take(static_cast<size_t>(L.P) * N * 4);
+  L.total = off;
+  return L;
+}
+
+}  // namespace kt
+
+struct kt_ctx {
+  kt_config cfg;
+  cudaStream_t stream;
+  int device;
+  int sm_count;
+  uint8_t* ws;
+  size_t ws_bytes;
+  kt::DeviceBlock* d_blk;
+  kt::DeviceBlock* h_blk;  // pinned
+  kt::EncodeTiledFn encode;
+  bool smem_attr_set;
+};
+
+namespace kt {
+
+#define KT_CUDA(call)                       \
+  do {                                      \
+    if ((call) != cudaSuccess) {            \
+      (void)cudaGetLastError();             \
+      return KT_ERR_CUDA;                   \
+    }                                       \
+  } while (0)
+#define KT_LAUNCH_CHECK() KT_CUDA(cudaGetLastError())
+#define KT_TRY(expr)                 \
+  do {                               \
+    kt_status st__ = (expr);         \
+    if (st__ != KT_OK) return st__;  \
+  } while (0)
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static kt_status check_x(const kt_mat& X, int64_t* N, int64_t* d) {
+  if (X.data == nullptr) return KT_ERR_INVALID_ARG;
+  if (X.dtype != KT_BF16 && X.dtype != KT_F32) return KT_ERR_INVALID_ARG;
+  if (X.rows < 1 || X.cols < 128 || X.cols % 128 != 0 || X.ld < X.cols) return KT_ERR_SHAPE;
+  if (X.rows > 0x7fffff00ll || X.cols > 65536) return KT_ERR_SHAPE;
+  const int64_t es = (X.dtype == KT_BF16) ? 2 : 4;
+  if (!aligned16(X.data) || (X.ld * es) % 16 != 0) return KT_ERR_ALIGN;
+  *N = X.rows;
+  *d = X.cols;
+  return KT_OK;
+}
+
+static kt_status check_ws(const kt_ctx* ctx, const WsLayout& L) {
+  if (ctx->ws == nullptr || ctx->ws_bytes < L.total) return KT_ERR_WORKSPACE;
+  return KT_OK;
+}
+
+// bf16 matrix of `rows` rows, `k_extent` valid elements per row, leading
+// dimension ld (elements); tiles of box_rows x 64 elements, 128-byte swizzle,
+// out-of-range elements read as zero.
+static kt_status make_tmap(const kt_ctx* ctx, CUtensorMap* tm, const void* base, uint64_t k_extent, uint64_t rows,
+                           uint64_t ld, uint32_t box_rows) {
+  cuuint64_t dims[2] = {k_extent, rows};
+  cuuint64_t strides[1] = {ld * 2};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(kBK), box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = ctx->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? KT_OK : KT_ERR_CUDA;
+}
+
+template <int BN, int EPI>
+static kt_status launch_gemm_inst(kt_ctx* ctx, const GemmParams& p) {
+  static bool attr_done[16] = {false};
+  const int smem = GemmSmem<BN>::kTotal;
+  if (!attr_done[ctx->device & 15]) {
+    KT_CUDA(cudaFuncSetAttribute(gemm_tn_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    attr_done[ctx->device & 15] = true;
+  }
+  const int tiles = p.m_tiles * p.n_tiles;
+  const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+  gemm_tn_kernel<BN, EPI><<<grid, kGemmThreads, smem, ctx->stream>>>(p);
+  KT_LAUNCH_CHECK();
+  return KT_OK;
+}
+
+struct Operand {
+  const void* base;
+  uint64_t ld;
+};
+
+// D (M x N) = sum_q A_q (M x K) * B_q (N x K)^T with the epilogue EPI.
+template <int EPI>
+static kt_status run_gemm(kt_ctx* ctx, int M, int N, int K, int terms, const Operand* A, const Operand* B,
+                          GemmParams& p) {
+  const int bn = (N % 256 == 0) ? 256 : 128;
+  p.terms = terms;
+  p.M = M;
+  p.N = N;
+  p.K = K;
+  p.m_tiles = (M + kBM - 1) / kBM;
+  p.n_tiles = N / bn;
+  p.err_word = &ctx->d_blk->sc.err_word;
+  for (int q = 0; q < terms; ++q) {
+    KT_TRY(make_tmap(ctx, &p.tmA[q], A[q].base, K, M, A[q].ld, kBM));
+    KT_TRY(make_tmap(ctx, &p.tmB[q], B[q].base, K, N, B[q].ld, bn));
+  }
+  if (bn == 256) return launch_gemm_inst<256, EPI>(ctx, p);
+  return launch_gemm_inst<128, EPI>(ctx, p);
+}
+
+static GemmParams blank_params() {
+  GemmParams p;
+  memset(&p, 0, sizeof(p));
+  return p;
+}
+
+template <typename T>
+static T* at(kt_ctx* ctx, size_t off) {
+  return reinterpret_cast<T*>(ctx->ws + off);
+}
+
+// ---------------------------------------------------------------- X ingest
+struct XView {
+  const __nv_bfloat16* xb;  // bf16 rows
+  long long ldx;
+};
+
+// forward-only view: bf16 X is used in place, float32 X is rounded into the workspace
+static kt_status ingest_x_forward(kt_ctx* ctx, const kt_mat& X, const WsLayout& L, XView* v) {
+  const int64_t N = X.rows, d = X.cols;
+  if (X.dtype == KT_BF16) {
+    v->xb = static_cast<const __nv_bfloat16*>(X.data);
+    v->ldx = X.ld;
+    return KT_OK;
+  }
+  __nv_bfloat16* xb = at<__nv_bfloat16>(ctx, L.xb);
+  const long long pairs = N * d / 2;
+  k_cast_x<<<static_cast<unsigned>((pairs + 255) / 256), 256, 0, ctx->stream>>>(static_cast<const float*>(X.data),
+                                                                                X.ld, N, static_cast<int>(d), xb);
+  KT_LAUNCH_CHECK();
+  v->xb = xb;
+  v->ldx = d;
+  return KT_OK;
+}
+
+// view for loss + gradient: also builds X^T (the token dimension becomes contiguous)
+static kt_status ingest_x_full(kt_ctx* ctx, const kt_mat& X, const WsLayout& L, XView* v) {
+  const int N = static_cast<int>(X.rows), d = static_cast<int>(X.cols);
+  dim3 grid(d / 64, (N + 63) / 64), block(32, 8);
+  __nv_bfloat16* xt = at<__nv_bfloat16>(ctx, L.xt);
+  if (X.dtype == KT_BF16) {
+    k_prepare_x<__nv_bfloat16><<<grid, block, 0, ctx->stream>>>(static_cast<const __nv_bfloat16*>(X.data), X.ld, N, d,
+                                                                xt, L.ldt, nullptr);
+    KT_LAUNCH_CHECK();
+    v->xb = static_cast<const __nv_bfloat16*>(X.data);
+    v->ldx = X.ld;
+  } else {
+    __nv_bfloat16* xb = at<__nv_bfloat16>(ctx, L.xb);
+    k_prepare_x<float><<<grid, block, 0, ctx->stream>>>(static_cast<const float*>(X.data), X.ld, N, d, xt, L.ldt, xb);
+    KT_LAUNCH_CHECK();
+    v->xb = xb;
+    v->ldx = d;
+  }
+  return KT_OK;
+}
+
+// ------------------------------------------------------------ forward pieces
+static kt_status cast_rt(kt_ctx* ctx, const float* R, int d, const WsLayout& L) {
+  dim3 grid(d / 32, d / 32), block(32, 8);
+  k_split_bf16<true><<<grid, block, 0, ctx->stream>>>(R, d, at<__nv_bfloat16>(ctx, L.rt_hi), nullptr, d);
+  KT_LAUNCH_CHECK();
+  return KT_OK;
+}
+
+// moments + loss for the rows of xv; R^T must already be in rt_hi.
+static kt_status forward_loss(kt_ctx* ctx, const XView& xv, int N, int d, const WsLayout& L, double* hist_slot) {
+  GemmParams p = blank_params();
+  p.partial = at<float4>(ctx, L.partial);
+  Operand A{xv.xb, static_cast<uint64_t>(xv.ldx)}, B{at<__nv_bfloat16>(ctx, L.rt_hi), static_cast<uint64_t>(d)};
+  KT_TRY(run_gemm<kMoments>(ctx, N, d, d, 1, &A, &B, p));
+  k_moments_finalize<<<L.loss_blocks, 256, 0, ctx->stream>>>(at<float4>(ctx, L.partial), L.P, N, d, L.bn,
+                                                            ctx->cfg.kappa_target, at<float4>(ctx, L.moments),
+                                                            at<float4>(ctx, L.coef), at<double>(ctx, L.block_loss),
+                                                            at<unsigned int>(ctx, L.block_deg));
+  KT_LAUNCH_CHECK();
+  k_final_sum<<<1, 256, 0, ctx->stream>>>(at<double>(ctx, L.block_loss), L.loss_blocks, 1.0 / N, &ctx->d_blk->sc.loss,
+                                          hist_slot, at<unsigned int>(ctx, L.block_deg), &ctx->d_blk->sc.deg_rows);
+  KT_LAUNCH_CHECK();
+  return KT_OK;
+}
+
+// dR = X^T G, G recomputed from the saved row coefficients.
+static kt_status backward(kt_ctx* ctx, const XView& xv, int N, int d, const WsLayout& L, float* dR) {
+  GemmParams p = blank_params();
+  p.coef = at<float4>(ctx, L.coef);
+  p.gt = at<__nv_bfloat16>(ctx, L.gt);
+  p.ldg = L.ldt;
+  Operand A{xv.xb, static_cast<uint64_t>(xv.ldx)}, B{at<__nv_bfloat16>(ctx, L.rt_hi), static_cast<uint64_t>(d)};
+  KT_TRY(run_gemm<kGrad>(ctx, N, d, d, 1, &A, &B, p));
+  GemmParams p2 = blank_params();
+  p2.out = dR;
+  p2.ldo = d;
+  Operand A2{at<__nv_bfloat16>(ctx, L.xt), static_cast<uint64_t>(L.ldt)},
+      B2{at<__nv_bfloat16>(ctx, L.gt), static_cast<uint64_t>(L.ldt)};
+  KT_TRY(run_gemm<kStoreF32>(ctx, d, d, N, 1, &A2, &B2, p2));
+  return KT_OK;
+}
+
+static kt_status loss_grad_async(kt_ctx* ctx, const XView& xv, int N, int d, const WsLayout& L, const float* R,
+                                 float* dR, double* hist_slot) {
+  KT_TRY(cast_rt(ctx, R, d, L));
+  KT_TRY(forward_loss(ctx, xv, N, d, L, hist_slot));
+  KT_TRY(backward(ctx, xv, N, d, L, dR));
+  return KT_OK;
+}
+
+// ---------------------------------------------------------- orthogonal step
+// E = R^T R - I from the bf16 splits of R^T (rt_hi, rt_lo) and, when
+// `with_polish`, R <- R - R E / 2 if max|E| > polish_thresh (needs r_hi).
+static kt_status guard(kt_ctx* ctx, float* R, int d, const WsLayout& L, bool with_polish) {
+  Scalars* sc = &ctx->d_blk->sc;
+  KT_CUDA(cudaMemsetAsync(&sc->max_e_bits, 0, sizeof(unsigned int), ctx->stream));
+  const uint64_t ld = static_cast<uint64_t>(d);
+  __nv_bfloat16* rt_hi = at<__nv_bfloat16>(ctx, L.rt_hi);
+  __nv_bfloat16* rt_lo = at<__nv_bfloat16>(ctx, L.rt_lo);
+  float* fbuf = at<float>(ctx, L.fbuf);
+  {
+    GemmParams p = blank_params();
+    p.out = fbuf;
+    p.ldo = d;
+    Operand A[3] = {{rt_hi, ld}, {rt_hi, ld}, {rt_lo, ld}};
+    Operand B[3] = {{rt_hi, ld}, {rt_lo, ld}, {rt_hi, ld}};
+    KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 3, A, B, p));
+  }
+  __nv_bfloat16* e_hi = at<__nv_bfloat16>(ctx, L.z_hi);
+  const unsigned blocks = static_cast<unsigned>(static_cast<long long>(d) * d / 4 / 256);
+  k_guard<<<blocks, 256, 0, ctx->stream>>>(fbuf, d, with_polish ? e_hi : nullptr, sc);
+  KT_LAUNCH_CHECK();
+  if (!with_polish) return KT_OK;
+  k_guard_decide<<<1, 1, 0, ctx->stream>>>(sc, ctx->cfg.polish_thresh);
+  KT_LAUNCH_CHECK();
+  {
+    GemmParams p = blank_params();
+    p.out = fbuf;
+    p.ldo = d;
+    p.gate = &sc->gate;
+    Operand A{at<__nv_bfloat16>(ctx, L.r_hi), ld}, B{e_hi, ld};  // (R E)[i][j] = sum_k R[i][k] E[j][k], E symmetric
+    KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 1, &A, &B, p));
+  }
+  k_polish_apply<<<blocks, 256, 0, ctx->stream>>>(R, fbuf, sc);
+  KT_LAUNCH_CHECK();
+  return KT_OK;
+}
+
+static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, float lr, const WsLayout& L,
+                                 bool run_guard) {
+  const kt_config& c = ctx->cfg;
+  Scalars* sc = &ctx->d_blk->sc;
+  const uint64_t ld = static_cast<uint64_t>(d);
+  dim3 tgrid(d / 32, d / 32), tblock(32, 8);
+  __nv_bfloat16* rt_hi = at<__nv_bfloat16>(ctx, L.rt_hi);
+  __nv_bfloat16* rt_lo = at<__nv_bfloat16>(ctx, L.rt_lo);
+  __nv_bfloat16* r_hi = at<__nv_bfloat16>(ctx, L.r_hi);
+  __nv_bfloat16* z_hi = at<__nv_bfloat16>(ctx, L.z_hi);
+  __nv_bfloat16* z_lo = at<__nv_bfloat16>(ctx, L.z_lo);
+  __nv_bfloat16* w_hi = at<__nv_bfloat16>(ctx, L.w_hi);
+  __nv_bfloat16* w_lo = at<__nv_bfloat16>(ctx, L.w_lo);
+  float* fbuf = at<float>(ctx, L.fbuf);
+  const int terms = c.retract_terms < 1 ? 1 : (c.retract_terms > 3 ? 3 : c.retract_terms);
+
+  // A = dR R^T (the gradient needs no more than bf16), W = (A - A^T)/2, alpha
+  k_split_bf16<false><<<tgrid, tblock, 0, ctx->stream>>>(dR, d, z_hi /* dR hi, free until the iterate is written */,
+                                                         nullptr, d);
+  KT_LAUNCH_CHECK();
+  k_split_bf16<false><<<tgrid, tblock, 0, ctx->stream>>>(R, d, r_hi, nullptr, d);
+  KT_LAUNCH_CHECK();
+  k_split_bf16<true><<<tgrid, tblock, 0, ctx->stream>>>(R, d, rt_hi, rt_lo, d);
+  KT_LAUNCH_CHECK();
+  {
+    GemmParams p = blank_params();
+    p.out = fbuf;
+    p.ldo = d;
+    Operand A{z_hi, ld}, B{r_hi, ld};
+    KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 1, &A, &B, p));
+  }
+  k_skew<<<tgrid, tblock, 0, ctx->stream>>>(fbuf, d, w_hi, terms == 3 ? w_lo : nullptr,
+                                            at<double>(ctx, L.norm_blocks));
+  KT_LAUNCH_CHECK();
+  k_step_size<<<1, 256, 0, ctx->stream>>>(at<double>(ctx, L.norm_blocks), L.norm_n, lr, c.q, c.eps, sc);
+  KT_LAUNCH_CHECK();
+
+  // P = W Z, Z^T given as bf16 hi/lo: (W Z)[i][j] = sum_k W[i][k] Zt[j][k]
+  auto product = [&](const __nv_bfloat16* zt_hi, const __nv_bfloat16* zt_lo) -> kt_status {
+    GemmParams p = blank_params();
+    p.out = fbuf;
+    p.ldo = d;
+    Operand A[3] = {{w_hi, ld}, {w_hi, ld}, {w_lo, ld}};
+    Operand B[3] = {{zt_hi, ld}, {zt_lo, ld}, {zt_hi, ld}};
+    return run_gemm<kStoreF32>(ctx, d, d, d, terms, A, B, p);
+  };
+  const int s = c.cayley_iters < 0 ? 0 : c.cayley_iters;
+  // Y0 = R - alpha W R
+  KT_TRY(product(rt_hi, rt_lo));
+  for (int i = 0; i <= s; ++i) {
+    const float cmul = (i == 0) ? 1.0f : 0.5f;
+    if (i < s) {
+      // Z = R + Y_i for the next product
+      k_axpy_split<<<tgrid, tblock, 0, ctx->stream>>>(R, fbuf, sc, cmul, 1.0f, d, nullptr, z_hi, z_lo, nullptr,
+                                                      nullptr);
+      KT_LAUNCH_CHECK();
+      KT_TRY(product(z_hi, z_lo));
+    } else {
+      // R <- Y_s, and its splits for the guard
+      k_axpy_split<<<tgrid, tblock, 0, ctx->stream>>>(R, fbuf, sc, cmul, 0.0f, d, R, rt_hi, rt_lo, r_hi, nullptr);
+      KT_LAUNCH_CHECK();
+    }
+  }
+  if (run_guard) KT_TRY(guard(ctx, R, d, L, true));
+  return KT_OK;
+}
+
+// Copies the scalar block back and synchronises; maps a recorded wait time-out.
+static kt_status sync_scalars(kt_ctx* ctx) {
+  KT_CUDA(cudaMemcpyAsync(&ctx->h_blk->sc, &ctx->d_blk->sc, sizeof(Scalars), cudaMemcpyDeviceToHost, ctx->stream));
+  KT_CUDA(cudaStreamSynchronize(ctx->stream));
+  if (ctx->h_blk->sc.err_word != 0) {
+    (void)cudaMemsetAsync(&ctx->d_blk->sc.err_word, 0, sizeof(unsigned int), ctx->stream);
+    return KT_ERR_TIMEOUT;
+  }
+  return KT_OK;
+}
+
+static kt_status check_d(int64_t d) {
+  if (d < 128 || d % 128 != 0 || d > 65536) return KT_ERR_SHAPE;
+  return KT_OK;
+}
+
+static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps, float lr, kt_fit_report* report) {
+  int64_t N64, d64;
+  KT_TRY(check_x(X, &N64, &d64));
+  if (R == nullptr || steps < 0) return KT_ERR_INVALID_ARG;
+  if (!aligned16(R)) return KT_ERR_ALIGN;
+  const WsLayout L = make_layout(N64, d64, X.dtype);
+  KT_TRY(check_ws(ctx, L));
+  const int N = static_cast<int>(N64), d = static_cast<int>(d64);
+  XView xv;
+  KT_TRY(ingest_x_full(ctx, X, L, &xv));
+  float* dR = at<float>(ctx, L.dr);
+  const int ge = ctx->cfg.guard_every < 1 ? 1 : ctx->cfg.guard_every;
+  double first = 0.0, last = 0.0;
+  int done = 0;
+  for (int k = 0; k < steps; ++k) {
+    const int slot = k % kHistMax;
+    if (k > 0 && slot == 0) {
+      // history block full: bring it to the host before it is overwritten
+      KT_CUDA(cudaMemcpyAsync(ctx->h_blk->hist, ctx->d_blk->hist, sizeof(double) * kHistMax, cudaMemcpyDeviceToHost,
+                              ctx->stream));
+      KT_CUDA(cudaStreamSynchronize(ctx->stream));
+      if (k == kHistMax) first = ctx->h_blk->hist[0];
+      if (report && report->loss_history)
+        memcpy(report->loss_history + (k - kHistMax), ctx->h_blk->hist, sizeof(double) * kHistMax);
+    }
+    KT_TRY(loss_grad_async(ctx, xv, N, d, L, R, dR, &ctx->d_blk->hist[slot]));
+    const bool run_guard = ((k + 1) % ge == 0) || (k + 1 == steps);
+    KT_TRY(orth_step_async(ctx, R, dR, d, lr, L, run_guard));
+    done = k + 1;
+  }
+  if (steps > 0) {
+    const int tail = (steps - 1) % kHistMax + 1;  // entries of the last history block
+    KT_CUDA(cudaMemcpyAsync(ctx->h_blk->hist, ctx->d_blk->hist, sizeof(double) * tail, cudaMemcpyDeviceToHost,
+                            ctx->stream));
+  }
+  kt_status st = sync_scalars(ctx);
+  if (steps > 0) {
+    const int tail = (steps - 1) % kHistMax + 1;
+    if (steps <= kHistMax) first = ctx->h_blk->hist[0];
+    last = ctx->h_blk->hist[tail - 1];
+    if (report && report->loss_history)
+      memcpy(report->loss_history + (steps - tail), ctx->h_blk->hist, sizeof(double) * tail);
+  }
+  if (report) {
+    report->steps_done = done;
+    report->degenerate_rows = static_cast<int32_t>(ctx->h_blk->sc.deg_rows);
+    report->loss_first = first;
+    report->loss_last = last;
+    report->orth_err = static_cast<double>(__builtin_bit_cast(float, ctx->h_blk->sc.max_e_bits));
+    report->alpha_last = ctx->h_blk->sc.alpha;
+    report->w_norm_last = ctx->h_blk->sc.wnorm;
+  }
+  if (st != KT_OK) return st;
+  if (steps > 0 && !isfinite(last)) return KT_ERR_NONFINITE;
+  return KT_OK;
+}
+
+}  // namespace kt
+
+using namespace kt;
+
+// ============================================================== C ABI
+extern "C" {
+
+void kt_default_config(kt_config* cfg) {
+  if (!cfg) return;
+  memset(cfg, 0, sizeof(*cfg));
+  cfg->kappa_target = 1.8f;
+  cfg->cayley_iters = 2;
+  cfg->q = 0.5f;
+  cfg->eps = 1e-8f;
+  cfg->polish_thresh = 1e-6f;
+  cfg->retract_terms = 2;
+  cfg->guard_every = 1;
+}
+
+const char* kt_status_string(kt_status s) {
+  switch (s) {
+    case KT_OK: return "ok";
+    case KT_ERR_INVALID_ARG: return "invalid argument";
+    case KT_ERR_SHAPE: return "unsupported shape";
+    case KT_ERR_ALIGN: return "pointer or leading dimension not 16-byte aligned";
+    case KT_ERR_WORKSPACE: return "workspace missing or too small";
+    case KT_ERR_ARCH: return "device is not sm_100";
+    case KT_ERR_CUDA: return "CUDA call failed";
+    case KT_ERR_NONFINITE: return "non-finite loss";
+    case KT_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+kt_status kt_create(kt_ctx** out, const kt_config* cfg, void* cuda_stream) {
+  if (!out) return KT_ERR_INVALID_ARG;
+  *out = nullptr;
+  int dev = 0;
+  KT_CUDA(cudaGetDevice(&dev));
+  int major = 0, sms = 0;
+  KT_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+  KT_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  if (major != 10) return KT_ERR_ARCH;
+  kt_ctx* c = new (std::nothrow) kt_ctx;
+  if (!c) return KT_ERR_CUDA;
+  memset(c, 0, sizeof(*c));
+  if (cfg) c->cfg = *cfg; else kt_default_config(&c->cfg);
+  c->stream = static_cast<cudaStream_t>(cuda_stream);
+  c->device = dev;
+  c->sm_count = sms;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+      qres != cudaDriverEntryPointSuccess) {
+    delete c;
+    return KT_ERR_CUDA;
+  }
+  c->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  if (cudaMalloc(&c->d_blk, sizeof(DeviceBlock)) != cudaSuccess) {
+    delete c;
+    return KT_ERR_CUDA;
+  }
+  if (cudaMallocHost(&c->h_blk, sizeof(DeviceBlock)) != cudaSuccess) {
+    cudaFree(c->d_blk);
+    delete c;
+    return KT_ERR_CUDA;
+  }
+  if (cudaMemset(c->d_blk, 0, sizeof(DeviceBlock)) != cudaSuccess) {
+    cudaFreeHost(c->h_blk);
+    cudaFree(c->d_blk);
+    delete c;
+    return KT_ERR_CUDA;
+  }
+  memset(c->h_blk, 0, sizeof(DeviceBlock));
+  *out = c;
+  return KT_OK;
+}
+
+void kt_destroy(kt_ctx* ctx) {
+  if (!ctx) return;
+  cudaStreamSynchronize(ctx->stream);
+  cudaFreeHost(ctx->h_blk);
+  cudaFree(ctx->d_blk);
+  delete ctx;
+}
+
+kt_status kt_workspace_bytes(const kt_ctx* ctx, int64_t N, int64_t d, int32_t x_dtype, size_t* bytes) {
+  (void)ctx;
+  if (!bytes) return KT_ERR_INVALID_ARG;
+  if (x_dtype != KT_BF16 && x_dtype != KT_F32) return KT_ERR_INVALID_ARG;
+  if (N < 1 || N > 0x7fffff00ll) return KT_ERR_SHAPE;
+  KT_TRY(check_d(d));
+  *bytes = make_layout(N, d, x_dtype).total;
+  return KT_OK;
+}
+
+kt_status kt_set_workspace(kt_ctx* ctx, void* dev_ptr, size_t bytes) {
+  if (!ctx) return KT_ERR_INVALID_ARG;
+  if (dev_ptr != nullptr && (reinterpret_cast<uintptr_t>(dev_ptr) & 255u) != 0) return KT_ERR_ALIGN;
+  ctx->ws = static_cast<uint8_t*>(dev_ptr);
+  ctx->ws_bytes = dev_ptr ? bytes : 0;
+  return KT_OK;
+}
+
+kt_status kt_init_rotation(kt_ctx* ctx, float* R, int64_t d, int32_t kind) {
+  if (!ctx || !R || (kind != 0 && kind != 1)) return KT_ERR_INVALID_ARG;
+  if (d < 1 || d > 65536) return KT_ERR_SHAPE;
+  if (kind == 1 && (d & (d - 1)) != 0) return KT_ERR_SHAPE;
+  const float scale = static_cast<float>(1.0 / sqrt(static_cast<double>(d)));
+  const long long n = d * d;
+  k_init_rotation<<<static_cast<unsigned>((n + 255) / 256), 256, 0, ctx->stream>>>(R, static_cast<int>(d), kind, scale);
+  KT_LAUNCH_CHECK();
+  return KT_OK;
+}
+
+kt_status kt_kurtosis_loss(kt_ctx* ctx, kt_mat X, const float* R, double* loss) {
+  if (!ctx || !R || !loss) return KT_ERR_INVALID_ARG;
+  int64_t N, d;
+  KT_TRY(check_x(X, &N, &d));
+  if (!aligned16(R)) return KT_ERR_ALIGN;
+  const WsLayout L = make_layout(N, d, X.dtype);
+  KT_TRY(check_ws(ctx, L));
+  XView xv;
+  KT_TRY(ingest_x_forward(ctx, X, L, &xv));
+  KT_TRY(cast_rt(ctx, R, static_cast<int>(d), L));
+  KT_TRY(forward_loss(ctx, xv, static_cast<int>(N), static_cast<int>(d), L, nullptr));
+  KT_TRY(sync_scalars(ctx));
+  *loss = ctx->h_blk->sc.loss;
+  return isfinite(*loss) ? KT_OK : KT_ERR_NONFINITE;
+}
+
+kt_status kt_row_moments(kt_ctx* ctx, kt_mat X, const float* R, float* moments) {
+  if (!ctx || !R || !moments) return KT_ERR_INVALID_ARG;
+  int64_t N, d;
+  KT_TRY(check_x(X, &N, &d));
+  if (!aligned16(R) || !aligned16(moments)) return KT_ERR_ALIGN;
+  const WsLayout L = make_layout(N, d, X.dtype);
+  KT_TRY(check_ws(ctx, L));
+  XView xv;
+  KT_TRY(ingest_x_forward(ctx, X, L, &xv));
+  KT_TRY(cast_rt(ctx, R, static_cast<int>(d), L));
+  KT_TRY(forward_loss(ctx, xv, static_cast<int>(N), static_cast<int>(d), L, nullptr));
+  KT_CUDA(cudaMemcpyAsync(moments, at<float4>(ctx, L.moments), static_cast<size_t>(N) * 16, cudaMemcpyDeviceToDevice,
+                          ctx->stream));
+  return KT_OK;
+}
+
+kt_status kt_rotate(kt_ctx* ctx, kt_mat X, const float* R, float* Y) {
+  if (!ctx || !R || !Y) return KT_ERR_INVALID_ARG;
+  int64_t N, d;
+  KT_TRY(check_x(X, &N, &d));
+  if (!aligned16(R) || !aligned16(Y)) return KT_ERR_ALIGN;
+  const WsLayout L = make_layout(N, d, X.dtype);
+  KT_TRY(check_ws(ctx, L));
+  XView xv;
+  KT_TRY(ingest_x_forward(ctx, X, L, &xv));
+  KT_TRY(cast_rt(ctx, R, static_cast<int>(d), L));
+  GemmParams p = blank_params();
+  p.out = Y;
+  p.ldo = d;
+  Operand A{xv.xb, static_cast<uint64_t>(xv.ldx)}, B{at<__nv_bfloat16>(ctx, L.rt_hi), static_cast<uint64_t>(d)};
+  return run_gemm<kStoreF32>(ctx, static_cast<int>(N), static_cast<int>(d), static_cast<int>(d), 1, &A, &B, p);
+}
+
+kt_status kt_loss_grad(kt_ctx* ctx, kt_mat X, const float* R, float* dR, double* loss) {
+  if (!ctx || !R || !dR) return KT_ERR_INVALID_ARG;
+  int64_t N, d;
+  KT_TRY(check_x(X, &N, &d));
+  if (!aligned16(R) || !aligned16(dR)) return KT_ERR_ALIGN;
+  const WsLayout L = make_layout(N, d, X.dtype);
+  KT_TRY(check_ws(ctx, L));
+  XView xv;
+  KT_TRY(ingest_x_full(ctx, X, L, &xv));
+  KT_TRY(loss_grad_async(ctx, xv, static_cast<int>(N), static_cast<int>(d), L, R, dR, nullptr));
+  if (!loss) return KT_OK;
+  KT_TRY(sync_scalars(ctx));
+  *loss = ctx->h_blk->sc.loss;
+  return isfinite(*loss) ? KT_OK : KT_ERR_NONFINITE;
+}
+
+kt_status kt_orth_step(kt_ctx* ctx, float* R, const float* dR, int64_t d, float lr) {
+  if (!ctx || !R || !dR || !(lr >= 0.f)) return KT_ERR_INVALID_ARG;
+  KT_TRY(check_d(d));
+  if (!aligned16(R) || !aligned16(dR)) return KT_ERR_ALIGN;
+  const WsLayout L = make_layout(1, d, KT_BF16);
+  KT_TRY(check_ws(ctx, L));
+  return orth_step_async(ctx, R, dR, static_cast<int>(d), lr, L, true);
+}
+
+kt_status kt_orth_error(kt_ctx* ctx, const float* R, int64_t d, double* err) {
+  if (!ctx || !R || !err) return KT_ERR_INVALID_ARG;
+  KT_TRY(check_d(d));
+  if (!aligned16(R)) return KT_ERR_ALIGN;
+  const WsLayout L = make_layout(1, d, KT_BF16);
+  KT_TRY(check_ws(ctx, L));
+  dim3 tgrid(static_cast<unsigned>(d / 32), static_cast<unsigned>(d / 32)), tblock(32, 8);
+  k_split_bf16<true><<<tgrid, tblock, 0, ctx->stream>>>(R, d, at<__nv_bfloat16>(ctx, L.rt_hi),
+                                                        at<__nv_bfloat16>(ctx, L.rt_lo), d);
+  KT_LAUNCH_CHECK();
+  KT_TRY(guard(ctx, nullptr, static_cast<int>(d), L, false));
+  KT_TRY(sync_scalars(ctx));
+  *err = static_cast<double>(__builtin_bit_cast(float, ctx->h_blk->sc.max_e_bits));
+  return KT_OK;
+}
+
+kt_status kt_fit(kt_ctx* ctx, kt_mat X, float* R, int32_t steps, float lr, kt_fit_report* report) {
+  if (!ctx || !(lr >= 0.f)) return KT_ERR_INVALID_ARG;
+  return fit_impl(ctx, X, R, steps, lr, report);
+}
+
+kt_status kt_fit_layers(kt_ctx* ctx, const kt_mat* X_layers, float* const* R_layers, int32_t L, int32_t first_layer,
+                        int32_t steps, float lr, kt_fit_report* per_layer) {
+  if (!ctx || !X_layers || !R_layers || L < 0 || first_layer < 0 || first_layer > L || !(lr >= 0.f))
+    return KT_ERR_INVALID_ARG;
+  // validate every layer before touching any
+  for (int l = first_layer; l < L; ++l) {
+    int64_t N, d;
+    KT_TRY(check_x(X_layers[l], &N, &d));
+    if (R_layers[l] == nullptr) return KT_ERR_INVALID_ARG;
+    if (!aligned16(R_layers[l])) return KT_ERR_ALIGN;
+    if (X_layers[l].rows != X_layers[first_layer].rows || X_layers[l].cols != X_layers[first_layer].cols ||
+        X_layers[l].dtype != X_layers[first_layer].dtype)
+      return KT_ERR_SHAPE;
+  }
+  for (int l = first_layer; l < L; ++l) {
+    KT_TRY(fit_impl(ctx, X_layers[l], R_layers[l], steps, lr, per_layer ? &per_layer[l] : nullptr));
+  }
+  return KT_OK;
+}
+
+kt_status kt_fit_host(kt_ctx* ctx, kt_mat X_host, void* X_dev_staging, float* R_host, float* R_dev, int32_t steps,
+                      float lr, kt_fit_report* report) {
+  if (!ctx || !X_dev_staging || !R_host || !R_dev || !(lr >= 0.f) || steps < 0) return KT_ERR_INVALID_ARG;
+  kt_mat Xd = X_host;
+  Xd.data = X_dev_staging;
+  int64_t N, d;
+  KT_TRY(check_x(Xd, &N, &d));
+  if (X_host.data == nullptr) return KT_ERR_INVALID_ARG;
+  if (!aligned16(R_dev)) return KT_ERR_ALIGN;
+  const WsLayout L = make_layout(N, d, Xd.dtype);
+  KT_TRY(check_ws(ctx, L));
+  const size_t es = (Xd.dtype == KT_BF16) ? 2 : 4;
+  KT_CUDA(cudaMemcpyAsync(X_dev_staging, X_host.data, static_cast<size_t>(N) * Xd.ld * es, cudaMemcpyHostToDevice,
+                          ctx->stream));
+  KT_CUDA(cudaMemcpyAsync(R_dev, R_host, static_cast<size_t>(d) * d * 4, cudaMemcpyHostToDevice, ctx->stream));
+  kt_status st = fit_impl(ctx, Xd, R_dev, steps, lr, report);
+  KT_CUDA(cudaMemcpyAsync(R_host, R_dev, static_cast<size_t>(d) * d * 4, cudaMemcpyDeviceToHost, ctx->stream));
+  KT_CUDA(cudaStreamSynchronize(ctx->stream));
+  return st;
+}
+
+kt_status kt_quant4_error(kt_ctx* ctx, kt_mat X, const float* R, double* mse) {
+  if (!ctx || !R || !mse) return KT_ERR_INVALID_ARG;
+  int64_t N64, d64;
+  KT_TRY(check_x(X, &N64, &d64));
+  if (!aligned16(R)) return KT_ERR_ALIGN;
+  const WsLayout L = make_layout(N64, d64, X.dtype);
+  KT_TRY(check_ws(ctx, L));
+  const int N = static_cast<int>(N64), d = static_cast<int>(d64);
+  XView xv;
+  KT_TRY(ingest_x_forward(ctx, X, L, &xv));
+  KT_TRY(cast_rt(ctx, R, d, L));
+  unsigned int* rowmax = at<unsigned int>(ctx, L.rowmax);
+  KT_CUDA(cudaMemsetAsync(rowmax, 0, static_cast<size_t>(N) * 4, ctx->stream));
+  Operand A{xv.xb, static_cast<uint64_t>(xv.ldx)}, B{at<__nv_bfloat16>(ctx, L.rt_hi), static_cast<uint64_t>(d)};
+  {
+    GemmParams p = blank_params();
+    p.rowmax = rowmax;
+    KT_TRY(run_gemm<kAbsMax>(ctx, N, d, d, 1, &A, &B, p));
+  }
+  {
+    GemmParams p = blank_params();
+    p.rowmax = rowmax;
+    p.qerr = at<float>(ctx, L.qerr);
+    KT_TRY(run_gemm<kQuantErr>(ctx, N, d, d, 1, &A, &B, p));
+  }
+  const long long n = static_cast<long long>(L.P) * N;
+  k_block_sums_f32<<<1024, 256, 0, ctx->stream>>>(at<float>(ctx, L.qerr), n, at<double>(ctx, L.norm_blocks));
+  KT_LAUNCH_CHECK();
+  k_final_sum<<<1, 256, 0, ctx->stream>>>(at<double>(ctx, L.norm_blocks), 1024, 1.0 / (static_cast<double>(N) * d),
+                                          &ctx->d_blk->sc.qmse, nullptr, nullptr, nullptr);
+  KT_LAUNCH_CHECK();
+  KT_TRY(sync_scalars(ctx));
+  *mse = ctx->h_blk->sc.qmse;
+  return isfinite(*mse) ? KT_OK : KT_ERR_NONFINITE;
+}
+
+kt_status kt_quant4_codes(kt_ctx* ctx, const float* Y, int64_t N, int64_t d, int8_t* codes, float* scales) {
+  if (!ctx || !Y || !codes || !scales) return KT_ERR_INVALID_ARG;
+  if (N < 1 || d < 1 || N > 0x7fffffffll || d > 0x7fffffffll) return KT_ERR_SHAPE;
+  k_quant4_codes<<<static_cast<unsigned>(N), 256, 0, ctx->stream>>>(Y, static_cast<int>(d), codes, scales);
+  KT_LAUNCH_CHECK();
+  return KT_OK;
+}
+
+}  // extern "C"

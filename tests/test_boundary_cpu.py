@@ -1,0 +1,78 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every
+symbol the header declares, and its host-only entry points behave."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2503_01483_b200 import build, kurtail
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    build.build()
+    return kurtail.lib()
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "kurtail.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(kt_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(L):
+    names = _declared_symbols()
+    assert len(names) >= 18
+    for n in names:
+        assert hasattr(L, n), n
+    assert sorted(kurtail.EXPORTS) == names
+
+
+def test_status_strings(L):
+    seen = set()
+    for code in range(9):
+        s = L.kt_status_string(code)
+        assert s and s not in seen
+        seen.add(s)
+    assert L.kt_status_string(0) == b"ok"
+
+
+def test_default_config(L):
+    cfg = kurtail.default_config()
+    assert cfg.kappa_target == pytest.approx(1.8)
+    assert cfg.cayley_iters == 2 and cfg.q == 0.5 and cfg.retract_terms == 2 and cfg.guard_every == 1
+
+
+def test_workspace_bytes_host_only(L):
+    n = C.c_size_t()
+    assert L.kt_workspace_bytes(None, 65536, 4096, kurtail.KT_BF16, C.byref(n)) == 0
+    big = n.value
+    # two transposed bf16 copies of X dominate: 2 * N * d * 2 bytes
+    assert big >= 2 * 65536 * 4096 * 2
+    assert big < 3 * 2**30
+    assert L.kt_workspace_bytes(None, 65536, 4096, kurtail.KT_F32, C.byref(n)) == 0
+    assert n.value >= big + 65536 * 4096 * 2
+    assert L.kt_workspace_bytes(None, 100, 100, 0, C.byref(n)) == 2      # d not a multiple of 128
+    assert L.kt_workspace_bytes(None, 0, 128, 0, C.byref(n)) == 2        # N < 1
+    assert L.kt_workspace_bytes(None, 10, 128, 7, C.byref(n)) == 1       # unknown dtype
+    assert L.kt_workspace_bytes(None, 10, 128, 0, None) == 1
+
+
+def test_null_context_is_rejected(L):
+    m = kurtail.kt_mat(0, 0, 0, 128, 128, 128)
+    out = C.c_double()
+    assert L.kt_kurtosis_loss(None, m, None, C.byref(out)) == 1
+    assert L.kt_set_workspace(None, None, 0) == 1
+    L.kt_destroy(None)  # must be a no-op
+
+
+def test_create_without_gpu_fails_cleanly(L):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    h = C.c_void_p()
+    st = L.kt_create(C.byref(h), None, None)
+    assert st in (5, 6) and not h.value
