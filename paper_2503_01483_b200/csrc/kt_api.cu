@@ -312,9 +312,10 @@ static kt_status guard(kt_ctx* ctx, float* R, int d, const WsLayout& L, bool wit
     GemmParams p = blank_params();
     p.out = fbuf;
     p.ldo = d;
-    Operand A[3] = {{rt_hi, ld}, {rt_hi, ld}, {rt_lo, ld}};
-    Operand B[3] = {{rt_hi, ld}, {rt_lo, ld}, {rt_hi, ld}};
-    KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 3, A, B, p));
+    // (H + L)^T (H + L) with all four products: dropping L^T L would bias the diagonal by sum_k L_ki^2 ~ 1e-6
+    Operand A[4] = {{rt_hi, ld}, {rt_hi, ld}, {rt_lo, ld}, {rt_lo, ld}};
+    Operand B[4] = {{rt_hi, ld}, {rt_lo, ld}, {rt_hi, ld}, {rt_lo, ld}};
+    KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 4, A, B, p));
   }
   __nv_bfloat16* e_hi = at<__nv_bfloat16>(ctx, L.z_hi);
   const unsigned blocks = static_cast<unsigned>(static_cast<long long>(d) * d / 4 / 256);
