@@ -15,8 +15,9 @@
  *   16 (the tiles are fetched by TMA).  R and dR are dense d x d float32,
  *   16-byte aligned.
  * Precision.  X is used as bfloat16 (float32 X is rounded once on entry), R is
- *   kept in float32 and rounded to bfloat16 for the token GEMMs; all products
- *   accumulate in float32 on the tensor cores.
+ *   kept in float32 and rounded to bfloat16 for the token GEMMs (see
+ *   kt_config.forward_terms); all products accumulate in float32 on the
+ *   tensor cores.
  * Stream.  All work is issued on the stream given to kt_create().  Calls that
  *   return a host scalar synchronise that stream; the others are stream
  *   ordered and return after enqueueing.
@@ -69,14 +70,20 @@ typedef struct {
   int32_t cayley_iters; /* [2]   fixed-point iterations s of the Cayley step    */
   float q;              /* [0.5] contraction bound: alpha <= 2q / ||W||_F       */
   float eps;            /* [1e-8] added to ||W||_F in that bound                */
-  float polish_thresh;  /* [1e-6] the Newton-Schulz polish runs when
+  float polish_thresh;  /* [1e-5] the Newton-Schulz polish runs when
                            max|R^T R - I| exceeds this; < 0: every step;
-                           +inf: never                                          */
+                           +inf: never.  (The guard measures R^T R from a
+                           two-term bf16 split: its noise floor is about
+                           2e-5/sqrt(d).)                                       */
   int32_t retract_terms;/* [2]   bf16 split terms (1..3) of the iterate in the
                            retraction products; more = closer to float32       */
   int32_t guard_every;  /* [1]   in kt_fit: run the orthogonality guard every
                            this many steps (and always after the last one)     */
-  int32_t reserved[5];
+  int32_t forward_terms;/* [0]   bf16 terms of R in the token GEMMs: 1 = R rounded
+                           to bf16; 2 = hi + lo (about 16 significant bits,
+                           twice the MMA work); 0 = 2 when d <= 512 (where the
+                           pass is memory bound anyway), else 1                */
+  int32_t reserved[4];
 } kt_config;
 
 /* Filled by kt_fit / kt_fit_layers (host memory). */

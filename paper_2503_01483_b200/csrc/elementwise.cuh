@@ -306,11 +306,38 @@ __global__ void k_axpy_split(const float* R, const float* __restrict__ P, const 
   }
 }
 
-// E = S - I (S = R^T R, d x d float32): max|E| into sc->max_e_bits (atomic max on
-// the bit pattern of a non-negative float: exact, order independent) and E as
-// bf16 when e_hi != null.  grid d*d/4/256, block 256; d*d a multiple of 1024.
-__global__ void k_guard(const float* __restrict__ S, int d, __nv_bfloat16* __restrict__ e_hi,
-                        Scalars* __restrict__ sc) {
+// Column sums of squares of a d x d float32 R, by row slabs of 32:
+// colpart[slab][j] = sum over the slab's 32 rows of R[i][j]^2.
+// grid (d/32, d/32), block (32, 8).
+__global__ void k_colnorm_partial(const float* __restrict__ R, int d, float* __restrict__ colpart) {
+  __shared__ float sh[8][33];
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  float acc = 0.f;
+  for (int r = ty; r < 32; r += 8) {
+    const float v = R[static_cast<long long>(r0 + r) * d + c0 + tx];
+    acc = fmaf(v, v, acc);
+  }
+  sh[ty][tx] = acc;
+  __syncthreads();
+  if (ty == 0) {
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s += sh[i][tx];
+    colpart[static_cast<long long>(blockIdx.y) * d + c0 + tx] = s;
+  }
+}
+
+// E = S - I (S = R^T R from the tensor cores, d x d float32): max|E| into
+// sc->max_e_bits (atomic max on the bit pattern of a non-negative float: exact,
+// order independent) and E as bf16 when e_hi != null.  The diagonal is NOT taken
+// from S: the tensor-core accumulator truncates, which biases a sum of d
+// positive terms near 1 by about one unit in the last place per MMA step; it is
+// rebuilt from the exact column norms, E_jj = sum_slabs colpart[slab][j] - 1
+// (accumulated in double).  Off-diagonal sums hover around 0 and carry no such
+// bias.  grid d*d/4/256, block 256; d*d a multiple of 1024.
+__global__ void k_guard(const float* __restrict__ S, int d, const float* __restrict__ colpart, int nslabs,
+                        __nv_bfloat16* __restrict__ e_hi, Scalars* __restrict__ sc) {
   const long long i4 = (static_cast<long long>(blockIdx.x) * 256 + threadIdx.x) * 4;
   const float4 s = *reinterpret_cast<const float4*>(S + i4);
   const int row = static_cast<int>(i4 / d), col = static_cast<int>(i4 % d);
@@ -319,7 +346,11 @@ __global__ void k_guard(const float* __restrict__ S, int d, __nv_bfloat16* __res
   bool bad = false;
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    if (col + j == row) e[j] -= 1.0f;
+    if (col + j == row) {
+      double n2 = 0.0;
+      for (int b = 0; b < nslabs; ++b) n2 += static_cast<double>(colpart[static_cast<long long>(b) * d + row]);
+      e[j] = static_cast<float>(n2 - 1.0);
+    }
     bad |= (e[j] != e[j]);
     mx = fmaxf(mx, fabsf(e[j]));
   }

@@ -26,7 +26,7 @@ namespace kt {
 constexpr int kBM = 128;           // rows per tile = tensor-memory lanes
 constexpr int kBK = 64;            // k elements per pipeline stage (one 128-byte swizzle row)
 constexpr int kGemmThreads = 192;  // 6 warps
-constexpr int kMaxTerms = 4;
+constexpr int kMaxTerms = 3;
 
 enum Epi : int { kStoreF32 = 0, kMoments = 1, kGrad = 2, kAbsMax = 3, kQuantErr = 4 };
 

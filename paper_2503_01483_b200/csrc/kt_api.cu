@@ -42,6 +42,7 @@ struct WsLayout {
   size_t coef, moments; // [N] float4 each
   size_t block_loss, block_deg, norm_blocks;
   size_t rowmax, qerr;  // quantizer: [N] uint, [P][N] float
+  size_t colpart;       // [d/32][d] float: column sums of squares of R by row slab
   size_t total;
   long long ldt;
   int P, bn, loss_blocks, norm_n;
@@ -83,6 +84,7 @@ static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype) {
   L.norm_blocks = take(static_cast<size_t>(L.norm_n > 1024 ? L.norm_n : 1024) * 8);
   L.rowmax = take(static_cast<size_t>(N) * 4);
   L.qerr = take(static_cast<size_t>(L.P) * N * 4);
+  L.colpart = take(static_cast<size_t>(d / 32) * d * 4);
   L.total = off;
   return L;
 }
@@ -249,19 +251,41 @@ static kt_status ingest_x_full(kt_ctx* ctx, const kt_mat& X, const WsLayout& L, 
 }
 
 // ------------------------------------------------------------ forward pieces
+// How many bf16 terms of R the token GEMMs use: 1 (R rounded to bf16) or 2 (hi + lo, ~16 significant bits).
+static int forward_terms(const kt_ctx* ctx, int d) {
+  const int t = ctx->cfg.forward_terms;
+  if (t == 1 || t == 2) return t;
+  return d <= 512 ? 2 : 1;
+}
+
 static kt_status cast_rt(kt_ctx* ctx, const float* R, int d, const WsLayout& L) {
   dim3 grid(d / 32, d / 32), block(32, 8);
-  k_split_bf16<true><<<grid, block, 0, ctx->stream>>>(R, d, at<__nv_bfloat16>(ctx, L.rt_hi), nullptr, d);
+  k_split_bf16<true><<<grid, block, 0, ctx->stream>>>(
+      R, d, at<__nv_bfloat16>(ctx, L.rt_hi), forward_terms(ctx, d) == 2 ? at<__nv_bfloat16>(ctx, L.rt_lo) : nullptr, d);
   KT_LAUNCH_CHECK();
   return KT_OK;
+}
+
+// Operands of Y = X R for the token GEMMs: X against R^T hi (and lo).
+struct FwdOperands {
+  Operand A[2], B[2];
+  int terms;
+};
+static FwdOperands fwd_operands(kt_ctx* ctx, const XView& xv, int d, const WsLayout& L) {
+  FwdOperands f;
+  f.terms = forward_terms(ctx, d);
+  f.A[0] = f.A[1] = Operand{xv.xb, static_cast<uint64_t>(xv.ldx)};
+  f.B[0] = Operand{at<__nv_bfloat16>(ctx, L.rt_hi), static_cast<uint64_t>(d)};
+  f.B[1] = Operand{at<__nv_bfloat16>(ctx, L.rt_lo), static_cast<uint64_t>(d)};
+  return f;
 }
 
 // moments + loss for the rows of xv; R^T must already be in rt_hi.
 static kt_status forward_loss(kt_ctx* ctx, const XView& xv, int N, int d, const WsLayout& L, double* hist_slot) {
   GemmParams p = blank_params();
   p.partial = at<float4>(ctx, L.partial);
-  Operand A{xv.xb, static_cast<uint64_t>(xv.ldx)}, B{at<__nv_bfloat16>(ctx, L.rt_hi), static_cast<uint64_t>(d)};
-  KT_TRY(run_gemm<kMoments>(ctx, N, d, d, 1, &A, &B, p));
+  const FwdOperands f = fwd_operands(ctx, xv, d, L);
+  KT_TRY(run_gemm<kMoments>(ctx, N, d, d, f.terms, f.A, f.B, p));
   k_moments_finalize<<<L.loss_blocks, 256, 0, ctx->stream>>>(at<float4>(ctx, L.partial), L.P, N, d, L.bn,
                                                             ctx->cfg.kappa_target, at<float4>(ctx, L.moments),
                                                             at<float4>(ctx, L.coef), at<double>(ctx, L.block_loss),
@@ -279,8 +303,8 @@ static kt_status backward(kt_ctx* ctx, const XView& xv, int N, int d, const WsLa
   p.coef = at<float4>(ctx, L.coef);
   p.gt = at<__nv_bfloat16>(ctx, L.gt);
   p.ldg = L.ldt;
-  Operand A{xv.xb, static_cast<uint64_t>(xv.ldx)}, B{at<__nv_bfloat16>(ctx, L.rt_hi), static_cast<uint64_t>(d)};
-  KT_TRY(run_gemm<kGrad>(ctx, N, d, d, 1, &A, &B, p));
+  const FwdOperands f = fwd_operands(ctx, xv, d, L);
+  KT_TRY(run_gemm<kGrad>(ctx, N, d, d, f.terms, f.A, f.B, p));
   GemmParams p2 = blank_params();
   p2.out = dR;
   p2.ldo = d;
@@ -301,8 +325,13 @@ static kt_status loss_grad_async(kt_ctx* ctx, const XView& xv, int N, int d, con
 // ---------------------------------------------------------- orthogonal step
 // E = R^T R - I from the bf16 splits of R^T (rt_hi, rt_lo) and, when
 // `with_polish`, R <- R - R E / 2 if max|E| > polish_thresh (needs r_hi).
-static kt_status guard(kt_ctx* ctx, float* R, int d, const WsLayout& L, bool with_polish) {
+static kt_status guard(kt_ctx* ctx, const float* R_in, float* R, int d, const WsLayout& L, bool with_polish) {
   Scalars* sc = &ctx->d_blk->sc;
+  {
+    dim3 tgrid(d / 32, d / 32), tblock(32, 8);
+    k_colnorm_partial<<<tgrid, tblock, 0, ctx->stream>>>(R_in, d, at<float>(ctx, L.colpart));
+    KT_LAUNCH_CHECK();
+  }
   KT_CUDA(cudaMemsetAsync(&sc->max_e_bits, 0, sizeof(unsigned int), ctx->stream));
   const uint64_t ld = static_cast<uint64_t>(d);
   __nv_bfloat16* rt_hi = at<__nv_bfloat16>(ctx, L.rt_hi);
@@ -312,14 +341,14 @@ static kt_status guard(kt_ctx* ctx, float* R, int d, const WsLayout& L, bool wit
     GemmParams p = blank_params();
     p.out = fbuf;
     p.ldo = d;
-    // (H + L)^T (H + L) with all four products: dropping L^T L would bias the diagonal by sum_k L_ki^2 ~ 1e-6
-    Operand A[4] = {{rt_hi, ld}, {rt_hi, ld}, {rt_lo, ld}, {rt_lo, ld}};
-    Operand B[4] = {{rt_hi, ld}, {rt_lo, ld}, {rt_hi, ld}, {rt_lo, ld}};
-    KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 4, A, B, p));
+    // (H + L)^T (H + L) without L^T L: that term only matters on the diagonal, which k_guard rebuilds exactly
+    Operand A[3] = {{rt_hi, ld}, {rt_hi, ld}, {rt_lo, ld}};
+    Operand B[3] = {{rt_hi, ld}, {rt_lo, ld}, {rt_hi, ld}};
+    KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 3, A, B, p));
   }
   __nv_bfloat16* e_hi = at<__nv_bfloat16>(ctx, L.z_hi);
   const unsigned blocks = static_cast<unsigned>(static_cast<long long>(d) * d / 4 / 256);
-  k_guard<<<blocks, 256, 0, ctx->stream>>>(fbuf, d, with_polish ? e_hi : nullptr, sc);
+  k_guard<<<blocks, 256, 0, ctx->stream>>>(fbuf, d, at<float>(ctx, L.colpart), d / 32, with_polish ? e_hi : nullptr, sc);
   KT_LAUNCH_CHECK();
   if (!with_polish) return KT_OK;
   k_guard_decide<<<1, 1, 0, ctx->stream>>>(sc, ctx->cfg.polish_thresh);
@@ -400,7 +429,7 @@ static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, 
       KT_LAUNCH_CHECK();
     }
   }
-  if (run_guard) KT_TRY(guard(ctx, R, d, L, true));
+  if (run_guard) KT_TRY(guard(ctx, R, R, d, L, true));
   return KT_OK;
 }
 
@@ -491,9 +520,10 @@ void kt_default_config(kt_config* cfg) {
   cfg->cayley_iters = 2;
   cfg->q = 0.5f;
   cfg->eps = 1e-8f;
-  cfg->polish_thresh = 1e-6f;
+  cfg->polish_thresh = 1e-5f;
   cfg->retract_terms = 2;
   cfg->guard_every = 1;
+  cfg->forward_terms = 0;
 }
 
 const char* kt_status_string(kt_status s) {
@@ -637,8 +667,8 @@ kt_status kt_rotate(kt_ctx* ctx, kt_mat X, const float* R, float* Y) {
   GemmParams p = blank_params();
   p.out = Y;
   p.ldo = d;
-  Operand A{xv.xb, static_cast<uint64_t>(xv.ldx)}, B{at<__nv_bfloat16>(ctx, L.rt_hi), static_cast<uint64_t>(d)};
-  return run_gemm<kStoreF32>(ctx, static_cast<int>(N), static_cast<int>(d), static_cast<int>(d), 1, &A, &B, p);
+  const FwdOperands f = fwd_operands(ctx, xv, static_cast<int>(d), L);
+  return run_gemm<kStoreF32>(ctx, static_cast<int>(N), static_cast<int>(d), static_cast<int>(d), f.terms, f.A, f.B, p);
 }
 
 kt_status kt_loss_grad(kt_ctx* ctx, kt_mat X, const float* R, float* dR, double* loss) {
@@ -676,7 +706,7 @@ kt_status kt_orth_error(kt_ctx* ctx, const float* R, int64_t d, double* err) {
   k_split_bf16<true><<<tgrid, tblock, 0, ctx->stream>>>(R, d, at<__nv_bfloat16>(ctx, L.rt_hi),
                                                         at<__nv_bfloat16>(ctx, L.rt_lo), d);
   KT_LAUNCH_CHECK();
-  KT_TRY(guard(ctx, nullptr, static_cast<int>(d), L, false));
+  KT_TRY(guard(ctx, R, nullptr, static_cast<int>(d), L, false));
   KT_TRY(sync_scalars(ctx));
   *err = static_cast<double>(__builtin_bit_cast(float, ctx->h_blk->sc.max_e_bits));
   return KT_OK;
@@ -741,17 +771,17 @@ kt_status kt_quant4_error(kt_ctx* ctx, kt_mat X, const float* R, double* mse) {
   KT_TRY(cast_rt(ctx, R, d, L));
   unsigned int* rowmax = at<unsigned int>(ctx, L.rowmax);
   KT_CUDA(cudaMemsetAsync(rowmax, 0, static_cast<size_t>(N) * 4, ctx->stream));
-  Operand A{xv.xb, static_cast<uint64_t>(xv.ldx)}, B{at<__nv_bfloat16>(ctx, L.rt_hi), static_cast<uint64_t>(d)};
+  const FwdOperands f = fwd_operands(ctx, xv, d, L);
   {
     GemmParams p = blank_params();
     p.rowmax = rowmax;
-    KT_TRY(run_gemm<kAbsMax>(ctx, N, d, d, 1, &A, &B, p));
+    KT_TRY(run_gemm<kAbsMax>(ctx, N, d, d, f.terms, f.A, f.B, p));
   }
   {
     GemmParams p = blank_params();
     p.rowmax = rowmax;
     p.qerr = at<float>(ctx, L.qerr);
-    KT_TRY(run_gemm<kQuantErr>(ctx, N, d, d, 1, &A, &B, p));
+    KT_TRY(run_gemm<kQuantErr>(ctx, N, d, d, f.terms, f.A, f.B, p));
   }
   const long long n = static_cast<long long>(L.P) * N;
   k_block_sums_f32<<<1024, 256, 0, ctx->stream>>>(at<float>(ctx, L.qerr), n, at<double>(ctx, L.norm_blocks));
