@@ -1,0 +1,350 @@
+#!/usr/bin/env python
+"""Benchmark of KurTail rotation learning on B200.
+
+One "step" is one pass of the whole hot path -- loss, gradient and the step on
+the orthogonal group -- over the resident calibration buffer, i.e. one
+iteration of kt_fit.  The default workload is the Llama-2-7B-like attention
+input (X bf16 65536 x 4096, Student-t(3) with 16 outlier channels x100, R
+initialised to the normalised Hadamard matrix).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+Prints ONE JSON line.  With --impl reference the float64 CPU checker is timed on
+the host cores on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "calibration tokens/s per rotation step"
+WORKLOADS = {
+    # name: (config name in synth, d, full N)
+    "llama2_7b_attn": ("llama2_7b_attn", 4096, 65536),
+    "tiny": ("tiny", 256, 2048),
+    "kv_heads": ("kv_heads", 128, 32 * 65536),
+    "llama3_8b_down": ("llama3_8b_down", 14336, 32768),
+    "llama3_70b_layer": ("llama3_70b_sweep", 8192, 32768),
+}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(tflops_sustained=p.get("bf16_tflops_sustained"), tflops_burst=p.get("bf16_tflops"),
+                    hbm_gbs=p.get("hbm_gbs"), source="measured")
+    return dict(tflops_sustained=1400.0, tflops_burst=1590.0, hbm_gbs=6650.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        for t, line in self.rows:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                clk = float(parts[0]); mx = float(parts[1])
+            except ValueError:
+                continue
+            if t0 <= t <= t1 + 0.1:
+                sm.append(clk)
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                     parts[3:7]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        sm.sort()
+        med = sm[len(sm) // 2] if sm else None
+        return dict(sm_mhz=med, sm_max_mhz=mx, samples=len(sm), reasons=sorted(reasons))
+
+
+def oracle_step_time(X64, R64, lr, repeats=1):
+    """Seconds for the oracle's loss+gradient on the sample rows, and for its orthogonal step."""
+    from oracle import kurtail_oracle as ko
+    t0 = time.perf_counter()
+    for _ in range(repeats):
+        _, dR = ko.loss_grad(X64, R64)
+    t_lg = (time.perf_counter() - t0) / repeats
+    t0 = time.perf_counter()
+    ko.orth_step(R64, dR, lr)
+    t_orth = time.perf_counter() - t0
+    return t_lg, t_orth
+
+
+def threads_in_use():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return len(os.sched_getaffinity(0))
+
+
+def cpu_baseline(sample_X, R_init, N_full, lr):
+    """The oracle as it stands, on the host cores, on a bounded row sample (rows are independent,
+    so loss+gradient time scales with N; the orthogonal step does not depend on N)."""
+    import numpy as np
+    X64 = sample_X.astype(np.float64)
+    R64 = R_init.astype(np.float64)
+    n_s = X64.shape[0]
+    t_lg, t_orth = oracle_step_time(X64, R64, lr)
+    t_full = t_lg * (N_full / n_s) + t_orth
+    return dict(value=N_full / t_full, unit="tokens/s", cores=threads_in_use(), kind="oracle",
+                sample="float64 loss+gradient on %d of %d rows at full d (%.2f s) scaled to N, plus one full "
+                       "orthogonal step (%.2f s)" % (n_s, N_full, t_lg, t_orth))
+
+
+def run_reference(args, wl_name, d, N_full):
+    """--impl reference: the CPU oracle, as it stands, on a bounded sample per step."""
+    import numpy as np
+    import torch
+    from paper_2503_01483_b200 import synth
+    from oracle import kurtail_oracle as ko
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n_s = min(N_full, max(64, int(2.0e10 / (4.0 * d * d))))   # ~2e10 f64 flops of GEMM per step
+    cfg = synth.config(WORKLOADS[wl_name][0], device="cpu", rows=n_s if wl_name != "kv_heads" else n_s // 32 * 32,
+                       **({"layers": 1} if wl_name == "llama3_70b_layer" else {}))
+    X = cfg["X"][0] if isinstance(cfg["X"], list) else cfg["X"]
+    X64 = X.float().numpy().astype(np.float64)
+    n_s = X64.shape[0]
+    R64 = ko.hadamard(d) if cfg["init"] == "hadamard" else np.eye(d)
+    lr = cfg["lr"]
+    times = []
+    for it in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        _, dR = ko.loss_grad(X64, R64)
+        t1 = time.perf_counter()
+        R64, _, _ = ko.orth_step(R64, dR, lr)
+        t2 = time.perf_counter()
+        if it >= args.warmup:
+            times.append(((t1 - t0) * (N_full / n_s) + (t2 - t1)))
+    t_step = sum(times) / len(times)
+    val = N_full / t_step
+    cores = threads_in_use()
+    sample = ("each step: float64 loss+gradient on %d of %d rows at full d, time scaled to N, plus one full "
+              "orthogonal step" % (n_s, N_full))
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC + " at d=%d" % d, "value": val, "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_step * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl_name, "N": N_full, "d": d},
+        "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama2_7b_attn", choices=sorted(WORKLOADS))
+    ap.add_argument("--rows", type=int, default=0, help="override N (profiling on a small case)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    wl_cfg, d, N_full = WORKLOADS[args.workload]
+    if args.rows:
+        N_full = args.rows
+    if args.impl == "reference":
+        run_reference(args, args.workload, d, N_full)
+        return
+
+    import numpy as np
+    import torch
+    from paper_2503_01483_b200 import build, kurtail, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local_rank)
+    dev = "cuda:%d" % local_rank
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    if rank == 0:
+        build.build()
+    if dist is not None:
+        dist.barrier()
+
+    # each rank fits its own layer buffer (layers are independent: no data-path collective)
+    kw = dict(device=dev, rows=N_full if wl_cfg != "kv_heads" else N_full)
+    if wl_cfg == "llama3_70b_sweep":
+        kw["layers"] = 1
+    cfg = synth.config(wl_cfg, **kw)
+    X = cfg["X"][0] if isinstance(cfg["X"], list) else cfg["X"]
+    if world > 1:
+        # different data per rank: re-draw with a rank-dependent seed by rolling rows
+        X = torch.roll(X, shifts=rank * 977, dims=0).contiguous()
+    N = X.shape[0]
+    lr = cfg["lr"]
+    ctx = kurtail.Context(dev)
+
+    def fresh_R():
+        if cfg["init"] == "hadamard":
+            return ctx.init_rotation(d, "hadamard")
+        if cfg["init"] == "random_orthogonal":
+            return synth.random_orthogonal(d, seed=3, device=dev).contiguous()
+        return ctx.init_rotation(d, "identity")
+
+    R = fresh_R()
+    R0_host = R.cpu().numpy()
+    ctx.fit(X, R, max(args.warmup, 1), lr)          # warm-up steps (also sizes the workspace)
+    torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ctx.profile_begin()
+    t_wall0 = time.time()
+    ev0.record()
+    rep = ctx.fit(X, R, args.steps, lr)
+    ev1.record()
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    prof = ctx.profile_end()
+    ms = ev0.elapsed_time(ev1)
+    if dist is not None:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+        dist.barrier()
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    ms_per_step = ms / args.steps
+    value = world * N * args.steps / (ms * 1e-3)
+
+    # ---- end to end through kt_fit_host: pinned host X and R in, R out, copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        Xh = X.cpu().pin_memory()
+        Rh = torch.from_numpy(R0_host.copy()).pin_memory()
+        stage = torch.empty_like(X)
+        Rdev = torch.empty_like(R)
+        ctx.fit_host(Xh, stage, Rh, Rdev, 1, lr)      # warm the copy path
+        Rh.copy_(torch.from_numpy(R0_host))
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        t0 = time.perf_counter()
+        ctx.fit_host(Xh, stage, Rh, Rdev, args.steps, lr)
+        torch.cuda.synchronize()
+        t_e2e = time.perf_counter() - t0
+        if dist is not None:
+            t = torch.tensor([t_e2e], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            t_e2e = float(t.item())
+        h2d = Xh.numel() * Xh.element_size() + Rh.numel() * 4
+        d2h = Rh.numel() * 4
+        e2e = {"value": world * N * args.steps / t_e2e, "unit": "tokens/s",
+               "h2d_bytes_per_step": h2d / args.steps, "d2h_bytes_per_step": d2h / args.steps,
+               "note": "one kt_fit_host call of %d steps: X and R copied host->device once, R copied back once; "
+                       "bytes are totals divided by steps" % args.steps}
+        del Xh, stage
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel: the three N x d x d tensor-core GEMMs of a step
+    peaks = measured_peaks()
+    g = prof["gemm"]
+    tok = [g[k] for k in ("forward", "backward_a", "backward_b")]
+    n_launch = sum(x["launches"] for x in tok)
+    t_tok = sum(x["ms"] for x in tok)
+    flops_per_launch = 2.0 * N * d * d
+    fwd_terms = 2 if d <= 512 else 1
+    achieved = flops_per_launch / (t_tok / max(n_launch, 1) * 1e-3) / 1e12 if t_tok > 0 else None
+    peak = peaks["tflops_sustained"]
+    roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": (achieved / peak) if achieved else None, "traffic": None,
+                "kernel": "gemm_tn_kernel (forward+moments, backward-A, backward-B): 2*N*d^2 flops per launch",
+                "peak_source": "%s bf16 GEMM, sustained (kernel timed inside a long step)" % peaks["source"],
+                "per_role_ms_per_launch": {k: (g[k]["ms"] / g[k]["launches"] if g[k]["launches"] else None)
+                                           for k in g},
+                "share_of_step": {k: g[k]["ms"] / ms for k in g}}
+
+    out = {
+        "metric": METRIC + " at d=%d" % d, "value": value, "unit": "tokens/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "steps_per_s": 1e3 / ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": args.workload, "N": N, "d": d, "R_init": cfg["init"], "lr": lr,
+                   "l2": "inputs (%.0f MiB of X per step) exceed the 126 MB L2" % (N * d * 2 / 2**20)
+                   if N * d * 2 > 126e6 else "inputs fit in L2; no flush (small case)",
+                   "parallelism": "one independent layer per GPU" if world > 1 else "single GPU"},
+        "algorithmic_tflops": (4.0 * N * d * d) * world / (ms_per_step * 1e-3) / 1e12,
+        "loss_first": rep["loss_first"], "loss_last": rep["loss_last"], "orth_err": rep["orth_err"],
+        "gpu_launches": prof["launches_total"], "clocks": clocks, "roofline": roofline, "e2e": e2e,
+    }
+
+    if not args.no_cpu_baseline and world == 1:
+        n_s = min(N, max(64, int(2.0e10 / (4.0 * d * d))))
+        sample = X[:n_s].float().cpu().numpy()
+        out["cpu_baseline"] = cpu_baseline(sample, R0_host, N, lr)
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

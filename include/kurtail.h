@@ -197,6 +197,24 @@ kt_status kt_quant4_error(kt_ctx* ctx, kt_mat X, const float* R, double* mse);
  * round-half-even decide the codes.  No workspace needed.  Stream ordered. */
 kt_status kt_quant4_codes(kt_ctx* ctx, const float* Y, int64_t N, int64_t d, int8_t* codes, float* scales);
 
+/* --- measurement ---------------------------------------------------------- */
+
+/* Device time of the tensor-core GEMM launches, by role, between
+ * kt_profile_begin() and kt_profile_end(): 0 forward (Y = X R with the moment
+ * epilogue; Section 2, Eq. 3), 1 backward-A (recompute Y, write dL/dY),
+ * 2 backward-B (dR = X^T dL/dY), 3 the d x d products of the Cayley step and its
+ * guard (Section 3), 4 the two quantizer passes (Section 2, Eq. 1).  Times come
+ * from CUDA events recorded on the context's stream around each launch (up to
+ * 8192 launches per window).  launches_total counts every kernel this library
+ * launched in the window.  kt_profile_end() synchronises; `out` is host memory. */
+typedef struct {
+  int64_t launches_total;
+  int32_t gemm_launches[8];
+  float gemm_ms[8];
+} kt_profile;
+kt_status kt_profile_begin(kt_ctx* ctx);
+kt_status kt_profile_end(kt_ctx* ctx, kt_profile* out);
+
 #ifdef __cplusplus
 }
 #endif

@@ -16,6 +16,8 @@
 namespace kt {
 
 constexpr int kHistMax = 4096;  // loss-history slots kept on the device between host read-backs
+constexpr int kProfPairs = 8192; // CUDA-event pairs available to one profiling window
+enum GemmCat : int { kCatForward = 0, kCatBackwardA = 1, kCatBackwardB = 2, kCatSquare = 3, kCatQuant = 4 };
 
 struct DeviceBlock {
   Scalars sc;
@@ -101,7 +103,12 @@ struct kt_ctx {
   kt::DeviceBlock* d_blk;
   kt::DeviceBlock* h_blk;  // pinned
   kt::EncodeTiledFn encode;
-  bool smem_attr_set;
+  // profiling (kt_profile_begin/kt_profile_end)
+  long long launches;       // kernels launched since kt_profile_begin
+  bool prof_on;
+  cudaEvent_t* prof_ev;     // 2 * kProfPairs events, created on first use
+  int prof_used;            // pairs recorded
+  unsigned char* prof_cat;  // category of each pair
 };
 
 namespace kt {
@@ -113,7 +120,11 @@ namespace kt {
       return KT_ERR_CUDA;                   \
     }                                       \
   } while (0)
-#define KT_LAUNCH_CHECK() KT_CUDA(cudaGetLastError())
+#define KT_LAUNCH_CHECK()          \
+  do {                             \
+    KT_CUDA(cudaGetLastError());   \
+    ++ctx->launches;               \
+  } while (0)
 #define KT_TRY(expr)                 \
   do {                               \
     kt_status st__ = (expr);         \
@@ -155,7 +166,7 @@ static kt_status make_tmap(const kt_ctx* ctx, CUtensorMap* tm, const void* base,
 }
 
 template <int BN, int EPI>
-static kt_status launch_gemm_inst(kt_ctx* ctx, const GemmParams& p) {
+static kt_status launch_gemm_inst(kt_ctx* ctx, const GemmParams& p, int cat) {
   static bool attr_done[16] = {false};
   const int smem = GemmSmem<BN>::kTotal;
   if (!attr_done[ctx->device & 15]) {
@@ -164,8 +175,14 @@ static kt_status launch_gemm_inst(kt_ctx* ctx, const GemmParams& p) {
   }
   const int tiles = p.m_tiles * p.n_tiles;
   const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+  const bool rec = ctx->prof_on && ctx->prof_used < kProfPairs;
+  if (rec) KT_CUDA(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], ctx->stream));
   gemm_tn_kernel<BN, EPI><<<grid, kGemmThreads, smem, ctx->stream>>>(p);
   KT_LAUNCH_CHECK();
+  if (rec) {
+    KT_CUDA(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used + 1], ctx->stream));
+    ctx->prof_cat[ctx->prof_used++] = static_cast<unsigned char>(cat);
+  }
   return KT_OK;
 }
 
@@ -177,7 +194,7 @@ struct Operand {
 // D (M x N) = sum_q A_q (M x K) * B_q (N x K)^T with the epilogue EPI.
 template <int EPI>
 static kt_status run_gemm(kt_ctx* ctx, int M, int N, int K, int terms, const Operand* A, const Operand* B,
-                          GemmParams& p) {
+                          GemmParams& p, int cat) {
   const int bn = (N % 256 == 0) ? 256 : 128;
   p.terms = terms;
   p.M = M;
@@ -190,8 +207,8 @@ static kt_status run_gemm(kt_ctx* ctx, int M, int N, int K, int terms, const Ope
     KT_TRY(make_tmap(ctx, &p.tmA[q], A[q].base, K, M, A[q].ld, kBM));
     KT_TRY(make_tmap(ctx, &p.tmB[q], B[q].base, K, N, B[q].ld, bn));
   }
-  if (bn == 256) return launch_gemm_inst<256, EPI>(ctx, p);
-  return launch_gemm_inst<128, EPI>(ctx, p);
+  if (bn == 256) return launch_gemm_inst<256, EPI>(ctx, p, cat);
+  return launch_gemm_inst<128, EPI>(ctx, p, cat);
 }
 
 static GemmParams blank_params() {
@@ -285,7 +302,7 @@ static kt_status forward_loss(kt_ctx* ctx, const XView& xv, int N, int d, const 
   GemmParams p = blank_params();
   p.partial = at<float4>(ctx, L.partial);
   const FwdOperands f = fwd_operands(ctx, xv, d, L);
-  KT_TRY(run_gemm<kMoments>(ctx, N, d, d, f.terms, f.A, f.B, p));
+  KT_TRY(run_gemm<kMoments>(ctx, N, d, d, f.terms, f.A, f.B, p, kCatForward));
   k_moments_finalize<<<L.loss_blocks, 256, 0, ctx->stream>>>(at<float4>(ctx, L.partial), L.P, N, d, L.bn,
                                                             ctx->cfg.kappa_target, at<float4>(ctx, L.moments),
                                                             at<float4>(ctx, L.coef), at<double>(ctx, L.block_loss),
@@ -304,13 +321,13 @@ static kt_status backward(kt_ctx* ctx, const XView& xv, int N, int d, const WsLa
   p.gt = at<__nv_bfloat16>(ctx, L.gt);
   p.ldg = L.ldt;
   const FwdOperands f = fwd_operands(ctx, xv, d, L);
-  KT_TRY(run_gemm<kGrad>(ctx, N, d, d, f.terms, f.A, f.B, p));
+  KT_TRY(run_gemm<kGrad>(ctx, N, d, d, f.terms, f.A, f.B, p, kCatBackwardA));
   GemmParams p2 = blank_params();
   p2.out = dR;
   p2.ldo = d;
   Operand A2{at<__nv_bfloat16>(ctx, L.xt), static_cast<uint64_t>(L.ldt)},
       B2{at<__nv_bfloat16>(ctx, L.gt), static_cast<uint64_t>(L.ldt)};
-  KT_TRY(run_gemm<kStoreF32>(ctx, d, d, N, 1, &A2, &B2, p2));
+  KT_TRY(run_gemm<kStoreF32>(ctx, d, d, N, 1, &A2, &B2, p2, kCatBackwardB));
   return KT_OK;
 }
 
@@ -344,7 +361,7 @@ static kt_status guard(kt_ctx* ctx, const float* R_in, float* R, int d, const Ws
     // (H + L)^T (H + L) without L^T L: that term only matters on the diagonal, which k_guard rebuilds exactly
     Operand A[3] = {{rt_hi, ld}, {rt_hi, ld}, {rt_lo, ld}};
     Operand B[3] = {{rt_hi, ld}, {rt_lo, ld}, {rt_hi, ld}};
-    KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 3, A, B, p));
+    KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 3, A, B, p, kCatSquare));
   }
   __nv_bfloat16* e_hi = at<__nv_bfloat16>(ctx, L.z_hi);
   const unsigned blocks = static_cast<unsigned>(static_cast<long long>(d) * d / 4 / 256);
@@ -359,7 +376,7 @@ static kt_status guard(kt_ctx* ctx, const float* R_in, float* R, int d, const Ws
     p.ldo = d;
     p.gate = &sc->gate;
     Operand A{at<__nv_bfloat16>(ctx, L.r_hi), ld}, B{e_hi, ld};  // (R E)[i][j] = sum_k R[i][k] E[j][k], E symmetric
-    KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 1, &A, &B, p));
+    KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 1, &A, &B, p, kCatSquare));
   }
   k_polish_apply<<<blocks, 256, 0, ctx->stream>>>(R, fbuf, sc);
   KT_LAUNCH_CHECK();
@@ -395,7 +412,7 @@ static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, 
     p.out = fbuf;
     p.ldo = d;
     Operand A{z_hi, ld}, B{r_hi, ld};
-    KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 1, &A, &B, p));
+    KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 1, &A, &B, p, kCatSquare));
   }
   k_skew<<<tgrid, tblock, 0, ctx->stream>>>(fbuf, d, w_hi, terms == 3 ? w_lo : nullptr,
                                             at<double>(ctx, L.norm_blocks));
@@ -410,7 +427,7 @@ static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, 
     p.ldo = d;
     Operand A[3] = {{w_hi, ld}, {w_hi, ld}, {w_lo, ld}};
     Operand B[3] = {{zt_hi, ld}, {zt_lo, ld}, {zt_hi, ld}};
-    return run_gemm<kStoreF32>(ctx, d, d, d, terms, A, B, p);
+    return run_gemm<kStoreF32>(ctx, d, d, d, terms, A, B, p, kCatSquare);
   };
   const int s = c.cayley_iters < 0 ? 0 : c.cayley_iters;
   // Y0 = R - alpha W R
@@ -588,6 +605,11 @@ kt_status kt_create(kt_ctx** out, const kt_config* cfg, void* cuda_stream) {
 void kt_destroy(kt_ctx* ctx) {
   if (!ctx) return;
   cudaStreamSynchronize(ctx->stream);
+  if (ctx->prof_ev) {
+    for (int i = 0; i < 2 * kProfPairs; ++i) cudaEventDestroy(ctx->prof_ev[i]);
+    delete[] ctx->prof_ev;
+    delete[] ctx->prof_cat;
+  }
   cudaFreeHost(ctx->h_blk);
   cudaFree(ctx->d_blk);
   delete ctx;
@@ -668,7 +690,8 @@ kt_status kt_rotate(kt_ctx* ctx, kt_mat X, const float* R, float* Y) {
   p.out = Y;
   p.ldo = d;
   const FwdOperands f = fwd_operands(ctx, xv, static_cast<int>(d), L);
-  return run_gemm<kStoreF32>(ctx, static_cast<int>(N), static_cast<int>(d), static_cast<int>(d), f.terms, f.A, f.B, p);
+  return run_gemm<kStoreF32>(ctx, static_cast<int>(N), static_cast<int>(d), static_cast<int>(d), f.terms, f.A, f.B, p,
+                             kCatForward);
 }
 
 kt_status kt_loss_grad(kt_ctx* ctx, kt_mat X, const float* R, float* dR, double* loss) {
@@ -775,13 +798,13 @@ kt_status kt_quant4_error(kt_ctx* ctx, kt_mat X, const float* R, double* mse) {
   {
     GemmParams p = blank_params();
     p.rowmax = rowmax;
-    KT_TRY(run_gemm<kAbsMax>(ctx, N, d, d, f.terms, f.A, f.B, p));
+    KT_TRY(run_gemm<kAbsMax>(ctx, N, d, d, f.terms, f.A, f.B, p, kCatQuant));
   }
   {
     GemmParams p = blank_params();
     p.rowmax = rowmax;
     p.qerr = at<float>(ctx, L.qerr);
-    KT_TRY(run_gemm<kQuantErr>(ctx, N, d, d, f.terms, f.A, f.B, p));
+    KT_TRY(run_gemm<kQuantErr>(ctx, N, d, d, f.terms, f.A, f.B, p, kCatQuant));
   }
   const long long n = static_cast<long long>(L.P) * N;
   k_block_sums_f32<<<1024, 256, 0, ctx->stream>>>(at<float>(ctx, L.qerr), n, at<double>(ctx, L.norm_blocks));
@@ -792,6 +815,36 @@ kt_status kt_quant4_error(kt_ctx* ctx, kt_mat X, const float* R, double* mse) {
   KT_TRY(sync_scalars(ctx));
   *mse = ctx->h_blk->sc.qmse;
   return isfinite(*mse) ? KT_OK : KT_ERR_NONFINITE;
+}
+
+kt_status kt_profile_begin(kt_ctx* ctx) {
+  if (!ctx) return KT_ERR_INVALID_ARG;
+  if (!ctx->prof_ev) {
+    ctx->prof_ev = new (std::nothrow) cudaEvent_t[2 * kProfPairs];
+    ctx->prof_cat = new (std::nothrow) unsigned char[kProfPairs];
+    if (!ctx->prof_ev || !ctx->prof_cat) return KT_ERR_CUDA;
+    for (int i = 0; i < 2 * kProfPairs; ++i) KT_CUDA(cudaEventCreate(&ctx->prof_ev[i]));
+  }
+  ctx->prof_used = 0;
+  ctx->launches = 0;
+  ctx->prof_on = true;
+  return KT_OK;
+}
+
+kt_status kt_profile_end(kt_ctx* ctx, kt_profile* out) {
+  if (!ctx || !out) return KT_ERR_INVALID_ARG;
+  memset(out, 0, sizeof(*out));
+  ctx->prof_on = false;
+  KT_CUDA(cudaStreamSynchronize(ctx->stream));
+  out->launches_total = ctx->launches;
+  for (int i = 0; i < ctx->prof_used; ++i) {
+    float ms = 0.f;
+    KT_CUDA(cudaEventElapsedTime(&ms, ctx->prof_ev[2 * i], ctx->prof_ev[2 * i + 1]));
+    const int c = ctx->prof_cat[i];
+    out->gemm_launches[c] += 1;
+    out->gemm_ms[c] += ms;
+  }
+  return KT_OK;
 }
 
 kt_status kt_quant4_codes(kt_ctx* ctx, const float* Y, int64_t N, int64_t d, int8_t* codes, float* scales) {

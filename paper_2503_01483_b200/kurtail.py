@@ -43,10 +43,14 @@ class kt_fit_report(C.Structure):
                 ("w_norm_last", C.c_float), ("loss_history", C.POINTER(C.c_double))]
 
 
+class kt_profile(C.Structure):
+    _fields_ = [("launches_total", C.c_int64), ("gemm_launches", C.c_int32 * 8), ("gemm_ms", C.c_float * 8)]
+
+
 EXPORTS = ["kt_default_config", "kt_create", "kt_destroy", "kt_status_string", "kt_workspace_bytes",
            "kt_set_workspace", "kt_init_rotation", "kt_kurtosis_loss", "kt_loss_grad", "kt_row_moments",
            "kt_rotate", "kt_orth_step", "kt_orth_error", "kt_fit", "kt_fit_layers", "kt_fit_host",
-           "kt_quant4_error", "kt_quant4_codes"]
+           "kt_quant4_error", "kt_quant4_codes", "kt_profile_begin", "kt_profile_end"]
 
 _lib = None
 
@@ -83,6 +87,8 @@ def lib():
     L.kt_fit_host.argtypes = [vp, kt_mat, vp, vp, vp, i32, f32, C.POINTER(kt_fit_report)]
     L.kt_quant4_error.argtypes = [vp, kt_mat, vp, dp]
     L.kt_quant4_codes.argtypes = [vp, vp, i64, i64, vp, vp]
+    L.kt_profile_begin.argtypes = [vp]
+    L.kt_profile_end.argtypes = [vp, C.POINTER(kt_profile)]
     for name in EXPORTS:
         fn = getattr(L, name)
         if name not in ("kt_default_config", "kt_destroy", "kt_status_string"):
@@ -247,6 +253,16 @@ class Context:
         out = C.c_double()
         _check(lib().kt_quant4_error(self._h, m, R.data_ptr(), C.byref(out)), "kt_quant4_error")
         return out.value
+
+    def profile_begin(self):
+        _check(lib().kt_profile_begin(self._h), "kt_profile_begin")
+
+    def profile_end(self):
+        pr = kt_profile()
+        _check(lib().kt_profile_end(self._h, C.byref(pr)), "kt_profile_end")
+        names = ["forward", "backward_a", "backward_b", "square", "quant"]
+        return dict(launches_total=pr.launches_total,
+                    gemm={n: dict(launches=pr.gemm_launches[i], ms=pr.gemm_ms[i]) for i, n in enumerate(names)})
 
     def quant4_codes(self, Y):
         N, d = Y.shape
