@@ -49,7 +49,8 @@ typedef enum {
   KT_ERR_ARCH = 5,        /* current device is not compute capability 10.x  */
   KT_ERR_CUDA = 6,        /* a CUDA runtime/driver call failed              */
   KT_ERR_NONFINITE = 7,   /* the loss came out NaN/Inf (outputs are written)*/
-  KT_ERR_TIMEOUT = 8      /* a bounded device-side wait ran out             */
+  KT_ERR_TIMEOUT = 8,     /* a bounded device-side wait ran out             */
+  KT_ERR_TOO_LARGE = 9    /* kt_kurtosis_loss_noalloc: N or d above its maximum */
 } kt_status;
 
 typedef enum { KT_BF16 = 0, KT_F32 = 1 } kt_dtype;
@@ -196,6 +197,41 @@ kt_status kt_quant4_error(kt_ctx* ctx, kt_mat X, const float* R, double* mse);
  * int8, device) and scales (N float32, device).  Float32 IEEE divide and
  * round-half-even decide the codes.  No workspace needed.  Stream ordered. */
 kt_status kt_quant4_codes(kt_ctx* ctx, const float* Y, int64_t N, int64_t d, int8_t* codes, float* scales);
+
+/* --- a loss call that allocates nothing ----------------------------------- */
+
+/* (The paper has no counterpart to this call; it exists for deployment.)
+ *
+ * kt_kurtosis_loss for callers that cannot allocate device memory: code running
+ * inside a memory pool that owns the whole GPU, a plug-in that is forbidden to
+ * call cudaMalloc because the host application budgets every byte, or a
+ * real-time loop where an allocation (an implicit device synchronisation) is not
+ * acceptable.  It needs no kt_ctx and no workspace: its scratch -- the bf16
+ * copies of R^T, the per-tile and per-row moment records, the block sums and the
+ * status words -- is a fixed 8 MiB array compiled into the library, which every
+ * GPU that loads the library holds until the process exits.  Neither this call
+ * nor anything it uses calls cudaMalloc, cudaFree or an allocating routine.
+ *
+ *   X        bf16 only, device, N <= KT_NOALLOC_MAX_N rows, d <= KT_NOALLOC_MAX_D
+ *            (same alignment rules as elsewhere); larger problems return
+ *            KT_ERR_TOO_LARGE and float32 X returns KT_ERR_INVALID_ARG, with
+ *            nothing enqueued.
+ *   R        d x d float32, device.
+ *   loss_dev DEVICE pointer to one double (8-byte aligned) that receives the
+ *            loss.  The call is stream ordered on `cuda_stream` and does not
+ *            synchronise; read the value after synchronising that stream.
+ *
+ * The first call on each device looks up the device address of the built-in
+ * array and a driver entry point, with that device current.  Make that first
+ * call before starting any stream capture.
+ * All calls on a device share the one array, which keeps the previous call's
+ * contents (the call clears the words that must start at zero itself).  Two
+ * calls that overlap on the GPU -- different streams, or different host threads
+ * without ordering between their streams -- race on it; order them yourself.
+ * The default configuration (kappa_target 1.8, forward_terms auto) applies. */
+#define KT_NOALLOC_MAX_N 16384
+#define KT_NOALLOC_MAX_D 1024
+kt_status kt_kurtosis_loss_noalloc(kt_mat X, const float* R, double* loss_dev, void* cuda_stream);
 
 /* --- measurement ---------------------------------------------------------- */
 

@@ -7,6 +7,7 @@
 #include <stdint.h>
 #include <string.h>
 
+#include <mutex>
 #include <new>
 
 #include "../../include/kurtail.h"
@@ -554,6 +555,7 @@ const char* kt_status_string(kt_status s) {
     case KT_ERR_CUDA: return "CUDA call failed";
     case KT_ERR_NONFINITE: return "non-finite loss";
     case KT_ERR_TIMEOUT: return "device-side wait timed out";
+    case KT_ERR_TOO_LARGE: return "problem exceeds the built-in scratch of the no-allocation entry point";
   }
   return "unknown status";
 }
@@ -853,6 +855,114 @@ kt_status kt_quant4_codes(kt_ctx* ctx, const float* Y, int64_t N, int64_t d, int
   k_quant4_codes<<<static_cast<unsigned>(N), 256, 0, ctx->stream>>>(Y, static_cast<int>(d), codes, scales);
   KT_LAUNCH_CHECK();
   return KT_OK;
+}
+
+// ------------------------------------------------------------------------
+// kt_kurtosis_loss_noalloc: the loss for callers that must not allocate.
+//
+// Scratch that kt_kurtosis_loss takes from the caller's workspace (the bf16
+// copies of R^T, the per-column-tile moment records, the per-row records, the
+// block sums) and the scalar block that kt_create() would cudaMalloc live here in
+// one fixed array inside the library image.  Every GPU that loads the library
+// carries these 8 MiB until the process exits.
+// ------------------------------------------------------------------------
+#define KT_NOALLOC_SCRATCH_BYTES (8u << 20)
+static __device__ __align__(256) unsigned char g_noalloc_scratch[KT_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+
+struct NoAllocDevice {
+  bool ready;
+  kt_ctx ctx;          // plain host struct; its device pointers point into g_noalloc_scratch
+  unsigned char* base; // device address of g_noalloc_scratch on this device
+};
+NoAllocDevice g_noalloc_dev[64];
+std::mutex g_noalloc_mutex;
+
+// One-time set-up for the current device: resolves the DEVICE address of the
+// scratch array (its name is only a host-side handle in host code and must not be
+// handed to a kernel), and looks up what the launches need.  Allocates nothing.
+kt_status noalloc_setup(int dev, NoAllocDevice** out) {
+  if (dev < 0 || dev >= 64) return KT_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  NoAllocDevice& nd = g_noalloc_dev[dev];
+  if (!nd.ready) {
+    int major = 0, sms = 0;
+    KT_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+    KT_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    if (major != 10) return KT_ERR_ARCH;
+    void* ptr = nullptr;
+    KT_CUDA(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
+    if (ptr == nullptr) return KT_ERR_CUDA;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+        qres != cudaDriverEntryPointSuccess)
+      return KT_ERR_CUDA;
+    memset(&nd.ctx, 0, sizeof(nd.ctx));
+    kt_default_config(&nd.ctx.cfg);
+    nd.ctx.device = dev;
+    nd.ctx.sm_count = sms;
+    nd.ctx.encode = reinterpret_cast<EncodeTiledFn>(fn);
+    nd.base = static_cast<unsigned char*>(ptr);
+    nd.ctx.d_blk = reinterpret_cast<DeviceBlock*>(nd.base);  // scalar block first
+    nd.ctx.ws = nd.base;
+    nd.ctx.ws_bytes = KT_NOALLOC_SCRATCH_BYTES;
+    nd.ready = true;
+  }
+  *out = &nd;
+  return KT_OK;
+}
+
+}  // namespace
+
+kt_status kt_kurtosis_loss_noalloc(kt_mat X, const float* R, double* loss_dev, void* cuda_stream) {
+  if (!R || !loss_dev) return KT_ERR_INVALID_ARG;
+  int64_t N, d;
+  KT_TRY(check_x(X, &N, &d));
+  if (X.dtype != KT_BF16) return KT_ERR_INVALID_ARG;  // a float32 X would need an N x d scratch copy
+  if (!aligned16(R) || (reinterpret_cast<uintptr_t>(loss_dev) & 7u) != 0) return KT_ERR_ALIGN;
+  if (N > KT_NOALLOC_MAX_N || d > KT_NOALLOC_MAX_D) return KT_ERR_TOO_LARGE;
+  int dev = 0;
+  KT_CUDA(cudaGetDevice(&dev));
+  NoAllocDevice* nd = nullptr;
+  KT_TRY(noalloc_setup(dev, &nd));
+
+  // carve the array: [scalar block][R^T hi][R^T lo][records ...]; sizes are bounded by the maxima above
+  WsLayout L;
+  memset(&L, 0, sizeof(L));
+  L.bn = (d % 256 == 0) ? 256 : 128;
+  L.P = static_cast<int>(d / L.bn);
+  L.loss_blocks = static_cast<int>((N + 255) / 256);
+  size_t off = align_up(sizeof(DeviceBlock), 256);
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes, 256);
+    return o;
+  };
+  const size_t dd = static_cast<size_t>(d) * d;
+  L.rt_hi = take(dd * 2);
+  L.rt_lo = take(dd * 2);
+  L.partial = take(static_cast<size_t>(L.P) * N * 16);
+  L.coef = take(static_cast<size_t>(N) * 16);
+  L.moments = take(static_cast<size_t>(N) * 16);
+  L.block_loss = take(static_cast<size_t>(L.loss_blocks) * 8);
+  L.block_deg = take(static_cast<size_t>(L.loss_blocks) * 4);
+  L.total = off;
+  if (L.total > KT_NOALLOC_SCRATCH_BYTES) return KT_ERR_TOO_LARGE;
+
+  // the shared host-side descriptor is used by one call at a time
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  kt_ctx* ctx = &nd->ctx;
+  ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+  // the array keeps whatever the previous call left: clear the one word that must start at zero
+  // (the time-out flag is only ever raised by atomicMax); everything else is written before it is read
+  KT_CUDA(cudaMemsetAsync(&ctx->d_blk->sc, 0, sizeof(Scalars), ctx->stream));
+  XView xv;
+  xv.xb = static_cast<const __nv_bfloat16*>(X.data);
+  xv.ldx = X.ld;
+  KT_TRY(cast_rt(ctx, R, static_cast<int>(d), L));
+  return forward_loss(ctx, xv, static_cast<int>(N), static_cast<int>(d), L, loss_dev);
 }
 
 }  // extern "C"

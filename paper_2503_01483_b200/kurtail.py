@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libkurtail.so")
 
 KT_BF16, KT_F32 = 0, 1
 STATUS = {0: "KT_OK", 1: "KT_ERR_INVALID_ARG", 2: "KT_ERR_SHAPE", 3: "KT_ERR_ALIGN", 4: "KT_ERR_WORKSPACE",
-          5: "KT_ERR_ARCH", 6: "KT_ERR_CUDA", 7: "KT_ERR_NONFINITE", 8: "KT_ERR_TIMEOUT"}
+          5: "KT_ERR_ARCH", 6: "KT_ERR_CUDA", 7: "KT_ERR_NONFINITE", 8: "KT_ERR_TIMEOUT", 9: "KT_ERR_TOO_LARGE"}
 
 
 class KtError(RuntimeError):
@@ -50,7 +50,8 @@ class kt_profile(C.Structure):
 EXPORTS = ["kt_default_config", "kt_create", "kt_destroy", "kt_status_string", "kt_workspace_bytes",
            "kt_set_workspace", "kt_init_rotation", "kt_kurtosis_loss", "kt_loss_grad", "kt_row_moments",
            "kt_rotate", "kt_orth_step", "kt_orth_error", "kt_fit", "kt_fit_layers", "kt_fit_host",
-           "kt_quant4_error", "kt_quant4_codes", "kt_profile_begin", "kt_profile_end"]
+           "kt_quant4_error", "kt_quant4_codes", "kt_profile_begin", "kt_profile_end",
+           "kt_kurtosis_loss_noalloc"]
 
 _lib = None
 
@@ -87,6 +88,7 @@ def lib():
     L.kt_fit_host.argtypes = [vp, kt_mat, vp, vp, vp, i32, f32, C.POINTER(kt_fit_report)]
     L.kt_quant4_error.argtypes = [vp, kt_mat, vp, dp]
     L.kt_quant4_codes.argtypes = [vp, vp, i64, i64, vp, vp]
+    L.kt_kurtosis_loss_noalloc.argtypes = [kt_mat, vp, vp, vp]
     L.kt_profile_begin.argtypes = [vp]
     L.kt_profile_end.argtypes = [vp, C.POINTER(kt_profile)]
     for name in EXPORTS:
@@ -127,6 +129,15 @@ def _rep_dict(rep, hist):
     return dict(steps_done=rep.steps_done, degenerate_rows=rep.degenerate_rows, loss_first=rep.loss_first,
                 loss_last=rep.loss_last, orth_err=rep.orth_err, alpha_last=rep.alpha_last,
                 w_norm_last=rep.w_norm_last, loss_history=list(hist) if hist is not None else None)
+
+
+def kurtosis_loss_noalloc(X, R, loss_dev, stream=None):
+    """kt_kurtosis_loss_noalloc: the loss without a context, a workspace or any allocation.
+    `loss_dev` is a caller-owned float64 device tensor of one element; the call is stream
+    ordered (synchronise before reading it).  Raises KtError(9) above N 16384 / d 1024."""
+    sp = C.c_void_p(stream.cuda_stream if stream is not None else 0)
+    _check(lib().kt_kurtosis_loss_noalloc(as_mat(X), R.data_ptr(), loss_dev.data_ptr(), sp),
+           "kt_kurtosis_loss_noalloc")
 
 
 class Context:
