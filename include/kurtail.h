@@ -156,9 +156,12 @@ kt_status kt_rotate(kt_ctx* ctx, kt_mat X, const float* R, float* Y);
 /* R <- retraction of R along -dR:  W = (dR R^T - R dR^T)/2,
  * alpha = min(lr, 2q/(||W||_F + eps)), Y0 = R - alpha W R,
  * Yi = R - alpha/2 W (R + Y(i-1)) for i = 1..cayley_iters, R <- Y(last), then
- * the orthogonality guard (see kt_config.polish_thresh).  Built from d x d
- * tensor-core products only.  R is updated in place; dR is read only.  Uses
- * the workspace (sized for any N >= 1 and this d).  Stream ordered. */
+ * the orthogonality guard (see kt_config.polish_thresh).  The iteration is
+ * evaluated as its Neumann series, which has the same partial sums:
+ * Y_s = R - alpha sum_{k<=s} (-alpha/2)^k W^k (W R).  Built from d x d
+ * tensor-core products only.  R is updated in place, one series term per
+ * kernel; dR is read only.  Uses the workspace (sized for any N >= 1 and this
+ * d).  Stream ordered. */
 kt_status kt_orth_step(kt_ctx* ctx, float* R, const float* dR, int64_t d, float lr);
 
 /* *err (host) = max|R^T R - I|.  Uses the workspace.  Synchronises. */
@@ -167,7 +170,8 @@ kt_status kt_orth_error(kt_ctx* ctx, const float* R, int64_t d, double* err);
 /* `steps` x (kt_loss_grad; kt_orth_step) on the context's stream with no host
  * synchronisation in between; bit-identical to composing those calls when
  * guard_every == 1.  R in/out.  `report` (host) may be NULL.  Synchronises at
- * the end.  On an error R holds the last completed step. */
+ * the end.  On an argument error R is untouched; after a CUDA failure in the
+ * middle of a step R may hold a partially applied step. */
 kt_status kt_fit(kt_ctx* ctx, kt_mat X, float* R, int32_t steps, float lr, kt_fit_report* report);
 
 /* Layer-wise driver (Section 3, "Training Cost": activations are stored per

@@ -223,6 +223,23 @@ __global__ void k_block_sums_f32(const float* __restrict__ v, long long n, doubl
   if (threadIdx.x == 0) block_out[blockIdx.x] = s;
 }
 
+// out[i] = sum over s of part[s * stride + i], s ascending (fixed order).  n a multiple of 4.
+// grid ceil(n/4/256), block 256.
+__global__ void k_sum_splits(const float* __restrict__ part, int splits, long long stride, long long n,
+                             float* __restrict__ out) {
+  const long long i4 = (static_cast<long long>(blockIdx.x) * 256 + threadIdx.x) * 4;
+  if (i4 >= n) return;
+  float4 acc = *reinterpret_cast<const float4*>(part + i4);
+  for (int s = 1; s < splits; ++s) {
+    const float4 v = *reinterpret_cast<const float4*>(part + s * stride + i4);
+    acc.x += v.x;
+    acc.y += v.y;
+    acc.z += v.z;
+    acc.w += v.w;
+  }
+  *reinterpret_cast<float4*>(out + i4) = acc;
+}
+
 // ------------------------------------------------------------- Cayley pieces
 // W = (A - A^T)/2 for a d x d float32 A, written as bf16 hi (and lo when asked;
 // the rounding is odd, so each bf16 part is exactly skew), plus per-block sums of W^2 (of the float32 W).
@@ -268,41 +285,82 @@ __global__ void k_step_size(const double* __restrict__ block_norm2, int n, float
   }
 }
 
-// Y = R - (alpha * cmul) P;  if dst: dst = Y;  Z = zr R + Y, written as bf16
-// hi/lo, transposed (zt_*) and/or as is (z_*).  All matrices d x d, dense.
-// grid (d/32, d/32), block (32, 8).  dst may alias R.
-__global__ void k_axpy_split(const float* R, const float* __restrict__ P, const Scalars* __restrict__ sc,
-                             float cmul, float zr, int d, float* dst, __nv_bfloat16* __restrict__ zt_hi,
-                             __nv_bfloat16* __restrict__ zt_lo, __nv_bfloat16* __restrict__ z_hi,
-                             __nv_bfloat16* __restrict__ z_lo) {
+// One term of the Cayley step written as its Neumann series:
+//   R_new = R - alpha * sum_{k=0..s} (-alpha/2)^k P_k,   P_0 = W R,  P_{k+1} = W P_k
+// (the partial sums are exactly the iterates Y_k of the fixed-point form Y_0 = R - alpha W R,
+// Y_k = R - alpha/2 W (R + Y_{k-1})).  This kernel adds term k in place, R += c_k P with
+// c_k = -alpha (-alpha/2)^k, writes P^T as bf16 for the next product when pt_hi != null, and, when
+// r_hi != null (last term), the bf16 forms of the new R: r_hi (as is), rt_hi/rt_lo (transposed hi/lo).
+// grid (d/32, d/32), block (32, 8).
+__global__ void k_series_term(float* __restrict__ R, const float* __restrict__ P, const Scalars* __restrict__ sc,
+                              int k, int d, __nv_bfloat16* __restrict__ pt_hi, __nv_bfloat16* __restrict__ r_hi,
+                              __nv_bfloat16* __restrict__ rt_hi, __nv_bfloat16* __restrict__ rt_lo) {
   __shared__ float tile[32][33];
   const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
   const int tx = threadIdx.x, ty = threadIdx.y;
-  const float beta = sc->alpha * cmul;
-  for (int r = ty; r < 32; r += 8) {
+  const float alpha = sc->alpha;
+  float ck = -alpha;
+  for (int i = 0; i < k; ++i) ck *= -0.5f * alpha;
+  float rn[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int r = ty + 8 * q;
     const long long o = static_cast<long long>(r0 + r) * d + c0 + tx;
-    const float rv = R[o];
-    const float y = fmaf(-beta, P[o], rv);
-    const float z = fmaf(zr, rv, y);
-    if (dst) dst[o] = y;
-    tile[r][tx] = z;
-    if (z_hi) {
-      __nv_bfloat16 h, l;
-      split_bf16(z, h, l);
-      z_hi[o] = h;
-      if (z_lo) z_lo[o] = l;
+    const float pv = P[o];
+    rn[q] = fmaf(ck, pv, R[o]);
+    R[o] = rn[q];
+    tile[r][tx] = pv;
+    if (r_hi) r_hi[o] = __float2bfloat16_rn(rn[q]);
+  }
+  if (pt_hi) {
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int c = ty + 8 * q;
+      pt_hi[static_cast<long long>(c0 + c) * d + r0 + tx] = __float2bfloat16_rn(tile[tx][c]);
     }
   }
-  if (zt_hi) {
+  if (rt_hi) {
     __syncthreads();
-    for (int c = ty; c < 32; c += 8) {
-      const float z = tile[tx][c];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) tile[ty + 8 * q][tx] = rn[q];
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int c = ty + 8 * q;
       __nv_bfloat16 h, l;
-      split_bf16(z, h, l);
+      split_bf16(tile[tx][c], h, l);
       const long long o = static_cast<long long>(c0 + c) * d + r0 + tx;
-      zt_hi[o] = h;
-      if (zt_lo) zt_lo[o] = l;
+      rt_hi[o] = h;
+      rt_lo[o] = l;
     }
+  }
+}
+
+// The bf16 forms of R that the step and the guard use: r_hi (as is) and rt_hi/rt_lo (transposed).
+// grid (d/32, d/32), block (32, 8).
+__global__ void k_split_r(const float* __restrict__ R, int d, __nv_bfloat16* __restrict__ r_hi,
+                          __nv_bfloat16* __restrict__ rt_hi, __nv_bfloat16* __restrict__ rt_lo) {
+  __shared__ float tile[32][33];
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int r = ty + 8 * q;
+    const long long o = static_cast<long long>(r0 + r) * d + c0 + tx;
+    const float v = R[o];
+    tile[r][tx] = v;
+    r_hi[o] = __float2bfloat16_rn(v);
+  }
+  __syncthreads();
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int c = ty + 8 * q;
+    __nv_bfloat16 h, l;
+    split_bf16(tile[tx][c], h, l);
+    const long long o = static_cast<long long>(c0 + c) * d + r0 + tx;
+    rt_hi[o] = h;
+    rt_lo[o] = l;
   }
 }
 
@@ -328,45 +386,62 @@ __global__ void k_colnorm_partial(const float* __restrict__ R, int d, float* __r
   }
 }
 
-// E = S - I (S = R^T R from the tensor cores, d x d float32): max|E| into
-// sc->max_e_bits (atomic max on the bit pattern of a non-negative float: exact,
-// order independent) and E as bf16 when e_hi != null.  The diagonal is NOT taken
-// from S: the tensor-core accumulator truncates, which biases a sum of d
-// positive terms near 1 by about one unit in the last place per MMA step; it is
-// rebuilt from the exact column norms, E_jj = sum_slabs colpart[slab][j] - 1
-// (accumulated in double).  Off-diagonal sums hover around 0 and carry no such
-// bias.  grid d*d/4/256, block 256; d*d a multiple of 1024.
-__global__ void k_guard(const float* __restrict__ S, int d, const float* __restrict__ colpart, int nslabs,
+// diag[j] = (sum over slabs of colpart[slab][j]) - 1, accumulated in double: the exact diagonal of
+// R^T R - I.  One warp per column; grid ceil(d/8), block 256.
+__global__ void k_colnorm_final(const float* __restrict__ colpart, int nslabs, int d, float* __restrict__ diag) {
+  const int j = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (j >= d) return;
+  double s = 0.0;
+  for (int b = threadIdx.x & 31; b < nslabs; b += 32) s += static_cast<double>(colpart[static_cast<long long>(b) * d + j]);
+  s = warp_sum(s);
+  if ((threadIdx.x & 31) == 0) diag[j] = static_cast<float>(s - 1.0);
+}
+
+// E = S - I for S = R^T R from the tensor cores (d x d float32, of which only the tiles that reach
+// the diagonal or lie above it were computed: tile rows of 128, tile columns of bn; the rest is
+// taken from the mirror entry).  max|E| goes into sc->max_e_bits (atomic max on the bit pattern of
+// a non-negative float: exact, order independent) and E as bf16 into e_hi when not null.
+// The diagonal is NOT taken from S: the tensor-core accumulator truncates, which biases a sum of d
+// positive terms near 1 by about one unit in the last place per MMA step; `diag` holds it exactly.
+// Off-diagonal sums hover around 0 and carry no such bias.  grid (d/32, d/32), block (32, 8).
+__global__ void k_guard(const float* __restrict__ S, int d, int bn, const float* __restrict__ diag,
                         __nv_bfloat16* __restrict__ e_hi, Scalars* __restrict__ sc) {
-  const long long i4 = (static_cast<long long>(blockIdx.x) * 256 + threadIdx.x) * 4;
-  const float4 s = *reinterpret_cast<const float4*>(S + i4);
-  const int row = static_cast<int>(i4 / d), col = static_cast<int>(i4 % d);
-  float e[4] = {s.x, s.y, s.z, s.w};
+  __shared__ float tile[32][33];
+  __shared__ float shm[8];
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  const bool computed = ((c0 / bn) + 1) * bn > (r0 / 128) * 128;
+  float e[4];
+  if (computed) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) e[q] = S[static_cast<long long>(r0 + ty + 8 * q) * d + c0 + tx];
+  } else {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) tile[ty + 8 * q][tx] = S[static_cast<long long>(c0 + ty + 8 * q) * d + r0 + tx];
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < 4; ++q) e[q] = tile[tx][ty + 8 * q];
+  }
   float mx = 0.f;
   bool bad = false;
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    if (col + j == row) {
-      double n2 = 0.0;
-      for (int b = 0; b < nslabs; ++b) n2 += static_cast<double>(colpart[static_cast<long long>(b) * d + row]);
-      e[j] = static_cast<float>(n2 - 1.0);
-    }
-    bad |= (e[j] != e[j]);
-    mx = fmaxf(mx, fabsf(e[j]));
+  for (int q = 0; q < 4; ++q) {
+    const int row = r0 + ty + 8 * q, col = c0 + tx;
+    if (row == col) e[q] = diag[row];
+    bad |= (e[q] != e[q]);
+    mx = fmaxf(mx, fabsf(e[q]));
+    if (e_hi) e_hi[static_cast<long long>(row) * d + col] = __float2bfloat16_rn(e[q]);
   }
   if (bad) mx = __uint_as_float(0x7f800000u);  // a NaN in R^T R reads as +inf
-  if (e_hi) {
-    __nv_bfloat162 a, b;
-    a.x = __float2bfloat16_rn(e[0]);
-    a.y = __float2bfloat16_rn(e[1]);
-    b.x = __float2bfloat16_rn(e[2]);
-    b.y = __float2bfloat16_rn(e[3]);
-    *reinterpret_cast<__nv_bfloat162*>(e_hi + i4) = a;
-    *reinterpret_cast<__nv_bfloat162*>(e_hi + i4 + 2) = b;
-  }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-  if ((threadIdx.x & 31) == 0 && mx > 0.f) atomicMax(&sc->max_e_bits, __float_as_uint(mx));
+  if (tx == 0) shm[ty] = mx;
+  __syncthreads();
+  if (tx == 0 && ty == 0) {
+#pragma unroll
+    for (int i = 1; i < 8; ++i) mx = fmaxf(mx, shm[i]);
+    if (mx > 0.f) atomicMax(&sc->max_e_bits, __float_as_uint(mx));
+  }
 }
 
 // gate = (max|E| > thresh).
@@ -375,17 +450,34 @@ __global__ void k_guard_decide(Scalars* sc, float thresh) {
   sc->gate = (mx > thresh) ? 1u : 0u;
 }
 
-// R <- R - Q/2 when the gate is open.  grid d*d/4/256, block 256.
-__global__ void k_polish_apply(float* __restrict__ R, const float* __restrict__ Q, const Scalars* __restrict__ sc) {
+// When the gate is open: R <- R - Q/2 (one Newton-Schulz step, Q = R E) and the bf16 forms of the
+// new R (r_hi, rt_hi, rt_lo) are rewritten.  grid (d/32, d/32), block (32, 8).
+__global__ void k_polish_apply(float* __restrict__ R, const float* __restrict__ Q, const Scalars* __restrict__ sc,
+                               int d, __nv_bfloat16* __restrict__ r_hi, __nv_bfloat16* __restrict__ rt_hi,
+                               __nv_bfloat16* __restrict__ rt_lo) {
   if (sc->gate == 0u) return;
-  const long long i4 = (static_cast<long long>(blockIdx.x) * 256 + threadIdx.x) * 4;
-  float4 r = *reinterpret_cast<float4*>(R + i4);
-  const float4 qv = *reinterpret_cast<const float4*>(Q + i4);
-  r.x = fmaf(-0.5f, qv.x, r.x);
-  r.y = fmaf(-0.5f, qv.y, r.y);
-  r.z = fmaf(-0.5f, qv.z, r.z);
-  r.w = fmaf(-0.5f, qv.w, r.w);
-  *reinterpret_cast<float4*>(R + i4) = r;
+  __shared__ float tile[32][33];
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int r = ty + 8 * q;
+    const long long o = static_cast<long long>(r0 + r) * d + c0 + tx;
+    const float v = fmaf(-0.5f, Q[o], R[o]);
+    R[o] = v;
+    tile[r][tx] = v;
+    r_hi[o] = __float2bfloat16_rn(v);
+  }
+  __syncthreads();
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int c = ty + 8 * q;
+    __nv_bfloat16 h, l;
+    split_bf16(tile[tx][c], h, l);
+    const long long o = static_cast<long long>(c0 + c) * d + r0 + tx;
+    rt_hi[o] = h;
+    rt_lo[o] = l;
+  }
 }
 
 // ------------------------------------------------------------------ quantizer

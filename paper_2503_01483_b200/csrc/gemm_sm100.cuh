@@ -36,6 +36,12 @@ struct GemmParams {
   int terms;
   int M, N, K;
   int m_tiles, n_tiles;
+  // split-K (kStoreF32 only): the k-blocks of every tile are cut into k_splits runs of kb_per_split blocks (all
+  // non-empty); run s writes its partial tile to out + s * split_stride.  k_splits = 1: no split.
+  int k_splits, kb_per_split;
+  long long split_stride;
+  // upper_only != 0 (square symmetric outputs): tiles that lie entirely below the diagonal are skipped
+  int upper_only;
   // epilogue operands (which are used depends on EPI)
   float* out;                 // kStoreF32: M x N, leading dimension ldo
   long long ldo;
@@ -85,9 +91,19 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int total_tiles = p.m_tiles * p.n_tiles;
+  const int total_tiles = p.m_tiles * p.n_tiles * p.k_splits;  // work units: (tile, k-run)
   const int k_blocks = (p.K + kBK - 1) / kBK;
-  const int iters = k_blocks * p.terms;
+  // k-block range and MMA/TMA iteration count of work unit u
+  // a tile whose last column is left of its first row holds only entries below the diagonal
+  auto skipped = [&](int tile) {
+    return p.upper_only != 0 && ((tile % p.n_tiles) + 1) * BN <= (tile / p.n_tiles) * kBM;
+  };
+  auto unit_kb0 = [&](int u) { return (u % p.k_splits) * p.kb_per_split; };
+  auto unit_iters = [&](int u) {
+    const int kb0 = (u % p.k_splits) * p.kb_per_split;
+    const int kb1 = (kb0 + p.kb_per_split < k_blocks) ? kb0 + p.kb_per_split : k_blocks;
+    return (kb1 - kb0) * p.terms;
+  };
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
@@ -125,12 +141,17 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
       uint32_t issued_mask = 0;  // stages that have had a load issued
       uint32_t last_parity = 0;  // parity of the last load issued, per stage
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      for (int unit = blockIdx.x; unit < total_tiles && ok; unit += gridDim.x) {
+        const int tile = unit / p.k_splits;
+        if (skipped(tile)) continue;
         const int m0 = (tile / p.n_tiles) * kBM;
         const int n0 = (tile % p.n_tiles) * BN;
+        const int kb0 = unit_kb0(unit);
+        const int iters = unit_iters(unit);
         for (int it = 0; it < iters; ++it) {
-          const int kb = it / p.terms;
-          const int q = it - kb * p.terms;
+          const int kbl = it / p.terms;
+          const int q = it - kbl * p.terms;
+          const int kb = kb0 + kbl;
           if (!mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, 1u)) {
             ok = false;
             break;
@@ -164,7 +185,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
       uint32_t phase = 0;
       int lt = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++lt) {
+      for (int unit = blockIdx.x; unit < total_tiles && ok; unit += gridDim.x) {
+        if (skipped(unit / p.k_splits)) continue;
+        const int iters = unit_iters(unit);
         const int buf = lt & 1;
         const uint32_t acc_phase = (lt >> 1) & 1;
         if (!mbar_wait_bounded(acc_empty_bar(buf), acc_phase ^ 1u, abort_flag, 2u)) {
@@ -193,6 +216,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
           }
         }
         if (ok) tc_commit(acc_full_bar(buf));  // accumulator complete
+        ++lt;
       }
     }
   } else {
@@ -200,7 +224,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
     const int lane_group = warp & 3;  // a warp may touch only tensor-memory lanes 32*(warp%4)..+31
     int lt = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++lt) {
+    for (int unit = blockIdx.x; unit < total_tiles && ok; unit += gridDim.x) {
+      const int tile = unit / p.k_splits;
+      if (skipped(tile)) continue;
       const int m_tile = tile / p.n_tiles;
       const int n_tile = tile % p.n_tiles;
       const int row = m_tile * kBM + lane_group * 32 + lane;
@@ -225,7 +251,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
           tmem_ld_32x32(t_addr + c0, v);
           tc_wait_ld();
           if (row_ok) {
-            float4* dst = reinterpret_cast<float4*>(p.out + static_cast<long long>(row) * p.ldo + n0 + c0);
+            float4* dst = reinterpret_cast<float4*>(p.out + static_cast<long long>(unit % p.k_splits) * p.split_stride +
+                                                    static_cast<long long>(row) * p.ldo + n0 + c0);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
               dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
@@ -326,6 +353,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(acc_empty_bar(buf));
+      ++lt;
     }
   }
 

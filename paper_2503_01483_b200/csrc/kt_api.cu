@@ -31,6 +31,40 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Split-K plan for the token contraction dR = X^T G (M = N = d, K = tokens).  The output has only
+// (d/128)*(d/BN) tiles, each walking all tokens: with few tiles (d = 128: one) most SMs would idle, and with
+// 512 tiles on 148 SMs the last of 3.46 waves is mostly empty.  Cutting K into s runs gives tiles*s work units.
+// s minimises a time model: (waves of units)/s tile times at ~10 TFLOP/s per SM, plus, for s > 1, the pass that
+// sums the s partial outputs ((2s+1) d^2 floats of traffic at ~6 TB/s and a launch).
+constexpr int kPlanSMs = 148;
+struct SplitPlan {
+  int splits, kb_per_split;
+};
+static SplitPlan plan_split_k(int64_t d, int64_t K) {
+  const int bn = (d % 256 == 0) ? 256 : 128;
+  const long long tiles = (d / 128) * (d / bn);
+  const int k_blocks = static_cast<int>((K + 63) / 64);
+  const double t_tile_us = 128.0 * bn * static_cast<double>(K) * 2.0 / 1.0e7;
+  const double dd_bytes = static_cast<double>(d) * d * 4.0;
+  int best = 1;
+  double best_cost = 1e300;
+  for (int s = 1; s <= 4 * kPlanSMs; ++s) {
+    const int per = (k_blocks + s - 1) / s;
+    if (s > 1 && (per < 16 || s * dd_bytes > 1073741824.0)) break;
+    const long long waves = (tiles * s + kPlanSMs - 1) / kPlanSMs;
+    double cost = static_cast<double>(waves) / s * t_tile_us;
+    if (s > 1) cost += (2.0 * s + 1.0) * dd_bytes / 6.0e6 + 5.0;
+    if (cost < best_cost * 0.98) {  // a larger s must win by 2 %
+      best_cost = cost;
+      best = s;
+    }
+  }
+  SplitPlan p;
+  p.kb_per_split = (k_blocks + best - 1) / best;
+  p.splits = (k_blocks + p.kb_per_split - 1) / p.kb_per_split;  // every run non-empty
+  return p;
+}
+
 // Where everything lives inside the caller's workspace for an (N, d) problem.
 struct WsLayout {
   size_t rt_hi, rt_lo;  // R^T as bf16 hi/lo  [d][d]
@@ -46,6 +80,8 @@ struct WsLayout {
   size_t block_loss, block_deg, norm_blocks;
   size_t rowmax, qerr;  // quantizer: [N] uint, [P][N] float
   size_t colpart;       // [d/32][d] float: column sums of squares of R by row slab
+  size_t diag;          // [d] float: exact diagonal of R^T R - I
+  size_t splitk;        // [splits][d][d] float: partial dR of the split-K backward-B (when splits > 1)
   size_t total;
   long long ldt;
   int P, bn, loss_blocks, norm_n;
@@ -88,6 +124,11 @@ static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype) {
   L.rowmax = take(static_cast<size_t>(N) * 4);
   L.qerr = take(static_cast<size_t>(L.P) * N * 4);
   L.colpart = take(static_cast<size_t>(d / 32) * d * 4);
+  L.diag = take(static_cast<size_t>(d) * 4);
+  {
+    const SplitPlan sp = plan_split_k(d, N);
+    L.splitk = take(sp.splits > 1 ? static_cast<size_t>(sp.splits) * dd * 4 : 0);
+  }
   L.total = off;
   return L;
 }
@@ -174,7 +215,7 @@ static kt_status launch_gemm_inst(kt_ctx* ctx, const GemmParams& p, int cat) {
     KT_CUDA(cudaFuncSetAttribute(gemm_tn_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     attr_done[ctx->device & 15] = true;
   }
-  const int tiles = p.m_tiles * p.n_tiles;
+  const int tiles = p.m_tiles * p.n_tiles * p.k_splits;
   const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
   const bool rec = ctx->prof_on && ctx->prof_used < kProfPairs;
   if (rec) KT_CUDA(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], ctx->stream));
@@ -203,6 +244,10 @@ static kt_status run_gemm(kt_ctx* ctx, int M, int N, int K, int terms, const Ope
   p.K = K;
   p.m_tiles = (M + kBM - 1) / kBM;
   p.n_tiles = N / bn;
+  if (p.k_splits < 1) {
+    p.k_splits = 1;
+    p.kb_per_split = (K + kBK - 1) / kBK;
+  }
   p.err_word = &ctx->d_blk->sc.err_word;
   for (int q = 0; q < terms; ++q) {
     KT_TRY(make_tmap(ctx, &p.tmA[q], A[q].base, K, M, A[q].ld, kBM));
@@ -324,49 +369,61 @@ static kt_status backward(kt_ctx* ctx, const XView& xv, int N, int d, const WsLa
   const FwdOperands f = fwd_operands(ctx, xv, d, L);
   KT_TRY(run_gemm<kGrad>(ctx, N, d, d, f.terms, f.A, f.B, p, kCatBackwardA));
   GemmParams p2 = blank_params();
-  p2.out = dR;
+  const SplitPlan sp = plan_split_k(d, N);
+  p2.out = sp.splits > 1 ? at<float>(ctx, L.splitk) : dR;
   p2.ldo = d;
+  p2.k_splits = sp.splits;
+  p2.kb_per_split = sp.kb_per_split;
+  p2.split_stride = static_cast<long long>(d) * d;
   Operand A2{at<__nv_bfloat16>(ctx, L.xt), static_cast<uint64_t>(L.ldt)},
       B2{at<__nv_bfloat16>(ctx, L.gt), static_cast<uint64_t>(L.ldt)};
   KT_TRY(run_gemm<kStoreF32>(ctx, d, d, N, 1, &A2, &B2, p2, kCatBackwardB));
+  if (sp.splits > 1) {
+    const long long n = static_cast<long long>(d) * d;
+    k_sum_splits<<<static_cast<unsigned>((n / 4 + 255) / 256), 256, 0, ctx->stream>>>(at<float>(ctx, L.splitk),
+                                                                                       sp.splits, n, n, dR);
+    KT_LAUNCH_CHECK();
+  }
   return KT_OK;
 }
 
 static kt_status loss_grad_async(kt_ctx* ctx, const XView& xv, int N, int d, const WsLayout& L, const float* R,
-                                 float* dR, double* hist_slot) {
-  KT_TRY(cast_rt(ctx, R, d, L));
+                                 float* dR, double* hist_slot, bool rt_current) {
+  if (!rt_current) KT_TRY(cast_rt(ctx, R, d, L));
   KT_TRY(forward_loss(ctx, xv, N, d, L, hist_slot));
   KT_TRY(backward(ctx, xv, N, d, L, dR));
   return KT_OK;
 }
 
 // ---------------------------------------------------------- orthogonal step
-// E = R^T R - I from the bf16 splits of R^T (rt_hi, rt_lo) and, when
-// `with_polish`, R <- R - R E / 2 if max|E| > polish_thresh (needs r_hi).
+// E = R^T R - I from the bf16 forms of R^T (rt_hi, rt_lo, which must be current) and, when
+// `with_polish`, R <- R - R E / 2 if max|E| > polish_thresh (needs r_hi; refreshes all three forms).
 static kt_status guard(kt_ctx* ctx, const float* R_in, float* R, int d, const WsLayout& L, bool with_polish) {
   Scalars* sc = &ctx->d_blk->sc;
-  {
-    dim3 tgrid(d / 32, d / 32), tblock(32, 8);
-    k_colnorm_partial<<<tgrid, tblock, 0, ctx->stream>>>(R_in, d, at<float>(ctx, L.colpart));
-    KT_LAUNCH_CHECK();
-  }
+  dim3 tgrid(d / 32, d / 32), tblock(32, 8);
+  k_colnorm_partial<<<tgrid, tblock, 0, ctx->stream>>>(R_in, d, at<float>(ctx, L.colpart));
+  KT_LAUNCH_CHECK();
+  k_colnorm_final<<<(d + 7) / 8, 256, 0, ctx->stream>>>(at<float>(ctx, L.colpart), d / 32, d, at<float>(ctx, L.diag));
+  KT_LAUNCH_CHECK();
   KT_CUDA(cudaMemsetAsync(&sc->max_e_bits, 0, sizeof(unsigned int), ctx->stream));
   const uint64_t ld = static_cast<uint64_t>(d);
   __nv_bfloat16* rt_hi = at<__nv_bfloat16>(ctx, L.rt_hi);
   __nv_bfloat16* rt_lo = at<__nv_bfloat16>(ctx, L.rt_lo);
+  __nv_bfloat16* r_hi = at<__nv_bfloat16>(ctx, L.r_hi);
   float* fbuf = at<float>(ctx, L.fbuf);
   {
     GemmParams p = blank_params();
     p.out = fbuf;
     p.ldo = d;
-    // (H + L)^T (H + L) without L^T L: that term only matters on the diagonal, which k_guard rebuilds exactly
+    p.upper_only = 1;  // R^T R is symmetric: tiles below the diagonal are mirrored by k_guard
+    // (H + L)^T (H + L) without L^T L: that term only matters on the diagonal, which k_guard takes from `diag`
     Operand A[3] = {{rt_hi, ld}, {rt_hi, ld}, {rt_lo, ld}};
     Operand B[3] = {{rt_hi, ld}, {rt_lo, ld}, {rt_hi, ld}};
     KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 3, A, B, p, kCatSquare));
   }
   __nv_bfloat16* e_hi = at<__nv_bfloat16>(ctx, L.z_hi);
-  const unsigned blocks = static_cast<unsigned>(static_cast<long long>(d) * d / 4 / 256);
-  k_guard<<<blocks, 256, 0, ctx->stream>>>(fbuf, d, at<float>(ctx, L.colpart), d / 32, with_polish ? e_hi : nullptr, sc);
+  k_guard<<<tgrid, tblock, 0, ctx->stream>>>(fbuf, d, (d % 256 == 0) ? 256 : 128, at<float>(ctx, L.diag),
+                                             with_polish ? e_hi : nullptr, sc);
   KT_LAUNCH_CHECK();
   if (!with_polish) return KT_OK;
   k_guard_decide<<<1, 1, 0, ctx->stream>>>(sc, ctx->cfg.polish_thresh);
@@ -376,16 +433,18 @@ static kt_status guard(kt_ctx* ctx, const float* R_in, float* R, int d, const Ws
     p.out = fbuf;
     p.ldo = d;
     p.gate = &sc->gate;
-    Operand A{at<__nv_bfloat16>(ctx, L.r_hi), ld}, B{e_hi, ld};  // (R E)[i][j] = sum_k R[i][k] E[j][k], E symmetric
+    Operand A{r_hi, ld}, B{e_hi, ld};  // (R E)[i][j] = sum_k R[i][k] E[j][k], E symmetric
     KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 1, &A, &B, p, kCatSquare));
   }
-  k_polish_apply<<<blocks, 256, 0, ctx->stream>>>(R, fbuf, sc);
+  k_polish_apply<<<tgrid, tblock, 0, ctx->stream>>>(R, fbuf, sc, d, r_hi, rt_hi, rt_lo);
   KT_LAUNCH_CHECK();
   return KT_OK;
 }
 
+// One Cayley-SGD step.  `forms_current`: r_hi / rt_hi / rt_lo already hold the bf16 forms of R (true from the
+// second step of kt_fit on: the previous step left them).  On return they hold the forms of the new R.
 static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, float lr, const WsLayout& L,
-                                 bool run_guard) {
+                                 bool run_guard, bool forms_current) {
   const kt_config& c = ctx->cfg;
   Scalars* sc = &ctx->d_blk->sc;
   const uint64_t ld = static_cast<uint64_t>(d);
@@ -394,20 +453,19 @@ static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, 
   __nv_bfloat16* rt_lo = at<__nv_bfloat16>(ctx, L.rt_lo);
   __nv_bfloat16* r_hi = at<__nv_bfloat16>(ctx, L.r_hi);
   __nv_bfloat16* z_hi = at<__nv_bfloat16>(ctx, L.z_hi);
-  __nv_bfloat16* z_lo = at<__nv_bfloat16>(ctx, L.z_lo);
   __nv_bfloat16* w_hi = at<__nv_bfloat16>(ctx, L.w_hi);
   __nv_bfloat16* w_lo = at<__nv_bfloat16>(ctx, L.w_lo);
   float* fbuf = at<float>(ctx, L.fbuf);
   const int terms = c.retract_terms < 1 ? 1 : (c.retract_terms > 3 ? 3 : c.retract_terms);
 
   // A = dR R^T (the gradient needs no more than bf16), W = (A - A^T)/2, alpha
-  k_split_bf16<false><<<tgrid, tblock, 0, ctx->stream>>>(dR, d, z_hi /* dR hi, free until the iterate is written */,
-                                                         nullptr, d);
+  k_split_bf16<false><<<tgrid, tblock, 0, ctx->stream>>>(dR, d, z_hi /* dR hi: free until P^T is written */, nullptr,
+                                                         d);
   KT_LAUNCH_CHECK();
-  k_split_bf16<false><<<tgrid, tblock, 0, ctx->stream>>>(R, d, r_hi, nullptr, d);
-  KT_LAUNCH_CHECK();
-  k_split_bf16<true><<<tgrid, tblock, 0, ctx->stream>>>(R, d, rt_hi, rt_lo, d);
-  KT_LAUNCH_CHECK();
+  if (!forms_current) {
+    k_split_r<<<tgrid, tblock, 0, ctx->stream>>>(R, d, r_hi, rt_hi, rt_lo);
+    KT_LAUNCH_CHECK();
+  }
   {
     GemmParams p = blank_params();
     p.out = fbuf;
@@ -421,31 +479,25 @@ static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, 
   k_step_size<<<1, 256, 0, ctx->stream>>>(at<double>(ctx, L.norm_blocks), L.norm_n, lr, c.q, c.eps, sc);
   KT_LAUNCH_CHECK();
 
-  // P = W Z, Z^T given as bf16 hi/lo: (W Z)[i][j] = sum_k W[i][k] Zt[j][k]
-  auto product = [&](const __nv_bfloat16* zt_hi, const __nv_bfloat16* zt_lo) -> kt_status {
+  // P_0 = W R with R^T as a bf16 split (it multiplies alpha directly); P_{k+1} = W P_k with P_k^T in plain bf16
+  // (these terms carry alpha^2 and higher).  (W Z)[i][j] = sum_k W[i][k] Zt[j][k].
+  const int s = c.cayley_iters < 0 ? 0 : c.cayley_iters;
+  for (int k = 0; k <= s; ++k) {
     GemmParams p = blank_params();
     p.out = fbuf;
     p.ldo = d;
-    Operand A[3] = {{w_hi, ld}, {w_hi, ld}, {w_lo, ld}};
-    Operand B[3] = {{zt_hi, ld}, {zt_lo, ld}, {zt_hi, ld}};
-    return run_gemm<kStoreF32>(ctx, d, d, d, terms, A, B, p, kCatSquare);
-  };
-  const int s = c.cayley_iters < 0 ? 0 : c.cayley_iters;
-  // Y0 = R - alpha W R
-  KT_TRY(product(rt_hi, rt_lo));
-  for (int i = 0; i <= s; ++i) {
-    const float cmul = (i == 0) ? 1.0f : 0.5f;
-    if (i < s) {
-      // Z = R + Y_i for the next product
-      k_axpy_split<<<tgrid, tblock, 0, ctx->stream>>>(R, fbuf, sc, cmul, 1.0f, d, nullptr, z_hi, z_lo, nullptr,
-                                                      nullptr);
-      KT_LAUNCH_CHECK();
-      KT_TRY(product(z_hi, z_lo));
+    if (k == 0) {
+      Operand A[3] = {{w_hi, ld}, {w_hi, ld}, {w_lo, ld}};
+      Operand B[3] = {{rt_hi, ld}, {rt_lo, ld}, {rt_hi, ld}};
+      KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, terms, A, B, p, kCatSquare));
     } else {
-      // R <- Y_s, and its splits for the guard
-      k_axpy_split<<<tgrid, tblock, 0, ctx->stream>>>(R, fbuf, sc, cmul, 0.0f, d, R, rt_hi, rt_lo, r_hi, nullptr);
-      KT_LAUNCH_CHECK();
+      Operand A{w_hi, ld}, B{z_hi, ld};
+      KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 1, &A, &B, p, kCatSquare));
     }
+    const bool last = (k == s);
+    k_series_term<<<tgrid, tblock, 0, ctx->stream>>>(R, fbuf, sc, k, d, last ? nullptr : z_hi, last ? r_hi : nullptr,
+                                                     last ? rt_hi : nullptr, last ? rt_lo : nullptr);
+    KT_LAUNCH_CHECK();
   }
   if (run_guard) KT_TRY(guard(ctx, R, R, d, L, true));
   return KT_OK;
@@ -492,9 +544,10 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
       if (report && report->loss_history)
         memcpy(report->loss_history + (k - kHistMax), ctx->h_blk->hist, sizeof(double) * kHistMax);
     }
-    KT_TRY(loss_grad_async(ctx, xv, N, d, L, R, dR, &ctx->d_blk->hist[slot]));
+    // from the second step on, the previous step left the bf16 forms of R in the workspace
+    KT_TRY(loss_grad_async(ctx, xv, N, d, L, R, dR, &ctx->d_blk->hist[slot], k > 0));
     const bool run_guard = ((k + 1) % ge == 0) || (k + 1 == steps);
-    KT_TRY(orth_step_async(ctx, R, dR, d, lr, L, run_guard));
+    KT_TRY(orth_step_async(ctx, R, dR, d, lr, L, run_guard, k > 0));
     done = k + 1;
   }
   if (steps > 0) {
@@ -705,7 +758,7 @@ kt_status kt_loss_grad(kt_ctx* ctx, kt_mat X, const float* R, float* dR, double*
   KT_TRY(check_ws(ctx, L));
   XView xv;
   KT_TRY(ingest_x_full(ctx, X, L, &xv));
-  KT_TRY(loss_grad_async(ctx, xv, static_cast<int>(N), static_cast<int>(d), L, R, dR, nullptr));
+  KT_TRY(loss_grad_async(ctx, xv, static_cast<int>(N), static_cast<int>(d), L, R, dR, nullptr, false));
   if (!loss) return KT_OK;
   KT_TRY(sync_scalars(ctx));
   *loss = ctx->h_blk->sc.loss;
@@ -718,7 +771,7 @@ kt_status kt_orth_step(kt_ctx* ctx, float* R, const float* dR, int64_t d, float 
   if (!aligned16(R) || !aligned16(dR)) return KT_ERR_ALIGN;
   const WsLayout L = make_layout(1, d, KT_BF16);
   KT_TRY(check_ws(ctx, L));
-  return orth_step_async(ctx, R, dR, static_cast<int>(d), lr, L, true);
+  return orth_step_async(ctx, R, dR, static_cast<int>(d), lr, L, true, false);
 }
 
 kt_status kt_orth_error(kt_ctx* ctx, const float* R, int64_t d, double* err) {

@@ -28,12 +28,13 @@ def _student_t(shape, nu, device):
     z = torch.randn(shape, device=device, dtype=torch.float32)
     # chi2(nu) = 2 * Gamma(nu/2, 1)
     g = torch._standard_gamma(torch.full(shape, nu / 2.0, device=device, dtype=torch.float32))
-    return z / torch.sqrt(2.0 * g / nu)
+    return z / torch.sqrt((2.0 * g / nu).clamp_(min=1e-20))
 
 
 def _laplace(shape, device):
     u = torch.rand(shape, device=device, dtype=torch.float32) - 0.5
-    return -torch.sign(u) * torch.log1p(-2.0 * u.abs())
+    # rand() can return exactly 0, i.e. |u| = 0.5 and log(0): keep the argument of the log positive
+    return -torch.sign(u) * torch.log1p(-(2.0 * u.abs()).clamp_(max=1.0 - 2.0 ** -24))
 
 
 def activations(N, d, dist="student_t", nu=3.0, n_outliers=0, outlier_scale=1.0,
