@@ -91,16 +91,18 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int total_tiles = p.m_tiles * p.n_tiles * p.k_splits;  // work units: (tile, k-run)
+  const int plain_tiles = p.m_tiles * p.n_tiles;
+  const int total_tiles = plain_tiles * p.k_splits;  // work units (k-run, tile), k-run major: CTAs that run
+                                                     // together walk the same k range and share operands in L2
   const int k_blocks = (p.K + kBK - 1) / kBK;
   // k-block range and MMA/TMA iteration count of work unit u
   // a tile whose last column is left of its first row holds only entries below the diagonal
   auto skipped = [&](int tile) {
     return p.upper_only != 0 && ((tile % p.n_tiles) + 1) * BN <= (tile / p.n_tiles) * kBM;
   };
-  auto unit_kb0 = [&](int u) { return (u % p.k_splits) * p.kb_per_split; };
+  auto unit_kb0 = [&](int u) { return (u / plain_tiles) * p.kb_per_split; };
   auto unit_iters = [&](int u) {
-    const int kb0 = (u % p.k_splits) * p.kb_per_split;
+    const int kb0 = (u / plain_tiles) * p.kb_per_split;
     const int kb1 = (kb0 + p.kb_per_split < k_blocks) ? kb0 + p.kb_per_split : k_blocks;
     return (kb1 - kb0) * p.terms;
   };
@@ -142,7 +144,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
       uint32_t last_parity = 0;  // parity of the last load issued, per stage
       bool ok = true;
       for (int unit = blockIdx.x; unit < total_tiles && ok; unit += gridDim.x) {
-        const int tile = unit / p.k_splits;
+        const int tile = unit % plain_tiles;
         if (skipped(tile)) continue;
         const int m0 = (tile / p.n_tiles) * kBM;
         const int n0 = (tile % p.n_tiles) * BN;
@@ -186,7 +188,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
       int lt = 0;
       bool ok = true;
       for (int unit = blockIdx.x; unit < total_tiles && ok; unit += gridDim.x) {
-        if (skipped(unit / p.k_splits)) continue;
+        if (skipped(unit % plain_tiles)) continue;
         const int iters = unit_iters(unit);
         const int buf = lt & 1;
         const uint32_t acc_phase = (lt >> 1) & 1;
@@ -225,7 +227,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
     int lt = 0;
     bool ok = true;
     for (int unit = blockIdx.x; unit < total_tiles && ok; unit += gridDim.x) {
-      const int tile = unit / p.k_splits;
+      const int tile = unit % plain_tiles;
       if (skipped(tile)) continue;
       const int m_tile = tile / p.n_tiles;
       const int n_tile = tile % p.n_tiles;
@@ -251,7 +253,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
           tmem_ld_32x32(t_addr + c0, v);
           tc_wait_ld();
           if (row_ok) {
-            float4* dst = reinterpret_cast<float4*>(p.out + static_cast<long long>(unit % p.k_splits) * p.split_stride +
+            float4* dst = reinterpret_cast<float4*>(p.out + static_cast<long long>(unit / plain_tiles) * p.split_stride +
                                                     static_cast<long long>(row) * p.ldo + n0 + c0);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
