@@ -84,7 +84,10 @@ typedef struct {
                            to bf16; 2 = hi + lo (about 16 significant bits,
                            twice the MMA work); 0 = 2 when d <= 512 (where the
                            pass is memory bound anyway), else 1                */
-  int32_t reserved[4];
+  int32_t small_d_fused;/* [1]   d == 128: kt_loss_grad / kt_fit use the single-pass
+                           kernel (X read once per evaluation); 0 = the general
+                           three-GEMM path                                      */
+  int32_t reserved[3];
 } kt_config;
 
 /* Filled by kt_fit / kt_fit_layers (host memory). */
@@ -243,7 +246,8 @@ kt_status kt_kurtosis_loss_noalloc(kt_mat X, const float* R, double* loss_dev, v
  * kt_profile_begin() and kt_profile_end(): 0 forward (Y = X R with the moment
  * epilogue; Section 2, Eq. 3), 1 backward-A (recompute Y, write dL/dY),
  * 2 backward-B (dR = X^T dL/dY), 3 the d x d products of the Cayley step and its
- * guard (Section 3), 4 the two quantizer passes (Section 2, Eq. 1).  Times come
+ * guard (Section 3), 4 the two quantizer passes (Section 2, Eq. 1), 5 the
+ * single-pass loss+gradient kernel used when d == 128.  Times come
  * from CUDA events recorded on the context's stream around each launch (up to
  * 8192 launches per window).  launches_total counts every kernel this library
  * launched in the window.  kt_profile_end() synchronises; `out` is host memory. */

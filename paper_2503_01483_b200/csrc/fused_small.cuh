@@ -1,0 +1,384 @@
+// Single-pass loss + gradient for d = 128 (one rotation shared by many short rows, e.g. the
+// value/KV rotation of Section 3, "Placement of the Rotations").
+//
+// A whole row of Y = X R fits one 128-column tensor-memory tile, so one CTA can take a tile of 128
+// tokens through the complete chain without leaving the SM:
+//
+//   TMA:  X tile (128 tokens x 128 channels, bf16)                     -> shared memory
+//   MMA1: Y = X R (R^T resident in shared memory, hi [+ lo])           -> tensor memory
+//   epilogue: per row mean, m2, m3, m4 (Eq. 3), kappa, loss term, then
+//             G = a c^3 - ab c - am3 as bf16                           -> shared memory
+//   MMA2: dR += X^T G  (both operands read token-major straight from the tiles above,
+//             "MN-major" shared-memory descriptors)                    -> one persistent accumulator
+//
+// X is read from HBM exactly once per evaluation; Y and G never leave the SM.  Each CTA ends by
+// writing its partial dR (128 x 128 float32) and partial loss; a fixed-order sum over CTAs follows.
+#pragma once
+#include <cuda.h>
+
+#include "sm100_prims.cuh"
+
+namespace kt {
+
+constexpr int kFsD = 128;          // channels = rows of a token tile
+constexpr int kFsThreads = 192;    // warp 0: TMA, warp 1: MMA, warps 2..5: epilogue
+constexpr int kFsXStages = 3;
+constexpr int kFsHalf = 128 * 64 * 2;      // bytes of one 128-row x 64-element swizzled block
+constexpr int kFsTile = 2 * kFsHalf;       // one 128 x 128 bf16 tile
+constexpr int kFsSmem = 1024 + 2 * kFsTile /*R^T hi, lo*/ + kFsXStages * kFsTile + 2 * kFsTile /*G*/ + 256;
+
+struct FusedParams {
+  CUtensorMap tmX;    // X  [N][128] bf16, box 128 rows x 64
+  CUtensorMap tmRhi;  // R^T hi [128][128] bf16, box 128 x 64
+  CUtensorMap tmRlo;  // R^T lo
+  int terms;          // 1: R^T hi only; 2: hi + lo
+  int N;
+  int tiles;          // ceil(N / 128)
+  float kappa_t;
+  float* dr_partial;        // [gridDim.x][128][128]
+  double* loss_partial;     // [gridDim.x]
+  unsigned int* deg_partial;// [gridDim.x]
+  unsigned int* err_word;
+};
+
+// Shared-memory descriptor for an "MN-major" bf16 operand stored as rows of 64 elements (128 bytes,
+// 128-byte swizzle) where the ROW index is the contraction index k and the 64 contiguous elements run
+// along M (or N): eight k-rows form a 1024-byte group (stride field), the next 64 elements of M/N live
+// `lead_bytes` further on (leading field).
+__device__ __forceinline__ uint64_t umma_desc_mnmajor_sw128(uint32_t smem_addr, uint32_t lead_bytes,
+                                                            uint32_t stride_bytes) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>(lead_bytes >> 4) << 16;
+  d |= static_cast<uint64_t>(stride_bytes >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+
+__global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid_constant__ FusedParams p) {
+  constexpr uint32_t kIdescK = umma_idesc_bf16_f32(128, 128);                            // both K-major
+  constexpr uint32_t kIdescMN = umma_idesc_bf16_f32(128, 128) | (1u << 15) | (1u << 16);  // both MN-major
+  constexpr uint32_t kTmemCols = 512;  // Y accumulators at columns 0 and 128, dR accumulator at 256
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t s_rhi = base;
+  const uint32_t s_rlo = base + kFsTile;
+  const uint32_t s_x = base + 2 * kFsTile;
+  const uint32_t s_g = s_x + kFsXStages * kFsTile;
+  const uint32_t bars = s_g + 2 * kFsTile;
+  auto x_full = [&](int s) { return bars + 8u * s; };
+  auto x_empty = [&](int s) { return bars + 8u * (kFsXStages + s); };
+  auto y_full = [&](int b) { return bars + 8u * (2 * kFsXStages + b); };
+  auto y_empty = [&](int b) { return bars + 8u * (2 * kFsXStages + 2 + b); };
+  auto g_full = [&](int b) { return bars + 8u * (2 * kFsXStages + 4 + b); };
+  auto g_empty = [&](int b) { return bars + 8u * (2 * kFsXStages + 6 + b); };
+  const uint32_t r_full = bars + 8u * (2 * kFsXStages + 8);
+  const uint32_t dr_full = bars + 8u * (2 * kFsXStages + 9);
+  uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gbase + (bars - base) + 192);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+  double* sh_loss = reinterpret_cast<double*>(gbase + (bars - base) + 208);          // 4 doubles
+  unsigned int* sh_deg = reinterpret_cast<unsigned int*>(gbase + (bars - base) + 240);  // 4 words
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  // tiles of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ...
+  const int my_tiles = (p.tiles > static_cast<int>(blockIdx.x))
+                           ? (p.tiles - 1 - static_cast<int>(blockIdx.x)) / static_cast<int>(gridDim.x) + 1
+                           : 0;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    prefetch_tensormap(&p.tmX);
+    prefetch_tensormap(&p.tmRhi);
+    prefetch_tensormap(&p.tmRlo);
+  }
+  if (warp == 1) {
+    if (lane == 0) {
+      for (int s = 0; s < kFsXStages; ++s) {
+        mbar_init(x_full(s), 1);
+        mbar_init(x_empty(s), 1);
+      }
+      for (int b = 0; b < 2; ++b) {
+        mbar_init(y_full(b), 1);
+        mbar_init(y_empty(b), 4);
+        mbar_init(g_full(b), 4);
+        mbar_init(g_empty(b), 1);
+      }
+      mbar_init(r_full, 1);
+      mbar_init(dr_full, 1);
+      fence_barrier_init();
+    }
+    __syncwarp();
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0 && my_tiles > 0) {
+      mbar_arrive_expect_tx(r_full, static_cast<uint32_t>(p.terms) * kFsTile);
+      tma_load_2d(s_rhi, &p.tmRhi, 0, 0, r_full);
+      tma_load_2d(s_rhi + kFsHalf, &p.tmRhi, 64, 0, r_full);
+      if (p.terms == 2) {
+        tma_load_2d(s_rlo, &p.tmRlo, 0, 0, r_full);
+        tma_load_2d(s_rlo + kFsHalf, &p.tmRlo, 64, 0, r_full);
+      }
+      bool ok = true;
+      uint32_t issued = 0, last_parity = 0;
+      for (int n = 0; n < my_tiles; ++n) {
+        const int s = n % kFsXStages;
+        const uint32_t ph = (n / kFsXStages) & 1;
+        if (!mbar_wait_bounded(x_empty(s), ph ^ 1u, abort_flag, 11u)) {
+          ok = false;
+          break;
+        }
+        const int row0 = (static_cast<int>(blockIdx.x) + n * static_cast<int>(gridDim.x)) * 128;
+        mbar_arrive_expect_tx(x_full(s), kFsTile);
+        tma_load_2d(s_x + s * kFsTile, &p.tmX, 0, row0, x_full(s));
+        tma_load_2d(s_x + s * kFsTile + kFsHalf, &p.tmX, 64, row0, x_full(s));
+        issued |= 1u << s;
+        last_parity = (last_parity & ~(1u << s)) | (ph << s);
+      }
+      if (!ok) {
+        for (int s = 0; s < kFsXStages; ++s) {
+          if (!(issued & (1u << s))) continue;
+          const uint64_t t0 = global_timer_ns();
+          while (!mbar_try_wait(x_full(s), (last_parity >> s) & 1u)) {
+            if (global_timer_ns() - t0 > 1000000ull) break;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // -------------------------------------------------------------- MMA issuer
+    if (lane == 0 && my_tiles > 0) {
+      bool ok = mbar_wait_bounded(r_full, 0u, abort_flag, 12u);
+      const uint32_t acc_dr = tmem_base + 256u;
+      for (int n = 0; n <= my_tiles && ok; ++n) {
+        if (n < my_tiles) {
+          // Y(n) = X(n) R
+          const int s = n % kFsXStages;
+          const int b = n & 1;
+          if (!mbar_wait_bounded(x_full(s), (n / kFsXStages) & 1, abort_flag, 13u) ||
+              !mbar_wait_bounded(y_empty(b), ((n >> 1) & 1) ^ 1u, abort_flag, 14u)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after_sync();
+          const uint32_t acc_y = tmem_base + static_cast<uint32_t>(b * 128);
+          uint32_t first = 1;
+          for (int q = 0; q < p.terms; ++q) {
+            const uint32_t rb = (q == 0) ? s_rhi : s_rlo;
+#pragma unroll
+            for (int kb = 0; kb < 2; ++kb) {
+              const uint64_t a_desc = umma_desc_kmajor_sw128(s_x + s * kFsTile + kb * kFsHalf, 1024);
+              const uint64_t b_desc = umma_desc_kmajor_sw128(rb + kb * kFsHalf, 1024);
+#pragma unroll
+              for (int kk = 0; kk < 4; ++kk) {
+                tc_mma_bf16(acc_y, a_desc + 2u * kk, b_desc + 2u * kk, kIdescK, first ? 0u : 1u);
+                first = 0;
+              }
+            }
+          }
+          tc_commit(y_full(b));
+        }
+        if (n >= 1) {
+          // dR += X(m)^T G(m): contraction over the tile's 128 tokens, 16 per MMA = two 8-row groups
+          const int m = n - 1;
+          const int s = m % kFsXStages;
+          const int b = m & 1;
+          if (!mbar_wait_bounded(g_full(b), (m >> 1) & 1, abort_flag, 15u)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after_sync();
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {
+            const uint64_t a_desc = umma_desc_mnmajor_sw128(s_x + s * kFsTile + ks * 2048, kFsHalf, 1024);
+            const uint64_t b_desc = umma_desc_mnmajor_sw128(s_g + b * kFsTile + ks * 2048, kFsHalf, 1024);
+            tc_mma_bf16(acc_dr, a_desc, b_desc, kIdescMN, (m > 0 || ks > 0) ? 1u : 0u);
+          }
+          tc_commit(x_empty(s));   // the X tile is free once these MMAs have read it
+          tc_commit(g_empty(b));
+        }
+      }
+      if (ok) tc_commit(dr_full);
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue
+    const int lg = warp & 3;                 // tensor-memory lane group of this warp
+    const int trow = lg * 32 + lane;         // row of the tile = token within the tile (and dR row at the end)
+    double loss_acc = 0.0;
+    unsigned int deg_acc = 0;
+    bool ok = true;
+    const float inv_nd = 1.0f;  // (kept in double below)
+    (void)inv_nd;
+    for (int n = 0; n < my_tiles && ok; ++n) {
+      const int b = n & 1;
+      const bool got = mbar_wait_bounded(y_full(b), (n >> 1) & 1, abort_flag, 16u);
+      if (!__all_sync(0xffffffffu, got)) {
+        ok = false;
+        break;
+      }
+      tc_fence_after_sync();
+      const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + static_cast<uint32_t>(b * 128);
+      uint32_t v[4][32];
+      tmem_ld_32x32(t_addr, v[0]);
+      tmem_ld_32x32(t_addr + 32, v[1]);
+      tmem_ld_32x32(t_addr + 64, v[2]);
+      tmem_ld_32x32(t_addr + 96, v[3]);
+      tc_wait_ld();
+      // the accumulator can be refilled while this tile is being reduced
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(y_empty(b));
+
+      // Eq. 3 on the row: mean, then central power sums about it
+      float s1 = 0.f;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) {
+          a0 += __uint_as_float(v[c][j]);
+          a1 += __uint_as_float(v[c][j + 1]);
+          a2 += __uint_as_float(v[c][j + 2]);
+          a3 += __uint_as_float(v[c][j + 3]);
+        }
+        s1 += (a0 + a1) + (a2 + a3);
+      }
+      const float mean = s1 * (1.0f / 128.0f);
+      float s2 = 0.f, s3 = 0.f, s4 = 0.f;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        float b2 = 0.f, b3 = 0.f, b4 = 0.f;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const float cc = __uint_as_float(v[c][j]) - mean;
+          const float c2 = cc * cc;
+          b2 += c2;
+          b3 = fmaf(c2, cc, b3);
+          b4 = fmaf(c2, c2, b4);
+        }
+        s2 += b2;
+        s3 += b3;
+        s4 += b4;
+      }
+      // kappa, loss term and the coefficients of dL/dY (same rules as the general path)
+      const int row = (static_cast<int>(blockIdx.x) + n * static_cast<int>(gridDim.x)) * 128 + trow;
+      const double m2 = static_cast<double>(s2) / 128.0, m3 = static_cast<double>(s3) / 128.0,
+                   m4 = static_cast<double>(s4) / 128.0;
+      const double mu = static_cast<double>(mean);
+      const double ms = m2 + mu * mu;
+      const bool degenerate = (ms == 0.0) || (m2 <= 1e-6 * ms);
+      float ca = 0.f, cab = 0.f, cam3 = 0.f;
+      if (!degenerate) {
+        const double kappa = m4 / (m2 * m2);
+        const double diff = kappa - static_cast<double>(p.kappa_t);
+        const double sgn = (diff > 0.0) ? 1.0 : ((diff < 0.0) ? -1.0 : 0.0);
+        const double a = sgn * 4.0 / (static_cast<double>(p.N) * 128.0 * m2 * m2);
+        ca = static_cast<float>(a);
+        cab = static_cast<float>(a * m4 / m2);
+        cam3 = static_cast<float>(a * m3);
+        if (row < p.N) loss_acc += fabs(diff);
+      } else if (row < p.N) {
+        ++deg_acc;
+      }
+
+      // G = a c^3 - ab c - am3 as bf16, token-major, into the swizzled tile MMA2 reads
+      const bool free_g = mbar_wait_bounded(g_empty(b), ((n >> 1) & 1) ^ 1u, abort_flag, 17u);
+      if (!__all_sync(0xffffffffu, free_g)) {
+        ok = false;
+        break;
+      }
+      const uint32_t g_row = s_g + b * kFsTile + static_cast<uint32_t>(trow) * 128u;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+#pragma unroll
+        for (int j8 = 0; j8 < 4; ++j8) {
+          uint32_t pk[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float c0 = __uint_as_float(v[c][j8 * 8 + 2 * e]) - mean;
+            const float c1 = __uint_as_float(v[c][j8 * 8 + 2 * e + 1]) - mean;
+            const float g0 = fmaf(c0, fmaf(ca * c0, c0, -cab), -cam3);
+            const float g1 = fmaf(c1, fmaf(ca * c1, c1, -cab), -cam3);
+            __nv_bfloat162 h = __floats2bfloat162_rn(g0, g1);
+            pk[e] = *reinterpret_cast<uint32_t*>(&h);
+          }
+          const int chunk = c * 4 + j8;                 // 16-byte chunk 0..15 of the 256-byte row
+          const uint32_t addr = g_row + static_cast<uint32_t>(chunk >> 3) * kFsHalf +
+                                (static_cast<uint32_t>((chunk & 7) ^ (trow & 7)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]),
+                       "r"(pk[3])
+                       : "memory");
+        }
+      }
+      fence_proxy_async_smem();  // make the generic-proxy stores visible to the tensor core
+      __syncwarp();
+      if (lane == 0) mbar_arrive(g_full(b));
+    }
+
+    // partial loss of this CTA (fixed order: lanes by shuffle tree, then warps 2,3,4,5 -> lane groups 2,3,0,1)
+    {
+      double l = loss_acc;
+      unsigned int dg = deg_acc;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        l += __shfl_down_sync(0xffffffffu, l, o);
+        dg += __shfl_down_sync(0xffffffffu, dg, o);
+      }
+      if (lane == 0) {
+        sh_loss[lg] = l;
+        sh_deg[lg] = dg;
+      }
+    }
+    // partial dR of this CTA
+    if (my_tiles > 0 && ok) {
+      const bool got = mbar_wait_bounded(dr_full, 0u, abort_flag, 18u);
+      if (__all_sync(0xffffffffu, got)) {
+        tc_fence_after_sync();
+        const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + 256u;
+        float* dst = p.dr_partial + (static_cast<long long>(blockIdx.x) * 128 + trow) * 128;
+        uint32_t w[32];
+#pragma unroll 1
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+          tmem_ld_32x32(t_addr + c0, w);
+          tc_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            reinterpret_cast<float4*>(dst + c0)[j] =
+                make_float4(__uint_as_float(w[4 * j]), __uint_as_float(w[4 * j + 1]), __uint_as_float(w[4 * j + 2]),
+                            __uint_as_float(w[4 * j + 3]));
+          }
+        }
+      }
+    } else if (my_tiles == 0) {
+      float* dst = p.dr_partial + (static_cast<long long>(blockIdx.x) * 128 + trow) * 128;
+      for (int j = 0; j < 32; ++j) reinterpret_cast<float4*>(dst)[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+  if (threadIdx.x == 0) {
+    p.loss_partial[blockIdx.x] = (sh_loss[0] + sh_loss[1]) + (sh_loss[2] + sh_loss[3]);
+    p.deg_partial[blockIdx.x] = sh_deg[0] + sh_deg[1] + sh_deg[2] + sh_deg[3];
+    if (*abort_flag != 0 && p.err_word != nullptr) atomicMax(p.err_word, *abort_flag);
+  }
+}
+
+}  // namespace kt

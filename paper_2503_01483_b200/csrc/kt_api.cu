@@ -12,13 +12,14 @@
 
 #include "../../include/kurtail.h"
 #include "elementwise.cuh"
+#include "fused_small.cuh"
 #include "gemm_sm100.cuh"
 
 namespace kt {
 
 constexpr int kHistMax = 4096;  // loss-history slots kept on the device between host read-backs
 constexpr int kProfPairs = 8192; // CUDA-event pairs available to one profiling window
-enum GemmCat : int { kCatForward = 0, kCatBackwardA = 1, kCatBackwardB = 2, kCatSquare = 3, kCatQuant = 4 };
+enum GemmCat : int { kCatForward = 0, kCatBackwardA = 1, kCatBackwardB = 2, kCatSquare = 3, kCatQuant = 4, kCatFused = 5 };
 
 struct DeviceBlock {
   Scalars sc;
@@ -118,8 +119,9 @@ static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype) {
   L.partial = take(static_cast<size_t>(L.P) * N * 16);
   L.coef = take(static_cast<size_t>(N) * 16);
   L.moments = take(static_cast<size_t>(N) * 16);
-  L.block_loss = take(static_cast<size_t>(L.loss_blocks) * 8);
-  L.block_deg = take(static_cast<size_t>(L.loss_blocks) * 4);
+  // at least 256 entries: the fused d = 128 kernel writes one partial per CTA here
+  L.block_loss = take(static_cast<size_t>(L.loss_blocks > 256 ? L.loss_blocks : 256) * 8);
+  L.block_deg = take(static_cast<size_t>(L.loss_blocks > 256 ? L.loss_blocks : 256) * 4);
   L.norm_blocks = take(static_cast<size_t>(L.norm_n > 1024 ? L.norm_n : 1024) * 8);
   L.rowmax = take(static_cast<size_t>(N) * 4);
   L.qerr = take(static_cast<size_t>(L.P) * N * 4);
@@ -127,7 +129,9 @@ static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype) {
   L.diag = take(static_cast<size_t>(d) * 4);
   {
     const SplitPlan sp = plan_split_k(d, N);
-    L.splitk = take(sp.splits > 1 ? static_cast<size_t>(sp.splits) * dd * 4 : 0);
+    int parts = sp.splits > 1 ? sp.splits : 0;
+    if (d == kFsD && parts < 256) parts = 256;  // per-CTA partial dR of the fused d = 128 kernel
+    L.splitk = take(static_cast<size_t>(parts) * dd * 4);
   }
   L.total = off;
   return L;
@@ -395,6 +399,50 @@ static kt_status loss_grad_async(kt_ctx* ctx, const XView& xv, int N, int d, con
   return KT_OK;
 }
 
+// d = 128: loss and gradient in one pass over X (fused_small_kernel), then fixed-order sums over the CTAs.
+static bool use_fused(const kt_ctx* ctx, int d) { return d == kFsD && ctx->cfg.small_d_fused != 0; }
+
+static kt_status fused_loss_grad_async(kt_ctx* ctx, const XView& xv, int N, const WsLayout& L, const float* R,
+                                       float* dR, double* hist_slot, bool rt_current) {
+  const int d = kFsD;
+  if (!rt_current) KT_TRY(cast_rt(ctx, R, d, L));
+  static bool attr_done[16] = {false};
+  if (!attr_done[ctx->device & 15]) {
+    KT_CUDA(cudaFuncSetAttribute(fused_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFsSmem));
+    attr_done[ctx->device & 15] = true;
+  }
+  FusedParams p;
+  memset(&p, 0, sizeof(p));
+  p.terms = forward_terms(ctx, d);
+  p.N = N;
+  p.tiles = (N + 127) / 128;
+  p.kappa_t = ctx->cfg.kappa_target;
+  p.dr_partial = at<float>(ctx, L.splitk);
+  p.loss_partial = at<double>(ctx, L.block_loss);
+  p.deg_partial = at<unsigned int>(ctx, L.block_deg);
+  p.err_word = &ctx->d_blk->sc.err_word;
+  KT_TRY(make_tmap(ctx, &p.tmX, xv.xb, d, N, xv.ldx, 128));
+  KT_TRY(make_tmap(ctx, &p.tmRhi, at<__nv_bfloat16>(ctx, L.rt_hi), d, d, d, 128));
+  KT_TRY(make_tmap(ctx, &p.tmRlo, at<__nv_bfloat16>(ctx, L.rt_lo), d, d, d, 128));
+  int grid = p.tiles < ctx->sm_count ? p.tiles : ctx->sm_count;
+  if (grid > 256) grid = 256;
+  const bool rec = ctx->prof_on && ctx->prof_used < kProfPairs;
+  if (rec) KT_CUDA(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], ctx->stream));
+  fused_small_kernel<<<grid, kFsThreads, kFsSmem, ctx->stream>>>(p);
+  KT_LAUNCH_CHECK();
+  if (rec) {
+    KT_CUDA(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used + 1], ctx->stream));
+    ctx->prof_cat[ctx->prof_used++] = static_cast<unsigned char>(kCatFused);
+  }
+  const long long n = static_cast<long long>(d) * d;
+  k_sum_splits<<<static_cast<unsigned>((n / 4 + 255) / 256), 256, 0, ctx->stream>>>(p.dr_partial, grid, n, n, dR);
+  KT_LAUNCH_CHECK();
+  k_final_sum<<<1, 256, 0, ctx->stream>>>(p.loss_partial, grid, 1.0 / N, &ctx->d_blk->sc.loss, hist_slot,
+                                          p.deg_partial, &ctx->d_blk->sc.deg_rows);
+  KT_LAUNCH_CHECK();
+  return KT_OK;
+}
+
 // ---------------------------------------------------------- orthogonal step
 // E = R^T R - I from the bf16 forms of R^T (rt_hi, rt_lo, which must be current) and, when
 // `with_polish`, R <- R - R E / 2 if max|E| > polish_thresh (needs r_hi; refreshes all three forms).
@@ -528,7 +576,8 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
   KT_TRY(check_ws(ctx, L));
   const int N = static_cast<int>(N64), d = static_cast<int>(d64);
   XView xv;
-  KT_TRY(ingest_x_full(ctx, X, L, &xv));
+  const bool fused = use_fused(ctx, d);
+  if (fused) KT_TRY(ingest_x_forward(ctx, X, L, &xv)); else KT_TRY(ingest_x_full(ctx, X, L, &xv));
   float* dR = at<float>(ctx, L.dr);
   const int ge = ctx->cfg.guard_every < 1 ? 1 : ctx->cfg.guard_every;
   double first = 0.0, last = 0.0;
@@ -545,7 +594,10 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
         memcpy(report->loss_history + (k - kHistMax), ctx->h_blk->hist, sizeof(double) * kHistMax);
     }
     // from the second step on, the previous step left the bf16 forms of R in the workspace
-    KT_TRY(loss_grad_async(ctx, xv, N, d, L, R, dR, &ctx->d_blk->hist[slot], k > 0));
+    if (fused)
+      KT_TRY(fused_loss_grad_async(ctx, xv, N, L, R, dR, &ctx->d_blk->hist[slot], k > 0));
+    else
+      KT_TRY(loss_grad_async(ctx, xv, N, d, L, R, dR, &ctx->d_blk->hist[slot], k > 0));
     const bool run_guard = ((k + 1) % ge == 0) || (k + 1 == steps);
     KT_TRY(orth_step_async(ctx, R, dR, d, lr, L, run_guard, k > 0));
     done = k + 1;
@@ -595,6 +647,7 @@ void kt_default_config(kt_config* cfg) {
   cfg->retract_terms = 2;
   cfg->guard_every = 1;
   cfg->forward_terms = 0;
+  cfg->small_d_fused = 1;
 }
 
 const char* kt_status_string(kt_status s) {
@@ -757,8 +810,13 @@ kt_status kt_loss_grad(kt_ctx* ctx, kt_mat X, const float* R, float* dR, double*
   const WsLayout L = make_layout(N, d, X.dtype);
   KT_TRY(check_ws(ctx, L));
   XView xv;
-  KT_TRY(ingest_x_full(ctx, X, L, &xv));
-  KT_TRY(loss_grad_async(ctx, xv, static_cast<int>(N), static_cast<int>(d), L, R, dR, nullptr, false));
+  if (use_fused(ctx, static_cast<int>(d))) {
+    KT_TRY(ingest_x_forward(ctx, X, L, &xv));
+    KT_TRY(fused_loss_grad_async(ctx, xv, static_cast<int>(N), L, R, dR, nullptr, false));
+  } else {
+    KT_TRY(ingest_x_full(ctx, X, L, &xv));
+    KT_TRY(loss_grad_async(ctx, xv, static_cast<int>(N), static_cast<int>(d), L, R, dR, nullptr, false));
+  }
   if (!loss) return KT_OK;
   KT_TRY(sync_scalars(ctx));
   *loss = ctx->h_blk->sc.loss;
@@ -999,8 +1057,9 @@ kt_status kt_kurtosis_loss_noalloc(kt_mat X, const float* R, double* loss_dev, v
   L.partial = take(static_cast<size_t>(L.P) * N * 16);
   L.coef = take(static_cast<size_t>(N) * 16);
   L.moments = take(static_cast<size_t>(N) * 16);
-  L.block_loss = take(static_cast<size_t>(L.loss_blocks) * 8);
-  L.block_deg = take(static_cast<size_t>(L.loss_blocks) * 4);
+  // at least 256 entries: the fused d = 128 kernel writes one partial per CTA here
+  L.block_loss = take(static_cast<size_t>(L.loss_blocks > 256 ? L.loss_blocks : 256) * 8);
+  L.block_deg = take(static_cast<size_t>(L.loss_blocks > 256 ? L.loss_blocks : 256) * 4);
   L.total = off;
   if (L.total > KT_NOALLOC_SCRATCH_BYTES) return KT_ERR_TOO_LARGE;
 

@@ -34,7 +34,7 @@ class kt_mat(C.Structure):
 class kt_config(C.Structure):
     _fields_ = [("kappa_target", C.c_float), ("cayley_iters", C.c_int32), ("q", C.c_float), ("eps", C.c_float),
                 ("polish_thresh", C.c_float), ("retract_terms", C.c_int32), ("guard_every", C.c_int32),
-                ("forward_terms", C.c_int32), ("reserved", C.c_int32 * 4)]
+                ("forward_terms", C.c_int32), ("small_d_fused", C.c_int32), ("reserved", C.c_int32 * 3)]
 
 
 class kt_fit_report(C.Structure):
@@ -271,7 +271,7 @@ class Context:
     def profile_end(self):
         pr = kt_profile()
         _check(lib().kt_profile_end(self._h, C.byref(pr)), "kt_profile_end")
-        names = ["forward", "backward_a", "backward_b", "square", "quant"]
+        names = ["forward", "backward_a", "backward_b", "square", "quant", "fused"]
         return dict(launches_total=pr.launches_total,
                     gemm={n: dict(launches=pr.gemm_launches[i], ms=pr.gemm_ms[i]) for i, n in enumerate(names)})
 

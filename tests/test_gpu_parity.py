@@ -188,6 +188,40 @@ def test_low_kurtosis_rows_flip_the_sign(ctx):
     assert np.linalg.norm(f64(dR) - dR_ref) / np.linalg.norm(dR_ref) <= 1e-2
 
 
+# ------------------------------------------- d = 128: the single-pass kernel
+@pytest.mark.parametrize("N", [128, 333, 5000, 128 * 300 + 17])
+def test_single_pass_kernel_d128(ctx, N):
+    X = synth.kv_heads(1, N, 128, 30.0, seed=N, device=DEV)
+    X[N // 2] = 0                                        # a degenerate row in the middle
+    R = rand_orth(128, seed=12)
+    loss, dR = ctx.loss_grad(X, R)
+    L_ref, dR_ref = ko.loss_grad(f64(X), f64(R))
+    assert abs(loss - L_ref) <= 1e-3 * abs(L_ref)
+    assert np.linalg.norm(f64(dR) - dR_ref) / np.linalg.norm(dR_ref) <= 1e-2
+    # the general three-GEMM path computes the same thing
+    gen = kurtail.Context(DEV, small_d_fused=0)
+    loss_g, dR_g = gen.loss_grad(X, R)
+    assert abs(loss - loss_g) <= 1e-6 * abs(loss_g)
+    assert np.linalg.norm(f64(dR) - f64(dR_g)) / np.linalg.norm(f64(dR_g)) <= 5e-3
+    gen.close()
+    # fixed-order reductions: a second evaluation is bit-identical
+    loss2, dR2 = ctx.loss_grad(X, R)
+    assert loss2 == loss and torch.equal(dR2, dR)
+
+
+def test_single_pass_kernel_fit_kv_heads(ctx):
+    cfg = synth.config("kv_heads", device=DEV, rows=32 * 1024)
+    X = cfg["X"]
+    R = ctx.init_rotation(128, "identity")
+    L0 = ctx.kurtosis_loss(X, R)
+    rep = ctx.fit(X, R, 20, cfg["lr"], history=True)
+    assert rep["loss_history"][0] == pytest.approx(L0, rel=1e-6)
+    assert rep["loss_history"][-1] < rep["loss_history"][0]
+    assert ctx.orth_error(R) <= 1e-4
+    L_ref = ko.kurtosis_loss(f64(X), f64(R))
+    assert abs(ctx.kurtosis_loss(X, R) - L_ref) <= 1e-3 * abs(L_ref)
+
+
 # ------------------------------------------------------------ the Cayley step
 @pytest.mark.parametrize("d,lr", [(128, 1e-2), (256, 1e-2), (512, 0.5), (1024, 5.0)])
 def test_orth_step_matches_stepwise_oracle(ctx, d, lr):
