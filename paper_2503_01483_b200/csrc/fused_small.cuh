@@ -6,7 +6,8 @@
 //
 //   TMA:  X tile (128 tokens x 128 channels, bf16)                     -> shared memory
 //   MMA1: Y = X R (R^T resident in shared memory, hi [+ lo])           -> tensor memory
-//   epilogue: per row mean, m2, m3, m4 (Eq. 3), kappa, loss term, then
+//   epilogue (two groups of 4 warps that take alternate tiles, one row per thread): mean, m2, m3, m4
+//             (Eq. 3), kappa, loss term, then
 //             G = a c^3 - ab c - am3 as bf16                           -> shared memory
 //   MMA2: dR += X^T G  (both operands read token-major straight from the tiles above,
 //             "MN-major" shared-memory descriptors)                    -> one persistent accumulator
@@ -21,11 +22,14 @@
 namespace kt {
 
 constexpr int kFsD = 128;          // channels = rows of a token tile
-constexpr int kFsThreads = 192;    // warp 0: TMA, warp 1: MMA, warps 2..5: epilogue
-constexpr int kFsXStages = 3;
+constexpr int kFsThreads = 320;    // warp 0: TMA, warp 1: MMA, warps 2..5 and 6..9: two epilogue groups
+constexpr int kFsXStages = 4;
 constexpr int kFsHalf = 128 * 64 * 2;      // bytes of one 128-row x 64-element swizzled block
 constexpr int kFsTile = 2 * kFsHalf;       // one 128 x 128 bf16 tile
-constexpr int kFsSmem = 1024 + 2 * kFsTile /*R^T hi, lo*/ + kFsXStages * kFsTile + 2 * kFsTile /*G*/ + 256;
+constexpr int kFsSmem = 1024 + 2 * kFsTile /*R^T hi, lo*/ + kFsXStages * kFsTile + kFsTile /*G*/ + 256;
+// Rows whose variance is below this are skipped like zero-variance rows: the coefficients of dL/dY are formed in
+// float32 (float64 is an order of magnitude slower on this part) and 1/m2^2 must stay finite.
+constexpr float kFsMinVariance = 1e-18f;
 
 struct FusedParams {
   CUtensorMap tmX;    // X  [N][128] bf16, box 128 rows x 64
@@ -59,7 +63,9 @@ __device__ __forceinline__ uint64_t umma_desc_mnmajor_sw128(uint32_t smem_addr, 
 __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid_constant__ FusedParams p) {
   constexpr uint32_t kIdescK = umma_idesc_bf16_f32(128, 128);                            // both K-major
   constexpr uint32_t kIdescMN = umma_idesc_bf16_f32(128, 128) | (1u << 15) | (1u << 16);  // both MN-major
-  constexpr uint32_t kTmemCols = 512;  // Y accumulators at columns 0 and 128, dR accumulator at 256
+  // tensor memory: Y accumulators at columns 0 (even tiles) and 128 (odd tiles), dR accumulator at 256
+  constexpr uint32_t kTmemCols = 512;
+  constexpr uint32_t kColDr = 256;
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -67,20 +73,22 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
   const uint32_t s_rlo = base + kFsTile;
   const uint32_t s_x = base + 2 * kFsTile;
   const uint32_t s_g = s_x + kFsXStages * kFsTile;
-  const uint32_t bars = s_g + 2 * kFsTile;
+  const uint32_t bars = s_g + kFsTile;
   auto x_full = [&](int s) { return bars + 8u * s; };
   auto x_empty = [&](int s) { return bars + 8u * (kFsXStages + s); };
   auto y_full = [&](int b) { return bars + 8u * (2 * kFsXStages + b); };
   auto y_empty = [&](int b) { return bars + 8u * (2 * kFsXStages + 2 + b); };
+  // one G buffer, but two barriers each way (even / odd tiles): a parity wait then cannot mistake the tile two
+  // back for the one it needs
   auto g_full = [&](int b) { return bars + 8u * (2 * kFsXStages + 4 + b); };
   auto g_empty = [&](int b) { return bars + 8u * (2 * kFsXStages + 6 + b); };
   const uint32_t r_full = bars + 8u * (2 * kFsXStages + 8);
   const uint32_t dr_full = bars + 8u * (2 * kFsXStages + 9);
   uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gbase + (bars - base) + 192);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gbase + (bars - base) + 152);
   volatile uint32_t* abort_flag = tmem_slot + 1;
-  double* sh_loss = reinterpret_cast<double*>(gbase + (bars - base) + 208);          // 4 doubles
-  unsigned int* sh_deg = reinterpret_cast<unsigned int*>(gbase + (bars - base) + 240);  // 4 words
+  double* sh_loss = reinterpret_cast<double*>(gbase + (bars - base) + 160);             // 8 doubles
+  unsigned int* sh_deg = reinterpret_cast<unsigned int*>(gbase + (bars - base) + 224);  // 8 words
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -104,6 +112,8 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
       for (int b = 0; b < 2; ++b) {
         mbar_init(y_full(b), 1);
         mbar_init(y_empty(b), 4);
+      }
+      for (int b = 0; b < 2; ++b) {
         mbar_init(g_full(b), 4);
         mbar_init(g_empty(b), 1);
       }
@@ -147,6 +157,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
         last_parity = (last_parity & ~(1u << s)) | (ph << s);
       }
       if (!ok) {
+        // leave no copy in flight behind: wait (bounded) for every load issued
         for (int s = 0; s < kFsXStages; ++s) {
           if (!(issued & (1u << s))) continue;
           const uint64_t t0 = global_timer_ns();
@@ -160,8 +171,9 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
     // -------------------------------------------------------------- MMA issuer
     if (lane == 0 && my_tiles > 0) {
       bool ok = mbar_wait_bounded(r_full, 0u, abort_flag, 12u);
-      const uint32_t acc_dr = tmem_base + 256u;
-      for (int n = 0; n <= my_tiles && ok; ++n) {
+      const uint32_t acc_dr = tmem_base + kColDr;
+      // MMA1 runs two tiles ahead of MMA2, so the tensor pipe has work while a tile is in the epilogue
+      for (int n = 0; n <= my_tiles + 1 && ok; ++n) {
         if (n < my_tiles) {
           // Y(n) = X(n) R
           const int s = n % kFsXStages;
@@ -189,12 +201,11 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
           }
           tc_commit(y_full(b));
         }
-        if (n >= 1) {
+        if (n >= 2) {
           // dR += X(m)^T G(m): contraction over the tile's 128 tokens, 16 per MMA = two 8-row groups
-          const int m = n - 1;
+          const int m = n - 2;
           const int s = m % kFsXStages;
-          const int b = m & 1;
-          if (!mbar_wait_bounded(g_full(b), (m >> 1) & 1, abort_flag, 15u)) {
+          if (!mbar_wait_bounded(g_full(m & 1), (m >> 1) & 1, abort_flag, 15u)) {
             ok = false;
             break;
           }
@@ -202,103 +213,119 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
             const uint64_t a_desc = umma_desc_mnmajor_sw128(s_x + s * kFsTile + ks * 2048, kFsHalf, 1024);
-            const uint64_t b_desc = umma_desc_mnmajor_sw128(s_g + b * kFsTile + ks * 2048, kFsHalf, 1024);
+            const uint64_t b_desc = umma_desc_mnmajor_sw128(s_g + ks * 2048, kFsHalf, 1024);
             tc_mma_bf16(acc_dr, a_desc, b_desc, kIdescMN, (m > 0 || ks > 0) ? 1u : 0u);
           }
           tc_commit(x_empty(s));   // the X tile is free once these MMAs have read it
-          tc_commit(g_empty(b));
+          tc_commit(g_empty(m & 1));  // and so is the G tile
         }
       }
       if (ok) tc_commit(dr_full);
     }
   } else {
     // ---------------------------------------------------------------- epilogue
-    const int lg = warp & 3;                 // tensor-memory lane group of this warp
-    const int trow = lg * 32 + lane;         // row of the tile = token within the tile (and dR row at the end)
+    // Group 0 (warps 2..5) takes this CTA's even tiles, group 1 (warps 6..9) the odd ones: two tiles are in
+    // flight per scheduler, so the latency of one tile's reduction hides behind the other's arithmetic.
+    const int lg = warp & 3;            // tensor-memory lane group of this warp
+    const int grp = (warp - 2) >> 2;    // = tile parity = Y accumulator = G buffer
+    const int trow = lg * 32 + lane;    // token within the tile (and row of dR at the end)
+    const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(lg * 32) << 16);
+    const float kscale = static_cast<float>(4.0 / (static_cast<double>(p.N) * 128.0));
     double loss_acc = 0.0;
     unsigned int deg_acc = 0;
     bool ok = true;
-    const float inv_nd = 1.0f;  // (kept in double below)
-    (void)inv_nd;
-    for (int n = 0; n < my_tiles && ok; ++n) {
-      const int b = n & 1;
-      const bool got = mbar_wait_bounded(y_full(b), (n >> 1) & 1, abort_flag, 16u);
+    for (int n = grp; n < my_tiles && ok; n += 2) {
+      const uint32_t par = (n >> 1) & 1;
+      const bool got = mbar_wait_bounded(y_full(grp), par, abort_flag, 16u);
       if (!__all_sync(0xffffffffu, got)) {
         ok = false;
         break;
       }
       tc_fence_after_sync();
-      const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + static_cast<uint32_t>(b * 128);
       uint32_t v[4][32];
-      tmem_ld_32x32(t_addr, v[0]);
-      tmem_ld_32x32(t_addr + 32, v[1]);
-      tmem_ld_32x32(t_addr + 64, v[2]);
-      tmem_ld_32x32(t_addr + 96, v[3]);
+      tmem_ld_32x32(lane_addr + static_cast<uint32_t>(grp * 128), v[0]);
+      tmem_ld_32x32(lane_addr + static_cast<uint32_t>(grp * 128 + 32), v[1]);
+      tmem_ld_32x32(lane_addr + static_cast<uint32_t>(grp * 128 + 64), v[2]);
+      tmem_ld_32x32(lane_addr + static_cast<uint32_t>(grp * 128 + 96), v[3]);
       tc_wait_ld();
       // the accumulator can be refilled while this tile is being reduced
       tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) mbar_arrive(y_empty(b));
+      if (lane == 0) mbar_arrive(y_empty(grp));
 
-      // Eq. 3 on the row: mean, then central power sums about it
-      float s1 = 0.f;
+      // Eq. 3 on the row: mean, then central power sums about it.  Two-wide arithmetic (packed f32x2
+      // add/mul/fma): this epilogue is bound by instruction issue and latency, not by memory.
+      float mean;
+      {
+        float2 a0 = make_float2(0.f, 0.f), a1 = a0, a2 = a0, a3 = a0;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        for (int c = 0; c < 4; ++c) {
 #pragma unroll
-        for (int j = 0; j < 32; j += 4) {
-          a0 += __uint_as_float(v[c][j]);
-          a1 += __uint_as_float(v[c][j + 1]);
-          a2 += __uint_as_float(v[c][j + 2]);
-          a3 += __uint_as_float(v[c][j + 3]);
+          for (int j = 0; j < 32; j += 8) {
+            a0 = __fadd2_rn(a0, make_float2(__uint_as_float(v[c][j]), __uint_as_float(v[c][j + 1])));
+            a1 = __fadd2_rn(a1, make_float2(__uint_as_float(v[c][j + 2]), __uint_as_float(v[c][j + 3])));
+            a2 = __fadd2_rn(a2, make_float2(__uint_as_float(v[c][j + 4]), __uint_as_float(v[c][j + 5])));
+            a3 = __fadd2_rn(a3, make_float2(__uint_as_float(v[c][j + 6]), __uint_as_float(v[c][j + 7])));
+          }
         }
-        s1 += (a0 + a1) + (a2 + a3);
+        a0 = __fadd2_rn(__fadd2_rn(a0, a1), __fadd2_rn(a2, a3));
+        mean = (a0.x + a0.y) * (1.0f / 128.0f);
       }
-      const float mean = s1 * (1.0f / 128.0f);
-      float s2 = 0.f, s3 = 0.f, s4 = 0.f;
+      float s2, s3, s4;
+      {
+        const float2 nm = make_float2(-mean, -mean);
+        float2 b2 = make_float2(0.f, 0.f), b3 = b2, b4 = b2, e2 = b2, e3 = b2, e4 = b2;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        float b2 = 0.f, b3 = 0.f, b4 = 0.f;
+        for (int c = 0; c < 4; ++c) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float cc = __uint_as_float(v[c][j]) - mean;
-          const float c2 = cc * cc;
-          b2 += c2;
-          b3 = fmaf(c2, cc, b3);
-          b4 = fmaf(c2, c2, b4);
+          for (int j = 0; j < 32; j += 4) {
+            const float2 c0 = __fadd2_rn(make_float2(__uint_as_float(v[c][j]), __uint_as_float(v[c][j + 1])), nm);
+            const float2 c1 = __fadd2_rn(make_float2(__uint_as_float(v[c][j + 2]), __uint_as_float(v[c][j + 3])), nm);
+            const float2 q0 = __fmul2_rn(c0, c0), q1 = __fmul2_rn(c1, c1);
+            b2 = __fadd2_rn(b2, q0);
+            e2 = __fadd2_rn(e2, q1);
+            b3 = __ffma2_rn(q0, c0, b3);
+            e3 = __ffma2_rn(q1, c1, e3);
+            b4 = __ffma2_rn(q0, q0, b4);
+            e4 = __ffma2_rn(q1, q1, e4);
+          }
         }
-        s2 += b2;
-        s3 += b3;
-        s4 += b4;
+        b2 = __fadd2_rn(b2, e2);
+        b3 = __fadd2_rn(b3, e3);
+        b4 = __fadd2_rn(b4, e4);
+        s2 = b2.x + b2.y;
+        s3 = b3.x + b3.y;
+        s4 = b4.x + b4.y;
       }
-      // kappa, loss term and the coefficients of dL/dY (same rules as the general path)
+      // kappa, the loss term and the coefficients of dL/dY (same rules as the general path, in float32)
       const int row = (static_cast<int>(blockIdx.x) + n * static_cast<int>(gridDim.x)) * 128 + trow;
-      const double m2 = static_cast<double>(s2) / 128.0, m3 = static_cast<double>(s3) / 128.0,
-                   m4 = static_cast<double>(s4) / 128.0;
-      const double mu = static_cast<double>(mean);
-      const double ms = m2 + mu * mu;
-      const bool degenerate = (ms == 0.0) || (m2 <= 1e-6 * ms);
+      const float m2 = s2 * (1.0f / 128.0f), m3 = s3 * (1.0f / 128.0f), m4 = s4 * (1.0f / 128.0f);
+      const float ms = fmaf(mean, mean, m2);
+      const bool degenerate = (ms == 0.f) || (m2 <= 1e-6f * ms) || (m2 < kFsMinVariance);
       float ca = 0.f, cab = 0.f, cam3 = 0.f;
       if (!degenerate) {
-        const double kappa = m4 / (m2 * m2);
-        const double diff = kappa - static_cast<double>(p.kappa_t);
-        const double sgn = (diff > 0.0) ? 1.0 : ((diff < 0.0) ? -1.0 : 0.0);
-        const double a = sgn * 4.0 / (static_cast<double>(p.N) * 128.0 * m2 * m2);
-        ca = static_cast<float>(a);
-        cab = static_cast<float>(a * m4 / m2);
-        cam3 = static_cast<float>(a * m3);
-        if (row < p.N) loss_acc += fabs(diff);
+        const float r = __frcp_rn(m2);
+        const float kappa = (m4 * r) * r;
+        const float diff = kappa - p.kappa_t;
+        const float sgn = (diff > 0.f) ? 1.0f : ((diff < 0.f) ? -1.0f : 0.0f);
+        ca = ((sgn * kscale) * r) * r;
+        cab = ca * (m4 * r);
+        cam3 = ca * m3;
+        if (row < p.N) loss_acc += static_cast<double>(fabsf(diff));
       } else if (row < p.N) {
         ++deg_acc;
       }
+      const float2 nmean2 = make_float2(-mean, -mean), ca2 = make_float2(ca, ca), ncab2 = make_float2(-cab, -cab),
+                   ncam32 = make_float2(-cam3, -cam3);
 
       // G = a c^3 - ab c - am3 as bf16, token-major, into the swizzled tile MMA2 reads
-      const bool free_g = mbar_wait_bounded(g_empty(b), ((n >> 1) & 1) ^ 1u, abort_flag, 17u);
+      // the single G tile is free once MMA2 of the previous tile (the other group's) has read it
+      const bool free_g = (n == 0) || mbar_wait_bounded(g_empty((n - 1) & 1), ((n - 1) >> 1) & 1, abort_flag, 17u);
       if (!__all_sync(0xffffffffu, free_g)) {
         ok = false;
         break;
       }
-      const uint32_t g_row = s_g + b * kFsTile + static_cast<uint32_t>(trow) * 128u;
+      const uint32_t g_row = s_g + static_cast<uint32_t>(trow) * 128u;
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
 #pragma unroll
@@ -306,14 +333,13 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
           uint32_t pk[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            const float c0 = __uint_as_float(v[c][j8 * 8 + 2 * e]) - mean;
-            const float c1 = __uint_as_float(v[c][j8 * 8 + 2 * e + 1]) - mean;
-            const float g0 = fmaf(c0, fmaf(ca * c0, c0, -cab), -cam3);
-            const float g1 = fmaf(c1, fmaf(ca * c1, c1, -cab), -cam3);
-            __nv_bfloat162 h = __floats2bfloat162_rn(g0, g1);
+            const float2 cc = __fadd2_rn(make_float2(__uint_as_float(v[c][j8 * 8 + 2 * e]),
+                                                     __uint_as_float(v[c][j8 * 8 + 2 * e + 1])), nmean2);
+            const float2 g = __ffma2_rn(cc, __ffma2_rn(__fmul2_rn(ca2, cc), cc, ncab2), ncam32);
+            __nv_bfloat162 h = __floats2bfloat162_rn(g.x, g.y);
             pk[e] = *reinterpret_cast<uint32_t*>(&h);
           }
-          const int chunk = c * 4 + j8;                 // 16-byte chunk 0..15 of the 256-byte row
+          const int chunk = c * 4 + j8;  // 16-byte chunk 0..15 of the 256-byte row
           const uint32_t addr = g_row + static_cast<uint32_t>(chunk >> 3) * kFsHalf +
                                 (static_cast<uint32_t>((chunk & 7) ^ (trow & 7)) << 4);
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]),
@@ -323,10 +349,10 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
       }
       fence_proxy_async_smem();  // make the generic-proxy stores visible to the tensor core
       __syncwarp();
-      if (lane == 0) mbar_arrive(g_full(b));
+      if (lane == 0) mbar_arrive(g_full(n & 1));
     }
 
-    // partial loss of this CTA (fixed order: lanes by shuffle tree, then warps 2,3,4,5 -> lane groups 2,3,0,1)
+    // partial loss of this CTA (fixed order: lanes by shuffle tree, then the eight warps)
     {
       double l = loss_acc;
       unsigned int dg = deg_acc;
@@ -336,21 +362,20 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
         dg += __shfl_down_sync(0xffffffffu, dg, o);
       }
       if (lane == 0) {
-        sh_loss[lg] = l;
-        sh_deg[lg] = dg;
+        sh_loss[grp * 4 + lg] = l;
+        sh_deg[grp * 4 + lg] = dg;
       }
     }
-    // partial dR of this CTA
+    // partial dR of this CTA: each warp writes its 32 rows x 64 columns (group 0 the left half)
+    float* dst = p.dr_partial + (static_cast<long long>(blockIdx.x) * 128 + trow) * 128 + grp * 64;
     if (my_tiles > 0 && ok) {
       const bool got = mbar_wait_bounded(dr_full, 0u, abort_flag, 18u);
       if (__all_sync(0xffffffffu, got)) {
         tc_fence_after_sync();
-        const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + 256u;
-        float* dst = p.dr_partial + (static_cast<long long>(blockIdx.x) * 128 + trow) * 128;
         uint32_t w[32];
 #pragma unroll 1
-        for (int c0 = 0; c0 < 128; c0 += 32) {
-          tmem_ld_32x32(t_addr + c0, w);
+        for (int c0 = 0; c0 < 64; c0 += 32) {
+          tmem_ld_32x32(lane_addr + kColDr + static_cast<uint32_t>(grp * 64 + c0), w);
           tc_wait_ld();
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
@@ -361,8 +386,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
         }
       }
     } else if (my_tiles == 0) {
-      float* dst = p.dr_partial + (static_cast<long long>(blockIdx.x) * 128 + trow) * 128;
-      for (int j = 0; j < 32; ++j) reinterpret_cast<float4*>(dst)[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int j = 0; j < 16; ++j) reinterpret_cast<float4*>(dst)[j] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
   }
 
@@ -375,8 +399,14 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
     tmem_dealloc(tmem_base, kTmemCols);
   }
   if (threadIdx.x == 0) {
-    p.loss_partial[blockIdx.x] = (sh_loss[0] + sh_loss[1]) + (sh_loss[2] + sh_loss[3]);
-    p.deg_partial[blockIdx.x] = sh_deg[0] + sh_deg[1] + sh_deg[2] + sh_deg[3];
+    double l = 0.0;
+    unsigned int dg = 0;
+    for (int i = 0; i < 8; ++i) {
+      l += sh_loss[i];
+      dg += sh_deg[i];
+    }
+    p.loss_partial[blockIdx.x] = l;
+    p.deg_partial[blockIdx.x] = dg;
     if (*abort_flag != 0 && p.err_word != nullptr) atomicMax(p.err_word, *abort_flag);
   }
 }
