@@ -87,7 +87,11 @@ typedef struct {
   int32_t small_d_fused;/* [1]   d == 128: kt_loss_grad / kt_fit use the single-pass
                            kernel (X read once per evaluation); 0 = the general
                            three-GEMM path                                      */
-  int32_t reserved[3];
+  int32_t small_d_orth; /* [1]   d <= 512: kt_orth_step runs as one cooperative
+                           launch in float32 on the CUDA cores (128 CTAs; the
+                           device must have at least 128 SMs free) instead of
+                           about twenty tensor-core launches; 0 = general path  */
+  int32_t reserved[2];
 } kt_config;
 
 /* Filled by kt_fit / kt_fit_layers (host memory). */

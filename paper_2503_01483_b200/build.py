@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libkurtail.so")
 SOURCES = ["kt_api.cu"]
-HEADERS = ["sm100_prims.cuh", "gemm_sm100.cuh", "elementwise.cuh", "fused_small.cuh"]
+HEADERS = ["sm100_prims.cuh", "gemm_sm100.cuh", "elementwise.cuh", "fused_small.cuh", "small_orth.cuh"]
 
 
 def _nvcc():

@@ -14,6 +14,7 @@
 #include "elementwise.cuh"
 #include "fused_small.cuh"
 #include "gemm_sm100.cuh"
+#include "small_orth.cuh"
 
 namespace kt {
 
@@ -83,6 +84,7 @@ struct WsLayout {
   size_t colpart;       // [d/32][d] float: column sums of squares of R by row slab
   size_t diag;          // [d] float: exact diagonal of R^T R - I
   size_t splitk;        // [splits][d][d] float: partial dR of the split-K backward-B (when splits > 1)
+  size_t small;         // d <= 512: scratch of the one-launch orthogonal step (5 d x d floats + per-CTA partials)
   size_t total;
   long long ldt;
   int P, bn, loss_blocks, norm_n;
@@ -133,6 +135,7 @@ static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype) {
     if (d == kFsD && parts < 256) parts = 256;  // per-CTA partial dR of the fused d = 128 kernel
     L.splitk = take(static_cast<size_t>(parts) * dd * 4);
   }
+  L.small = take(d <= 512 ? 5 * dd * 4 + 4096 : 0);
   L.total = off;
   return L;
 }
@@ -489,10 +492,54 @@ static kt_status guard(kt_ctx* ctx, const float* R_in, float* R, int d, const Ws
   return KT_OK;
 }
 
+// d <= 512: the whole step and its guard in one cooperative launch (float32 on the CUDA cores).
+static bool use_small_orth(const kt_ctx* ctx, int d) { return d <= 512 && ctx->cfg.small_d_orth != 0; }
+
+static kt_status small_orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, float lr, const WsLayout& L,
+                                       bool run_guard) {
+  const kt_config& c = ctx->cfg;
+  SmallOrthParams p;
+  memset(&p, 0, sizeof(p));
+  const size_t dd = static_cast<size_t>(d) * d;
+  float* sm = at<float>(ctx, L.small);
+  p.R = R;
+  p.dR = dR;
+  p.d = d;
+  p.iters = c.cayley_iters < 0 ? 0 : c.cayley_iters;
+  p.run_guard = run_guard ? 1 : 0;
+  p.lr = lr;
+  p.q = c.q;
+  p.eps = c.eps;
+  p.thresh = c.polish_thresh;
+  p.Rt = sm;
+  p.A = sm + dd;
+  p.W = sm + 2 * dd;
+  p.P0 = sm + 3 * dd;
+  p.P1 = sm + 4 * dd;
+  p.norm_part = reinterpret_cast<double*>(sm + 5 * dd);
+  p.max_part = reinterpret_cast<float*>(p.norm_part + kSoGrid);
+  p.sc = &ctx->d_blk->sc;
+  p.r_hi = at<__nv_bfloat16>(ctx, L.r_hi);
+  p.rt_hi = at<__nv_bfloat16>(ctx, L.rt_hi);
+  p.rt_lo = at<__nv_bfloat16>(ctx, L.rt_lo);
+  void* args[] = {&p};
+  const void* fn = nullptr;
+  switch (d / 128) {
+    case 1: fn = reinterpret_cast<const void*>(small_orth_kernel<1>); break;
+    case 2: fn = reinterpret_cast<const void*>(small_orth_kernel<2>); break;
+    case 3: fn = reinterpret_cast<const void*>(small_orth_kernel<3>); break;
+    default: fn = reinterpret_cast<const void*>(small_orth_kernel<4>); break;
+  }
+  KT_CUDA(cudaLaunchCooperativeKernel(fn, dim3(kSoGrid), dim3(d), args, 0, ctx->stream));
+  KT_LAUNCH_CHECK();
+  return KT_OK;
+}
+
 // One Cayley-SGD step.  `forms_current`: r_hi / rt_hi / rt_lo already hold the bf16 forms of R (true from the
 // second step of kt_fit on: the previous step left them).  On return they hold the forms of the new R.
 static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, float lr, const WsLayout& L,
                                  bool run_guard, bool forms_current) {
+  if (use_small_orth(ctx, d)) return small_orth_step_async(ctx, R, dR, d, lr, L, run_guard);
   const kt_config& c = ctx->cfg;
   Scalars* sc = &ctx->d_blk->sc;
   const uint64_t ld = static_cast<uint64_t>(d);
@@ -648,6 +695,7 @@ void kt_default_config(kt_config* cfg) {
   cfg->guard_every = 1;
   cfg->forward_terms = 0;
   cfg->small_d_fused = 1;
+  cfg->small_d_orth = 1;
 }
 
 const char* kt_status_string(kt_status s) {

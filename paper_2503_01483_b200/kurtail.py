@@ -34,7 +34,7 @@ class kt_mat(C.Structure):
 class kt_config(C.Structure):
     _fields_ = [("kappa_target", C.c_float), ("cayley_iters", C.c_int32), ("q", C.c_float), ("eps", C.c_float),
                 ("polish_thresh", C.c_float), ("retract_terms", C.c_int32), ("guard_every", C.c_int32),
-                ("forward_terms", C.c_int32), ("small_d_fused", C.c_int32), ("reserved", C.c_int32 * 3)]
+                ("forward_terms", C.c_int32), ("small_d_fused", C.c_int32), ("small_d_orth", C.c_int32), ("reserved", C.c_int32 * 2)]
 
 
 class kt_fit_report(C.Structure):
