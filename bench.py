@@ -205,21 +205,16 @@ def main():
     import torch
     from paper_2503_01483_b200 import build, kurtail, synth
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    from paper_2503_01483_b200 import dist_util
+    rank, local_rank, world = dist_util.env_rank()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
     torch.cuda.set_device(local_rank)
     dev = "cuda:%d" % local_rank
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device(dev))
+    dist = dist_util.init("nccl", dev)
     if rank == 0:
         build.build()
-    if dist is not None:
-        dist.barrier()
+    dist_util.barrier(dist)
 
     # each rank fits its own layer buffer (layers are independent: no data-path collective)
     kw = dict(device=dev, rows=N_full if wl_cfg != "kv_heads" else N_full)
@@ -250,8 +245,7 @@ def main():
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    if dist is not None:
-        dist.barrier()
+    dist_util.barrier(dist)
     torch.cuda.synchronize()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ctx.profile_begin()
@@ -263,11 +257,8 @@ def main():
     t_wall1 = time.time()
     prof = ctx.profile_end()
     ms = ev0.elapsed_time(ev1)
-    if dist is not None:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-        dist.barrier()
+    ms = dist_util.max_over_ranks(dist, ms, dev)
+    dist_util.barrier(dist)
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
     ms_per_step = ms / args.steps
     value = world * N * args.steps / (ms * 1e-3)
@@ -282,16 +273,12 @@ def main():
         ctx.fit_host(Xh, stage, Rh, Rdev, 1, lr)      # warm the copy path
         Rh.copy_(torch.from_numpy(R0_host))
         torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
+        dist_util.barrier(dist)
         t0 = time.perf_counter()
         ctx.fit_host(Xh, stage, Rh, Rdev, args.steps, lr)
         torch.cuda.synchronize()
         t_e2e = time.perf_counter() - t0
-        if dist is not None:
-            t = torch.tensor([t_e2e], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            t_e2e = float(t.item())
+        t_e2e = dist_util.max_over_ranks(dist, t_e2e, dev)
         h2d = Xh.numel() * Xh.element_size() + Rh.numel() * 4
         d2h = Rh.numel() * 4
         e2e = {"value": world * N * args.steps / t_e2e, "unit": "tokens/s",
@@ -301,8 +288,7 @@ def main():
         del Xh, stage
 
     if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
+        dist_util.finalize(dist)
         return
 
     # ---- roofline of the dominant kernel: the three N x d x d tensor-core GEMMs of a step
@@ -342,8 +328,7 @@ def main():
         sample = X[:n_s].float().cpu().numpy()
         out["cpu_baseline"] = cpu_baseline(sample, R0_host, N, lr)
     print(json.dumps(out))
-    if dist is not None:
-        dist.destroy_process_group()
+    dist_util.finalize(dist)
 
 
 if __name__ == "__main__":
