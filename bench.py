@@ -184,7 +184,7 @@ def run_reference(args, wl_name, d, N_full):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2_7b_attn", choices=sorted(WORKLOADS))
@@ -320,6 +320,7 @@ def main():
                    "parallelism": "one independent layer per GPU" if world > 1 else "single GPU"},
         "algorithmic_tflops": (4.0 * N * d * d) * world / (ms_per_step * 1e-3) / 1e12,
         "loss_first": rep["loss_first"], "loss_last": rep["loss_last"], "orth_err": rep["orth_err"],
+        "alpha_last": rep["alpha_last"], "w_norm_last": rep["w_norm_last"],
         "gpu_launches": prof["launches_total"], "clocks": clocks, "roofline": roofline, "e2e": e2e,
     }
 

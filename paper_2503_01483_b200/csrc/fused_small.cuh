@@ -26,7 +26,12 @@ constexpr int kFsThreads = 320;    // warp 0: TMA, warp 1: MMA, warps 2..5 and 6
 constexpr int kFsXStages = 4;
 constexpr int kFsHalf = 128 * 64 * 2;      // bytes of one 128-row x 64-element swizzled block
 constexpr int kFsTile = 2 * kFsHalf;       // one 128 x 128 bf16 tile
-constexpr int kFsSmem = 1024 + 2 * kFsTile /*R^T hi, lo*/ + kFsXStages * kFsTile + kFsTile /*G*/ + 256;
+// TERMS = 1: R^T hi only, which leaves room for a second G tile; TERMS = 2: R^T hi + lo and one G tile.
+template <int TERMS>
+struct FusedCfg {
+  static constexpr int kGBufs = (TERMS == 1) ? 2 : 1;
+  static constexpr int kSmem = 1024 + TERMS * kFsTile /*R^T*/ + kFsXStages * kFsTile + kGBufs * kFsTile /*G*/ + 256;
+};
 // Rows whose variance is below this are skipped like zero-variance rows: the coefficients of dL/dY are formed in
 // float32 (float64 is an order of magnitude slower on this part) and 1/m2^2 must stay finite.
 constexpr float kFsMinVariance = 1e-18f;
@@ -35,7 +40,6 @@ struct FusedParams {
   CUtensorMap tmX;    // X  [N][128] bf16, box 128 rows x 64
   CUtensorMap tmRhi;  // R^T hi [128][128] bf16, box 128 x 64
   CUtensorMap tmRlo;  // R^T lo
-  int terms;          // 1: R^T hi only; 2: hi + lo
   int N;
   int tiles;          // ceil(N / 128)
   float kappa_t;
@@ -60,7 +64,9 @@ __device__ __forceinline__ uint64_t umma_desc_mnmajor_sw128(uint32_t smem_addr, 
   return d;
 }
 
+template <int TERMS>
 __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid_constant__ FusedParams p) {
+  constexpr int kGBufs = FusedCfg<TERMS>::kGBufs;
   constexpr uint32_t kIdescK = umma_idesc_bf16_f32(128, 128);                            // both K-major
   constexpr uint32_t kIdescMN = umma_idesc_bf16_f32(128, 128) | (1u << 15) | (1u << 16);  // both MN-major
   // tensor memory: Y accumulators at columns 0 (even tiles) and 128 (odd tiles), dR accumulator at 256
@@ -70,16 +76,16 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t s_rhi = base;
-  const uint32_t s_rlo = base + kFsTile;
-  const uint32_t s_x = base + 2 * kFsTile;
+  const uint32_t s_rlo = base + kFsTile;  // only when TERMS == 2
+  const uint32_t s_x = base + TERMS * kFsTile;
   const uint32_t s_g = s_x + kFsXStages * kFsTile;
-  const uint32_t bars = s_g + kFsTile;
+  const uint32_t bars = s_g + kGBufs * kFsTile;
   auto x_full = [&](int s) { return bars + 8u * s; };
   auto x_empty = [&](int s) { return bars + 8u * (kFsXStages + s); };
   auto y_full = [&](int b) { return bars + 8u * (2 * kFsXStages + b); };
   auto y_empty = [&](int b) { return bars + 8u * (2 * kFsXStages + 2 + b); };
-  // one G buffer, but two barriers each way (even / odd tiles): a parity wait then cannot mistake the tile two
-  // back for the one it needs
+  // one or two G tiles, and in either case two barriers each way (even / odd tiles): with one tile a parity
+  // wait then cannot mistake the tile two back for the one it needs
   auto g_full = [&](int b) { return bars + 8u * (2 * kFsXStages + 4 + b); };
   auto g_empty = [&](int b) { return bars + 8u * (2 * kFsXStages + 6 + b); };
   const uint32_t r_full = bars + 8u * (2 * kFsXStages + 8);
@@ -133,10 +139,10 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0 && my_tiles > 0) {
-      mbar_arrive_expect_tx(r_full, static_cast<uint32_t>(p.terms) * kFsTile);
+      mbar_arrive_expect_tx(r_full, static_cast<uint32_t>(TERMS) * kFsTile);
       tma_load_2d(s_rhi, &p.tmRhi, 0, 0, r_full);
       tma_load_2d(s_rhi + kFsHalf, &p.tmRhi, 64, 0, r_full);
-      if (p.terms == 2) {
+      if (TERMS == 2) {
         tma_load_2d(s_rlo, &p.tmRlo, 0, 0, r_full);
         tma_load_2d(s_rlo + kFsHalf, &p.tmRlo, 64, 0, r_full);
       }
@@ -186,7 +192,8 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
           tc_fence_after_sync();
           const uint32_t acc_y = tmem_base + static_cast<uint32_t>(b * 128);
           uint32_t first = 1;
-          for (int q = 0; q < p.terms; ++q) {
+#pragma unroll
+          for (int q = 0; q < TERMS; ++q) {
             const uint32_t rb = (q == 0) ? s_rhi : s_rlo;
 #pragma unroll
             for (int kb = 0; kb < 2; ++kb) {
@@ -213,7 +220,8 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
             const uint64_t a_desc = umma_desc_mnmajor_sw128(s_x + s * kFsTile + ks * 2048, kFsHalf, 1024);
-            const uint64_t b_desc = umma_desc_mnmajor_sw128(s_g + ks * 2048, kFsHalf, 1024);
+            const uint64_t b_desc =
+                umma_desc_mnmajor_sw128(s_g + (kGBufs == 2 ? (m & 1) * kFsTile : 0) + ks * 2048, kFsHalf, 1024);
             tc_mma_bf16(acc_dr, a_desc, b_desc, kIdescMN, (m > 0 || ks > 0) ? 1u : 0u);
           }
           tc_commit(x_empty(s));   // the X tile is free once these MMAs have read it
@@ -319,13 +327,15 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
                    ncam32 = make_float2(-cam3, -cam3);
 
       // G = a c^3 - ab c - am3 as bf16, token-major, into the swizzled tile MMA2 reads
-      // the single G tile is free once MMA2 of the previous tile (the other group's) has read it
-      const bool free_g = (n == 0) || mbar_wait_bounded(g_empty((n - 1) & 1), ((n - 1) >> 1) & 1, abort_flag, 17u);
+      // with one G tile it is free once MMA2 of the previous tile (the other group's) has read it; with two,
+      // once MMA2 of this group's previous tile has
+      const int gw = (kGBufs == 2) ? n - 2 : n - 1;
+      const bool free_g = (gw < 0) || mbar_wait_bounded(g_empty(gw & 1), (gw >> 1) & 1, abort_flag, 17u);
       if (!__all_sync(0xffffffffu, free_g)) {
         ok = false;
         break;
       }
-      const uint32_t g_row = s_g + static_cast<uint32_t>(trow) * 128u;
+      const uint32_t g_row = s_g + (kGBufs == 2 ? static_cast<uint32_t>(grp) * kFsTile : 0u) + static_cast<uint32_t>(trow) * 128u;
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
 #pragma unroll

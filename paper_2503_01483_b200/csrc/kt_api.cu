@@ -322,16 +322,18 @@ static kt_status ingest_x_full(kt_ctx* ctx, const kt_mat& X, const WsLayout& L, 
 
 // ------------------------------------------------------------ forward pieces
 // How many bf16 terms of R the token GEMMs use: 1 (R rounded to bf16) or 2 (hi + lo, ~16 significant bits).
-static int forward_terms(const kt_ctx* ctx, int d) {
+// Automatic choice: 2 for small problems (d <= 512 and N d <= 2^24), where the doubled MMA work costs nothing.
+static int forward_terms(const kt_ctx* ctx, int d, long long N) {
   const int t = ctx->cfg.forward_terms;
   if (t == 1 || t == 2) return t;
-  return d <= 512 ? 2 : 1;
+  return (d <= 512 && N * d <= (1ll << 24)) ? 2 : 1;
 }
 
-static kt_status cast_rt(kt_ctx* ctx, const float* R, int d, const WsLayout& L) {
+static kt_status cast_rt(kt_ctx* ctx, const float* R, int d, long long N, const WsLayout& L) {
   dim3 grid(d / 32, d / 32), block(32, 8);
   k_split_bf16<true><<<grid, block, 0, ctx->stream>>>(
-      R, d, at<__nv_bfloat16>(ctx, L.rt_hi), forward_terms(ctx, d) == 2 ? at<__nv_bfloat16>(ctx, L.rt_lo) : nullptr, d);
+      R, d, at<__nv_bfloat16>(ctx, L.rt_hi), forward_terms(ctx, d, N) == 2 ? at<__nv_bfloat16>(ctx, L.rt_lo) : nullptr,
+      d);
   KT_LAUNCH_CHECK();
   return KT_OK;
 }
@@ -341,9 +343,9 @@ struct FwdOperands {
   Operand A[2], B[2];
   int terms;
 };
-static FwdOperands fwd_operands(kt_ctx* ctx, const XView& xv, int d, const WsLayout& L) {
+static FwdOperands fwd_operands(kt_ctx* ctx, const XView& xv, int d, long long N, const WsLayout& L) {
   FwdOperands f;
-  f.terms = forward_terms(ctx, d);
+  f.terms = forward_terms(ctx, d, N);
   f.A[0] = f.A[1] = Operand{xv.xb, static_cast<uint64_t>(xv.ldx)};
   f.B[0] = Operand{at<__nv_bfloat16>(ctx, L.rt_hi), static_cast<uint64_t>(d)};
   f.B[1] = Operand{at<__nv_bfloat16>(ctx, L.rt_lo), static_cast<uint64_t>(d)};
@@ -354,7 +356,7 @@ static FwdOperands fwd_operands(kt_ctx* ctx, const XView& xv, int d, const WsLay
 static kt_status forward_loss(kt_ctx* ctx, const XView& xv, int N, int d, const WsLayout& L, double* hist_slot) {
   GemmParams p = blank_params();
   p.partial = at<float4>(ctx, L.partial);
-  const FwdOperands f = fwd_operands(ctx, xv, d, L);
+  const FwdOperands f = fwd_operands(ctx, xv, d, N, L);
   KT_TRY(run_gemm<kMoments>(ctx, N, d, d, f.terms, f.A, f.B, p, kCatForward));
   k_moments_finalize<<<L.loss_blocks, 256, 0, ctx->stream>>>(at<float4>(ctx, L.partial), L.P, N, d, L.bn,
                                                             ctx->cfg.kappa_target, at<float4>(ctx, L.moments),
@@ -373,7 +375,7 @@ static kt_status backward(kt_ctx* ctx, const XView& xv, int N, int d, const WsLa
   p.coef = at<float4>(ctx, L.coef);
   p.gt = at<__nv_bfloat16>(ctx, L.gt);
   p.ldg = L.ldt;
-  const FwdOperands f = fwd_operands(ctx, xv, d, L);
+  const FwdOperands f = fwd_operands(ctx, xv, d, N, L);
   KT_TRY(run_gemm<kGrad>(ctx, N, d, d, f.terms, f.A, f.B, p, kCatBackwardA));
   GemmParams p2 = blank_params();
   const SplitPlan sp = plan_split_k(d, N);
@@ -396,7 +398,7 @@ static kt_status backward(kt_ctx* ctx, const XView& xv, int N, int d, const WsLa
 
 static kt_status loss_grad_async(kt_ctx* ctx, const XView& xv, int N, int d, const WsLayout& L, const float* R,
                                  float* dR, double* hist_slot, bool rt_current) {
-  if (!rt_current) KT_TRY(cast_rt(ctx, R, d, L));
+  if (!rt_current) KT_TRY(cast_rt(ctx, R, d, N, L));
   KT_TRY(forward_loss(ctx, xv, N, d, L, hist_slot));
   KT_TRY(backward(ctx, xv, N, d, L, dR));
   return KT_OK;
@@ -408,15 +410,18 @@ static bool use_fused(const kt_ctx* ctx, int d) { return d == kFsD && ctx->cfg.s
 static kt_status fused_loss_grad_async(kt_ctx* ctx, const XView& xv, int N, const WsLayout& L, const float* R,
                                        float* dR, double* hist_slot, bool rt_current) {
   const int d = kFsD;
-  if (!rt_current) KT_TRY(cast_rt(ctx, R, d, L));
+  if (!rt_current) KT_TRY(cast_rt(ctx, R, d, N, L));
   static bool attr_done[16] = {false};
   if (!attr_done[ctx->device & 15]) {
-    KT_CUDA(cudaFuncSetAttribute(fused_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFsSmem));
+    KT_CUDA(cudaFuncSetAttribute(fused_small_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 FusedCfg<1>::kSmem));
+    KT_CUDA(cudaFuncSetAttribute(fused_small_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 FusedCfg<2>::kSmem));
     attr_done[ctx->device & 15] = true;
   }
   FusedParams p;
   memset(&p, 0, sizeof(p));
-  p.terms = forward_terms(ctx, d);
+  const int terms = forward_terms(ctx, d, N);
   p.N = N;
   p.tiles = (N + 127) / 128;
   p.kappa_t = ctx->cfg.kappa_target;
@@ -431,7 +436,10 @@ static kt_status fused_loss_grad_async(kt_ctx* ctx, const XView& xv, int N, cons
   if (grid > 256) grid = 256;
   const bool rec = ctx->prof_on && ctx->prof_used < kProfPairs;
   if (rec) KT_CUDA(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], ctx->stream));
-  fused_small_kernel<<<grid, kFsThreads, kFsSmem, ctx->stream>>>(p);
+  if (terms == 2)
+    fused_small_kernel<2><<<grid, kFsThreads, FusedCfg<2>::kSmem, ctx->stream>>>(p);
+  else
+    fused_small_kernel<1><<<grid, kFsThreads, FusedCfg<1>::kSmem, ctx->stream>>>(p);
   KT_LAUNCH_CHECK();
   if (rec) {
     KT_CUDA(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used + 1], ctx->stream));
@@ -809,7 +817,7 @@ kt_status kt_kurtosis_loss(kt_ctx* ctx, kt_mat X, const float* R, double* loss) 
   KT_TRY(check_ws(ctx, L));
   XView xv;
   KT_TRY(ingest_x_forward(ctx, X, L, &xv));
-  KT_TRY(cast_rt(ctx, R, static_cast<int>(d), L));
+  KT_TRY(cast_rt(ctx, R, static_cast<int>(d), N, L));
   KT_TRY(forward_loss(ctx, xv, static_cast<int>(N), static_cast<int>(d), L, nullptr));
   KT_TRY(sync_scalars(ctx));
   *loss = ctx->h_blk->sc.loss;
@@ -825,7 +833,7 @@ kt_status kt_row_moments(kt_ctx* ctx, kt_mat X, const float* R, float* moments) 
   KT_TRY(check_ws(ctx, L));
   XView xv;
   KT_TRY(ingest_x_forward(ctx, X, L, &xv));
-  KT_TRY(cast_rt(ctx, R, static_cast<int>(d), L));
+  KT_TRY(cast_rt(ctx, R, static_cast<int>(d), N, L));
   KT_TRY(forward_loss(ctx, xv, static_cast<int>(N), static_cast<int>(d), L, nullptr));
   KT_CUDA(cudaMemcpyAsync(moments, at<float4>(ctx, L.moments), static_cast<size_t>(N) * 16, cudaMemcpyDeviceToDevice,
                           ctx->stream));
@@ -841,11 +849,11 @@ kt_status kt_rotate(kt_ctx* ctx, kt_mat X, const float* R, float* Y) {
   KT_TRY(check_ws(ctx, L));
   XView xv;
   KT_TRY(ingest_x_forward(ctx, X, L, &xv));
-  KT_TRY(cast_rt(ctx, R, static_cast<int>(d), L));
+  KT_TRY(cast_rt(ctx, R, static_cast<int>(d), N, L));
   GemmParams p = blank_params();
   p.out = Y;
   p.ldo = d;
-  const FwdOperands f = fwd_operands(ctx, xv, static_cast<int>(d), L);
+  const FwdOperands f = fwd_operands(ctx, xv, static_cast<int>(d), N, L);
   return run_gemm<kStoreF32>(ctx, static_cast<int>(N), static_cast<int>(d), static_cast<int>(d), f.terms, f.A, f.B, p,
                              kCatForward);
 }
@@ -952,10 +960,10 @@ kt_status kt_quant4_error(kt_ctx* ctx, kt_mat X, const float* R, double* mse) {
   const int N = static_cast<int>(N64), d = static_cast<int>(d64);
   XView xv;
   KT_TRY(ingest_x_forward(ctx, X, L, &xv));
-  KT_TRY(cast_rt(ctx, R, d, L));
+  KT_TRY(cast_rt(ctx, R, d, N, L));
   unsigned int* rowmax = at<unsigned int>(ctx, L.rowmax);
   KT_CUDA(cudaMemsetAsync(rowmax, 0, static_cast<size_t>(N) * 4, ctx->stream));
-  const FwdOperands f = fwd_operands(ctx, xv, d, L);
+  const FwdOperands f = fwd_operands(ctx, xv, d, N, L);
   {
     GemmParams p = blank_params();
     p.rowmax = rowmax;
@@ -1121,7 +1129,7 @@ kt_status kt_kurtosis_loss_noalloc(kt_mat X, const float* R, double* loss_dev, v
   XView xv;
   xv.xb = static_cast<const __nv_bfloat16*>(X.data);
   xv.ldx = X.ld;
-  KT_TRY(cast_rt(ctx, R, static_cast<int>(d), L));
+  KT_TRY(cast_rt(ctx, R, static_cast<int>(d), N, L));
   return forward_loss(ctx, xv, static_cast<int>(N), static_cast<int>(d), L, loss_dev);
 }
 
