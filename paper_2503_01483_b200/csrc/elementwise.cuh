@@ -61,22 +61,27 @@ __global__ void k_split_bf16(const float* __restrict__ src, long long ld, __nv_b
   __shared__ float tile[32][33];
   const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
   const int tx = threadIdx.x, ty = threadIdx.y;
+  float x[4];  // four independent loads in flight per thread
+#pragma unroll
+  for (int q = 0; q < 4; ++q) x[q] = src[static_cast<long long>(r0 + ty + 8 * q) * ld + c0 + tx];
   if (!TRANSPOSE) {
-    for (int r = ty; r < 32; r += 8) {
-      const float x = src[static_cast<long long>(r0 + r) * ld + c0 + tx];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
       __nv_bfloat16 h, l;
-      split_bf16(x, h, l);
-      const long long o = static_cast<long long>(r0 + r) * ldo + c0 + tx;
+      split_bf16(x[q], h, l);
+      const long long o = static_cast<long long>(r0 + ty + 8 * q) * ldo + c0 + tx;
       hi[o] = h;
       if (lo) lo[o] = l;
     }
   } else {
-    for (int r = ty; r < 32; r += 8) tile[r][tx] = src[static_cast<long long>(r0 + r) * ld + c0 + tx];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) tile[ty + 8 * q][tx] = x[q];
     __syncthreads();
-    for (int c = ty; c < 32; c += 8) {
-      const float x = tile[tx][c];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int c = ty + 8 * q;
       __nv_bfloat16 h, l;
-      split_bf16(x, h, l);
+      split_bf16(tile[tx][c], h, l);
       const long long o = static_cast<long long>(c0 + c) * ldo + r0 + tx;
       hi[o] = h;
       if (lo) lo[o] = l;
@@ -250,13 +255,22 @@ __global__ void k_skew(const float* __restrict__ A, int d, __nv_bfloat16* __rest
   __shared__ double sh[8];
   const int bj = blockIdx.x, bi = blockIdx.y;
   const int tx = threadIdx.x, ty = threadIdx.y;
-  // tile (bj, bi) of A, to be read transposed
-  for (int r = ty; r < 32; r += 8) tT[r][tx] = A[static_cast<long long>(bj * 32 + r) * d + bi * 32 + tx];
+  // eight independent loads per thread: four of tile (bi, bj), four of tile (bj, bi) (to be read transposed)
+  float av[4], tv[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    av[q] = A[static_cast<long long>(bi * 32 + ty + 8 * q) * d + bj * 32 + tx];
+    tv[q] = A[static_cast<long long>(bj * 32 + ty + 8 * q) * d + bi * 32 + tx];
+  }
+#pragma unroll
+  for (int q = 0; q < 4; ++q) tT[ty + 8 * q][tx] = tv[q];
   __syncthreads();
   double acc = 0.0;
-  for (int r = ty; r < 32; r += 8) {
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int r = ty + 8 * q;
     const long long o = static_cast<long long>(bi * 32 + r) * d + bj * 32 + tx;
-    const float w = 0.5f * (A[o] - tT[tx][r]);
+    const float w = 0.5f * (av[q] - tT[tx][r]);
     __nv_bfloat16 h, l;
     split_bf16(w, h, l);
     w_hi[o] = h;
@@ -371,11 +385,12 @@ __global__ void k_colnorm_partial(const float* __restrict__ R, int d, float* __r
   __shared__ float sh[8][33];
   const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
   const int tx = threadIdx.x, ty = threadIdx.y;
+  float v[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) v[q] = R[static_cast<long long>(r0 + ty + 8 * q) * d + c0 + tx];
   float acc = 0.f;
-  for (int r = ty; r < 32; r += 8) {
-    const float v = R[static_cast<long long>(r0 + r) * d + c0 + tx];
-    acc = fmaf(v, v, acc);
-  }
+#pragma unroll
+  for (int q = 0; q < 4; ++q) acc = fmaf(v[q], v[q], acc);
   sh[ty][tx] = acc;
   __syncthreads();
   if (ty == 0) {
