@@ -189,6 +189,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2_7b_attn", choices=sorted(WORKLOADS))
     ap.add_argument("--rows", type=int, default=0, help="override N (profiling on a small case)")
+    ap.add_argument("--forward-terms", type=int, default=0, help="kt_config.forward_terms (0 = automatic)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -227,7 +228,7 @@ def main():
         X = torch.roll(X, shifts=rank * 977, dims=0).contiguous()
     N = X.shape[0]
     lr = cfg["lr"]
-    ctx = kurtail.Context(dev)
+    ctx = kurtail.Context(dev, forward_terms=args.forward_terms)
 
     def fresh_R():
         if cfg["init"] == "hadamard":

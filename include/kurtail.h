@@ -82,9 +82,10 @@ typedef struct {
                            this many steps (and always after the last one)     */
   int32_t forward_terms;/* [0]   bf16 terms of R in the token GEMMs: 1 = R rounded
                            to bf16; 2 = hi + lo (about 16 significant bits,
-                           twice the MMA work); 0 = automatic: 2 for small
-                           problems (d <= 512 and N*d <= 2^24, where the extra
-                           work is free), else 1                                */
+                           twice the MMA work); 0 = automatic: 2 when d <= 512
+                           (with few channels the rounding error of R is
+                           systematic over tokens and one term can miss the
+                           1e-3 loss tolerance), else 1                         */
   int32_t small_d_fused;/* [1]   d == 128: kt_loss_grad / kt_fit use the single-pass
                            kernel (X read once per evaluation); 0 = the general
                            three-GEMM path                                      */

@@ -287,8 +287,16 @@ __global__ void k_skew(const float* __restrict__ A, int d, __nv_bfloat16* __rest
 __global__ void k_step_size(const double* __restrict__ block_norm2, int n, float lr, float q, float eps,
                             Scalars* __restrict__ sc) {
   __shared__ double sh[8];
-  double s = 0.0;
-  for (int i = threadIdx.x; i < n; i += 256) s += block_norm2[i];
+  double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;  // four chains: the loads of a thread overlap
+  int i = threadIdx.x;
+  for (; i + 768 < n; i += 1024) {
+    s0 += block_norm2[i];
+    s1 += block_norm2[i + 256];
+    s2 += block_norm2[i + 512];
+    s3 += block_norm2[i + 768];
+  }
+  for (; i < n; i += 256) s0 += block_norm2[i];
+  double s = (s0 + s1) + (s2 + s3);
   s = block_sum_256(s, sh, threadIdx.x);
   if (threadIdx.x == 0) {
     const double nrm = sqrt(s);
@@ -466,32 +474,44 @@ __global__ void k_guard_decide(Scalars* sc, float thresh) {
 }
 
 // When the gate is open: R <- R - Q/2 (one Newton-Schulz step, Q = R E) and the bf16 forms of the
-// new R (r_hi, rt_hi, rt_lo) are rewritten.  grid (d/32, d/32), block (32, 8).
+// new R (r_hi, rt_hi, rt_lo) are rewritten.  grid (d/32, 16), block (32, 8): each block walks the row tiles
+// blockIdx.y, blockIdx.y + 16, ... (a small grid, because in most steps the gate is closed and the kernel only
+// has to find that out).
 __global__ void k_polish_apply(float* __restrict__ R, const float* __restrict__ Q, const Scalars* __restrict__ sc,
                                int d, __nv_bfloat16* __restrict__ r_hi, __nv_bfloat16* __restrict__ rt_hi,
                                __nv_bfloat16* __restrict__ rt_lo) {
   if (sc->gate == 0u) return;
   __shared__ float tile[32][33];
-  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  const int c0 = blockIdx.x * 32;
   const int tx = threadIdx.x, ty = threadIdx.y;
+  for (int r0 = blockIdx.y * 32; r0 < d; r0 += gridDim.y * 32) {
+    float rv[4], qv[4];
 #pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const int r = ty + 8 * q;
-    const long long o = static_cast<long long>(r0 + r) * d + c0 + tx;
-    const float v = fmaf(-0.5f, Q[o], R[o]);
-    R[o] = v;
-    tile[r][tx] = v;
-    r_hi[o] = __float2bfloat16_rn(v);
-  }
-  __syncthreads();
+    for (int q = 0; q < 4; ++q) {
+      const long long o = static_cast<long long>(r0 + ty + 8 * q) * d + c0 + tx;
+      rv[q] = R[o];
+      qv[q] = Q[o];
+    }
 #pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const int c = ty + 8 * q;
-    __nv_bfloat16 h, l;
-    split_bf16(tile[tx][c], h, l);
-    const long long o = static_cast<long long>(c0 + c) * d + r0 + tx;
-    rt_hi[o] = h;
-    rt_lo[o] = l;
+    for (int q = 0; q < 4; ++q) {
+      const int r = ty + 8 * q;
+      const long long o = static_cast<long long>(r0 + r) * d + c0 + tx;
+      const float v = fmaf(-0.5f, qv[q], rv[q]);
+      R[o] = v;
+      tile[r][tx] = v;
+      r_hi[o] = __float2bfloat16_rn(v);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int c = ty + 8 * q;
+      __nv_bfloat16 h, l;
+      split_bf16(tile[tx][c], h, l);
+      const long long o = static_cast<long long>(c0 + c) * d + r0 + tx;
+      rt_hi[o] = h;
+      rt_lo[o] = l;
+    }
+    __syncthreads();
   }
 }
 
