@@ -34,6 +34,8 @@ WORKLOADS = {
     "kv_heads": ("kv_heads", 128, 32 * 65536),
     "llama3_8b_down": ("llama3_8b_down", 14336, 32768),
     "llama3_70b_layer": ("llama3_70b_sweep", 8192, 32768),
+    # the whole layer-wise sweep: --layers resident layer buffers (80 by default), --steps steps per layer
+    "llama3_70b_sweep": ("llama3_70b_sweep", 8192, 32768),
 }
 
 
@@ -189,6 +191,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2_7b_attn", choices=sorted(WORKLOADS))
     ap.add_argument("--rows", type=int, default=0, help="override N (profiling on a small case)")
+    ap.add_argument("--layers", type=int, default=80, help="layers of the llama3_70b_sweep workload")
     ap.add_argument("--forward-terms", type=int, default=0, help="kt_config.forward_terms (0 = automatic)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -218,11 +221,13 @@ def main():
     dist_util.barrier(dist)
 
     # each rank fits its own layer buffer (layers are independent: no data-path collective)
+    sweep = args.workload == "llama3_70b_sweep"
     kw = dict(device=dev, rows=N_full if wl_cfg != "kv_heads" else N_full)
     if wl_cfg == "llama3_70b_sweep":
-        kw["layers"] = 1
+        kw["layers"] = args.layers if sweep else 1
     cfg = synth.config(wl_cfg, **kw)
-    X = cfg["X"][0] if isinstance(cfg["X"], list) else cfg["X"]
+    Xs = cfg["X"] if isinstance(cfg["X"], list) else [cfg["X"]]   # all layer buffers stay resident in HBM
+    X = Xs[0]
     if world > 1:
         # different data per rank: re-draw with a rank-dependent seed by rolling rows
         X = torch.roll(X, shifts=rank * 977, dims=0).contiguous()
@@ -252,7 +257,14 @@ def main():
     ctx.profile_begin()
     t_wall0 = time.time()
     ev0.record()
-    rep = ctx.fit(X, R, args.steps, lr)
+    if sweep:
+        Rs = [R] + [fresh_R() for _ in Xs[1:]]
+        torch.cuda.synchronize()
+        ev0.record()
+        reps = ctx.fit_layers(Xs, Rs, args.steps, lr)
+        rep = reps[-1]
+    else:
+        rep = ctx.fit(X, R, args.steps, lr)
     ev1.record()
     torch.cuda.synchronize()
     t_wall1 = time.time()
@@ -261,12 +273,13 @@ def main():
     ms = dist_util.max_over_ranks(dist, ms, dev)
     dist_util.barrier(dist)
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
-    ms_per_step = ms / args.steps
-    value = world * N * args.steps / (ms * 1e-3)
+    n_layers = len(Xs) if sweep else 1
+    ms_per_step = ms / (args.steps * n_layers)
+    value = world * N * args.steps * n_layers / (ms * 1e-3)
 
     # ---- end to end through kt_fit_host: pinned host X and R in, R out, copies inside the timed region
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not sweep:
         Xh = X.cpu().pin_memory()
         Rh = torch.from_numpy(R0_host.copy()).pin_memory()
         stage = torch.empty_like(X)
@@ -339,7 +352,9 @@ def main():
         "config": {"workload": args.workload, "N": N, "d": d, "R_init": cfg["init"], "lr": lr,
                    "l2": "inputs (%.0f MiB of X per step) exceed the 126 MB L2" % (N * d * 2 / 2**20)
                    if N * d * 2 > 126e6 else "inputs fit in L2; no flush (small case)",
-                   "parallelism": "one independent layer per GPU" if world > 1 else "single GPU"},
+                   "parallelism": "one independent layer per GPU" if world > 1 else "single GPU",
+                   **({"layers": n_layers, "steps_per_layer": args.steps, "resident_gib": n_layers * N * d * 2 / 2**30,
+                       "sweep_seconds": ms * 1e-3} if sweep else {})},
         "algorithmic_tflops": (4.0 * N * d * d) * world / (ms_per_step * 1e-3) / 1e12,
         "loss_first": rep["loss_first"], "loss_last": rep["loss_last"], "orth_err": rep["orth_err"],
         "alpha_last": rep["alpha_last"], "w_norm_last": rep["w_norm_last"],

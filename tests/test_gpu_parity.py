@@ -209,6 +209,20 @@ def test_single_pass_kernel_d128(ctx, N):
     assert loss2 == loss and torch.equal(dR2, dR)
 
 
+def test_single_head_rows_meet_the_loss_tolerance(ctx):
+    # every token puts its energy into the same two channels: the rounding of R is then systematic over tokens,
+    # which is why R is used as a two-term bf16 split at small d (one term gives 2e-3 here)
+    X = synth.kv_heads(1, 200000, 128, 30.0, seed=200000, device=DEV)
+    R = rand_orth(128, seed=12)
+    loss, dR = ctx.loss_grad(X, R)
+    L_ref, dR_ref = ko.loss_grad(f64(X), f64(R))
+    assert abs(loss - L_ref) <= 1e-3 * abs(L_ref)
+    assert np.linalg.norm(f64(dR) - dR_ref) / np.linalg.norm(dR_ref) <= 1e-2
+    gen = kurtail.Context(DEV, small_d_fused=0)
+    assert abs(gen.kurtosis_loss(X, R) - L_ref) <= 1e-3 * abs(L_ref)
+    gen.close()
+
+
 def test_single_pass_kernel_fit_kv_heads(ctx):
     cfg = synth.config("kv_heads", device=DEV, rows=32 * 1024)
     X = cfg["X"]
