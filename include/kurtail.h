@@ -76,10 +76,18 @@ typedef struct {
                            +inf: never.  (The guard measures R^T R from a
                            two-term bf16 split: its noise floor is about
                            2e-5/sqrt(d).)                                       */
-  int32_t retract_terms;/* [2]   bf16 split terms (1..3) of the iterate in the
-                           retraction products; more = closer to float32       */
-  int32_t guard_every;  /* [1]   in kt_fit: run the orthogonality guard every
-                           this many steps (and always after the last one)     */
+  int32_t retract_terms;/* [0]   bf16 split terms of R in the product P0 = W R of
+                           the retraction: 1..3 forces a count; 0 = chosen on
+                           the device per step (one term while alpha*||W||_F *
+                           2^-9 < 2.5e-6, else hi + lo), and series terms that
+                           fall below float32 resolution are skipped           */
+  int32_t guard_every;  /* [0]   kt_fit: k >= 1 measures R^T R - I every k-th step
+                           (and after the last one); 0 = on the first and the
+                           last step and in between whenever a device-side
+                           bound on the accumulated drift reaches half of
+                           polish_thresh; in this mode the polish already runs
+                           at a quarter of polish_thresh, so that measurements
+                           stay rare.  kt_orth_step always measures           */
   int32_t forward_terms;/* [0]   bf16 terms of R in the token GEMMs: 1 = R rounded
                            to bf16; 2 = hi + lo (about 16 significant bits,
                            twice the MMA work); 0 = automatic: 2 when d <= 512
@@ -102,8 +110,8 @@ typedef struct {
   int32_t degenerate_rows; /* rows skipped in the last evaluated loss          */
   double loss_first;       /* loss at R before the first step                   */
   double loss_last;        /* loss at R before the last step                    */
-  double orth_err;         /* max|R^T R - I| seen by the last guard, before its
-                              polish                                            */
+  double orth_err;         /* max|R^T R - I| seen by the last measuring step,
+                              before its polish                                 */
   float alpha_last;        /* step size used by the last step                   */
   float w_norm_last;       /* ||W||_F of the last step                          */
   double* loss_history;    /* optional host array of `steps` entries, or NULL   */
@@ -178,7 +186,8 @@ kt_status kt_orth_error(kt_ctx* ctx, const float* R, int64_t d, double* err);
 
 /* `steps` x (kt_loss_grad; kt_orth_step) on the context's stream with no host
  * synchronisation in between; bit-identical to composing those calls when
- * guard_every == 1.  R in/out.  `report` (host) may be NULL.  Synchronises at
+ * guard_every == 1 (with the default 0 the two differ only in which steps
+ * measure orthogonality).  R in/out.  `report` (host) may be NULL.  Synchronises at
  * the end.  On an argument error R is untouched; after a CUDA failure in the
  * middle of a step R may hold a partially applied step. */
 kt_status kt_fit(kt_ctx* ctx, kt_mat X, float* R, int32_t steps, float lr, kt_fit_report* report);

@@ -21,6 +21,11 @@ struct Scalars {
   unsigned int gate;        // 1 = the polish runs
   unsigned int err_word;    // != 0: a bounded wait ran out (code of the waiting role)
   unsigned int deg_rows;    // rows skipped by the last loss
+  // adaptive Cayley step (written by k_step_size, read by the kernels of the step)
+  unsigned int n_terms;     // series terms P_0 .. P_{n_terms-1} are evaluated (the rest are below float32 resolution)
+  unsigned int p0_terms;    // bf16 terms of R used for P_0 = W R
+  unsigned int gate_guard;  // 1 = this step measures R^T R - I
+  float drift;              // bound on the orthogonality error accumulated since the last measurement
   unsigned int pad[2];
 };
 
@@ -282,10 +287,18 @@ __global__ void k_skew(const float* __restrict__ A, int d, __nv_bfloat16* __rest
   if (lin == 0) block_norm2[blockIdx.y * gridDim.x + blockIdx.x] = acc;
 }
 
-// One block: ||W||_F and alpha = min(lr, 2q/(||W||_F + eps)); also clears the
-// guard's running maximum for this step.
+// One block: ||W||_F, alpha = min(lr, 2q/(||W||_F + eps)), and the decisions that depend on x = alpha ||W||_F:
+//  * n_terms: term k of the series changes R by at most x (x/2)^k (Frobenius bounds the spectral norm, ||R|| = 1);
+//    terms below a quarter unit in the last place of a typical entry (2^-26 / sqrt(d)) are skipped (`gate_terms`);
+//  * p0_terms: P_0 = W R multiplies alpha directly; with R as a single bf16 term its error is x 2^-9, which is
+//    accepted while that is below 2.5e-6 (a quarter of the default polish threshold), else hi + lo
+//    (`cfg_terms` 1..3 forces a count, 0 = this rule);
+//  * gate_guard: guard_mode 1 = measure R^T R - I in this step, 2 = do not, 0 = only when the drift bound, which
+//    grows by x^2 + x 2^-9 (or x 2^-17 with two terms) + 4e-7 per step (truncation of the series; rounding of R in
+//    P_0; float32 rounding of the update), has reached half the polish threshold.  A measuring step also clears the running maximum.
 __global__ void k_step_size(const double* __restrict__ block_norm2, int n, float lr, float q, float eps,
-                            Scalars* __restrict__ sc) {
+                            Scalars* __restrict__ sc, int d, int iters, int cfg_terms, int gate_terms, int guard_mode,
+                            float thresh) {
   __shared__ double sh[8];
   double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;  // four chains: the loads of a thread overlap
   int i = threadIdx.x;
@@ -304,58 +317,91 @@ __global__ void k_step_size(const double* __restrict__ block_norm2, int n, float
     const double a = (static_cast<double>(lr) < cap) ? static_cast<double>(lr) : cap;
     sc->alpha = static_cast<float>(a);
     sc->wnorm = static_cast<float>(nrm);
+    const double x = a * nrm;
+    unsigned int nt = 1;
+    const double floor_k = ldexp(1.0, -26) / sqrt(static_cast<double>(d));
+    double bound = x;
+    for (int k = 1; k <= iters; ++k) {
+      bound *= 0.5 * x;
+      if (gate_terms && bound < floor_k) break;
+      ++nt;
+    }
+    sc->n_terms = nt;
+    const unsigned int p0t =
+        cfg_terms > 0 ? static_cast<unsigned int>(cfg_terms) : ((x * ldexp(1.0, -9) >= 2.5e-6) ? 2u : 1u);
+    sc->p0_terms = p0t;
+    unsigned int gg;
+    if (guard_mode == 1) {
+      gg = 1u;
+    } else if (guard_mode == 2) {
+      gg = 0u;
+    } else {
+      const float drift = sc->drift + static_cast<float>(x * x + x * ldexp(1.0, p0t == 1u ? -9 : -17)) + 4e-7f;
+      sc->drift = drift;
+      gg = (thresh <= 0.f || drift >= 0.5f * thresh) ? 1u : 0u;
+    }
+    sc->gate_guard = gg;
+    if (gg) sc->max_e_bits = 0u;
   }
+}
+
+// Before a measurement outside a step (kt_orth_error): open the guard's gate and clear its running maximum.
+__global__ void k_force_guard(Scalars* sc) {
+  sc->gate_guard = 1u;
+  sc->max_e_bits = 0u;
 }
 
 // One term of the Cayley step written as its Neumann series:
 //   R_new = R - alpha * sum_{k=0..s} (-alpha/2)^k P_k,   P_0 = W R,  P_{k+1} = W P_k
 // (the partial sums are exactly the iterates Y_k of the fixed-point form Y_0 = R - alpha W R,
 // Y_k = R - alpha/2 W (R + Y_{k-1})).  This kernel adds term k in place, R += c_k P with
-// c_k = -alpha (-alpha/2)^k, writes P^T as bf16 for the next product when pt_hi != null, and, when
-// r_hi != null (last term), the bf16 forms of the new R: r_hi (as is), rt_hi/rt_lo (transposed hi/lo).
-// grid (d/32, d/32), block (32, 8).
+// c_k = -alpha (-alpha/2)^k.  Terms k >= sc->n_terms do nothing.  A term that is not the last one evaluated writes
+// P^T as bf16 (pt_hi) for the next product; the last one writes the bf16 forms of the new R instead: r_hi (as is),
+// rt_hi/rt_lo (transposed hi/lo).  grid (d/32, min(d/32, 32)), block (32, 8); each block walks row tiles.
 __global__ void k_series_term(float* __restrict__ R, const float* __restrict__ P, const Scalars* __restrict__ sc,
                               int k, int d, __nv_bfloat16* __restrict__ pt_hi, __nv_bfloat16* __restrict__ r_hi,
                               __nv_bfloat16* __restrict__ rt_hi, __nv_bfloat16* __restrict__ rt_lo) {
+  const unsigned int n_terms = sc->n_terms;
+  if (static_cast<unsigned int>(k) >= n_terms) return;
+  const bool last = (static_cast<unsigned int>(k) + 1u == n_terms);
   __shared__ float tile[32][33];
-  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  const int c0 = blockIdx.x * 32;
   const int tx = threadIdx.x, ty = threadIdx.y;
   const float alpha = sc->alpha;
   float ck = -alpha;
   for (int i = 0; i < k; ++i) ck *= -0.5f * alpha;
-  float rn[4];
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const int r = ty + 8 * q;
-    const long long o = static_cast<long long>(r0 + r) * d + c0 + tx;
-    const float pv = P[o];
-    rn[q] = fmaf(ck, pv, R[o]);
-    R[o] = rn[q];
-    tile[r][tx] = pv;
-    if (r_hi) r_hi[o] = __float2bfloat16_rn(rn[q]);
-  }
-  if (pt_hi) {
-    __syncthreads();
+  for (int r0 = blockIdx.y * 32; r0 < d; r0 += gridDim.y * 32) {
+    float pv[4], rv[4], rn[4];
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      const int c = ty + 8 * q;
-      pt_hi[static_cast<long long>(c0 + c) * d + r0 + tx] = __float2bfloat16_rn(tile[tx][c]);
+      const long long o = static_cast<long long>(r0 + ty + 8 * q) * d + c0 + tx;
+      pv[q] = P[o];
+      rv[q] = R[o];
     }
-  }
-  if (rt_hi) {
-    __syncthreads();
 #pragma unroll
-    for (int q = 0; q < 4; ++q) tile[ty + 8 * q][tx] = rn[q];
+    for (int q = 0; q < 4; ++q) {
+      const int r = ty + 8 * q;
+      const long long o = static_cast<long long>(r0 + r) * d + c0 + tx;
+      rn[q] = fmaf(ck, pv[q], rv[q]);
+      R[o] = rn[q];
+      tile[r][tx] = last ? rn[q] : pv[q];
+      if (last) r_hi[o] = __float2bfloat16_rn(rn[q]);
+    }
     __syncthreads();
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const int c = ty + 8 * q;
-      __nv_bfloat16 h, l;
-      split_bf16(tile[tx][c], h, l);
       const long long o = static_cast<long long>(c0 + c) * d + r0 + tx;
-      rt_hi[o] = h;
-      rt_lo[o] = l;
+      if (last) {
+        __nv_bfloat16 h, l;
+        split_bf16(tile[tx][c], h, l);
+        rt_hi[o] = h;
+        rt_lo[o] = l;
+      } else {
+        pt_hi[o] = __float2bfloat16_rn(tile[tx][c]);
+      }
     }
+    __syncthreads();
   }
 }
 
@@ -387,31 +433,39 @@ __global__ void k_split_r(const float* __restrict__ R, int d, __nv_bfloat16* __r
 }
 
 // Column sums of squares of a d x d float32 R, by row slabs of 32:
-// colpart[slab][j] = sum over the slab's 32 rows of R[i][j]^2.
-// grid (d/32, d/32), block (32, 8).
-__global__ void k_colnorm_partial(const float* __restrict__ R, int d, float* __restrict__ colpart) {
+// colpart[slab][j] = sum over the slab's 32 rows of R[i][j]^2.  Does nothing when the guard's gate is closed.
+// grid (d/32, min(d/32, 32)), block (32, 8); each block walks row slabs.
+__global__ void k_colnorm_partial(const float* __restrict__ R, int d, float* __restrict__ colpart,
+                                  const Scalars* __restrict__ sc) {
+  if (sc->gate_guard == 0u) return;
   __shared__ float sh[8][33];
-  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  const int c0 = blockIdx.x * 32;
   const int tx = threadIdx.x, ty = threadIdx.y;
-  float v[4];
+  for (int slab = blockIdx.y; slab * 32 < d; slab += gridDim.y) {
+    const int r0 = slab * 32;
+    float v[4];
 #pragma unroll
-  for (int q = 0; q < 4; ++q) v[q] = R[static_cast<long long>(r0 + ty + 8 * q) * d + c0 + tx];
-  float acc = 0.f;
+    for (int q = 0; q < 4; ++q) v[q] = R[static_cast<long long>(r0 + ty + 8 * q) * d + c0 + tx];
+    float acc = 0.f;
 #pragma unroll
-  for (int q = 0; q < 4; ++q) acc = fmaf(v[q], v[q], acc);
-  sh[ty][tx] = acc;
-  __syncthreads();
-  if (ty == 0) {
-    float s = 0.f;
+    for (int q = 0; q < 4; ++q) acc = fmaf(v[q], v[q], acc);
+    sh[ty][tx] = acc;
+    __syncthreads();
+    if (ty == 0) {
+      float s = 0.f;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) s += sh[i][tx];
-    colpart[static_cast<long long>(blockIdx.y) * d + c0 + tx] = s;
+      for (int i = 0; i < 8; ++i) s += sh[i][tx];
+      colpart[static_cast<long long>(slab) * d + c0 + tx] = s;
+    }
+    __syncthreads();
   }
 }
 
 // diag[j] = (sum over slabs of colpart[slab][j]) - 1, accumulated in double: the exact diagonal of
 // R^T R - I.  One warp per column; grid ceil(d/8), block 256.
-__global__ void k_colnorm_final(const float* __restrict__ colpart, int nslabs, int d, float* __restrict__ diag) {
+__global__ void k_colnorm_final(const float* __restrict__ colpart, int nslabs, int d, float* __restrict__ diag,
+                                const Scalars* __restrict__ sc) {
+  if (sc->gate_guard == 0u) return;
   const int j = blockIdx.x * 8 + (threadIdx.x >> 5);
   if (j >= d) return;
   double s = 0.0;
@@ -429,31 +483,38 @@ __global__ void k_colnorm_final(const float* __restrict__ colpart, int nslabs, i
 // Off-diagonal sums hover around 0 and carry no such bias.  grid (d/32, d/32), block (32, 8).
 __global__ void k_guard(const float* __restrict__ S, int d, int bn, const float* __restrict__ diag,
                         __nv_bfloat16* __restrict__ e_hi, Scalars* __restrict__ sc) {
+  if (sc->gate_guard == 0u) return;
   __shared__ float tile[32][33];
   __shared__ float shm[8];
-  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  const int c0 = blockIdx.x * 32;
   const int tx = threadIdx.x, ty = threadIdx.y;
-  const bool computed = ((c0 / bn) + 1) * bn > (r0 / 128) * 128;
-  float e[4];
-  if (computed) {
-#pragma unroll
-    for (int q = 0; q < 4; ++q) e[q] = S[static_cast<long long>(r0 + ty + 8 * q) * d + c0 + tx];
-  } else {
-#pragma unroll
-    for (int q = 0; q < 4; ++q) tile[ty + 8 * q][tx] = S[static_cast<long long>(c0 + ty + 8 * q) * d + r0 + tx];
-    __syncthreads();
-#pragma unroll
-    for (int q = 0; q < 4; ++q) e[q] = tile[tx][ty + 8 * q];
-  }
   float mx = 0.f;
   bool bad = false;
+  for (int r0 = blockIdx.y * 32; r0 < d; r0 += gridDim.y * 32) {
+    const bool computed = ((c0 / bn) + 1) * bn > (r0 / 128) * 128;
+    float e[4];
+    if (computed) {
 #pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const int row = r0 + ty + 8 * q, col = c0 + tx;
-    if (row == col) e[q] = diag[row];
-    bad |= (e[q] != e[q]);
-    mx = fmaxf(mx, fabsf(e[q]));
-    if (e_hi) e_hi[static_cast<long long>(row) * d + col] = __float2bfloat16_rn(e[q]);
+      for (int q = 0; q < 4; ++q) e[q] = S[static_cast<long long>(r0 + ty + 8 * q) * d + c0 + tx];
+    } else {
+      float t[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) t[q] = S[static_cast<long long>(c0 + ty + 8 * q) * d + r0 + tx];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) tile[ty + 8 * q][tx] = t[q];
+      __syncthreads();
+#pragma unroll
+      for (int q = 0; q < 4; ++q) e[q] = tile[tx][ty + 8 * q];
+      __syncthreads();
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int row = r0 + ty + 8 * q, col = c0 + tx;
+      if (row == col) e[q] = diag[row];
+      bad |= (e[q] != e[q]);
+      mx = fmaxf(mx, fabsf(e[q]));
+      if (e_hi) e_hi[static_cast<long long>(row) * d + col] = __float2bfloat16_rn(e[q]);
+    }
   }
   if (bad) mx = __uint_as_float(0x7f800000u);  // a NaN in R^T R reads as +inf
 #pragma unroll
@@ -467,10 +528,18 @@ __global__ void k_guard(const float* __restrict__ S, int d, int bn, const float*
   }
 }
 
-// gate = (max|E| > thresh).
-__global__ void k_guard_decide(Scalars* sc, float thresh) {
+// gate = (max|E| > thresh) when this step measured E.
+// `polish_at` <= thresh: inside kt_fit's adaptive cadence the polish already runs at a quarter of the threshold, so
+// that the drift bound restarts low and the next measurements can be skipped.
+__global__ void k_guard_decide(Scalars* sc, float polish_at) {
+  if (sc->gate_guard == 0u) {  // nothing was measured in this step: no polish, the last measurement stands
+    sc->gate = 0u;
+    return;
+  }
   const float mx = __uint_as_float(sc->max_e_bits);
-  sc->gate = (mx > thresh) ? 1u : 0u;
+  const unsigned int polish = (mx > polish_at) ? 1u : 0u;
+  sc->gate = polish;
+  sc->drift = polish ? 0.f : mx;  // the drift bound restarts from what was just measured
 }
 
 // When the gate is open: R <- R - Q/2 (one Newton-Schulz step, Q = R E) and the bf16 forms of the

@@ -51,7 +51,9 @@ struct GemmParams {
   long long ldg;
   unsigned int* rowmax;       // kAbsMax (out) / kQuantErr (in): per-row max|D| as float bits
   float* qerr;                // kQuantErr: [n_tiles][M] partial squared errors
-  const unsigned int* gate;   // when not null and *gate == 0 the kernel does nothing
+  const unsigned int* gate;   // when not null and *gate < gate_min the kernel does nothing
+  unsigned int gate_min;
+  const unsigned int* terms_dev;  // when not null, min(terms, *terms_dev) operand pairs are used
   unsigned int* err_word;     // receives the code of a wait that ran out
 };
 
@@ -72,7 +74,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
   constexpr uint32_t kTmemCols = 2 * BN;  // two accumulators: 256 or 512 columns
   constexpr uint32_t kIdesc = umma_idesc_bf16_f32(kBM, BN);
 
-  if (p.gate != nullptr && *p.gate == 0u) return;  // uniform over the grid
+  if (p.gate != nullptr && *p.gate < p.gate_min) return;  // uniform over the grid
+  int n_terms = p.terms;
+  if (p.terms_dev != nullptr) {
+    const int t = static_cast<int>(*p.terms_dev);
+    n_terms = t < n_terms ? (t < 1 ? 1 : t) : n_terms;
+  }
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -104,7 +111,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
   auto unit_iters = [&](int u) {
     const int kb0 = (u / plain_tiles) * p.kb_per_split;
     const int kb1 = (kb0 + p.kb_per_split < k_blocks) ? kb0 + p.kb_per_split : k_blocks;
-    return (kb1 - kb0) * p.terms;
+    return (kb1 - kb0) * n_terms;
   };
 
   if (threadIdx.x == 0) {
@@ -151,8 +158,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
         const int kb0 = unit_kb0(unit);
         const int iters = unit_iters(unit);
         for (int it = 0; it < iters; ++it) {
-          const int kbl = it / p.terms;
-          const int q = it - kbl * p.terms;
+          const int kbl = it / n_terms;
+          const int q = it - kbl * n_terms;
           const int kb = kb0 + kbl;
           if (!mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, 1u)) {
             ok = false;

@@ -460,14 +460,18 @@ static kt_status fused_loss_grad_async(kt_ctx* ctx, const XView& xv, int N, cons
 // ---------------------------------------------------------- orthogonal step
 // E = R^T R - I from the bf16 forms of R^T (rt_hi, rt_lo, which must be current) and, when
 // `with_polish`, R <- R - R E / 2 if max|E| > polish_thresh (needs r_hi; refreshes all three forms).
-static kt_status guard(kt_ctx* ctx, const float* R_in, float* R, int d, const WsLayout& L, bool with_polish) {
+// Every kernel here looks at the device-side gate sc->gate_guard (set by k_step_size or k_force_guard, which also
+// clear the running maximum) and does nothing when it is closed.
+static kt_status guard(kt_ctx* ctx, const float* R_in, float* R, int d, const WsLayout& L, bool with_polish,
+                       float polish_at) {
   Scalars* sc = &ctx->d_blk->sc;
-  dim3 tgrid(d / 32, d / 32), tblock(32, 8);
-  k_colnorm_partial<<<tgrid, tblock, 0, ctx->stream>>>(R_in, d, at<float>(ctx, L.colpart));
+  const int gy = d / 32 < 32 ? d / 32 : 32;
+  dim3 lgrid(d / 32, gy), tblock(32, 8);
+  k_colnorm_partial<<<lgrid, tblock, 0, ctx->stream>>>(R_in, d, at<float>(ctx, L.colpart), sc);
   KT_LAUNCH_CHECK();
-  k_colnorm_final<<<(d + 7) / 8, 256, 0, ctx->stream>>>(at<float>(ctx, L.colpart), d / 32, d, at<float>(ctx, L.diag));
+  k_colnorm_final<<<(d + 7) / 8, 256, 0, ctx->stream>>>(at<float>(ctx, L.colpart), d / 32, d, at<float>(ctx, L.diag),
+                                                        sc);
   KT_LAUNCH_CHECK();
-  KT_CUDA(cudaMemsetAsync(&sc->max_e_bits, 0, sizeof(unsigned int), ctx->stream));
   const uint64_t ld = static_cast<uint64_t>(d);
   __nv_bfloat16* rt_hi = at<__nv_bfloat16>(ctx, L.rt_hi);
   __nv_bfloat16* rt_lo = at<__nv_bfloat16>(ctx, L.rt_lo);
@@ -478,27 +482,31 @@ static kt_status guard(kt_ctx* ctx, const float* R_in, float* R, int d, const Ws
     p.out = fbuf;
     p.ldo = d;
     p.upper_only = 1;  // R^T R is symmetric: tiles below the diagonal are mirrored by k_guard
+    p.gate = &sc->gate_guard;
+    p.gate_min = 1;
     // (H + L)^T (H + L) without L^T L: that term only matters on the diagonal, which k_guard takes from `diag`
     Operand A[3] = {{rt_hi, ld}, {rt_hi, ld}, {rt_lo, ld}};
     Operand B[3] = {{rt_hi, ld}, {rt_lo, ld}, {rt_hi, ld}};
     KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 3, A, B, p, kCatSquare));
   }
   __nv_bfloat16* e_hi = at<__nv_bfloat16>(ctx, L.z_hi);
-  k_guard<<<tgrid, tblock, 0, ctx->stream>>>(fbuf, d, (d % 256 == 0) ? 256 : 128, at<float>(ctx, L.diag),
+  k_guard<<<lgrid, tblock, 0, ctx->stream>>>(fbuf, d, (d % 256 == 0) ? 256 : 128, at<float>(ctx, L.diag),
                                              with_polish ? e_hi : nullptr, sc);
   KT_LAUNCH_CHECK();
   if (!with_polish) return KT_OK;
-  k_guard_decide<<<1, 1, 0, ctx->stream>>>(sc, ctx->cfg.polish_thresh);
+  k_guard_decide<<<1, 1, 0, ctx->stream>>>(sc, polish_at);
   KT_LAUNCH_CHECK();
   {
     GemmParams p = blank_params();
     p.out = fbuf;
     p.ldo = d;
     p.gate = &sc->gate;
+    p.gate_min = 1;
     Operand A{r_hi, ld}, B{e_hi, ld};  // (R E)[i][j] = sum_k R[i][k] E[j][k], E symmetric
     KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 1, &A, &B, p, kCatSquare));
   }
-  k_polish_apply<<<dim3(d / 32, d / 32 < 16 ? d / 32 : 16), tblock, 0, ctx->stream>>>(R, fbuf, sc, d, r_hi, rt_hi, rt_lo);
+  k_polish_apply<<<dim3(d / 32, d / 32 < 16 ? d / 32 : 16), tblock, 0, ctx->stream>>>(R, fbuf, sc, d, r_hi, rt_hi,
+                                                                                         rt_lo);
   KT_LAUNCH_CHECK();
   return KT_OK;
 }
@@ -548,13 +556,16 @@ static kt_status small_orth_step_async(kt_ctx* ctx, float* R, const float* dR, i
 
 // One Cayley-SGD step.  `forms_current`: r_hi / rt_hi / rt_lo already hold the bf16 forms of R (true from the
 // second step of kt_fit on: the previous step left them).  On return they hold the forms of the new R.
+// guard_mode: 1 = measure R^T R - I (and polish if needed) in this step, 2 = do not, 0 = let the device decide from
+// its drift bound (see k_step_size).
 static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, float lr, const WsLayout& L,
-                                 bool run_guard, bool forms_current) {
-  if (use_small_orth(ctx, d)) return small_orth_step_async(ctx, R, dR, d, lr, L, run_guard);
+                                 int guard_mode, bool forms_current, bool adaptive = false) {
+  if (use_small_orth(ctx, d)) return small_orth_step_async(ctx, R, dR, d, lr, L, guard_mode != 2);
   const kt_config& c = ctx->cfg;
   Scalars* sc = &ctx->d_blk->sc;
   const uint64_t ld = static_cast<uint64_t>(d);
-  dim3 tgrid(d / 32, d / 32), tblock(32, 8);
+  const int gy = d / 32 < 32 ? d / 32 : 32;
+  dim3 tgrid(d / 32, d / 32), lgrid(d / 32, gy), tblock(32, 8);
   __nv_bfloat16* rt_hi = at<__nv_bfloat16>(ctx, L.rt_hi);
   __nv_bfloat16* rt_lo = at<__nv_bfloat16>(ctx, L.rt_lo);
   __nv_bfloat16* r_hi = at<__nv_bfloat16>(ctx, L.r_hi);
@@ -562,9 +573,11 @@ static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, 
   __nv_bfloat16* w_hi = at<__nv_bfloat16>(ctx, L.w_hi);
   __nv_bfloat16* w_lo = at<__nv_bfloat16>(ctx, L.w_lo);
   float* fbuf = at<float>(ctx, L.fbuf);
-  const int terms = c.retract_terms < 1 ? 1 : (c.retract_terms > 3 ? 3 : c.retract_terms);
+  const int cfg_terms = c.retract_terms < 0 ? 0 : (c.retract_terms > 3 ? 3 : c.retract_terms);  // 0 = automatic
+  const int max_terms = cfg_terms > 0 ? cfg_terms : 2;
+  const int s = c.cayley_iters < 0 ? 0 : c.cayley_iters;
 
-  // A = dR R^T (the gradient needs no more than bf16), W = (A - A^T)/2, alpha
+  // A = dR R^T (the gradient needs no more than bf16), W = (A - A^T)/2, alpha and the step's gates
   k_split_bf16<false><<<tgrid, tblock, 0, ctx->stream>>>(dR, d, z_hi /* dR hi: free until P^T is written */, nullptr,
                                                          d);
   KT_LAUNCH_CHECK();
@@ -579,33 +592,38 @@ static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, 
     Operand A{z_hi, ld}, B{r_hi, ld};
     KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 1, &A, &B, p, kCatSquare));
   }
-  k_skew<<<tgrid, tblock, 0, ctx->stream>>>(fbuf, d, w_hi, terms == 3 ? w_lo : nullptr,
+  k_skew<<<tgrid, tblock, 0, ctx->stream>>>(fbuf, d, w_hi, max_terms == 3 ? w_lo : nullptr,
                                             at<double>(ctx, L.norm_blocks));
   KT_LAUNCH_CHECK();
-  k_step_size<<<1, 256, 0, ctx->stream>>>(at<double>(ctx, L.norm_blocks), L.norm_n, lr, c.q, c.eps, sc);
+  k_step_size<<<1, 256, 0, ctx->stream>>>(at<double>(ctx, L.norm_blocks), L.norm_n, lr, c.q, c.eps, sc, d, s,
+                                          cfg_terms, cfg_terms == 0 ? 1 : 0, guard_mode, c.polish_thresh);
   KT_LAUNCH_CHECK();
 
-  // P_0 = W R with R^T as a bf16 split (it multiplies alpha directly); P_{k+1} = W P_k with P_k^T in plain bf16
-  // (these terms carry alpha^2 and higher).  (W Z)[i][j] = sum_k W[i][k] Zt[j][k].
-  const int s = c.cayley_iters < 0 ? 0 : c.cayley_iters;
+  // P_0 = W R with R^T as a bf16 split (it multiplies alpha directly; the device picks one or two terms);
+  // P_{k+1} = W P_k with P_k^T in plain bf16 (these terms carry alpha^2 and higher), skipped on the device once
+  // they are below float32 resolution.  (W Z)[i][j] = sum_k W[i][k] Zt[j][k].
   for (int k = 0; k <= s; ++k) {
     GemmParams p = blank_params();
     p.out = fbuf;
     p.ldo = d;
     if (k == 0) {
+      p.terms_dev = &sc->p0_terms;
       Operand A[3] = {{w_hi, ld}, {w_hi, ld}, {w_lo, ld}};
       Operand B[3] = {{rt_hi, ld}, {rt_lo, ld}, {rt_hi, ld}};
-      KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, terms, A, B, p, kCatSquare));
+      KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, max_terms, A, B, p, kCatSquare));
     } else {
+      p.gate = &sc->n_terms;
+      p.gate_min = static_cast<unsigned int>(k + 1);
       Operand A{w_hi, ld}, B{z_hi, ld};
       KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 1, &A, &B, p, kCatSquare));
     }
-    const bool last = (k == s);
-    k_series_term<<<tgrid, tblock, 0, ctx->stream>>>(R, fbuf, sc, k, d, last ? nullptr : z_hi, last ? r_hi : nullptr,
-                                                     last ? rt_hi : nullptr, last ? rt_lo : nullptr);
+    k_series_term<<<lgrid, tblock, 0, ctx->stream>>>(R, fbuf, sc, k, d, z_hi, r_hi, rt_hi, rt_lo);
     KT_LAUNCH_CHECK();
   }
-  if (run_guard) KT_TRY(guard(ctx, R, R, d, L, true));
+  if (guard_mode != 2) {
+    const float th = ctx->cfg.polish_thresh;
+    KT_TRY(guard(ctx, R, R, d, L, true, (adaptive && th > 0.f) ? 0.25f * th : th));
+  }
   return KT_OK;
 }
 
@@ -656,8 +674,14 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
       KT_TRY(fused_loss_grad_async(ctx, xv, N, L, R, dR, &ctx->d_blk->hist[slot], k > 0));
     else
       KT_TRY(loss_grad_async(ctx, xv, N, d, L, R, dR, &ctx->d_blk->hist[slot], k > 0));
-    const bool run_guard = ((k + 1) % ge == 0) || (k + 1 == steps);
-    KT_TRY(orth_step_async(ctx, R, dR, d, lr, L, run_guard, k > 0));
+    // guard: a fixed cadence when guard_every >= 1; otherwise measured on the first and the last step and in between
+    // whenever the device's drift bound asks for it
+    int guard_mode;
+    if (ctx->cfg.guard_every >= 1)
+      guard_mode = (((k + 1) % ge == 0) || (k + 1 == steps)) ? 1 : 2;
+    else
+      guard_mode = (k == 0 || k + 1 == steps) ? 1 : 0;
+    KT_TRY(orth_step_async(ctx, R, dR, d, lr, L, guard_mode, k > 0, ctx->cfg.guard_every < 1));
     done = k + 1;
   }
   if (steps > 0) {
@@ -702,8 +726,8 @@ void kt_default_config(kt_config* cfg) {
   cfg->q = 0.5f;
   cfg->eps = 1e-8f;
   cfg->polish_thresh = 1e-5f;
-  cfg->retract_terms = 2;
-  cfg->guard_every = 1;
+  cfg->retract_terms = 0;
+  cfg->guard_every = 0;
   cfg->forward_terms = 0;
   cfg->small_d_fused = 1;
   cfg->small_d_orth = 1;
@@ -888,7 +912,7 @@ kt_status kt_orth_step(kt_ctx* ctx, float* R, const float* dR, int64_t d, float 
   if (!aligned16(R) || !aligned16(dR)) return KT_ERR_ALIGN;
   const WsLayout L = make_layout(1, d, KT_BF16);
   KT_TRY(check_ws(ctx, L));
-  return orth_step_async(ctx, R, dR, static_cast<int>(d), lr, L, true, false);
+  return orth_step_async(ctx, R, dR, static_cast<int>(d), lr, L, 1, false);
 }
 
 kt_status kt_orth_error(kt_ctx* ctx, const float* R, int64_t d, double* err) {
@@ -901,7 +925,9 @@ kt_status kt_orth_error(kt_ctx* ctx, const float* R, int64_t d, double* err) {
   k_split_bf16<true><<<tgrid, tblock, 0, ctx->stream>>>(R, d, at<__nv_bfloat16>(ctx, L.rt_hi),
                                                         at<__nv_bfloat16>(ctx, L.rt_lo), d);
   KT_LAUNCH_CHECK();
-  KT_TRY(guard(ctx, R, nullptr, static_cast<int>(d), L, false));
+  k_force_guard<<<1, 1, 0, ctx->stream>>>(&ctx->d_blk->sc);
+  KT_LAUNCH_CHECK();
+  KT_TRY(guard(ctx, R, nullptr, static_cast<int>(d), L, false, 0.f));
   KT_TRY(sync_scalars(ctx));
   *err = static_cast<double>(__builtin_bit_cast(float, ctx->h_blk->sc.max_e_bits));
   return KT_OK;

@@ -43,7 +43,7 @@ def test_status_strings(L):
 def test_default_config(L):
     cfg = kurtail.default_config()
     assert cfg.kappa_target == pytest.approx(1.8)
-    assert cfg.cayley_iters == 2 and cfg.q == 0.5 and cfg.retract_terms == 2 and cfg.guard_every == 1 and cfg.forward_terms == 0
+    assert cfg.cayley_iters == 2 and cfg.q == 0.5 and cfg.retract_terms == 0 and cfg.guard_every == 0 and cfg.forward_terms == 0
 
 
 def test_workspace_bytes_host_only(L):

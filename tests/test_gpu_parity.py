@@ -310,9 +310,12 @@ def test_fit_100_steps_stays_orthogonal_and_descends(ctx):
     assert rep["loss_first"] == pytest.approx(L0, rel=1e-12)
 
 
-def test_fit_equals_composed_calls(ctx):
-    X = make_x(1500, 256, seed=71)
-    Ra = ctx.init_rotation(256, "hadamard")
+@pytest.mark.parametrize("d", [256, 1024])
+def test_fit_equals_composed_calls(d):
+    # the identity holds when every step measures orthogonality (guard_every = 1), as kt_orth_step always does
+    ctx = kurtail.Context(DEV, guard_every=1)
+    X = make_x(1500, d, seed=71)
+    Ra = ctx.init_rotation(d, "hadamard")
     Rb = Ra.clone()
     rep = ctx.fit(X, Ra, 4, 1e-2, history=True)
     losses = []
@@ -322,6 +325,27 @@ def test_fit_equals_composed_calls(ctx):
         ctx.orth_step(Rb, dR, 1e-2)
     assert torch.equal(Ra, Rb)
     assert losses == rep["loss_history"]
+    ctx.close()
+
+
+def test_adaptive_step_matches_forced_precision():
+    # default: the device picks the number of series terms and of bf16 terms of R, and measures orthogonality only
+    # when its drift bound asks; forcing everything must give the same trajectory to well within the step's tolerance
+    d = 1024
+    X = make_x(2048, d, seed=72, n_out=8, scale=100.0)
+    auto = kurtail.Context(DEV)
+    full = kurtail.Context(DEV, retract_terms=2, guard_every=1)
+    Ra = auto.init_rotation(d, "hadamard")
+    Rf = Ra.clone()
+    R0 = Ra.clone()
+    ra = auto.fit(X, Ra, 30, 1e-2, history=True)
+    rf = full.fit(X, Rf, 30, 1e-2, history=True)
+    moved = float((Rf - R0).norm())
+    assert float((Ra - Rf).norm()) <= 2e-2 * moved
+    assert ra["loss_history"][-1] == pytest.approx(rf["loss_history"][-1], rel=1e-4)
+    assert auto.orth_error(Ra) <= 1e-4 and ko.orthogonality_error(f64(Ra)) <= 1e-4
+    auto.close()
+    full.close()
 
 
 def test_fit_teacher_forced_steps(ctx):
