@@ -361,6 +361,15 @@ def main():
         "gpu_launches": prof["launches_total"], "clocks": clocks, "roofline": roofline, "e2e": e2e,
     }
 
+    if world == 1 and not sweep:
+        # the 4-bit fake-quantisation error of the fitted rotation (two GEMM passes; outside the timed region)
+        q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ctx.quant4_error(X, R)
+        q0.record()
+        mse = ctx.quant4_error(X, R)
+        q1.record()
+        torch.cuda.synchronize()
+        out["quant4_error"] = {"mse": mse, "ms": q0.elapsed_time(q1)}
     if not args.no_cpu_baseline and world == 1:
         n_s = min(N, max(64, int(2.0e10 / (4.0 * d * d))))
         sample = X[:n_s].float().cpu().numpy()
