@@ -287,7 +287,7 @@ __global__ void k_skew(const float* __restrict__ A, int d, __nv_bfloat16* __rest
   if (lin == 0) block_norm2[blockIdx.y * gridDim.x + blockIdx.x] = acc;
 }
 
-// One block: ||W||_F, alpha = min(lr, 2q/(||W||_F + eps)), and the decisions that depend on x = alpha ||W||_F:
+// One block of 1024 threads: ||W||_F, alpha = min(lr, 2q/(||W||_F + eps)), and the decisions that depend on x = alpha ||W||_F:
 //  * n_terms: term k of the series changes R by at most x (x/2)^k (Frobenius bounds the spectral norm, ||R|| = 1);
 //    terms below a quarter unit in the last place of a typical entry (2^-26 / sqrt(d)) are skipped (`gate_terms`);
 //  * p0_terms: P_0 = W R multiplies alpha directly; with R as a single bf16 term its error is x 2^-9, which is
@@ -299,18 +299,17 @@ __global__ void k_skew(const float* __restrict__ A, int d, __nv_bfloat16* __rest
 __global__ void k_step_size(const double* __restrict__ block_norm2, int n, float lr, float q, float eps,
                             Scalars* __restrict__ sc, int d, int iters, int cfg_terms, int gate_terms, int guard_mode,
                             float thresh) {
-  __shared__ double sh[8];
-  double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;  // four chains: the loads of a thread overlap
-  int i = threadIdx.x;
-  for (; i + 768 < n; i += 1024) {
-    s0 += block_norm2[i];
-    s1 += block_norm2[i + 256];
-    s2 += block_norm2[i + 512];
-    s3 += block_norm2[i + 768];
+  // 1024 threads; fixed-order sum: per-thread strided partial, warp shuffle tree, then the 32 warp sums in order
+  __shared__ double sh[32];
+  double s = 0.0;
+  for (int i = threadIdx.x; i < n; i += 1024) s += block_norm2[i];
+  s = warp_sum(s);
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    s = 0.0;
+    for (int w = 0; w < 32; ++w) s += sh[w];
   }
-  for (; i < n; i += 256) s0 += block_norm2[i];
-  double s = (s0 + s1) + (s2 + s3);
-  s = block_sum_256(s, sh, threadIdx.x);
   if (threadIdx.x == 0) {
     const double nrm = sqrt(s);
     const double cap = 2.0 * static_cast<double>(q) / (nrm + static_cast<double>(eps));

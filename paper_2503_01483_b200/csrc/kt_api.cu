@@ -595,7 +595,7 @@ static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, 
   k_skew<<<tgrid, tblock, 0, ctx->stream>>>(fbuf, d, w_hi, max_terms == 3 ? w_lo : nullptr,
                                             at<double>(ctx, L.norm_blocks));
   KT_LAUNCH_CHECK();
-  k_step_size<<<1, 256, 0, ctx->stream>>>(at<double>(ctx, L.norm_blocks), L.norm_n, lr, c.q, c.eps, sc, d, s,
+  k_step_size<<<1, 1024, 0, ctx->stream>>>(at<double>(ctx, L.norm_blocks), L.norm_n, lr, c.q, c.eps, sc, d, s,
                                           cfg_terms, cfg_terms == 0 ? 1 : 0, guard_mode, c.polish_thresh);
   KT_LAUNCH_CHECK();
 
