@@ -309,15 +309,19 @@ def main():
     peaks = measured_peaks()
     g = prof["gemm"]
     per_role = {k: (g[k]["ms"] / g[k]["launches"] if g[k]["launches"] else None) for k in g}
-    share = {k: g[k]["ms"] / ms for k in g}
+    # every step launches exactly one forward (or one single-pass) kernel: the steps the event window covered
+    # (it holds 8192 launches; the 80-layer sweep overruns it, and then the split describes the steps it holds)
+    steps_seen = max(g["fused"]["launches"] or g["forward"]["launches"], 1)
+    share = {k: g[k]["ms"] / steps_seen / ms_per_step for k in g}
     if g["fused"]["launches"] > 0:
         # d = 128: the single-pass kernel reads X once; HBM bound.  Algorithmic bytes per launch = N * d * 2.
         t_f = g["fused"]["ms"] / g["fused"]["launches"] * 1e-3
         alg_bytes = 2.0 * N * d
         achieved = alg_bytes / t_f / 1e9
         peak = peaks["hbm_gbs"]
-        # DRAM bytes per launch: ncu capture at 1 048 576 rows (272.0 MB for 268.4 MB algorithmic), scaled by N
-        traffic = alg_bytes * (272.0 / 268.435)
+        # DRAM bytes per launch: ncu capture at 1 048 576 rows (268.4 MB algorithmic; read + written 272.8 MB with
+        # R as two bf16 terms, the default, and 272.0 MB with one), scaled by N
+        traffic = alg_bytes * ((272.0 if args.forward_terms == 1 else 272.8) / 268.435)
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "traffic": traffic,
                     "kernel": "fused_small_kernel (loss + gradient in one pass over X): N*d*2 bytes per launch",
@@ -335,7 +339,7 @@ def main():
         if args.workload == "llama2_7b_attn":
             # mean DRAM bytes per launch of the three kernels: ncu capture at N = 16384 (same d); the part that
             # grows with N (everything but the 33.5 MB of R^T read by forward and backward-A) is scaled by N / 16384
-            var_mb = (167.8 + 7.7 - 33.5) + (172.4 + 117.0 - 33.5) + (683.9 + 62.0)
+            var_mb = (167.8 + 7.3 - 33.5) + (174.8 + 116.5 - 33.5) + (683.8 + 62.2)
             traffic = (var_mb * (N / 16384.0) + 2 * 33.5) / 3.0 * 1e6
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                     "frac": (achieved / peak) if achieved else None, "traffic": traffic,
