@@ -193,6 +193,8 @@ def main():
     ap.add_argument("--rows", type=int, default=0, help="override N (profiling on a small case)")
     ap.add_argument("--layers", type=int, default=80, help="layers of the llama3_70b_sweep workload")
     ap.add_argument("--forward-terms", type=int, default=0, help="kt_config.forward_terms (0 = automatic)")
+    ap.add_argument("--optimizer", default="sgd", choices=["sgd", "adam"],
+                    help="kt_config.optimizer: Cayley SGD (the headline configuration) or Cayley Adam")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -233,7 +235,7 @@ def main():
         X = torch.roll(X, shifts=rank * 977, dims=0).contiguous()
     N = X.shape[0]
     lr = cfg["lr"]
-    ctx = kurtail.Context(dev, forward_terms=args.forward_terms)
+    ctx = kurtail.Context(dev, forward_terms=args.forward_terms, optimizer=1 if args.optimizer == "adam" else 0)
 
     def fresh_R():
         if cfg["init"] == "hadamard":
@@ -354,6 +356,7 @@ def main():
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": args.workload, "N": N, "d": d, "R_init": cfg["init"], "lr": lr,
+                   "optimizer": "cayley_" + args.optimizer,
                    "l2": "inputs (%.0f MiB of X per step) exceed the 126 MB L2" % (N * d * 2 / 2**20)
                    if N * d * 2 > 126e6 else "inputs fit in L2; no flush (small case)",
                    "parallelism": "one independent layer per GPU" if world > 1 else "single GPU",

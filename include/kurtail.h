@@ -101,6 +101,12 @@ typedef struct {
                            launch in float32 on the CUDA cores (128 CTAs; the
                            device must have at least 128 SMs free) instead of
                            about twenty tensor-core launches; 0 = general path  */
+  int32_t optimizer;    /* [0]   kt_fit: 0 = Cayley SGD (kt_orth_step per step);
+                           1 = Cayley Adam (kt_adam_step per step; the
+                           workspace then also holds the d x d momentum)       */
+  float beta1;          /* [0.9]  Cayley Adam: decay of the momentum M          */
+  float beta2;          /* [0.99] Cayley Adam: decay of the scalar second moment */
+  float adam_eps;       /* [1e-8] Cayley Adam: added under the square root      */
   int32_t reserved[2];
 } kt_config;
 
@@ -181,10 +187,33 @@ kt_status kt_rotate(kt_ctx* ctx, kt_mat X, const float* R, float* Y);
  * d).  Stream ordered. */
 kt_status kt_orth_step(kt_ctx* ctx, float* R, const float* dR, int64_t d, float lr);
 
+/* Cayley Adam (Section 3, "Optimization in the Orthogonal Space", names it as
+ * the optimiser of the paper's runs and defers to the publication it cites;
+ * the update below is that publication's algorithm for a square orthogonal
+ * R).  With k = st->step + 1:
+ *   M <- beta1 M + (1 - beta1) dR;   v <- beta2 v + (1 - beta2) ||dR||_F^2;
+ *   r = (1 - beta1^k) sqrt(v / (1 - beta2^k) + adam_eps);
+ *   W = (M R^T - R M^T) / (2 r);     M <- r W R   (momentum back on the tangent space);
+ *   alpha = min(lr, 2q/(||W||_F + eps)); then the same fixed-point iteration
+ *   and guard as kt_orth_step, started from Y0 = R - alpha W R.
+ * R (device, d x d) and M (device, d x d float32, caller-owned, zero before
+ * the first step) are updated in place; dR is read only.  *st (host) carries
+ * v and the step count between calls: zero it before the first step; it is
+ * read on entry and written on return.  beta1, beta2, adam_eps come from the
+ * context's configuration.  Always runs the general tensor-core path.  Uses
+ * the workspace (sized for any N >= 1 and this d).  Synchronises. */
+typedef struct {
+  double v;        /* running mean of ||dR||_F^2 */
+  int32_t step;    /* steps taken so far */
+  int32_t reserved;
+} kt_adam_state;
+kt_status kt_adam_step(kt_ctx* ctx, float* R, const float* dR, float* M, kt_adam_state* st, int64_t d, float lr);
+
 /* *err (host) = max|R^T R - I|.  Uses the workspace.  Synchronises. */
 kt_status kt_orth_error(kt_ctx* ctx, const float* R, int64_t d, double* err);
 
-/* `steps` x (kt_loss_grad; kt_orth_step) on the context's stream with no host
+/* `steps` x (kt_loss_grad; kt_orth_step) -- or kt_adam_step from a zero state
+ * when kt_config.optimizer == 1 -- on the context's stream with no host
  * synchronisation in between; bit-identical to composing those calls when
  * guard_every == 1 (with the default 0 the two differ only in which steps
  * measure orthogonality).  R in/out.  `report` (host) may be NULL.  Synchronises at

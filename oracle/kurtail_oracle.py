@@ -33,8 +33,10 @@ What follows the paper, and where:
 Parity status: every function above is pinned by tests/test_oracle_pins.py
 against closed forms, invariants, finite differences, library routines or
 brute force.  Cayley *Adam* (``cayley_adam_step``) is "parity unpinned" as far
-as the paper goes: its constants and exact form are nowhere in the paper; it is
-pinned only by invariants (orthogonality, reduction to the SGD step).
+as the paper goes: its constants and exact form are nowhere in the paper.  As a
+restatement of the cited publication's algorithm it is pinned by its reduction
+to the SGD step (first step; zero decays), by the scalar recursion followed by
+hand at d = 2, and by invariants (orthogonality, tangency of the momentum).
 
 All floating point is float64 except the quantizer, which works in float32
 because the integer codes are decided in float32 on both sides.
@@ -206,9 +208,15 @@ def fit(X, R, steps, lr, kappa_target=KAPPA_UNIFORM, iters=2, q=0.5, eps=1e-8, p
 
 def cayley_adam_step(R, dR, state, lr, beta1=0.9, beta2=0.99, adam_eps=1e-8,
                      iters=2, q=0.5, eps=1e-8, polish_thresh=0.0):
-    """Cayley Adam (published algorithm of Li et al. 2020, square orthogonal
-    case).  PARITY UNPINNED against the paper: the paper names the optimiser
-    only.  state = dict(M=d x d, v=scalar, k=step count)."""
+    """Cayley Adam (Section 3, "Optimization in the Orthogonal Space", names the
+    optimiser only; the update is the algorithm of the publication it cites, Li
+    et al. 2020, for a square orthogonal R, with the fixed-point iteration
+    started from Y0 = R - alpha W R as in cayley_stepwise).
+    state = dict(M=d x d, v=scalar, k=step count), updated in place.
+    Pins (tests): reduction to the SGD step along G/||G|| on the first step and
+    with zero decays, the scalar recursion followed by hand at d = 2, tangency
+    of M and orthogonality.  What no test can pin is the paper's own choice of
+    beta1, beta2, learning rate and iteration count: it prints none."""
     R = np.asarray(R, dtype=np.float64)
     dR = np.asarray(dR, dtype=np.float64)
     state["k"] += 1

@@ -26,7 +26,10 @@ struct Scalars {
   unsigned int p0_terms;    // bf16 terms of R used for P_0 = W R
   unsigned int gate_guard;  // 1 = this step measures R^T R - I
   float drift;              // bound on the orthogonality error accumulated since the last measurement
-  unsigned int pad[2];
+  unsigned int adam_k;      // Cayley Adam: steps taken
+  unsigned int pad;
+  double adam_v;            // Cayley Adam: running mean of ||dR||_F^2
+  double adam_r;            // Cayley Adam: (1 - beta1^k) sqrt(v / (1 - beta2^k) + eps) of the current step
 };
 
 constexpr float kDegenerateRel = 1e-6f;
@@ -250,16 +253,76 @@ __global__ void k_sum_splits(const float* __restrict__ part, int splits, long lo
   *reinterpret_cast<float4*>(out + i4) = acc;
 }
 
+// --------------------------------------------------------------- Cayley Adam
+// M <- beta1 M + (1 - beta1) dR, m_hi = bf16(M), and per-block sums of dR^2.
+// grid (d/32, d/32), block (32, 8).
+__global__ void k_adam_moment(float* __restrict__ M, const float* __restrict__ dR, float beta1, int d,
+                              __nv_bfloat16* __restrict__ m_hi, double* __restrict__ block_g2) {
+  __shared__ double sh[8];
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  float mv[4], gv[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const long long o = static_cast<long long>(r0 + ty + 8 * q) * d + c0 + tx;
+    mv[q] = M[o];
+    gv[q] = dR[o];
+  }
+  double acc = 0.0;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const long long o = static_cast<long long>(r0 + ty + 8 * q) * d + c0 + tx;
+    const float m = fmaf(beta1, mv[q], (1.f - beta1) * gv[q]);
+    M[o] = m;
+    m_hi[o] = __float2bfloat16_rn(m);
+    acc += static_cast<double>(gv[q]) * gv[q];
+  }
+  const int lin = ty * 32 + tx;
+  acc = block_sum_256(acc, sh, lin);
+  if (lin == 0) block_g2[blockIdx.y * gridDim.x + blockIdx.x] = acc;
+}
+
+// One block of 1024 threads: ||dR||_F^2 in fixed order, then the scalar recurrences of Cayley Adam.
+__global__ void k_adam_scalars(const double* __restrict__ block_g2, int n, float beta1, float beta2, float adam_eps,
+                               Scalars* __restrict__ sc) {
+  __shared__ double sh[32];
+  double s = 0.0;
+  for (int i = threadIdx.x; i < n; i += 1024) s += block_g2[i];
+  s = warp_sum(s);
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    s = 0.0;
+    for (int w = 0; w < 32; ++w) s += sh[w];
+    const unsigned int k = sc->adam_k + 1u;
+    const double b1 = static_cast<double>(beta1), b2 = static_cast<double>(beta2);
+    const double v = b2 * sc->adam_v + (1.0 - b2) * s;
+    const double vhat = v / (1.0 - pow(b2, static_cast<double>(k)));
+    sc->adam_k = k;
+    sc->adam_v = v;
+    sc->adam_r = (1.0 - pow(b1, static_cast<double>(k))) * sqrt(vhat + static_cast<double>(adam_eps));
+  }
+}
+
+// Loads the Cayley Adam state that lives on the host between kt_adam_step calls.
+__global__ void k_adam_set(Scalars* sc, double v, unsigned int k) {
+  sc->adam_v = v;
+  sc->adam_k = k;
+}
+
 // ------------------------------------------------------------- Cayley pieces
-// W = (A - A^T)/2 for a d x d float32 A, written as bf16 hi (and lo when asked;
+// W = (A - A^T)/2 (divided by adam->adam_r when `adam` is given) for a d x d float32 A, written as bf16 hi (and lo when asked;
 // the rounding is odd, so each bf16 part is exactly skew), plus per-block sums of W^2 (of the float32 W).
 // grid (d/32, d/32), block (32, 8).
 __global__ void k_skew(const float* __restrict__ A, int d, __nv_bfloat16* __restrict__ w_hi,
-                       __nv_bfloat16* __restrict__ w_lo, double* __restrict__ block_norm2) {
+                       __nv_bfloat16* __restrict__ w_lo, double* __restrict__ block_norm2,
+                       const Scalars* __restrict__ adam) {
   __shared__ float tT[32][33];
   __shared__ double sh[8];
   const int bj = blockIdx.x, bi = blockIdx.y;
   const int tx = threadIdx.x, ty = threadIdx.y;
+  // Cayley Adam divides the skew part by r (same float for (i, j) and (j, i): W stays exactly skew)
+  const float half_scale = adam ? static_cast<float>(0.5 / adam->adam_r) : 0.5f;
   // eight independent loads per thread: four of tile (bi, bj), four of tile (bj, bi) (to be read transposed)
   float av[4], tv[4];
 #pragma unroll
@@ -275,7 +338,7 @@ __global__ void k_skew(const float* __restrict__ A, int d, __nv_bfloat16* __rest
   for (int q = 0; q < 4; ++q) {
     const int r = ty + 8 * q;
     const long long o = static_cast<long long>(bi * 32 + r) * d + bj * 32 + tx;
-    const float w = 0.5f * (av[q] - tT[tx][r]);
+    const float w = half_scale * (av[q] - tT[tx][r]);
     __nv_bfloat16 h, l;
     split_bf16(w, h, l);
     w_hi[o] = h;
@@ -356,10 +419,12 @@ __global__ void k_force_guard(Scalars* sc) {
 // Y_k = R - alpha/2 W (R + Y_{k-1})).  This kernel adds term k in place, R += c_k P with
 // c_k = -alpha (-alpha/2)^k.  Terms k >= sc->n_terms do nothing.  A term that is not the last one evaluated writes
 // P^T as bf16 (pt_hi) for the next product; the last one writes the bf16 forms of the new R instead: r_hi (as is),
-// rt_hi/rt_lo (transposed hi/lo).  grid (d/32, min(d/32, 32)), block (32, 8); each block walks row tiles.
+// rt_hi/rt_lo (transposed hi/lo).  adam_m != null (given with k = 0 only): also M <- adam_r * P.
+// grid (d/32, min(d/32, 32)), block (32, 8); each block walks row tiles.
 __global__ void k_series_term(float* __restrict__ R, const float* __restrict__ P, const Scalars* __restrict__ sc,
                               int k, int d, __nv_bfloat16* __restrict__ pt_hi, __nv_bfloat16* __restrict__ r_hi,
-                              __nv_bfloat16* __restrict__ rt_hi, __nv_bfloat16* __restrict__ rt_lo) {
+                              __nv_bfloat16* __restrict__ rt_hi, __nv_bfloat16* __restrict__ rt_lo,
+                              float* __restrict__ adam_m) {
   const unsigned int n_terms = sc->n_terms;
   if (static_cast<unsigned int>(k) >= n_terms) return;
   const bool last = (static_cast<unsigned int>(k) + 1u == n_terms);
@@ -369,6 +434,7 @@ __global__ void k_series_term(float* __restrict__ R, const float* __restrict__ P
   const float alpha = sc->alpha;
   float ck = -alpha;
   for (int i = 0; i < k; ++i) ck *= -0.5f * alpha;
+  const float adam_r = adam_m ? static_cast<float>(sc->adam_r) : 0.f;
   for (int r0 = blockIdx.y * 32; r0 < d; r0 += gridDim.y * 32) {
     float pv[4], rv[4], rn[4];
 #pragma unroll
@@ -383,6 +449,7 @@ __global__ void k_series_term(float* __restrict__ R, const float* __restrict__ P
       const long long o = static_cast<long long>(r0 + r) * d + c0 + tx;
       rn[q] = fmaf(ck, pv[q], rv[q]);
       R[o] = rn[q];
+      if (adam_m) adam_m[o] = adam_r * pv[q];  // Cayley Adam (k = 0 only): M <- r W R
       tile[r][tx] = last ? rn[q] : pv[q];
       if (last) r_hi[o] = __float2bfloat16_rn(rn[q]);
     }

@@ -85,12 +85,13 @@ struct WsLayout {
   size_t diag;          // [d] float: exact diagonal of R^T R - I
   size_t splitk;        // [splits][d][d] float: partial dR of the split-K backward-B (when splits > 1)
   size_t small;         // d <= 512: scratch of the one-launch orthogonal step (5 d x d floats + per-CTA partials)
+  size_t adam_m;        // d x d float32: momentum of Cayley Adam inside kt_fit (only when asked for)
   size_t total;
   long long ldt;
   int P, bn, loss_blocks, norm_n;
 };
 
-static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype) {
+static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, bool adam = false) {
   WsLayout L;
   memset(&L, 0, sizeof(L));
   L.bn = (d % 256 == 0) ? 256 : 128;
@@ -136,6 +137,7 @@ static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype) {
     L.splitk = take(static_cast<size_t>(parts) * dd * 4);
   }
   L.small = take(d <= 512 ? 5 * dd * 4 + 4096 : 0);
+  L.adam_m = take(adam ? dd * 4 : 0);
   L.total = off;
   return L;
 }
@@ -558,9 +560,10 @@ static kt_status small_orth_step_async(kt_ctx* ctx, float* R, const float* dR, i
 // second step of kt_fit on: the previous step left them).  On return they hold the forms of the new R.
 // guard_mode: 1 = measure R^T R - I (and polish if needed) in this step, 2 = do not, 0 = let the device decide from
 // its drift bound (see k_step_size).
+// adam_m != null: Cayley Adam (momentum buffer; v and the step count live in the device scalar block).
 static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, float lr, const WsLayout& L,
-                                 int guard_mode, bool forms_current, bool adaptive = false) {
-  if (use_small_orth(ctx, d)) return small_orth_step_async(ctx, R, dR, d, lr, L, guard_mode != 2);
+                                 int guard_mode, bool forms_current, bool adaptive = false, float* adam_m = nullptr) {
+  if (!adam_m && use_small_orth(ctx, d)) return small_orth_step_async(ctx, R, dR, d, lr, L, guard_mode != 2);
   const kt_config& c = ctx->cfg;
   Scalars* sc = &ctx->d_blk->sc;
   const uint64_t ld = static_cast<uint64_t>(d);
@@ -578,9 +581,18 @@ static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, 
   const int s = c.cayley_iters < 0 ? 0 : c.cayley_iters;
 
   // A = dR R^T (the gradient needs no more than bf16), W = (A - A^T)/2, alpha and the step's gates
-  k_split_bf16<false><<<tgrid, tblock, 0, ctx->stream>>>(dR, d, z_hi /* dR hi: free until P^T is written */, nullptr,
-                                                         d);
-  KT_LAUNCH_CHECK();
+  if (adam_m) {
+    // Cayley Adam: the direction comes from the momentum M <- beta1 M + (1 - beta1) dR, scaled by 1/r
+    k_adam_moment<<<tgrid, tblock, 0, ctx->stream>>>(adam_m, dR, c.beta1, d, z_hi, at<double>(ctx, L.norm_blocks));
+    KT_LAUNCH_CHECK();
+    k_adam_scalars<<<1, 1024, 0, ctx->stream>>>(at<double>(ctx, L.norm_blocks), L.norm_n, c.beta1, c.beta2, c.adam_eps,
+                                                sc);
+    KT_LAUNCH_CHECK();
+  } else {
+    k_split_bf16<false><<<tgrid, tblock, 0, ctx->stream>>>(dR, d, z_hi /* dR hi: free until P^T is written */,
+                                                           nullptr, d);
+    KT_LAUNCH_CHECK();
+  }
   if (!forms_current) {
     k_split_r<<<tgrid, tblock, 0, ctx->stream>>>(R, d, r_hi, rt_hi, rt_lo);
     KT_LAUNCH_CHECK();
@@ -593,7 +605,7 @@ static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, 
     KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 1, &A, &B, p, kCatSquare));
   }
   k_skew<<<tgrid, tblock, 0, ctx->stream>>>(fbuf, d, w_hi, max_terms == 3 ? w_lo : nullptr,
-                                            at<double>(ctx, L.norm_blocks));
+                                            at<double>(ctx, L.norm_blocks), adam_m ? sc : nullptr);
   KT_LAUNCH_CHECK();
   k_step_size<<<1, 1024, 0, ctx->stream>>>(at<double>(ctx, L.norm_blocks), L.norm_n, lr, c.q, c.eps, sc, d, s,
                                           cfg_terms, cfg_terms == 0 ? 1 : 0, guard_mode, c.polish_thresh);
@@ -617,7 +629,8 @@ static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, 
       Operand A{w_hi, ld}, B{z_hi, ld};
       KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 1, &A, &B, p, kCatSquare));
     }
-    k_series_term<<<lgrid, tblock, 0, ctx->stream>>>(R, fbuf, sc, k, d, z_hi, r_hi, rt_hi, rt_lo);
+    k_series_term<<<lgrid, tblock, 0, ctx->stream>>>(R, fbuf, sc, k, d, z_hi, r_hi, rt_hi, rt_lo,
+                                                     k == 0 ? adam_m : nullptr);
     KT_LAUNCH_CHECK();
   }
   if (guard_mode != 2) {
@@ -648,9 +661,17 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
   KT_TRY(check_x(X, &N64, &d64));
   if (R == nullptr || steps < 0) return KT_ERR_INVALID_ARG;
   if (!aligned16(R)) return KT_ERR_ALIGN;
-  const WsLayout L = make_layout(N64, d64, X.dtype);
+  const bool adam = ctx->cfg.optimizer == 1;
+  const WsLayout L = make_layout(N64, d64, X.dtype, adam);
   KT_TRY(check_ws(ctx, L));
   const int N = static_cast<int>(N64), d = static_cast<int>(d64);
+  float* adam_m = nullptr;
+  if (adam) {  // every fit starts Cayley Adam from a zero state
+    adam_m = at<float>(ctx, L.adam_m);
+    KT_CUDA(cudaMemsetAsync(adam_m, 0, static_cast<size_t>(d) * d * 4, ctx->stream));
+    k_adam_set<<<1, 1, 0, ctx->stream>>>(&ctx->d_blk->sc, 0.0, 0u);
+    KT_LAUNCH_CHECK();
+  }
   XView xv;
   const bool fused = use_fused(ctx, d);
   if (fused) KT_TRY(ingest_x_forward(ctx, X, L, &xv)); else KT_TRY(ingest_x_full(ctx, X, L, &xv));
@@ -681,7 +702,7 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
       guard_mode = (((k + 1) % ge == 0) || (k + 1 == steps)) ? 1 : 2;
     else
       guard_mode = (k == 0 || k + 1 == steps) ? 1 : 0;
-    KT_TRY(orth_step_async(ctx, R, dR, d, lr, L, guard_mode, k > 0, ctx->cfg.guard_every < 1));
+    KT_TRY(orth_step_async(ctx, R, dR, d, lr, L, guard_mode, k > 0, ctx->cfg.guard_every < 1, adam_m));
     done = k + 1;
   }
   if (steps > 0) {
@@ -731,6 +752,10 @@ void kt_default_config(kt_config* cfg) {
   cfg->forward_terms = 0;
   cfg->small_d_fused = 1;
   cfg->small_d_orth = 1;
+  cfg->optimizer = 0;
+  cfg->beta1 = 0.9f;
+  cfg->beta2 = 0.99f;
+  cfg->adam_eps = 1e-8f;
 }
 
 const char* kt_status_string(kt_status s) {
@@ -807,12 +832,11 @@ void kt_destroy(kt_ctx* ctx) {
 }
 
 kt_status kt_workspace_bytes(const kt_ctx* ctx, int64_t N, int64_t d, int32_t x_dtype, size_t* bytes) {
-  (void)ctx;
   if (!bytes) return KT_ERR_INVALID_ARG;
   if (x_dtype != KT_BF16 && x_dtype != KT_F32) return KT_ERR_INVALID_ARG;
   if (N < 1 || N > 0x7fffff00ll) return KT_ERR_SHAPE;
   KT_TRY(check_d(d));
-  *bytes = make_layout(N, d, x_dtype).total;
+  *bytes = make_layout(N, d, x_dtype, ctx != nullptr && ctx->cfg.optimizer == 1).total;
   return KT_OK;
 }
 
@@ -915,6 +939,24 @@ kt_status kt_orth_step(kt_ctx* ctx, float* R, const float* dR, int64_t d, float 
   return orth_step_async(ctx, R, dR, static_cast<int>(d), lr, L, 1, false);
 }
 
+kt_status kt_adam_step(kt_ctx* ctx, float* R, const float* dR, float* M, kt_adam_state* st, int64_t d, float lr) {
+  if (!ctx || !R || !dR || !M || !st || !(lr >= 0.f) || st->step < 0 || !(st->v >= 0.0)) return KT_ERR_INVALID_ARG;
+  const kt_config& c = ctx->cfg;
+  if (!(c.beta1 >= 0.f && c.beta1 < 1.f) || !(c.beta2 >= 0.f && c.beta2 < 1.f) || !(c.adam_eps > 0.f))
+    return KT_ERR_INVALID_ARG;
+  KT_TRY(check_d(d));
+  if (!aligned16(R) || !aligned16(dR) || !aligned16(M)) return KT_ERR_ALIGN;
+  const WsLayout L = make_layout(1, d, KT_BF16);
+  KT_TRY(check_ws(ctx, L));
+  k_adam_set<<<1, 1, 0, ctx->stream>>>(&ctx->d_blk->sc, st->v, static_cast<unsigned int>(st->step));
+  KT_LAUNCH_CHECK();
+  KT_TRY(orth_step_async(ctx, R, dR, static_cast<int>(d), lr, L, 1, false, false, M));
+  KT_TRY(sync_scalars(ctx));
+  st->v = ctx->h_blk->sc.adam_v;
+  st->step = static_cast<int32_t>(ctx->h_blk->sc.adam_k);
+  return KT_OK;
+}
+
 kt_status kt_orth_error(kt_ctx* ctx, const float* R, int64_t d, double* err) {
   if (!ctx || !R || !err) return KT_ERR_INVALID_ARG;
   KT_TRY(check_d(d));
@@ -967,7 +1009,7 @@ kt_status kt_fit_host(kt_ctx* ctx, kt_mat X_host, void* X_dev_staging, float* R_
   KT_TRY(check_x(Xd, &N, &d));
   if (X_host.data == nullptr) return KT_ERR_INVALID_ARG;
   if (!aligned16(R_dev)) return KT_ERR_ALIGN;
-  const WsLayout L = make_layout(N, d, Xd.dtype);
+  const WsLayout L = make_layout(N, d, Xd.dtype, ctx->cfg.optimizer == 1);
   KT_TRY(check_ws(ctx, L));
   const size_t es = (Xd.dtype == KT_BF16) ? 2 : 4;
   KT_CUDA(cudaMemcpyAsync(X_dev_staging, X_host.data, static_cast<size_t>(N) * Xd.ld * es, cudaMemcpyHostToDevice,

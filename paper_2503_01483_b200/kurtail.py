@@ -34,7 +34,13 @@ class kt_mat(C.Structure):
 class kt_config(C.Structure):
     _fields_ = [("kappa_target", C.c_float), ("cayley_iters", C.c_int32), ("q", C.c_float), ("eps", C.c_float),
                 ("polish_thresh", C.c_float), ("retract_terms", C.c_int32), ("guard_every", C.c_int32),
-                ("forward_terms", C.c_int32), ("small_d_fused", C.c_int32), ("small_d_orth", C.c_int32), ("reserved", C.c_int32 * 2)]
+                ("forward_terms", C.c_int32), ("small_d_fused", C.c_int32), ("small_d_orth", C.c_int32),
+                ("optimizer", C.c_int32), ("beta1", C.c_float), ("beta2", C.c_float), ("adam_eps", C.c_float),
+                ("reserved", C.c_int32 * 2)]
+
+
+class kt_adam_state(C.Structure):
+    _fields_ = [("v", C.c_double), ("step", C.c_int32), ("reserved", C.c_int32)]
 
 
 class kt_fit_report(C.Structure):
@@ -49,7 +55,7 @@ class kt_profile(C.Structure):
 
 EXPORTS = ["kt_default_config", "kt_create", "kt_destroy", "kt_status_string", "kt_workspace_bytes",
            "kt_set_workspace", "kt_init_rotation", "kt_kurtosis_loss", "kt_loss_grad", "kt_row_moments",
-           "kt_rotate", "kt_orth_step", "kt_orth_error", "kt_fit", "kt_fit_layers", "kt_fit_host",
+           "kt_rotate", "kt_orth_step", "kt_adam_step", "kt_orth_error", "kt_fit", "kt_fit_layers", "kt_fit_host",
            "kt_quant4_error", "kt_quant4_codes", "kt_profile_begin", "kt_profile_end",
            "kt_kurtosis_loss_noalloc"]
 
@@ -82,6 +88,7 @@ def lib():
     L.kt_row_moments.argtypes = [vp, kt_mat, vp, vp]
     L.kt_rotate.argtypes = [vp, kt_mat, vp, vp]
     L.kt_orth_step.argtypes = [vp, vp, vp, i64, f32]
+    L.kt_adam_step.argtypes = [vp, vp, vp, vp, C.POINTER(kt_adam_state), i64, f32]
     L.kt_orth_error.argtypes = [vp, vp, i64, dp]
     L.kt_fit.argtypes = [vp, kt_mat, vp, i32, f32, C.POINTER(kt_fit_report)]
     L.kt_fit_layers.argtypes = [vp, C.POINTER(kt_mat), C.POINTER(vp), i32, i32, i32, f32, C.POINTER(kt_fit_report)]
@@ -224,6 +231,16 @@ class Context:
         d = R.shape[0]
         self.ensure_workspace(1, d, KT_BF16)
         _check(lib().kt_orth_step(self._h, R.data_ptr(), dR.data_ptr(), d, lr), "kt_orth_step")
+        return R
+
+    def adam_step(self, R, dR, M, state, lr):
+        """kt_adam_step.  `state` is a dict(v=float, step=int), zero before the first step; updated in place."""
+        d = R.shape[0]
+        self.ensure_workspace(1, d, KT_BF16)
+        st = kt_adam_state(float(state["v"]), int(state["step"]), 0)
+        _check(lib().kt_adam_step(self._h, R.data_ptr(), dR.data_ptr(), M.data_ptr(), C.byref(st), d, lr),
+               "kt_adam_step")
+        state["v"], state["step"] = st.v, st.step
         return R
 
     def orth_error(self, R):

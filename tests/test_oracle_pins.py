@@ -280,6 +280,65 @@ def test_cayley_adam_invariants():
         assert abs((st["M"] * Rprev).sum()) < 1e-12  # momentum is tangent at the old point: <W R, R> = 0
 
 
+def test_cayley_adam_first_step_is_scale_free_normalised_sgd():
+    # From a zero state the bias corrections cancel the decays: M = (1 - b1) G, r = (1 - b1) ||G||_F, so
+    # W = skew(G R^T) / ||G||_F whatever b1, b2 and the scale of G are: the first step equals the (pinned) SGD step
+    # along G / ||G||_F.  A missing bias correction, a wrong power or a misplaced square root breaks this.
+    rng = np.random.default_rng(15)
+    d = 10
+    R = scipy.stats.ortho_group.rvs(d, random_state=10)
+    G = rng.normal(size=(d, d))
+    want, _, _ = ko.orth_step(R, G / np.linalg.norm(G), 3e-2, polish_thresh=0.0)
+    for b1, b2, scale in [(0.9, 0.99, 1.0), (0.5, 0.999, 1e3), (0.0, 0.0, 1e-3)]:
+        st = dict(M=np.zeros((d, d)), v=0.0, k=0)
+        got = ko.cayley_adam_step(R, scale * G, st, 3e-2, beta1=b1, beta2=b2, adam_eps=1e-30)
+        assert np.abs(got - want).max() < 1e-12
+        assert st["k"] == 1 and st["v"] == pytest.approx((1 - b2) * scale ** 2 * (G * G).sum(), rel=1e-12)
+        # the stored momentum is the tangent projection of (1 - b1) G: r W R = (1 - b1) skew(G R^T) R
+        assert np.abs(st["M"] - (1 - b1) * scale * ko.skew_direction(R, G) @ R).max() < 1e-12 * scale
+
+
+def test_cayley_adam_without_decay_is_normalised_sgd_every_step():
+    # b1 = b2 = 0: no memory; each step is SGD along G / sqrt(||G||^2 + eps)
+    rng = np.random.default_rng(16)
+    d = 6
+    R = scipy.stats.ortho_group.rvs(d, random_state=11)
+    st = dict(M=rng.normal(size=(d, d)), v=123.0, k=7)  # stale state must not matter
+    for _ in range(3):
+        G = rng.normal(size=(d, d))
+        want, _, _ = ko.orth_step(R, G / np.sqrt((G * G).sum() + 1e-8), 1e-2, polish_thresh=0.0)
+        R = ko.cayley_adam_step(R, G, st, 1e-2, beta1=0.0, beta2=0.0, adam_eps=1e-8)
+        assert np.abs(R - want).max() < 1e-12
+
+
+def test_cayley_adam_second_moment_and_momentum_recurrences_d2():
+    # d = 2: every skew matrix is w J, so the whole recursion is scalar and can be followed by hand.
+    # With R_k = rotation(theta_k) and G = g_k J R_k: skew(G R_k^T) = g_k J.  The stored momentum m_{k-1} J R_{k-1} sits
+    # at the previous point; seen from R_k its skew part is m_{k-1} cos(theta_k - theta_{k-1}) J (the algorithm does
+    # no parallel transport), so m_k = b1 m_{k-1} cos(dtheta_{k-1}) + (1-b1) g_k; v_k = b2 v_{k-1} + (1-b2) 2 g_k^2;
+    # w_k = m_k / r_k; theta moves by the angle of the s-step iterate.
+    J = np.array([[0.0, -1.0], [1.0, 0.0]])
+    th = 0.3
+    R = np.array([[np.cos(th), -np.sin(th)], [np.sin(th), np.cos(th)]])
+    b1, b2, eps_a, lr = 0.8, 0.95, 1e-12, 1e-3
+    st = dict(M=np.zeros((2, 2)), v=0.0, k=0)
+    m = v = dth = 0.0
+    for k, g in enumerate([2.0, -1.0, 0.5], start=1):
+        G = g * J @ R
+        Rn = ko.cayley_adam_step(R, G, st, lr, beta1=b1, beta2=b2, adam_eps=eps_a, polish_thresh=np.inf)
+        m = b1 * m * np.cos(dth) + (1 - b1) * g
+        v = b2 * v + (1 - b2) * 2 * g * g
+        r = (1 - b1 ** k) * np.sqrt(v / (1 - b2 ** k) + eps_a)
+        w = m / r
+        alpha = min(lr, 2 * 0.5 / (abs(w) * np.sqrt(2) + 1e-8))
+        assert st["v"] == pytest.approx(v, rel=1e-13)
+        assert np.abs(st["M"] - m * J @ R).max() < 1e-13      # r * (w J) R = m J R
+        # exact Cayley rotates by -2 atan(alpha w / 2); the two-iteration form differs at order (alpha w / 2)^3
+        dth = np.arctan2(Rn[1, 0], Rn[0, 0]) - np.arctan2(R[1, 0], R[0, 0])
+        assert dth == pytest.approx(-2 * np.arctan(alpha * w / 2), abs=2 * abs(alpha * w / 2) ** 3 + 1e-15)
+        R = Rn
+
+
 # ---------------- quantizer ----------------
 def _golden_quant_cases():
     rows, codes = [], []
