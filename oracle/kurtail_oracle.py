@@ -17,6 +17,10 @@ What follows the paper, and where:
   readings list in the design notes for why.
 * ``loss_grad``  -- the derivative of that loss through Y = X R (Section 3,
   "Learning the Rotations": the rotation is the weight of a linear layer).
+* ``kurtosis_loss_flat`` / ``loss_grad_flat``  -- the same loss equation read
+  literally: kappa of the concatenation of all tokens' activations of the layer.
+  ``rmsnorm_rows`` / ``small_network``  -- Section 3, "Learning the Rotations":
+  the trained network is the linear layer followed by an RMSNorm.
 * ``skew_direction``, ``cayley_exact``, ``cayley_stepwise``, ``orth_step`` --
   Section 3, "Optimization in the Orthogonal Space": Cayley SGD on the
   Stiefel manifold.  The paper gives the method by citation only (Li et al.
@@ -119,6 +123,45 @@ def loss_grad(X, R, kappa_target=KAPPA_UNIFORM):
     G = (sgn / N)[:, None] * dk
     L = float((np.where(deg, 0.0, np.abs(kappa - kappa_target))).sum() / N)
     return L, X.T @ G
+
+
+# --------------------------------------------------------------------------
+# The loss equation of Section 2 taken literally: one kurtosis per layer over
+# the concatenation of all tokens' activations; and the RMSNorm of the small
+# network of Section 3, "Learning the Rotations"
+# --------------------------------------------------------------------------
+def rmsnorm_rows(X, rms_eps=1e-6):
+    """Unit-gain RMSNorm of each row: x / sqrt(mean(x^2) + rms_eps)."""
+    X = np.asarray(X, dtype=np.float64)
+    return X / np.sqrt((X * X).mean(axis=1, keepdims=True) + rms_eps)
+
+
+def small_network(X, R, rms_eps=1e-6):
+    """The network the paper trains for R1: a linear layer (the rotation)
+    followed by an RMSNorm (unit gain)."""
+    return rmsnorm_rows(rotate(X, R), rms_eps)
+
+
+def kurtosis_flat(Y):
+    """Eq. 3 over all N*n entries of Y as one sample.  NaN when Y has no spread."""
+    v = np.asarray(Y, dtype=np.float64).reshape(1, -1)
+    return float(kurtosis_rows(v)[0])
+
+
+def kurtosis_loss_flat(X, R, kappa_target=KAPPA_UNIFORM):
+    """|kappa(concatenation over tokens of Y_t) - kappa_u|, Y = X R (one layer, L = 1)."""
+    k = kurtosis_flat(rotate(X, R))
+    return 0.0 if np.isnan(k) else abs(k - kappa_target)
+
+
+def loss_grad_flat(X, R, kappa_target=KAPPA_UNIFORM):
+    """(L, dR) of kurtosis_loss_flat: the per-row derivative of loss_grad with
+    the row replaced by the whole layer (n = N*d entries, one mean, one set of
+    moments): dL/dY = sgn(kappa - kappa_u) 4/(n m2^2) (c^3 - m3 - kappa m2 c)."""
+    X = np.asarray(X, dtype=np.float64)
+    Y = rotate(X, R)
+    g = loss_dY(Y.reshape(1, -1), kappa_target).reshape(Y.shape)
+    return kurtosis_loss_flat(X, R, kappa_target), X.T @ g
 
 
 def loss_dY(Y, kappa_target=KAPPA_UNIFORM):

@@ -339,6 +339,82 @@ def test_cayley_adam_second_moment_and_momentum_recurrences_d2():
         R = Rn
 
 
+# ---------------- flattened (whole-layer) kurtosis and the RMSNorm ----------------
+def test_flat_kurtosis_library_and_closed_forms():
+    rng = np.random.default_rng(21)
+    Y = rng.standard_t(5, size=(37, 12)) + 0.3
+    assert ko.kurtosis_flat(Y) == pytest.approx(scipy.stats.kurtosis(Y.ravel(), fisher=False, bias=True), rel=1e-12)
+    # the integers 0..n-1 laid out as a matrix: 3 - 1.2 (n^2 + 1)/(n^2 - 1)
+    n = 24 * 16
+    assert ko.kurtosis_flat(np.arange(n, dtype=float).reshape(24, 16)) == pytest.approx(
+        3 - 1.2 * (n * n + 1) / (n * n - 1), rel=1e-12)
+    # one token: the layer is the row
+    X = rng.normal(size=(1, 16)); R = scipy.stats.ortho_group.rvs(16, random_state=3)
+    assert ko.kurtosis_loss_flat(X, R) == pytest.approx(ko.kurtosis_loss(X, R), rel=1e-13)
+    # rows with different means and scales: not the mean of the rows' kurtoses
+    Y2 = np.vstack([rng.normal(size=(1, 4000)), 10 + 5 * rng.normal(size=(1, 4000))])
+    assert abs(ko.kurtosis_flat(Y2) - np.nanmean(ko.kurtosis_rows(Y2))) > 0.3
+    assert np.isnan(ko.kurtosis_flat(np.full((3, 4), 2.5)))
+    assert ko.kurtosis_loss_flat(np.zeros((4, 4)), np.eye(4)) == 0.0
+
+
+def test_flat_gradient_finite_differences_and_orthogonality_to_r():
+    rng = np.random.default_rng(22)
+    N, d = 12, 6
+    X = rng.standard_t(4, size=(N, d)); X[:, 2] *= 7
+    R = scipy.stats.ortho_group.rvs(d, random_state=4) + 0.01 * rng.normal(size=(d, d))
+    L, dR = ko.loss_grad_flat(X, R)
+    assert L == pytest.approx(ko.kurtosis_loss_flat(X, R), rel=1e-14)
+    h = 1e-6
+    num = np.zeros_like(dR)
+    for i in range(d):
+        for j in range(d):
+            E = np.zeros((d, d)); E[i, j] = h
+            num[i, j] = (ko.kurtosis_loss_flat(X, R + E) - ko.kurtosis_loss_flat(X, R - E)) / (2 * h)
+    assert np.abs(num - dR).max() <= 1e-6 * np.abs(dR).max()
+    # kurtosis is scale and shift invariant: <Y, dL/dY> = 0 and sum dL/dY = 0, hence <R, dR> = 0
+    assert abs((R * dR).sum()) <= 1e-12 * np.abs(dR).sum()
+    # below the target the sign flips (uniform-ish data, kappa < 1.8 needs a two-point law)
+    Xl = rng.choice([-1.0, 1.0], size=(N, d)) + 0.01 * rng.normal(size=(N, d))
+    Ll, dRl = ko.loss_grad_flat(Xl, np.eye(d))
+    assert ko.kurtosis_flat(Xl) < 1.8
+    E = 1e-6 * rng.normal(size=(d, d))
+    num = (ko.kurtosis_loss_flat(Xl, np.eye(d) + E) - ko.kurtosis_loss_flat(Xl, np.eye(d) - E)) / 2
+    assert num == pytest.approx((dRl * E).sum(), rel=1e-4)
+
+
+def test_rmsnorm_commutes_with_a_rotation_and_drops_out_of_the_tangent_gradient():
+    rng = np.random.default_rng(23)
+    N, d = 10, 8
+    X = rng.standard_t(3, size=(N, d)); X[:, 1] *= 20
+    R = scipy.stats.ortho_group.rvs(d, random_state=5)
+    Z = ko.rmsnorm_rows(X, rms_eps=0.0)
+    assert np.allclose((Z * Z).mean(axis=1), 1.0, rtol=1e-13)
+    assert np.allclose(ko.rmsnorm_rows(3.7 * X, rms_eps=0.0), Z, rtol=1e-13)
+    eps = 1e-6
+    # orthogonal R keeps row norms: RMSNorm(X R) = RMSNorm(X) R
+    assert np.abs(ko.small_network(X, R, eps) - ko.rmsnorm_rows(X, eps) @ R).max() <= 1e-13
+    # Along any direction that stays on the group, R(t) = (I - t W) R with W skew, the row norms do not change to
+    # first order, so the derivative of the loss of the true network (linear layer, then RMSNorm) equals the one
+    # computed from the pre-normalised X with the RMSNorm left out:  d/dt = -<dR_pre, W R>.
+    _, dR_pre = ko.loss_grad_flat(ko.rmsnorm_rows(X, eps), R)
+    _, dR_row = ko.loss_grad(ko.rmsnorm_rows(X, eps), R)
+    for seed in range(3):
+        A = np.random.default_rng(seed).normal(size=(d, d))
+        W = A - A.T
+        t = 1e-6
+
+        def net_loss(tt, flat):
+            Y = ko.small_network(X, (np.eye(d) - tt * W) @ R, eps)
+            if flat:
+                return abs(ko.kurtosis_flat(Y) - ko.KAPPA_UNIFORM)
+            return float(np.abs(ko.kurtosis_rows(Y) - ko.KAPPA_UNIFORM).mean())
+
+        for flat, g in ((True, dR_pre), (False, dR_row)):
+            num = (net_loss(t, flat) - net_loss(-t, flat)) / (2 * t)
+            assert num == pytest.approx(-(g * (W @ R)).sum(), rel=1e-5, abs=1e-9)
+
+
 # ---------------- quantizer ----------------
 def _golden_quant_cases():
     rows, codes = [], []
