@@ -195,6 +195,9 @@ def main():
     ap.add_argument("--forward-terms", type=int, default=0, help="kt_config.forward_terms (0 = automatic)")
     ap.add_argument("--optimizer", default="sgd", choices=["sgd", "adam"],
                     help="kt_config.optimizer: Cayley SGD (the headline configuration) or Cayley Adam")
+    ap.add_argument("--loss-mode", default="token", choices=["token", "layer"],
+                    help="kt_config.loss_mode: one kurtosis per token (headline) or one over the whole layer")
+    ap.add_argument("--rmsnorm", action="store_true", help="kt_config.rmsnorm: row-normalise X first")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -235,7 +238,8 @@ def main():
         X = torch.roll(X, shifts=rank * 977, dims=0).contiguous()
     N = X.shape[0]
     lr = cfg["lr"]
-    ctx = kurtail.Context(dev, forward_terms=args.forward_terms, optimizer=1 if args.optimizer == "adam" else 0)
+    ctx = kurtail.Context(dev, forward_terms=args.forward_terms, optimizer=1 if args.optimizer == "adam" else 0,
+                          loss_mode=1 if args.loss_mode == "layer" else 0, rmsnorm=1 if args.rmsnorm else 0)
 
     def fresh_R():
         if cfg["init"] == "hadamard":
@@ -356,7 +360,7 @@ def main():
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": args.workload, "N": N, "d": d, "R_init": cfg["init"], "lr": lr,
-                   "optimizer": "cayley_" + args.optimizer,
+                   "optimizer": "cayley_" + args.optimizer, "loss_mode": args.loss_mode, "rmsnorm": bool(args.rmsnorm),
                    "l2": "inputs (%.0f MiB of X per step) exceed the 126 MB L2" % (N * d * 2 / 2**20)
                    if N * d * 2 > 126e6 else "inputs fit in L2; no flush (small case)",
                    "parallelism": "one independent layer per GPU" if world > 1 else "single GPU",

@@ -107,6 +107,19 @@ typedef struct {
   float beta1;          /* [0.9]  Cayley Adam: decay of the momentum M          */
   float beta2;          /* [0.99] Cayley Adam: decay of the scalar second moment */
   float adam_eps;       /* [1e-8] Cayley Adam: added under the square root      */
+  int32_t loss_mode;    /* [0]   0 = one kurtosis per token (row) over its d
+                           entries, loss = mean over tokens; 1 = the loss
+                           equation of Section 2 taken literally: one kurtosis
+                           over the concatenation of all N d entries of the
+                           layer, loss = |kappa - kappa_target| (zero rows are
+                           then part of the distribution; d == 128 uses the
+                           general path)                                        */
+  int32_t rmsnorm;      /* [0]   1 = every call that takes X first replaces it by
+                           its row-normalised bf16 copy x / sqrt(mean(x^2) +
+                           rms_eps) in the workspace: the unit-gain RMSNorm of
+                           the small network of Section 3, "Learning the
+                           Rotations", which commutes with an orthogonal R     */
+  float rms_eps;        /* [1e-6] */
   int32_t reserved[2];
 } kt_config;
 

@@ -205,6 +205,115 @@ __global__ void k_moments_finalize(const float4* __restrict__ partial, int P, in
   }
 }
 
+// ------------------------------------------- flattened (whole-layer) kurtosis
+// The loss of Section 2 taken literally: one kurtosis over the concatenation of all tokens' entries (N*d values).
+// The rows' means and central moments (k_moments_finalize) are merged in two fixed-order passes: the global mean
+// first, then the central sums about it with the exact shift formulas, all in float64.
+// Stage 1: per-block sums of the row means.  grid ceil(N/256), block 256.
+__global__ void k_flat_mean(const float4* __restrict__ moments, int N, double* __restrict__ block_out) {
+  __shared__ double sh[8];
+  const int row = blockIdx.x * 256 + threadIdx.x;
+  const double v = (row < N) ? static_cast<double>(moments[row].x) : 0.0;
+  const double b = block_sum_256(v, sh, threadIdx.x);
+  if (threadIdx.x == 0) block_out[blockIdx.x] = b;
+}
+
+// Stage 2: per-block sums of the rows' second, third and fourth central moments shifted to the global mean *mean.
+// grid ceil(N/256), block 256; b2/b3/b4 hold one double per block.
+__global__ void k_flat_central(const float4* __restrict__ moments, int N, const double* __restrict__ mean,
+                               double* __restrict__ b2, double* __restrict__ b3, double* __restrict__ b4) {
+  __shared__ double sh[8];
+  const int row = blockIdx.x * 256 + threadIdx.x;
+  double s2 = 0.0, s3 = 0.0, s4 = 0.0;
+  if (row < N) {
+    const float4 m = moments[row];
+    const double dl = static_cast<double>(m.x) - *mean, dl2 = dl * dl;
+    s2 = m.y + dl2;
+    s3 = m.z + 3.0 * dl * m.y + dl2 * dl;
+    s4 = m.w + 4.0 * dl * m.z + 6.0 * dl2 * m.y + dl2 * dl2;
+  }
+  s2 = block_sum_256(s2, sh, threadIdx.x);
+  s3 = block_sum_256(s3, sh, threadIdx.x);
+  s4 = block_sum_256(s4, sh, threadIdx.x);
+  if (threadIdx.x == 0) {
+    b2[blockIdx.x] = s2;
+    b3[blockIdx.x] = s3;
+    b4[blockIdx.x] = s4;
+  }
+}
+
+// One block of 256 threads: global m2, m3, m4, kappa, the loss |kappa - kappa_t| and the coefficients of
+// dL/dY = a c^3 - ab c - am3 with c = Y - mean and a = sgn 4/(N d m2^2) (one kurtosis over n = N d values).
+// A layer with (numerically) no variance gives loss 0, zero coefficients and deg_rows = N.
+__global__ void k_flat_finalize(const double* __restrict__ b2, const double* __restrict__ b3,
+                                const double* __restrict__ b4, int nb, int N, int d, float kappa_t,
+                                const double* __restrict__ mean, Scalars* __restrict__ sc,
+                                double* __restrict__ hist_slot, float4* __restrict__ coef_global) {
+  __shared__ double sh[8];
+  double s2 = 0.0, s3 = 0.0, s4 = 0.0;
+  for (int i = threadIdx.x; i < nb; i += 256) {
+    s2 += b2[i];
+    s3 += b3[i];
+    s4 += b4[i];
+  }
+  s2 = block_sum_256(s2, sh, threadIdx.x);
+  s3 = block_sum_256(s3, sh, threadIdx.x);
+  s4 = block_sum_256(s4, sh, threadIdx.x);
+  if (threadIdx.x == 0) {
+    const double mu = *mean;
+    const double m2 = s2 / N, m3 = s3 / N, m4 = s4 / N;
+    const double ms = m2 + mu * mu;
+    float4 cf = make_float4(static_cast<float>(mu), 0.f, 0.f, 0.f);
+    double loss = 0.0;
+    unsigned int deg = 0u;
+    if (ms == 0.0 || m2 <= static_cast<double>(kDegenerateRel) * ms) {
+      deg = static_cast<unsigned int>(N);
+    } else {
+      const double kappa = m4 / (m2 * m2);
+      const double diff = kappa - static_cast<double>(kappa_t);
+      loss = fabs(diff);
+      const double sgn = (diff > 0.0) ? 1.0 : ((diff < 0.0) ? -1.0 : 0.0);
+      const double a = sgn * 4.0 / (static_cast<double>(N) * d * m2 * m2);
+      cf.y = static_cast<float>(a);
+      cf.z = static_cast<float>(a * m4 / m2);
+      cf.w = static_cast<float>(a * m3);
+    }
+    *coef_global = cf;
+    sc->loss = loss;
+    sc->deg_rows = deg;
+    if (hist_slot) *hist_slot = loss;
+  }
+}
+
+// Every row gets the layer's coefficients.  grid ceil(N/256), block 256.
+__global__ void k_flat_fill(const float4* __restrict__ coef_global, int N, float4* __restrict__ coef) {
+  const int row = blockIdx.x * 256 + threadIdx.x;
+  if (row < N) coef[row] = *coef_global;
+}
+
+// ------------------------------------------------------- RMSNorm of the rows
+// xb[t][:] = bf16( X[t][:] / sqrt(mean_j X[t][j]^2 + eps) ) -- the RMSNorm (unit gain) that follows the rotation in
+// the paper's small network (Section 3, "Learning the Rotations"); an orthogonal R keeps every row's norm, so it
+// can be applied to X once.  One block of 256 threads per row; T = float or bf16; xb dense N x d.
+template <typename T>
+__global__ void k_rmsnorm_rows(const T* __restrict__ X, long long ld, int d, float eps,
+                               __nv_bfloat16* __restrict__ xb) {
+  __shared__ double sh[8];
+  __shared__ float scale_sh;
+  const T* x = X + static_cast<long long>(blockIdx.x) * ld;
+  float part = 0.f;  // at most d/256 terms per thread in float32, the 256 partials in float64
+  for (int j = threadIdx.x; j < d; j += 256) {
+    const float v = to_f32(x[j]);
+    part = fmaf(v, v, part);
+  }
+  double acc = block_sum_256(static_cast<double>(part), sh, threadIdx.x);
+  if (threadIdx.x == 0) scale_sh = static_cast<float>(1.0 / sqrt(acc / d + static_cast<double>(eps)));
+  __syncthreads();
+  const float sc = scale_sh;
+  __nv_bfloat16* o = xb + static_cast<long long>(blockIdx.x) * d;
+  for (int j = threadIdx.x; j < d; j += 256) o[j] = __float2bfloat16_rn(to_f32(x[j]) * sc);
+}
+
 // One block: *dst = scale * sum(vals[0..n)) (also to *dst2 when not null);
 // *count_dst = sum(counts) when counts != null.
 __global__ void k_final_sum(const double* __restrict__ vals, int n, double scale, double* __restrict__ dst,

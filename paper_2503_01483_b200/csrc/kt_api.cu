@@ -75,7 +75,7 @@ struct WsLayout {
   size_t w_hi, w_lo;    // skew direction W as bf16
   size_t fbuf;          // d x d float32: A, then P, then R^T R, then R E
   size_t dr;            // d x d float32: gradient inside kt_fit
-  size_t xb;            // dense bf16 copy of a float32 X  [N][d]
+  size_t xb;            // dense bf16 copy of a float32 X, or of any X after RMSNorm  [N][d]
   size_t xt, gt;        // X^T and G^T as bf16  [d][ldt]
   size_t partial;       // [P][N] float4 partial moment records
   size_t coef, moments; // [N] float4 each
@@ -86,12 +86,16 @@ struct WsLayout {
   size_t splitk;        // [splits][d][d] float: partial dR of the split-K backward-B (when splits > 1)
   size_t small;         // d <= 512: scratch of the one-launch orthogonal step (5 d x d floats + per-CTA partials)
   size_t adam_m;        // d x d float32: momentum of Cayley Adam inside kt_fit (only when asked for)
+  size_t flat;          // flattened-kurtosis mode: the global coefficients, the global mean, 3 x [blocks] doubles
   size_t total;
   long long ldt;
   int P, bn, loss_blocks, norm_n;
 };
 
-static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, bool adam = false) {
+// cfg == null: the default configuration (no momentum buffer, no normalised copy of a bf16 X).
+static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, const kt_config* cfg = nullptr) {
+  const bool adam = cfg != nullptr && cfg->optimizer == 1;
+  const bool xcopy = x_dtype == KT_F32 || (cfg != nullptr && cfg->rmsnorm != 0);
   WsLayout L;
   memset(&L, 0, sizeof(L));
   L.bn = (d % 256 == 0) ? 256 : 128;
@@ -116,7 +120,7 @@ static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, bool adam = f
   L.w_lo = take(dd * 2);
   L.fbuf = take(dd * 4);
   L.dr = take(dd * 4);
-  L.xb = take(x_dtype == KT_F32 ? static_cast<size_t>(N) * d * 2 : 0);
+  L.xb = take(xcopy ? static_cast<size_t>(N) * d * 2 : 0);
   L.xt = take(static_cast<size_t>(d) * L.ldt * 2);
   L.gt = take(static_cast<size_t>(d) * L.ldt * 2);
   L.partial = take(static_cast<size_t>(L.P) * N * 16);
@@ -138,6 +142,7 @@ static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, bool adam = f
   }
   L.small = take(d <= 512 ? 5 * dd * 4 + 4096 : 0);
   L.adam_m = take(adam ? dd * 4 : 0);
+  L.flat = take(static_cast<size_t>(L.loss_blocks) * 8 * 3 + 64);
   L.total = off;
   return L;
 }
@@ -284,8 +289,26 @@ struct XView {
 };
 
 // forward-only view: bf16 X is used in place, float32 X is rounded into the workspace
+// RMSNorm mode: the row-normalised bf16 copy of X (any dtype) that every later kernel reads instead of X.
+static kt_status rmsnorm_x(kt_ctx* ctx, const kt_mat& X, const WsLayout& L, XView* v) {
+  const int d = static_cast<int>(X.cols);
+  __nv_bfloat16* xb = at<__nv_bfloat16>(ctx, L.xb);
+  const unsigned rows = static_cast<unsigned>(X.rows);
+  if (X.dtype == KT_BF16)
+    k_rmsnorm_rows<__nv_bfloat16><<<rows, 256, 0, ctx->stream>>>(static_cast<const __nv_bfloat16*>(X.data), X.ld, d,
+                                                                 ctx->cfg.rms_eps, xb);
+  else
+    k_rmsnorm_rows<float><<<rows, 256, 0, ctx->stream>>>(static_cast<const float*>(X.data), X.ld, d, ctx->cfg.rms_eps,
+                                                         xb);
+  KT_LAUNCH_CHECK();
+  v->xb = xb;
+  v->ldx = d;
+  return KT_OK;
+}
+
 static kt_status ingest_x_forward(kt_ctx* ctx, const kt_mat& X, const WsLayout& L, XView* v) {
   const int64_t N = X.rows, d = X.cols;
+  if (ctx->cfg.rmsnorm != 0) return rmsnorm_x(ctx, X, L, v);
   if (X.dtype == KT_BF16) {
     v->xb = static_cast<const __nv_bfloat16*>(X.data);
     v->ldx = X.ld;
@@ -306,7 +329,11 @@ static kt_status ingest_x_full(kt_ctx* ctx, const kt_mat& X, const WsLayout& L, 
   const int N = static_cast<int>(X.rows), d = static_cast<int>(X.cols);
   dim3 grid(d / 64, (N + 63) / 64), block(32, 8);
   __nv_bfloat16* xt = at<__nv_bfloat16>(ctx, L.xt);
-  if (X.dtype == KT_BF16) {
+  if (ctx->cfg.rmsnorm != 0) {
+    KT_TRY(rmsnorm_x(ctx, X, L, v));
+    k_prepare_x<__nv_bfloat16><<<grid, block, 0, ctx->stream>>>(v->xb, v->ldx, N, d, xt, L.ldt, nullptr);
+    KT_LAUNCH_CHECK();
+  } else if (X.dtype == KT_BF16) {
     k_prepare_x<__nv_bfloat16><<<grid, block, 0, ctx->stream>>>(static_cast<const __nv_bfloat16*>(X.data), X.ld, N, d,
                                                                 xt, L.ldt, nullptr);
     KT_LAUNCH_CHECK();
@@ -368,6 +395,30 @@ static kt_status forward_loss(kt_ctx* ctx, const XView& xv, int N, int d, const 
                                                             at<float4>(ctx, L.coef), at<double>(ctx, L.block_loss),
                                                             at<unsigned int>(ctx, L.block_deg));
   KT_LAUNCH_CHECK();
+  if (ctx->cfg.loss_mode == 1) {
+    // one kurtosis over all N d entries: merge the rows' moments, then hand every row the layer's coefficients
+    const int nb = L.loss_blocks;
+    // L.flat is 256-byte aligned: the float4 of global coefficients first (16-byte aligned), the mean at +16,
+    // the three per-block arrays from +64
+    float4* cg = at<float4>(ctx, L.flat);
+    double* mean = at<double>(ctx, L.flat + 16);
+    double* b2 = at<double>(ctx, L.flat + 64);
+    double* b3 = b2 + nb;
+    double* b4 = b3 + nb;
+    k_flat_mean<<<nb, 256, 0, ctx->stream>>>(at<float4>(ctx, L.moments), N, at<double>(ctx, L.block_loss));
+    KT_LAUNCH_CHECK();
+    k_final_sum<<<1, 256, 0, ctx->stream>>>(at<double>(ctx, L.block_loss), nb, 1.0 / N, mean, nullptr, nullptr,
+                                            nullptr);
+    KT_LAUNCH_CHECK();
+    k_flat_central<<<nb, 256, 0, ctx->stream>>>(at<float4>(ctx, L.moments), N, mean, b2, b3, b4);
+    KT_LAUNCH_CHECK();
+    k_flat_finalize<<<1, 256, 0, ctx->stream>>>(b2, b3, b4, nb, N, d, ctx->cfg.kappa_target, mean, &ctx->d_blk->sc,
+                                                hist_slot, cg);
+    KT_LAUNCH_CHECK();
+    k_flat_fill<<<nb, 256, 0, ctx->stream>>>(cg, N, at<float4>(ctx, L.coef));
+    KT_LAUNCH_CHECK();
+    return KT_OK;
+  }
   k_final_sum<<<1, 256, 0, ctx->stream>>>(at<double>(ctx, L.block_loss), L.loss_blocks, 1.0 / N, &ctx->d_blk->sc.loss,
                                           hist_slot, at<unsigned int>(ctx, L.block_deg), &ctx->d_blk->sc.deg_rows);
   KT_LAUNCH_CHECK();
@@ -410,7 +461,10 @@ static kt_status loss_grad_async(kt_ctx* ctx, const XView& xv, int N, int d, con
 }
 
 // d = 128: loss and gradient in one pass over X (fused_small_kernel), then fixed-order sums over the CTAs.
-static bool use_fused(const kt_ctx* ctx, int d) { return d == kFsD && ctx->cfg.small_d_fused != 0; }
+// (the single-pass kernel needs each row's coefficients before the row leaves the SM: per-token loss only)
+static bool use_fused(const kt_ctx* ctx, int d) {
+  return d == kFsD && ctx->cfg.small_d_fused != 0 && ctx->cfg.loss_mode == 0;
+}
 
 static kt_status fused_loss_grad_async(kt_ctx* ctx, const XView& xv, int N, const WsLayout& L, const float* R,
                                        float* dR, double* hist_slot, bool rt_current) {
@@ -662,7 +716,7 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
   if (R == nullptr || steps < 0) return KT_ERR_INVALID_ARG;
   if (!aligned16(R)) return KT_ERR_ALIGN;
   const bool adam = ctx->cfg.optimizer == 1;
-  const WsLayout L = make_layout(N64, d64, X.dtype, adam);
+  const WsLayout L = make_layout(N64, d64, X.dtype, &ctx->cfg);
   KT_TRY(check_ws(ctx, L));
   const int N = static_cast<int>(N64), d = static_cast<int>(d64);
   float* adam_m = nullptr;
@@ -756,6 +810,9 @@ void kt_default_config(kt_config* cfg) {
   cfg->beta1 = 0.9f;
   cfg->beta2 = 0.99f;
   cfg->adam_eps = 1e-8f;
+  cfg->loss_mode = 0;
+  cfg->rmsnorm = 0;
+  cfg->rms_eps = 1e-6f;
 }
 
 const char* kt_status_string(kt_status s) {
@@ -836,7 +893,7 @@ kt_status kt_workspace_bytes(const kt_ctx* ctx, int64_t N, int64_t d, int32_t x_
   if (x_dtype != KT_BF16 && x_dtype != KT_F32) return KT_ERR_INVALID_ARG;
   if (N < 1 || N > 0x7fffff00ll) return KT_ERR_SHAPE;
   KT_TRY(check_d(d));
-  *bytes = make_layout(N, d, x_dtype, ctx != nullptr && ctx->cfg.optimizer == 1).total;
+  *bytes = make_layout(N, d, x_dtype, ctx ? &ctx->cfg : nullptr).total;
   return KT_OK;
 }
 
@@ -864,7 +921,7 @@ kt_status kt_kurtosis_loss(kt_ctx* ctx, kt_mat X, const float* R, double* loss) 
   int64_t N, d;
   KT_TRY(check_x(X, &N, &d));
   if (!aligned16(R)) return KT_ERR_ALIGN;
-  const WsLayout L = make_layout(N, d, X.dtype);
+  const WsLayout L = make_layout(N, d, X.dtype, &ctx->cfg);
   KT_TRY(check_ws(ctx, L));
   XView xv;
   KT_TRY(ingest_x_forward(ctx, X, L, &xv));
@@ -880,7 +937,7 @@ kt_status kt_row_moments(kt_ctx* ctx, kt_mat X, const float* R, float* moments) 
   int64_t N, d;
   KT_TRY(check_x(X, &N, &d));
   if (!aligned16(R) || !aligned16(moments)) return KT_ERR_ALIGN;
-  const WsLayout L = make_layout(N, d, X.dtype);
+  const WsLayout L = make_layout(N, d, X.dtype, &ctx->cfg);
   KT_TRY(check_ws(ctx, L));
   XView xv;
   KT_TRY(ingest_x_forward(ctx, X, L, &xv));
@@ -896,7 +953,7 @@ kt_status kt_rotate(kt_ctx* ctx, kt_mat X, const float* R, float* Y) {
   int64_t N, d;
   KT_TRY(check_x(X, &N, &d));
   if (!aligned16(R) || !aligned16(Y)) return KT_ERR_ALIGN;
-  const WsLayout L = make_layout(N, d, X.dtype);
+  const WsLayout L = make_layout(N, d, X.dtype, &ctx->cfg);
   KT_TRY(check_ws(ctx, L));
   XView xv;
   KT_TRY(ingest_x_forward(ctx, X, L, &xv));
@@ -914,7 +971,7 @@ kt_status kt_loss_grad(kt_ctx* ctx, kt_mat X, const float* R, float* dR, double*
   int64_t N, d;
   KT_TRY(check_x(X, &N, &d));
   if (!aligned16(R) || !aligned16(dR)) return KT_ERR_ALIGN;
-  const WsLayout L = make_layout(N, d, X.dtype);
+  const WsLayout L = make_layout(N, d, X.dtype, &ctx->cfg);
   KT_TRY(check_ws(ctx, L));
   XView xv;
   if (use_fused(ctx, static_cast<int>(d))) {
@@ -934,7 +991,7 @@ kt_status kt_orth_step(kt_ctx* ctx, float* R, const float* dR, int64_t d, float 
   if (!ctx || !R || !dR || !(lr >= 0.f)) return KT_ERR_INVALID_ARG;
   KT_TRY(check_d(d));
   if (!aligned16(R) || !aligned16(dR)) return KT_ERR_ALIGN;
-  const WsLayout L = make_layout(1, d, KT_BF16);
+  const WsLayout L = make_layout(1, d, KT_BF16, &ctx->cfg);
   KT_TRY(check_ws(ctx, L));
   return orth_step_async(ctx, R, dR, static_cast<int>(d), lr, L, 1, false);
 }
@@ -946,7 +1003,7 @@ kt_status kt_adam_step(kt_ctx* ctx, float* R, const float* dR, float* M, kt_adam
     return KT_ERR_INVALID_ARG;
   KT_TRY(check_d(d));
   if (!aligned16(R) || !aligned16(dR) || !aligned16(M)) return KT_ERR_ALIGN;
-  const WsLayout L = make_layout(1, d, KT_BF16);
+  const WsLayout L = make_layout(1, d, KT_BF16, &ctx->cfg);
   KT_TRY(check_ws(ctx, L));
   k_adam_set<<<1, 1, 0, ctx->stream>>>(&ctx->d_blk->sc, st->v, static_cast<unsigned int>(st->step));
   KT_LAUNCH_CHECK();
@@ -961,7 +1018,7 @@ kt_status kt_orth_error(kt_ctx* ctx, const float* R, int64_t d, double* err) {
   if (!ctx || !R || !err) return KT_ERR_INVALID_ARG;
   KT_TRY(check_d(d));
   if (!aligned16(R)) return KT_ERR_ALIGN;
-  const WsLayout L = make_layout(1, d, KT_BF16);
+  const WsLayout L = make_layout(1, d, KT_BF16, &ctx->cfg);
   KT_TRY(check_ws(ctx, L));
   dim3 tgrid(static_cast<unsigned>(d / 32), static_cast<unsigned>(d / 32)), tblock(32, 8);
   k_split_bf16<true><<<tgrid, tblock, 0, ctx->stream>>>(R, d, at<__nv_bfloat16>(ctx, L.rt_hi),
@@ -1009,7 +1066,7 @@ kt_status kt_fit_host(kt_ctx* ctx, kt_mat X_host, void* X_dev_staging, float* R_
   KT_TRY(check_x(Xd, &N, &d));
   if (X_host.data == nullptr) return KT_ERR_INVALID_ARG;
   if (!aligned16(R_dev)) return KT_ERR_ALIGN;
-  const WsLayout L = make_layout(N, d, Xd.dtype, ctx->cfg.optimizer == 1);
+  const WsLayout L = make_layout(N, d, Xd.dtype, &ctx->cfg);
   KT_TRY(check_ws(ctx, L));
   const size_t es = (Xd.dtype == KT_BF16) ? 2 : 4;
   KT_CUDA(cudaMemcpyAsync(X_dev_staging, X_host.data, static_cast<size_t>(N) * Xd.ld * es, cudaMemcpyHostToDevice,

@@ -1,0 +1,126 @@
+"""Whole-layer (flattened) kurtosis mode and the RMSNorm pre-scaling on the GPU against the float64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import kurtail_oracle as ko
+from paper_2503_01483_b200 import kurtail, synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def f64(t):
+    return t.detach().to(torch.float32).cpu().numpy().astype(np.float64)
+
+
+def make_x(N, d, seed, dist="student_t", dtype=torch.bfloat16, n_out=4, scale=50.0):
+    return synth.activations(N, d, dist=dist, nu=3.0, n_outliers=n_out, outlier_scale=scale, seed=seed, dtype=dtype,
+                             device=DEV)
+
+
+def init_r(ctx, d, kind):
+    if kind == "orth":
+        return synth.random_orthogonal(d, seed=5, device=DEV).contiguous()
+    return ctx.init_rotation(d, kind)
+
+
+@pytest.fixture(scope="module")
+def flat():
+    c = kurtail.Context(DEV, loss_mode=1)
+    yield c
+    c.close()
+
+
+@pytest.mark.parametrize("N,d,init", [(2048, 256, "identity"), (1000, 256, "hadamard"), (700, 1024, "orth"),
+                                      (128 * 40 + 9, 128, "orth"), (333, 4096, "hadamard")])
+def test_flat_loss_and_gradient(flat, N, d, init):
+    X = make_x(N, d, seed=101)
+    R = init_r(flat, d, init)
+    L_ref, dR_ref = ko.loss_grad_flat(f64(X), f64(R))
+    assert abs(flat.kurtosis_loss(X, R) - L_ref) <= 1e-3 * abs(L_ref)
+    L, dR = flat.loss_grad(X, R)
+    assert abs(L - L_ref) <= 1e-3 * abs(L_ref)
+    assert np.linalg.norm(f64(dR) - dR_ref) <= 1e-2 * np.linalg.norm(dR_ref)
+    # shift and scale invariance of the kurtosis: <R, dR> = 0 (checked relative to the gradient's own size)
+    assert abs(float((R * dR).sum())) <= 1e-2 * float(dR.norm()) * float(R.norm()) / np.sqrt(d)
+
+
+def test_flat_differs_from_per_token_mode(flat):
+    # rows of very different scale: the layer's kurtosis is not the mean of the rows' kurtoses
+    X = make_x(1024, 256, seed=102)
+    X[::2] *= 8.0
+    R = flat.init_rotation(256, "hadamard")
+    per = kurtail.Context(DEV)
+    a, b = flat.kurtosis_loss(X, R), per.kurtosis_loss(X, R)
+    assert a == pytest.approx(ko.kurtosis_loss_flat(f64(X), f64(R)), rel=1e-3)
+    assert b == pytest.approx(ko.kurtosis_loss(f64(X), f64(R)), rel=1e-3)
+    assert abs(a - b) > 0.1 * b
+    per.close()
+
+
+def test_flat_float32_input_and_sign_below_target(flat):
+    # a two-point layer has kurtosis 1 < 1.8: the gradient points the other way
+    g = torch.Generator(device="cpu").manual_seed(7)
+    X = (torch.randint(0, 2, (512, 256), generator=g).float() * 2 - 1 + 0.05 * torch.randn((512, 256), generator=g))
+    X = X.to(DEV)
+    R = synth.random_orthogonal(256, seed=6, device=DEV).contiguous()
+    L, dR = flat.loss_grad(X, R)
+    Xb = f64(X.to(torch.bfloat16))          # float32 X is rounded to bf16 on entry
+    L_ref, dR_ref = ko.loss_grad_flat(Xb, f64(R))
+    assert abs(L - L_ref) <= 1e-3 * abs(L_ref)
+    assert np.linalg.norm(f64(dR) - dR_ref) <= 1e-2 * np.linalg.norm(dR_ref)
+
+
+def test_flat_layer_without_spread(flat):
+    X = torch.zeros((256, 256), dtype=torch.bfloat16, device=DEV)
+    R = flat.init_rotation(256, "identity")
+    L, dR = flat.loss_grad(X, R)
+    assert L == 0.0 and float(dR.abs().max()) == 0.0
+
+
+def test_flat_fit_descends_and_equals_composed_calls():
+    c = kurtail.Context(DEV, loss_mode=1, guard_every=1)
+    X = make_x(2048, 256, seed=103, n_out=8, scale=100.0)
+    Ra = c.init_rotation(256, "identity")
+    Rb = Ra.clone()
+    rep = c.fit(X, Ra, 6, 1e-2, history=True)
+    losses = []
+    for _ in range(6):
+        l, dR = c.loss_grad(X, Rb)
+        losses.append(l)
+        c.orth_step(Rb, dR, 1e-2)
+    assert torch.equal(Ra, Rb) and losses == rep["loss_history"]
+    assert rep["loss_history"][-1] < rep["loss_history"][0]
+    # from the identity the first steps run at the step-size cap (alpha ||W|| = 2q = 1), where one polish per step
+    # leaves more than the 1e-4 that the long runs settle to
+    assert ko.orthogonality_error(f64(Ra)) <= 1e-3
+    c.close()
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_rmsnorm_prescaling(mode, dtype):
+    c = kurtail.Context(DEV, loss_mode=mode, rmsnorm=1, rms_eps=1e-6)
+    N, d = 1500, 512
+    X = make_x(N, d, seed=104, dtype=dtype)
+    X[::3] *= 5.0
+    R = synth.random_orthogonal(d, seed=8, device=DEV).contiguous()
+    Xn = ko.rmsnorm_rows(f64(X), 1e-6)
+    # the library stores the normalised rows as bf16: the oracle is given the same rounding of its own float64 rows
+    Xn_b = torch.from_numpy(Xn).to(torch.bfloat16).to(torch.float64).numpy()
+    ref = ko.loss_grad_flat if mode == 1 else ko.loss_grad
+    L_ref, dR_ref = ref(Xn_b, f64(R))
+    L, dR = c.loss_grad(X, R)
+    assert abs(L - L_ref) <= 1e-3 * abs(L_ref)
+    assert np.linalg.norm(f64(dR) - dR_ref) <= 1e-2 * np.linalg.norm(dR_ref)
+    # and against the network as the paper draws it (linear layer, then RMSNorm), without any bf16 rounding of
+    # the normalised rows: same loss to the tolerance
+    Y = ko.small_network(f64(X), f64(R), 1e-6)
+    L_net = abs(ko.kurtosis_flat(Y) - 1.8) if mode == 1 else float(np.abs(ko.kurtosis_rows(Y) - 1.8).mean())
+    assert abs(L - L_net) <= 2e-3 * abs(L_net)
+    # rotated rows of the library: unit mean square, up to the bf16 rounding of the few channels that hold most of a
+    # row's energy (half an ulp is 2^-8 relative, twice that in the square)
+    Yg = f64(c.rotate(X, R))
+    assert np.allclose((Yg * Yg).mean(axis=1), 1.0, atol=1e-2)
+    c.close()
