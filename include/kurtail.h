@@ -107,6 +107,15 @@ typedef struct {
   float beta1;          /* [0.9]  Cayley Adam: decay of the momentum M          */
   float beta2;          /* [0.99] Cayley Adam: decay of the scalar second moment */
   float adam_eps;       /* [1e-8] Cayley Adam: added under the square root      */
+  int32_t norm_iters;   /* [2]   the per-step choices of retract_terms = 0 and
+                           guard_every = 0 depend on the size of W as an
+                           operator.  k >= 1: 2k products W v (a power
+                           iteration from a fixed vector) estimate ||W||_2
+                           from below; twice the estimate, capped by ||W||_F,
+                           is used.  0: ||W||_F alone (a strict bound, but
+                           loose by up to sqrt(d): more terms and more
+                           measurements than needed).  alpha always uses
+                           ||W||_F.  Ignored by the d <= 512 one-launch step   */
   int32_t loss_mode;    /* [0]   0 = one kurtosis per token (row) over its d
                            entries, loss = mean over tokens; 1 = the loss
                            equation of Section 2 taken literally: one kurtosis
@@ -134,6 +143,11 @@ typedef struct {
   float alpha_last;        /* step size used by the last step                   */
   float w_norm_last;       /* ||W||_F of the last step                          */
   double* loss_history;    /* optional host array of `steps` entries, or NULL   */
+  float w_op_last;         /* the size of W as an operator that the last step's
+                              choices used (see kt_config.norm_iters)           */
+  int32_t series_terms_last; /* series terms the last step evaluated            */
+  int32_t p0_terms_last;   /* bf16 terms of R in the last step's product W R    */
+  int32_t guards_run;      /* steps of this fit that measured R^T R - I         */
 } kt_fit_report;
 
 /* --- life cycle ---------------------------------------------------------- */

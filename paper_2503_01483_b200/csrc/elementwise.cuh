@@ -27,9 +27,11 @@ struct Scalars {
   unsigned int gate_guard;  // 1 = this step measures R^T R - I
   float drift;              // bound on the orthogonality error accumulated since the last measurement
   unsigned int adam_k;      // Cayley Adam: steps taken
-  unsigned int pad;
+  unsigned int guards;      // measurements of R^T R - I since the fit began
   double adam_v;            // Cayley Adam: running mean of ||dR||_F^2
   double adam_r;            // Cayley Adam: (1 - beta1^k) sqrt(v / (1 - beta2^k) + eps) of the current step
+  float wop;                // size of W as an operator used by the current step's choices
+  unsigned int pad;
 };
 
 constexpr float kDegenerateRel = 1e-6f;
@@ -459,7 +461,49 @@ __global__ void k_skew(const float* __restrict__ A, int d, __nv_bfloat16* __rest
   if (lin == 0) block_norm2[blockIdx.y * gridDim.x + blockIdx.x] = acc;
 }
 
-// One block of 1024 threads: ||W||_F, alpha = min(lr, 2q/(||W||_F + eps)), and the decisions that depend on x = alpha ||W||_F:
+// y = W v for the d x d bf16 matrix W (row-major) and a float32 vector v; v == null stands for a fixed vector of
+// +-1 entries (a hash of the index), the start of the power iteration below.  One warp per row, 8 rows per block:
+// grid d/8, block 256.  d is a multiple of 128 (each lane reads 8 consecutive bf16 = 16 bytes at a time).
+__device__ __forceinline__ float start_sign(int j) {
+  unsigned int h = static_cast<unsigned int>(j) * 2654435761u;
+  h ^= h >> 15;
+  h *= 2246822519u;
+  return ((h >> 13) & 1u) ? 1.f : -1.f;
+}
+__global__ void k_skew_matvec(const __nv_bfloat16* __restrict__ W, int d, const float* __restrict__ v,
+                              float* __restrict__ y) {
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const __nv_bfloat16* w = W + static_cast<long long>(row) * d;
+  float acc0 = 0.f, acc1 = 0.f;
+  for (int j = lane * 8; j < d; j += 256) {
+    const uint4 raw = *reinterpret_cast<const uint4*>(w + j);
+    const __nv_bfloat162* pr = reinterpret_cast<const __nv_bfloat162*>(&raw);
+    float vv[8];
+    if (v) {
+      const float4 a = *reinterpret_cast<const float4*>(v + j);
+      const float4 b = *reinterpret_cast<const float4*>(v + j + 4);
+      vv[0] = a.x; vv[1] = a.y; vv[2] = a.z; vv[3] = a.w;
+      vv[4] = b.x; vv[5] = b.y; vv[6] = b.z; vv[7] = b.w;
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) vv[e] = start_sign(j + e);
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float2 f = __bfloat1622float2(pr[e]);
+      acc0 = fmaf(f.x, vv[2 * e], acc0);
+      acc1 = fmaf(f.y, vv[2 * e + 1], acc1);
+    }
+  }
+  float acc = acc0 + acc1;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, o);
+  if (lane == 0) y[row] = acc;
+}
+
+// One block of 1024 threads: ||W||_F, alpha = min(lr, 2q/(||W||_F + eps)), and the decisions that depend on
+// x = alpha ||W||_2 (bounded by alpha ||W||_F; estimated by a short power iteration when pv_prev/pv_last are given):
 //  * n_terms: term k of the series changes R by at most x (x/2)^k (Frobenius bounds the spectral norm, ||R|| = 1);
 //    terms below a quarter unit in the last place of a typical entry (2^-26 / sqrt(d)) are skipped (`gate_terms`);
 //  * p0_terms: P_0 = W R multiplies alpha directly; with R as a single bf16 term its error is x 2^-9, which is
@@ -470,25 +514,44 @@ __global__ void k_skew(const float* __restrict__ A, int d, __nv_bfloat16* __rest
 //    P_0; float32 rounding of the update), has reached half the polish threshold.  A measuring step also clears the running maximum.
 __global__ void k_step_size(const double* __restrict__ block_norm2, int n, float lr, float q, float eps,
                             Scalars* __restrict__ sc, int d, int iters, int cfg_terms, int gate_terms, int guard_mode,
-                            float thresh) {
-  // 1024 threads; fixed-order sum: per-thread strided partial, warp shuffle tree, then the 32 warp sums in order
+                            float thresh, const float* __restrict__ pv_prev, const float* __restrict__ pv_last) {
+  // 1024 threads; fixed-order sums: per-thread strided partial, warp shuffle tree, then the 32 warp sums in order
   __shared__ double sh[32];
-  double s = 0.0;
-  for (int i = threadIdx.x; i < n; i += 1024) s += block_norm2[i];
-  s = warp_sum(s);
-  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = s;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    s = 0.0;
-    for (int w = 0; w < 32; ++w) s += sh[w];
+  __shared__ double tot[3];
+  for (int what = 0; what < 3; ++what) {
+    double s = 0.0;
+    if (what == 0) {
+      for (int i = threadIdx.x; i < n; i += 1024) s += block_norm2[i];
+    } else if (pv_prev) {
+      const float* v = (what == 1) ? pv_prev : pv_last;
+      for (int i = threadIdx.x; i < d; i += 1024) s += static_cast<double>(v[i]) * v[i];
+    }
+    s = warp_sum(s);
+    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      s = 0.0;
+      for (int w = 0; w < 32; ++w) s += sh[w];
+      tot[what] = s;
+    }
+    __syncthreads();
   }
   if (threadIdx.x == 0) {
-    const double nrm = sqrt(s);
+    const double nrm = sqrt(tot[0]);
     const double cap = 2.0 * static_cast<double>(q) / (nrm + static_cast<double>(eps));
     const double a = (static_cast<double>(lr) < cap) ? static_cast<double>(lr) : cap;
     sc->alpha = static_cast<float>(a);
     sc->wnorm = static_cast<float>(nrm);
-    const double x = a * nrm;
+    // The step itself uses ||W||_F (above).  The decisions below only need the size of W as an operator: when the
+    // power iteration ran, pv_last = W pv_prev, and ||pv_last|| / ||pv_prev|| <= ||W||_2 is its estimate from
+    // below; twice that (the iteration is short), capped by the Frobenius norm, stands in for ||W||_2.
+    double wop = nrm;
+    if (pv_prev && tot[1] > 0.0) {
+      const double est = 2.0 * sqrt(tot[2] / tot[1]);
+      if (est < wop) wop = est;
+    }
+    sc->wop = static_cast<float>(wop);
+    const double x = a * wop;
     unsigned int nt = 1;
     const double floor_k = ldexp(1.0, -26) / sqrt(static_cast<double>(d));
     double bound = x;
@@ -512,9 +575,15 @@ __global__ void k_step_size(const double* __restrict__ block_norm2, int n, float
       gg = (thresh <= 0.f || drift >= 0.5f * thresh) ? 1u : 0u;
     }
     sc->gate_guard = gg;
-    if (gg) sc->max_e_bits = 0u;
+    if (gg) {
+      sc->max_e_bits = 0u;
+      sc->guards += 1u;
+    }
   }
 }
+
+// Start of a fit: no measurement counted yet.
+__global__ void k_fit_begin(Scalars* sc) { sc->guards = 0u; }
 
 // Before a measurement outside a step (kt_orth_error): open the guard's gate and clear its running maximum.
 __global__ void k_force_guard(Scalars* sc) {

@@ -83,6 +83,7 @@ struct WsLayout {
   size_t rowmax, qerr;  // quantizer: [N] uint, [P][N] float
   size_t colpart;       // [d/32][d] float: column sums of squares of R by row slab
   size_t diag;          // [d] float: exact diagonal of R^T R - I
+  size_t pvec;          // [2][d] float: the last two vectors of the power iteration on W
   size_t splitk;        // [splits][d][d] float: partial dR of the split-K backward-B (when splits > 1)
   size_t small;         // d <= 512: scratch of the one-launch orthogonal step (5 d x d floats + per-CTA partials)
   size_t adam_m;        // d x d float32: momentum of Cayley Adam inside kt_fit (only when asked for)
@@ -134,6 +135,7 @@ static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, const kt_conf
   L.qerr = take(static_cast<size_t>(L.P) * N * 4);
   L.colpart = take(static_cast<size_t>(d / 32) * d * 4);
   L.diag = take(static_cast<size_t>(d) * 4);
+  L.pvec = take(static_cast<size_t>(d) * 4 * 2);
   {
     const SplitPlan sp = plan_split_k(d, N);
     int parts = sp.splits > 1 ? sp.splits : 0;
@@ -661,8 +663,23 @@ static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, 
   k_skew<<<tgrid, tblock, 0, ctx->stream>>>(fbuf, d, w_hi, max_terms == 3 ? w_lo : nullptr,
                                             at<double>(ctx, L.norm_blocks), adam_m ? sc : nullptr);
   KT_LAUNCH_CHECK();
+  // a short power iteration on W^T W = -W^2 (W is skew): v <- W v, 2 * norm_iters times from a fixed +-1 vector;
+  // the growth of the last application estimates ||W||_2 for the step's decisions (not for alpha)
+  const float* pv_prev = nullptr;
+  const float* pv_last = nullptr;
+  const int n_mv = c.norm_iters > 0 ? 2 * (c.norm_iters > 16 ? 16 : c.norm_iters) : 0;
+  if (n_mv > 0) {
+    float* pv[2] = {at<float>(ctx, L.pvec), at<float>(ctx, L.pvec) + d};
+    for (int i = 0; i < n_mv; ++i) {
+      k_skew_matvec<<<d / 8, 256, 0, ctx->stream>>>(w_hi, d, i == 0 ? nullptr : pv[(i + 1) & 1], pv[i & 1]);
+      KT_LAUNCH_CHECK();
+    }
+    pv_prev = pv[n_mv & 1];        // written by application n_mv - 2
+    pv_last = pv[(n_mv + 1) & 1];  // written by application n_mv - 1
+  }
   k_step_size<<<1, 1024, 0, ctx->stream>>>(at<double>(ctx, L.norm_blocks), L.norm_n, lr, c.q, c.eps, sc, d, s,
-                                          cfg_terms, cfg_terms == 0 ? 1 : 0, guard_mode, c.polish_thresh);
+                                          cfg_terms, cfg_terms == 0 ? 1 : 0, guard_mode, c.polish_thresh, pv_prev,
+                                          pv_last);
   KT_LAUNCH_CHECK();
 
   // P_0 = W R with R^T as a bf16 split (it multiplies alpha directly; the device picks one or two terms);
@@ -726,6 +743,8 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
     k_adam_set<<<1, 1, 0, ctx->stream>>>(&ctx->d_blk->sc, 0.0, 0u);
     KT_LAUNCH_CHECK();
   }
+  k_fit_begin<<<1, 1, 0, ctx->stream>>>(&ctx->d_blk->sc);
+  KT_LAUNCH_CHECK();
   XView xv;
   const bool fused = use_fused(ctx, d);
   if (fused) KT_TRY(ingest_x_forward(ctx, X, L, &xv)); else KT_TRY(ingest_x_full(ctx, X, L, &xv));
@@ -780,6 +799,10 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
     report->orth_err = static_cast<double>(__builtin_bit_cast(float, ctx->h_blk->sc.max_e_bits));
     report->alpha_last = ctx->h_blk->sc.alpha;
     report->w_norm_last = ctx->h_blk->sc.wnorm;
+    report->w_op_last = ctx->h_blk->sc.wop;
+    report->series_terms_last = static_cast<int32_t>(ctx->h_blk->sc.n_terms);
+    report->p0_terms_last = static_cast<int32_t>(ctx->h_blk->sc.p0_terms);
+    report->guards_run = static_cast<int32_t>(ctx->h_blk->sc.guards);
   }
   if (st != KT_OK) return st;
   if (steps > 0 && !isfinite(last)) return KT_ERR_NONFINITE;
@@ -810,6 +833,7 @@ void kt_default_config(kt_config* cfg) {
   cfg->beta1 = 0.9f;
   cfg->beta2 = 0.99f;
   cfg->adam_eps = 1e-8f;
+  cfg->norm_iters = 2;
   cfg->loss_mode = 0;
   cfg->rmsnorm = 0;
   cfg->rms_eps = 1e-6f;

@@ -120,6 +120,10 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
     if (blockIdx.x == 0 && threadIdx.x == 0) {
       p.sc->alpha = alpha;
       p.sc->wnorm = static_cast<float>(nrm);
+      p.sc->wop = static_cast<float>(nrm);  // this path evaluates every term in float32 and decides nothing
+      p.sc->n_terms = static_cast<unsigned int>(p.iters + 1);
+      p.sc->p0_terms = 0u;
+      if (p.run_guard) p.sc->guards += 1u;
     }
   }
 

@@ -36,7 +36,7 @@ class kt_config(C.Structure):
                 ("polish_thresh", C.c_float), ("retract_terms", C.c_int32), ("guard_every", C.c_int32),
                 ("forward_terms", C.c_int32), ("small_d_fused", C.c_int32), ("small_d_orth", C.c_int32),
                 ("optimizer", C.c_int32), ("beta1", C.c_float), ("beta2", C.c_float), ("adam_eps", C.c_float),
-                ("loss_mode", C.c_int32), ("rmsnorm", C.c_int32), ("rms_eps", C.c_float),
+                ("norm_iters", C.c_int32), ("loss_mode", C.c_int32), ("rmsnorm", C.c_int32), ("rms_eps", C.c_float),
                 ("reserved", C.c_int32 * 2)]
 
 
@@ -47,7 +47,8 @@ class kt_adam_state(C.Structure):
 class kt_fit_report(C.Structure):
     _fields_ = [("steps_done", C.c_int32), ("degenerate_rows", C.c_int32), ("loss_first", C.c_double),
                 ("loss_last", C.c_double), ("orth_err", C.c_double), ("alpha_last", C.c_float),
-                ("w_norm_last", C.c_float), ("loss_history", C.POINTER(C.c_double))]
+                ("w_norm_last", C.c_float), ("loss_history", C.POINTER(C.c_double)), ("w_op_last", C.c_float),
+                ("series_terms_last", C.c_int32), ("p0_terms_last", C.c_int32), ("guards_run", C.c_int32)]
 
 
 class kt_profile(C.Structure):
@@ -136,7 +137,9 @@ def as_mat(X: torch.Tensor) -> kt_mat:
 def _rep_dict(rep, hist):
     return dict(steps_done=rep.steps_done, degenerate_rows=rep.degenerate_rows, loss_first=rep.loss_first,
                 loss_last=rep.loss_last, orth_err=rep.orth_err, alpha_last=rep.alpha_last,
-                w_norm_last=rep.w_norm_last, loss_history=list(hist) if hist is not None else None)
+                w_norm_last=rep.w_norm_last, loss_history=list(hist) if hist is not None else None,
+                w_op_last=rep.w_op_last, series_terms_last=rep.series_terms_last, p0_terms_last=rep.p0_terms_last,
+                guards_run=rep.guards_run)
 
 
 def kurtosis_loss_noalloc(X, R, loss_dev, stream=None):
