@@ -24,6 +24,10 @@
 namespace kt {
 
 constexpr int kBM = 128;           // rows per tile = tensor-memory lanes
+#ifndef KT_GROUP_M
+#define KT_GROUP_M 16
+#endif
+constexpr int kGroupM = KT_GROUP_M;  // row tiles per group of the tile order
 constexpr int kBK = 64;            // k elements per pipeline stage (one 128-byte swizzle row)
 constexpr int kGemmThreads = 192;  // 6 warps
 constexpr int kMaxTerms = 3;
@@ -104,8 +108,23 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
   const int k_blocks = (p.K + kBK - 1) / kBK;
   // k-block range and MMA/TMA iteration count of work unit u
   // a tile whose last column is left of its first row holds only entries below the diagonal
+  // Tile order: row tiles are taken in groups of kGroupM; inside a group the column tile is the slow index.  The
+  // CTAs that run together then cover about kGroupM x (CTAs / kGroupM) tiles, so a wave reads kGroupM row panels of
+  // A and CTAs/kGroupM column panels of B instead of a few row panels and all of B (which, once B no longer fits
+  // in L2, streamed the whole of B from memory for every two or three row tiles).
+  auto tile_mn = [&](int tile, int& mt, int& nt) {
+    const int per_group = kGroupM * p.n_tiles;
+    const int g = tile / per_group, r = tile - g * per_group;
+    const int rem = p.m_tiles - g * kGroupM;
+    const int gm = rem < kGroupM ? rem : kGroupM;
+    nt = r / gm;
+    mt = g * kGroupM + (r - nt * gm);
+  };
   auto skipped = [&](int tile) {
-    return p.upper_only != 0 && ((tile % p.n_tiles) + 1) * BN <= (tile / p.n_tiles) * kBM;
+    if (p.upper_only == 0) return false;
+    int mt, nt;
+    tile_mn(tile, mt, nt);
+    return (nt + 1) * BN <= mt * kBM;
   };
   auto unit_kb0 = [&](int u) { return (u / plain_tiles) * p.kb_per_split; };
   auto unit_iters = [&](int u) {
@@ -153,8 +172,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
       for (int unit = blockIdx.x; unit < total_tiles && ok; unit += gridDim.x) {
         const int tile = unit % plain_tiles;
         if (skipped(tile)) continue;
-        const int m0 = (tile / p.n_tiles) * kBM;
-        const int n0 = (tile % p.n_tiles) * BN;
+        int m_tile, n_tile;
+        tile_mn(tile, m_tile, n_tile);
+        const int m0 = m_tile * kBM;
+        const int n0 = n_tile * BN;
         const int kb0 = unit_kb0(unit);
         const int iters = unit_iters(unit);
         for (int it = 0; it < iters; ++it) {
@@ -236,8 +257,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
     for (int unit = blockIdx.x; unit < total_tiles && ok; unit += gridDim.x) {
       const int tile = unit % plain_tiles;
       if (skipped(tile)) continue;
-      const int m_tile = tile / p.n_tiles;
-      const int n_tile = tile % p.n_tiles;
+      int m_tile, n_tile;
+      tile_mn(tile, m_tile, n_tile);
       const int row = m_tile * kBM + lane_group * 32 + lane;
       const int n0 = n_tile * BN;
       const int buf = lt & 1;
