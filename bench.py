@@ -36,7 +36,12 @@ WORKLOADS = {
     "llama3_70b_layer": ("llama3_70b_sweep", 8192, 32768),
     # the whole layer-wise sweep: --layers resident layer buffers (80 by default), --steps steps per layer
     "llama3_70b_sweep": ("llama3_70b_sweep", 8192, 32768),
+    # the paper's procedure for the shared rotation R1: 64 stored buffers (32 layers x 2 blocks) of 8192 tokens, every
+    # step a shuffled minibatch of 32 samples of 2048 tokens (N = 65536 tokens per step), Cayley Adam, whole-batch
+    # kurtosis after RMSNorm
+    "llama2_7b_r1_shared": ("llama2_7b_r1_shared", 4096, 65536),
 }
+SHARED_RPS, SHARED_BATCH = 2048, 32
 
 
 def measured_peaks():
@@ -230,13 +235,17 @@ def main():
     kw = dict(device=dev, rows=N_full if wl_cfg != "kv_heads" else N_full)
     if wl_cfg == "llama3_70b_sweep":
         kw["layers"] = args.layers if sweep else 1
+    shared = args.workload == "llama2_7b_r1_shared"
+    if shared:
+        args.optimizer, args.loss_mode, args.rmsnorm = "adam", "layer", True
+        kw["rows"] = None
     cfg = synth.config(wl_cfg, **kw)
     Xs = cfg["X"] if isinstance(cfg["X"], list) else [cfg["X"]]   # all layer buffers stay resident in HBM
     X = Xs[0]
     if world > 1:
         # different data per rank: re-draw with a rank-dependent seed by rolling rows
         X = torch.roll(X, shifts=rank * 977, dims=0).contiguous()
-    N = X.shape[0]
+    N = SHARED_RPS * SHARED_BATCH if shared else X.shape[0]
     lr = cfg["lr"]
     ctx = kurtail.Context(dev, forward_terms=args.forward_terms, optimizer=1 if args.optimizer == "adam" else 0,
                           loss_mode=1 if args.loss_mode == "layer" else 0, rmsnorm=1 if args.rmsnorm else 0)
@@ -250,7 +259,17 @@ def main():
 
     R = fresh_R()
     R0_host = R.cpu().numpy()
-    ctx.fit(X, R, max(args.warmup, 1), lr)          # warm-up steps (also sizes the workspace)
+    if shared:
+        # the shuffle: epochs of a seeded permutation of all stored samples, cut into minibatches
+        n_samples = len(Xs) * (Xs[0].shape[0] // SHARED_RPS)
+        rng = np.random.default_rng(1234 + rank)
+        need = (max(args.warmup, 1) + args.steps) * SHARED_BATCH
+        order = np.concatenate([rng.permutation(n_samples) for _ in range(need // n_samples + 1)])[:need].tolist()
+        w = max(args.warmup, 1)
+        ctx.fit_shared(Xs, SHARED_RPS, order[:w * SHARED_BATCH], SHARED_BATCH, R, w, lr)
+        order = order[w * SHARED_BATCH:]
+    else:
+        ctx.fit(X, R, max(args.warmup, 1), lr)          # warm-up steps (also sizes the workspace)
     torch.cuda.synchronize()
 
     sampler = ClockSampler(local_rank)
@@ -269,6 +288,8 @@ def main():
         ev0.record()
         reps = ctx.fit_layers(Xs, Rs, args.steps, lr)
         rep = reps[-1]
+    elif shared:
+        rep = ctx.fit_shared(Xs, SHARED_RPS, order, SHARED_BATCH, R, args.steps, lr)
     else:
         rep = ctx.fit(X, R, args.steps, lr)
     ev1.record()
@@ -285,7 +306,7 @@ def main():
 
     # ---- end to end through kt_fit_host: pinned host X and R in, R out, copies inside the timed region
     e2e = None
-    if not args.no_e2e and not sweep:
+    if not args.no_e2e and not sweep and not shared:
         Xh = X.cpu().pin_memory()
         Rh = torch.from_numpy(R0_host.copy()).pin_memory()
         stage = torch.empty_like(X)
@@ -369,6 +390,7 @@ def main():
         "algorithmic_tflops": (4.0 * N * d * d) * world / (ms_per_step * 1e-3) / 1e12,
         "loss_first": rep["loss_first"], "loss_last": rep["loss_last"], "orth_err": rep["orth_err"],
         "alpha_last": rep["alpha_last"], "w_norm_last": rep["w_norm_last"],
+        "step_choices": {k: rep[k] for k in ("w_op_last", "series_terms_last", "p0_terms_last", "guards_run")},
         "gpu_launches": prof["launches_total"], "clocks": clocks, "roofline": roofline, "e2e": e2e,
     }
 
@@ -381,7 +403,11 @@ def main():
         q1.record()
         torch.cuda.synchronize()
         out["quant4_error"] = {"mse": mse, "ms": q0.elapsed_time(q1)}
-    if not args.no_cpu_baseline and world == 1:
+    if shared:
+        out["config"].update({"buffers": len(Xs), "rows_per_buffer": int(Xs[0].shape[0]),
+                              "rows_per_sample": SHARED_RPS, "batch_samples": SHARED_BATCH,
+                              "resident_gib": len(Xs) * Xs[0].shape[0] * d * 2 / 2**30})
+    if not args.no_cpu_baseline and world == 1 and not shared:
         n_s = min(N, max(64, int(2.0e10 / (4.0 * d * d))))
         sample = X[:n_s].float().cpu().numpy()
         out["cpu_baseline"] = cpu_baseline(sample, R0_host, N, lr)

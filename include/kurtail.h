@@ -256,6 +256,26 @@ kt_status kt_fit(kt_ctx* ctx, kt_mat X, float* R, int32_t steps, float lr, kt_fi
 kt_status kt_fit_layers(kt_ctx* ctx, const kt_mat* X_layers, float* const* R_layers, int32_t L,
                         int32_t first_layer, int32_t steps, float lr, kt_fit_report* per_layer);
 
+/* One rotation shared by several activation buffers (Section 3, "Learning the
+ * Rotations": the stored inputs of all transformer layers and of both blocks
+ * are shuffled and a single R1 is trained on them).  X_bufs[0..n_bufs) are
+ * device matrices of equal rows, cols, ld and dtype (n_bufs <= 4096); a
+ * "sample" is a run of rows_per_sample consecutive rows (rows must be a
+ * multiple of it), numbered id = buffer * (rows / rows_per_sample) + index
+ * within the buffer.  Step k fits on the minibatch of the `batch` samples
+ * order[k*batch .. (k+1)*batch): their rows are gathered (in that order) into
+ * a dense bf16 matrix of batch*rows_per_sample rows in the workspace, and the
+ * step is the one kt_fit takes on that matrix (loss_mode, rmsnorm, optimizer
+ * as configured).  The shuffle is the caller's: `order` (host, steps*batch
+ * entries) is an input, so that a run can be reproduced exactly.  Needs a
+ * workspace of kt_fit_shared_workspace_bytes().  KT_ERR_INVALID_ARG if an id
+ * is out of range (checked before any work).  Synchronises at the end. */
+kt_status kt_fit_shared_workspace_bytes(const kt_ctx* ctx, int64_t rows_per_sample, int32_t batch, int64_t d,
+                                        size_t* bytes);
+kt_status kt_fit_shared(kt_ctx* ctx, const kt_mat* X_bufs, int32_t n_bufs, int64_t rows_per_sample,
+                        const int32_t* order, int32_t batch, float* R, int32_t steps, float lr,
+                        kt_fit_report* report);
+
 /* kt_fit with HOST buffers: copies X_host (N x d, pinned or pageable host
  * memory) into X_dev_staging (device, N*ld elements), R_host (d x d float32)
  * into R_dev, fits, and copies R back to R_host.  The copies run on the

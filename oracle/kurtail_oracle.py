@@ -21,6 +21,8 @@ What follows the paper, and where:
   literally: kappa of the concatenation of all tokens' activations of the layer.
   ``rmsnorm_rows`` / ``small_network``  -- Section 3, "Learning the Rotations":
   the trained network is the linear layer followed by an RMSNorm.
+  ``gather_samples`` / ``fit_shared``  -- same paragraph: one rotation trained on
+  shuffled minibatches of the stored inputs of all layers and both blocks.
 * ``skew_direction``, ``cayley_exact``, ``cayley_stepwise``, ``orth_step`` --
   Section 3, "Optimization in the Orthogonal Space": Cayley SGD on the
   Stiefel manifold.  The paper gives the method by citation only (Li et al.
@@ -275,6 +277,50 @@ def cayley_adam_step(R, dR, state, lr, beta1=0.9, beta2=0.99, adam_eps=1e-8,
     if orthogonality_error(Rn) > polish_thresh:
         Rn = polish(Rn)
     return Rn
+
+
+# --------------------------------------------------------------------------
+# Section 3, "Learning the Rotations": one rotation for the stored inputs of
+# all layers and both blocks, trained on shuffled minibatches
+# --------------------------------------------------------------------------
+def gather_samples(X_bufs, rows_per_sample, ids):
+    """The minibatch named by `ids`: sample id = buffer * samples_per_buffer +
+    index within the buffer; a sample is rows_per_sample consecutive rows.  The
+    samples' rows are stacked in the order of `ids`."""
+    spb = X_bufs[0].shape[0] // rows_per_sample
+    parts = []
+    for i in ids:
+        b, s = divmod(int(i), spb)
+        parts.append(np.asarray(X_bufs[b], dtype=np.float64)[s * rows_per_sample:(s + 1) * rows_per_sample])
+    return np.concatenate(parts, axis=0)
+
+
+def fit_shared(X_bufs, rows_per_sample, order, batch, R, steps, lr, flat=False, rmsnorm=False, adam=False,
+               rms_eps=1e-6, kappa_target=KAPPA_UNIFORM, polish_thresh=0.0, round_batch=None):
+    """steps x (gather the step's minibatch; [RMSNorm its rows]; loss and
+    gradient, per token or over the whole minibatch; Cayley SGD or Cayley Adam
+    step).  `order` holds steps*batch sample ids: the shuffle is an input.
+    `round_batch`, if given, is applied to the normalised minibatch (the tests
+    pass the bfloat16 rounding the library applies to its stored copy).
+    Returns (R_final, [loss per step])."""
+    R = np.asarray(R, dtype=np.float64).copy()
+    d = R.shape[0]
+    state = dict(M=np.zeros((d, d)), v=0.0, k=0)
+    lg = loss_grad_flat if flat else loss_grad
+    losses = []
+    for k in range(steps):
+        Xk = gather_samples(X_bufs, rows_per_sample, order[k * batch:(k + 1) * batch])
+        if rmsnorm:
+            Xk = rmsnorm_rows(Xk, rms_eps)
+            if round_batch is not None:
+                Xk = round_batch(Xk)
+        L, dR = lg(Xk, R, kappa_target)
+        losses.append(L)
+        if adam:
+            R = cayley_adam_step(R, dR, state, lr, polish_thresh=polish_thresh)
+        else:
+            R, _, _ = orth_step(R, dR, lr, polish_thresh=polish_thresh)
+    return R, losses
 
 
 # --------------------------------------------------------------------------

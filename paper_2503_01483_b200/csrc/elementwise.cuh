@@ -293,13 +293,43 @@ __global__ void k_flat_fill(const float4* __restrict__ coef_global, int N, float
   if (row < N) coef[row] = *coef_global;
 }
 
+// ------------------------------------------------ minibatch of stored samples
+// Gathers one minibatch for a rotation shared by several activation buffers: sample ids[b] (b < batch) lives in
+// buffer ids[b] / samples_per_buf at rows (ids[b] % samples_per_buf) * rps .. + rps; its rows are copied (and
+// rounded to bf16 when T = float) to rows b * rps .. of the dense bf16 matrix out (batch*rps x d).
+// grid batch * rps (one block per row), block 256; d a multiple of 8.
+template <typename T>
+__global__ void k_gather_samples(const void* const* __restrict__ bases, long long ld, int samples_per_buf, int rps,
+                                 const int* __restrict__ ids, int d, __nv_bfloat16* __restrict__ out) {
+  const int b = blockIdx.x / rps, r = blockIdx.x - b * rps;
+  const int id = ids[b];
+  const int buf = id / samples_per_buf, smp = id - buf * samples_per_buf;
+  const T* src = static_cast<const T*>(bases[buf]) + (static_cast<long long>(smp) * rps + r) * ld;
+  __nv_bfloat16* dst = out + static_cast<long long>(blockIdx.x) * d;
+  for (int j = threadIdx.x * 8; j < d; j += 256 * 8) {
+    uint4 o;
+    __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&o);
+    if (sizeof(T) == 2) {
+      o = *reinterpret_cast<const uint4*>(src + j);
+    } else {
+      const float4 a = *reinterpret_cast<const float4*>(src + j);
+      const float4 c = *reinterpret_cast<const float4*>(src + j + 4);
+      po[0] = __floats2bfloat162_rn(a.x, a.y);
+      po[1] = __floats2bfloat162_rn(a.z, a.w);
+      po[2] = __floats2bfloat162_rn(c.x, c.y);
+      po[3] = __floats2bfloat162_rn(c.z, c.w);
+    }
+    *reinterpret_cast<uint4*>(dst + j) = o;
+  }
+}
+
 // ------------------------------------------------------- RMSNorm of the rows
 // xb[t][:] = bf16( X[t][:] / sqrt(mean_j X[t][j]^2 + eps) ) -- the RMSNorm (unit gain) that follows the rotation in
 // the paper's small network (Section 3, "Learning the Rotations"); an orthogonal R keeps every row's norm, so it
-// can be applied to X once.  One block of 256 threads per row; T = float or bf16; xb dense N x d.
+// can be applied to X once.  One block of 256 threads per row; T = float or bf16; xb dense N x d.  xb may be X
+// itself (bf16, ld == d): a thread writes only elements it has read, after the row's sum is complete.
 template <typename T>
-__global__ void k_rmsnorm_rows(const T* __restrict__ X, long long ld, int d, float eps,
-                               __nv_bfloat16* __restrict__ xb) {
+__global__ void k_rmsnorm_rows(const T* X, long long ld, int d, float eps, __nv_bfloat16* xb) {
   __shared__ double sh[8];
   __shared__ float scale_sh;
   const T* x = X + static_cast<long long>(blockIdx.x) * ld;

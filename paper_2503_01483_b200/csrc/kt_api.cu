@@ -19,6 +19,8 @@
 namespace kt {
 
 constexpr int kHistMax = 4096;  // loss-history slots kept on the device between host read-backs
+constexpr int kIdsChunk = 256;  // kt_fit_shared: steps whose sample ids are on the device at a time
+constexpr int kMaxSharedBufs = 4096;  // kt_fit_shared: activation buffers one rotation can be shared by
 constexpr int kProfPairs = 8192; // CUDA-event pairs available to one profiling window
 enum GemmCat : int { kCatForward = 0, kCatBackwardA = 1, kCatBackwardB = 2, kCatSquare = 3, kCatQuant = 4, kCatFused = 5 };
 
@@ -87,6 +89,8 @@ struct WsLayout {
   size_t splitk;        // [splits][d][d] float: partial dR of the split-K backward-B (when splits > 1)
   size_t small;         // d <= 512: scratch of the one-launch orthogonal step (5 d x d floats + per-CTA partials)
   size_t adam_m;        // d x d float32: momentum of Cayley Adam inside kt_fit (only when asked for)
+  size_t gather_ids;    // kt_fit_shared: [kIdsChunk][batch] int sample ids
+  size_t gather_bases;  // kt_fit_shared: [kMaxSharedBufs] buffer base pointers
   size_t flat;          // flattened-kurtosis mode: the global coefficients, the global mean, 3 x [blocks] doubles
   size_t total;
   long long ldt;
@@ -94,9 +98,12 @@ struct WsLayout {
 };
 
 // cfg == null: the default configuration (no momentum buffer, no normalised copy of a bf16 X).
-static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, const kt_config* cfg = nullptr) {
+// gather_batch > 0: the layout of kt_fit_shared (N = batch * rows per sample): the dense bf16 matrix is the gathered
+// minibatch, and the sample ids of kIdsChunk steps and the buffers' base pointers live in the workspace too.
+static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, const kt_config* cfg = nullptr,
+                            int gather_batch = 0) {
   const bool adam = cfg != nullptr && cfg->optimizer == 1;
-  const bool xcopy = x_dtype == KT_F32 || (cfg != nullptr && cfg->rmsnorm != 0);
+  const bool xcopy = x_dtype == KT_F32 || (cfg != nullptr && cfg->rmsnorm != 0) || gather_batch > 0;
   WsLayout L;
   memset(&L, 0, sizeof(L));
   L.bn = (d % 256 == 0) ? 256 : 128;
@@ -144,6 +151,8 @@ static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, const kt_conf
   }
   L.small = take(d <= 512 ? 5 * dd * 4 + 4096 : 0);
   L.adam_m = take(adam ? dd * 4 : 0);
+  L.gather_ids = take(gather_batch > 0 ? static_cast<size_t>(kIdsChunk) * gather_batch * 4 : 0);
+  L.gather_bases = take(gather_batch > 0 ? static_cast<size_t>(kMaxSharedBufs) * 8 : 0);
   L.flat = take(static_cast<size_t>(L.loss_blocks) * 8 * 3 + 64);
   L.total = off;
   return L;
@@ -727,15 +736,37 @@ static kt_status check_d(int64_t d) {
   return KT_OK;
 }
 
-static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps, float lr, kt_fit_report* report) {
+// A rotation shared by several equally shaped activation buffers: every step works on a minibatch of `batch`
+// samples (runs of `rps` consecutive rows) named by `order` (host; steps * batch ids, id = buffer * samples per
+// buffer + sample within the buffer).
+struct SharedSrc {
+  const kt_mat* bufs;
+  int n_bufs;
+  int64_t rps;
+  const int32_t* order;
+  int batch;
+};
+
+// X is the calibration matrix, or (sh != null) the first of the shared buffers, which stands for their common shape.
+static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps, float lr, kt_fit_report* report,
+                          const SharedSrc* sh = nullptr) {
   int64_t N64, d64;
   KT_TRY(check_x(X, &N64, &d64));
   if (R == nullptr || steps < 0) return KT_ERR_INVALID_ARG;
   if (!aligned16(R)) return KT_ERR_ALIGN;
   const bool adam = ctx->cfg.optimizer == 1;
-  const WsLayout L = make_layout(N64, d64, X.dtype, &ctx->cfg);
+  const int spb = sh ? static_cast<int>(N64 / sh->rps) : 0;  // samples per buffer
+  if (sh) N64 = static_cast<int64_t>(sh->batch) * sh->rps;
+  const WsLayout L = make_layout(N64, d64, X.dtype, &ctx->cfg, sh ? sh->batch : 0);
   KT_TRY(check_ws(ctx, L));
   const int N = static_cast<int>(N64), d = static_cast<int>(d64);
+  if (sh) {
+    const void* bases[kMaxSharedBufs];
+    for (int b = 0; b < sh->n_bufs; ++b) bases[b] = sh->bufs[b].data;
+    KT_CUDA(cudaMemcpyAsync(ctx->ws + L.gather_bases, bases, sizeof(void*) * sh->n_bufs, cudaMemcpyHostToDevice,
+                            ctx->stream));
+    KT_CUDA(cudaStreamSynchronize(ctx->stream));  // `bases` is a stack array
+  }
   float* adam_m = nullptr;
   if (adam) {  // every fit starts Cayley Adam from a zero state
     adam_m = at<float>(ctx, L.adam_m);
@@ -747,7 +778,9 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
   KT_LAUNCH_CHECK();
   XView xv;
   const bool fused = use_fused(ctx, d);
-  if (fused) KT_TRY(ingest_x_forward(ctx, X, L, &xv)); else KT_TRY(ingest_x_full(ctx, X, L, &xv));
+  if (!sh) {
+    if (fused) KT_TRY(ingest_x_forward(ctx, X, L, &xv)); else KT_TRY(ingest_x_full(ctx, X, L, &xv));
+  }
   float* dR = at<float>(ctx, L.dr);
   const int ge = ctx->cfg.guard_every < 1 ? 1 : ctx->cfg.guard_every;
   double first = 0.0, last = 0.0;
@@ -762,6 +795,34 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
       if (k == kHistMax) first = ctx->h_blk->hist[0];
       if (report && report->loss_history)
         memcpy(report->loss_history + (k - kHistMax), ctx->h_blk->hist, sizeof(double) * kHistMax);
+    }
+    if (sh) {
+      // this step's minibatch: gather its samples into the dense bf16 matrix, normalise, transpose
+      const int cslot = k % kIdsChunk;
+      if (cslot == 0) {
+        const int n_steps = (steps - k < kIdsChunk) ? steps - k : kIdsChunk;
+        if (k > 0) KT_CUDA(cudaStreamSynchronize(ctx->stream));  // the previous chunk's ids are still being read
+        KT_CUDA(cudaMemcpyAsync(ctx->ws + L.gather_ids, sh->order + static_cast<size_t>(k) * sh->batch,
+                                sizeof(int32_t) * n_steps * sh->batch, cudaMemcpyHostToDevice, ctx->stream));
+      }
+      __nv_bfloat16* xb = at<__nv_bfloat16>(ctx, L.xb);
+      const void* const* bases = at<const void*>(ctx, L.gather_bases);
+      const int* ids = at<int>(ctx, L.gather_ids) + static_cast<size_t>(cslot) * sh->batch;
+      const int rps = static_cast<int>(sh->rps);
+      if (X.dtype == KT_BF16)
+        k_gather_samples<__nv_bfloat16><<<N, 256, 0, ctx->stream>>>(bases, X.ld, spb, rps, ids, d, xb);
+      else
+        k_gather_samples<float><<<N, 256, 0, ctx->stream>>>(bases, X.ld, spb, rps, ids, d, xb);
+      KT_LAUNCH_CHECK();
+      kt_mat Xb;
+      Xb.data = xb;
+      Xb.dtype = KT_BF16;
+      Xb.reserved = 0;
+      Xb.rows = N;
+      Xb.cols = d;
+      Xb.ld = d;
+      // (with rmsnorm the rows are normalised in place: each block reads its whole row before it writes it)
+      if (fused) KT_TRY(ingest_x_forward(ctx, Xb, L, &xv)); else KT_TRY(ingest_x_full(ctx, Xb, L, &xv));
     }
     // from the second step on, the previous step left the bf16 forms of R in the workspace
     if (fused)
@@ -1079,6 +1140,36 @@ kt_status kt_fit_layers(kt_ctx* ctx, const kt_mat* X_layers, float* const* R_lay
     KT_TRY(fit_impl(ctx, X_layers[l], R_layers[l], steps, lr, per_layer ? &per_layer[l] : nullptr));
   }
   return KT_OK;
+}
+
+kt_status kt_fit_shared_workspace_bytes(const kt_ctx* ctx, int64_t rows_per_sample, int32_t batch, int64_t d,
+                                        size_t* bytes) {
+  if (!ctx || !bytes) return KT_ERR_INVALID_ARG;
+  if (rows_per_sample < 1 || batch < 1 || batch > 65536 || rows_per_sample * batch > 0x7fffff00ll) return KT_ERR_SHAPE;
+  KT_TRY(check_d(d));
+  *bytes = make_layout(rows_per_sample * batch, d, KT_BF16, &ctx->cfg, batch).total;
+  return KT_OK;
+}
+
+kt_status kt_fit_shared(kt_ctx* ctx, const kt_mat* X_bufs, int32_t n_bufs, int64_t rows_per_sample,
+                        const int32_t* order, int32_t batch, float* R, int32_t steps, float lr,
+                        kt_fit_report* report) {
+  if (!ctx || !X_bufs || !order || !R || n_bufs < 1 || n_bufs > kMaxSharedBufs || steps < 0 || !(lr >= 0.f))
+    return KT_ERR_INVALID_ARG;
+  if (rows_per_sample < 1 || batch < 1 || batch > 65536 || rows_per_sample * batch > 0x7fffff00ll) return KT_ERR_SHAPE;
+  int64_t N0, d0;
+  KT_TRY(check_x(X_bufs[0], &N0, &d0));
+  if (N0 % rows_per_sample != 0) return KT_ERR_SHAPE;
+  for (int b = 1; b < n_bufs; ++b) {
+    int64_t N, d;
+    KT_TRY(check_x(X_bufs[b], &N, &d));
+    if (N != N0 || d != d0 || X_bufs[b].dtype != X_bufs[0].dtype || X_bufs[b].ld != X_bufs[0].ld) return KT_ERR_SHAPE;
+  }
+  const int64_t n_samples = static_cast<int64_t>(n_bufs) * (N0 / rows_per_sample);
+  for (int64_t i = 0; i < static_cast<int64_t>(steps) * batch; ++i)
+    if (order[i] < 0 || order[i] >= n_samples) return KT_ERR_INVALID_ARG;
+  SharedSrc sh{X_bufs, n_bufs, rows_per_sample, order, batch};
+  return fit_impl(ctx, X_bufs[0], R, steps, lr, report, &sh);
 }
 
 kt_status kt_fit_host(kt_ctx* ctx, kt_mat X_host, void* X_dev_staging, float* R_host, float* R_dev, int32_t steps,

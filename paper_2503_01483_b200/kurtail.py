@@ -57,7 +57,8 @@ class kt_profile(C.Structure):
 
 EXPORTS = ["kt_default_config", "kt_create", "kt_destroy", "kt_status_string", "kt_workspace_bytes",
            "kt_set_workspace", "kt_init_rotation", "kt_kurtosis_loss", "kt_loss_grad", "kt_row_moments",
-           "kt_rotate", "kt_orth_step", "kt_adam_step", "kt_orth_error", "kt_fit", "kt_fit_layers", "kt_fit_host",
+           "kt_rotate", "kt_orth_step", "kt_adam_step", "kt_orth_error", "kt_fit", "kt_fit_layers",
+           "kt_fit_shared_workspace_bytes", "kt_fit_shared", "kt_fit_host",
            "kt_quant4_error", "kt_quant4_codes", "kt_profile_begin", "kt_profile_end",
            "kt_kurtosis_loss_noalloc"]
 
@@ -94,6 +95,9 @@ def lib():
     L.kt_orth_error.argtypes = [vp, vp, i64, dp]
     L.kt_fit.argtypes = [vp, kt_mat, vp, i32, f32, C.POINTER(kt_fit_report)]
     L.kt_fit_layers.argtypes = [vp, C.POINTER(kt_mat), C.POINTER(vp), i32, i32, i32, f32, C.POINTER(kt_fit_report)]
+    L.kt_fit_shared_workspace_bytes.argtypes = [vp, i64, i32, i64, C.POINTER(C.c_size_t)]
+    L.kt_fit_shared.argtypes = [vp, C.POINTER(kt_mat), i32, i64, C.POINTER(i32), i32, vp, i32, f32,
+                                C.POINTER(kt_fit_report)]
     L.kt_fit_host.argtypes = [vp, kt_mat, vp, vp, vp, i32, f32, C.POINTER(kt_fit_report)]
     L.kt_quant4_error.argtypes = [vp, kt_mat, vp, dp]
     L.kt_quant4_codes.argtypes = [vp, vp, i64, i64, vp, vp]
@@ -271,6 +275,28 @@ class Context:
         reps = (kt_fit_report * L)()
         _check(lib().kt_fit_layers(self._h, mats, ptrs, L, first_layer, steps, lr, reps), "kt_fit_layers")
         return [_rep_dict(r, None) for r in reps]
+
+    def fit_shared(self, Xs, rows_per_sample, order, batch, R, steps, lr, history=False):
+        """kt_fit_shared: one R for the equally shaped buffers Xs; `order` is a sequence of steps*batch sample ids."""
+        nb = len(Xs)
+        mats = (kt_mat * nb)(*[as_mat(X) for X in Xs])
+        need = C.c_size_t()
+        _check(lib().kt_fit_shared_workspace_bytes(self._h, rows_per_sample, batch, mats[0].cols, C.byref(need)),
+               "kt_fit_shared_workspace_bytes")
+        if need.value > self._ws_bytes:
+            self._ws = None
+            self._ws = torch.empty(need.value + 256, dtype=torch.uint8, device=self.device)
+            base = (self._ws.data_ptr() + 255) // 256 * 256
+            _check(lib().kt_set_workspace(self._h, C.c_void_p(base), need.value), "kt_set_workspace")
+            self._ws_bytes = need.value
+        ids = (C.c_int32 * (steps * batch))(*[int(v) for v in order[:steps * batch]])
+        rep = kt_fit_report()
+        hist = (C.c_double * steps)() if history and steps > 0 else None
+        if hist is not None:
+            rep.loss_history = C.cast(hist, C.POINTER(C.c_double))
+        _check(lib().kt_fit_shared(self._h, mats, nb, rows_per_sample, ids, batch, R.data_ptr(), steps, lr,
+                                   C.byref(rep)), "kt_fit_shared")
+        return _rep_dict(rep, hist)
 
     def fit_host(self, X_host, X_staging, R_host, R_dev, steps, lr):
         m = as_mat(X_host)

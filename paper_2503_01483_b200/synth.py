@@ -119,6 +119,13 @@ def config(name, device="cpu", rows=None, layers=None):
         L = layers or 80
         Xs = [activations(N, 8192, "student_t", 2.5, 32, 200.0, seed=1000 + l, device=device) for l in range(L)]
         return dict(X=Xs, d=8192, init="hadamard", steps=50, lr=1e-2)
+    if name == "llama2_7b_r1_shared":
+        # stored inputs of 32 layers x 2 blocks: same outlier channels everywhere, scale growing with depth
+        N = rows or 8192
+        L = layers or 64
+        Xs = [(activations(N, 4096, "student_t", 3.0, 16, 100.0, seed=2000 + l, device=device).float()
+               * (1.0 + l / 16.0)).to(torch.bfloat16) for l in range(L)]
+        return dict(X=Xs, d=4096, init="hadamard", steps=100, lr=1e-2)
     raise ValueError(name)
 
 

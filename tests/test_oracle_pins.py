@@ -415,6 +415,41 @@ def test_rmsnorm_commutes_with_a_rotation_and_drops_out_of_the_tangent_gradient(
             assert num == pytest.approx(-(g * (W @ R)).sum(), rel=1e-5, abs=1e-9)
 
 
+# ---------------- shared rotation on shuffled minibatches ----------------
+def test_fit_shared_reduces_to_fit_and_gathers_the_named_rows():
+    rng = np.random.default_rng(31)
+    d, rps, spb, nb = 8, 4, 3, 2
+    bufs = [rng.standard_t(3, size=(rps * spb, d)) for _ in range(nb)]
+    # the gather: buffer and row range of every id, in the order given
+    G = ko.gather_samples(bufs, rps, [4, 0, 5])
+    assert np.array_equal(G[:rps], bufs[1][rps:2 * rps])
+    assert np.array_equal(G[rps:2 * rps], bufs[0][:rps])
+    assert np.array_equal(G[2 * rps:], bufs[1][2 * rps:])
+    R0 = scipy.stats.ortho_group.rvs(d, random_state=6)
+    # one buffer, every step the whole buffer in order: the plain full-batch fit
+    one = [np.concatenate(bufs, axis=0)]
+    order = list(range(nb * spb)) * 5
+    Ra, la = ko.fit_shared(one, rps, order, nb * spb, R0, 5, 1e-2)
+    Rb, lb = ko.fit(one[0], R0, 5, 1e-2)
+    assert np.array_equal(Ra, Rb) and la == lb
+    # the per-token loss does not care about the order of the rows: a permuted batch gives the same step
+    perm = rng.permutation(nb * spb).tolist()
+    Rc, lc = ko.fit_shared(one, rps, perm, nb * spb, R0, 1, 1e-2)
+    Rd, ld = ko.fit_shared(one, rps, sorted(perm), nb * spb, R0, 1, 1e-2)
+    assert np.abs(Rc - Rd).max() < 1e-13 and lc[0] == pytest.approx(ld[0], rel=1e-13)
+    # step k sees only its own minibatch: losses equal the loss of that batch at the R of that step
+    order2 = rng.integers(0, nb * spb, size=3 * 2).tolist()
+    R = R0.copy()
+    Rf, lf = ko.fit_shared(bufs, rps, order2, 2, R0, 3, 1e-2, flat=True, adam=True)
+    st = dict(M=np.zeros((d, d)), v=0.0, k=0)
+    for k in range(3):
+        Xk = ko.gather_samples(bufs, rps, order2[2 * k:2 * k + 2])
+        L, dR = ko.loss_grad_flat(Xk, R)
+        assert L == lf[k]
+        R = ko.cayley_adam_step(R, dR, st, 1e-2)
+    assert np.array_equal(R, Rf)
+
+
 # ---------------- quantizer ----------------
 def _golden_quant_cases():
     rows, codes = [], []
