@@ -34,6 +34,9 @@ What follows the paper, and where:
 * ``quant4_codes`` / ``quant4_error``  -- Section 2, "Uniform Quantization
   for k-bit Precision" (symmetric case, k = 4) and Eq. 1 (MSE); one scale
   per token as in Section 4 "Setup".
+  ``quant_codes`` / ``quant_error``: the same paragraph for k bits, symmetric
+  or asymmetric, with the clip ratio of Section 4 "Setup"; ``rowmax_success``:
+  the success rate of Section 3 (per-token maxima).
 * ``hadamard``  -- Section 3 (Hadamard rotations), Sylvester construction.
 
 Parity status: every function above is pinned by tests/test_oracle_pins.py
@@ -348,6 +351,53 @@ def quant4_error(Y32):
     deq = (codes.astype(np.float32) * s[:, None]).astype(np.float32)
     diff = Y.astype(np.float64) - deq.astype(np.float64)
     return float((diff * diff).sum() / Y.size)
+
+
+def quant_codes(Y32, bits=4, asymmetric=False, clip=1.0):
+    """The k-bit quantizer of Section 2, "Uniform Quantization for k-bit
+    Precision", per row, in float32 throughout:
+      symmetric:  b = 0, s = clip*max|y| / (2^(k-1) - 1), codes in [-(2^(k-1)-1), 2^(k-1)-1];
+      asymmetric: b = clip*min(y), s = (clip*max(y) - b) / (2^k - 1), codes in [0, 2^k - 1];
+      code = clamp(rint((y - b) / s), lo, hi), ties to even; s == 0 gives code 0.
+    `clip` in (0, 1] shrinks the range towards zero (Section 4, "Setup" clips
+    activations).  Returns (codes int16 N x n, s float32 N, b float32 N)."""
+    Y = np.asarray(Y32, dtype=np.float32)
+    c = np.float32(clip)
+    if asymmetric:
+        den = np.float32(2 ** bits - 1)
+        lo, hi = np.float32(0.0), den
+        b = (c * Y.min(axis=1)).astype(np.float32)
+        rng = ((c * Y.max(axis=1)).astype(np.float32) - b).astype(np.float32)
+    else:
+        den = np.float32(2 ** (bits - 1) - 1)
+        lo, hi = -den, den
+        b = np.zeros(Y.shape[0], dtype=np.float32)
+        rng = (c * np.abs(Y).max(axis=1)).astype(np.float32)
+    s = (rng / den).astype(np.float32)
+    safe = np.where(s == 0, np.float32(1.0), s).astype(np.float32)
+    q = np.rint(((Y - b[:, None]).astype(np.float32) / safe[:, None]).astype(np.float32))
+    q = np.clip(q, lo, hi)
+    q = np.where((s == 0)[:, None], 0.0, q)
+    return q.astype(np.int16), s, b
+
+
+def quant_error(Y32, bits=4, asymmetric=False, clip=1.0):
+    """Eq. 1 for quant_codes: mean (Y - Q(Y))^2 with Q(Y) = code*s + b formed in
+    float32, the difference and the sum in float64."""
+    Y = np.asarray(Y32, dtype=np.float32)
+    codes, s, b = quant_codes(Y, bits, asymmetric, clip)
+    deq = ((codes.astype(np.float32) * s[:, None]).astype(np.float32) + b[:, None]).astype(np.float32)
+    diff = Y.astype(np.float64) - deq.astype(np.float64)
+    return float((diff * diff).sum() / Y.size)
+
+
+def rowmax_success(X, R_a, R_b=None):
+    """Section 3's success rate: the fraction of tokens whose largest magnitude
+    after rotation R_a is smaller than after R_b (R_b None: the un-rotated token)."""
+    X = np.asarray(X, dtype=np.float64)
+    a = np.abs(rotate(X, R_a)).max(axis=1)
+    b = np.abs(X if R_b is None else rotate(X, R_b)).max(axis=1)
+    return float((a < b).mean())
 
 
 def quant4_error_rotated(X, R):

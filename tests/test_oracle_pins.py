@@ -516,3 +516,69 @@ def test_quant4_error_rotated_uses_the_product():
     A = rng.normal(size=(16, 16))
     assert ko.quant4_error_rotated(X, A) == pytest.approx(ko.quant4_error((X @ A).astype(np.float32)))
     assert ko.quant4_error_rotated(X, A) != pytest.approx(ko.quant4_error((X @ A.T).astype(np.float32)))
+
+
+# ---------------- general k-bit quantizer and the success rate ----------------
+def test_quant_general_reduces_to_the_4bit_case_and_hits_the_grid():
+    rng = np.random.default_rng(41)
+    Y = rng.normal(size=(20, 64)).astype(np.float32)
+    c4, s4 = ko.quant4_codes(Y)
+    c, s, b = ko.quant_codes(Y, 4, False, 1.0)
+    assert np.array_equal(c, c4) and np.array_equal(s, s4) and not b.any()
+    assert ko.quant_error(Y, 4, False, 1.0) == ko.quant4_error(Y)
+    for bits in (2, 3, 8):
+        # asymmetric: a row that already sits on the grid b + i*s is reproduced exactly, with codes i
+        lv = 2 ** bits
+        i = rng.integers(0, lv, size=(6, 40)); i[:, 0] = 0; i[:, 1] = lv - 1
+        step, shift = np.float32(0.25), np.float32(-3.0)
+        G = (shift + i.astype(np.float32) * step).astype(np.float32)
+        c, s, b = ko.quant_codes(G, bits, True, 1.0)
+        assert np.array_equal(c, i) and np.all(s == step) and np.all(b == shift)
+        assert ko.quant_error(G, bits, True, 1.0) == 0.0
+        # symmetric: integer multiples of max/L
+        L = 2 ** (bits - 1) - 1
+        k = rng.integers(-L, L + 1, size=(6, 40)); k[:, 0] = L
+        S = (k * np.float32(0.5)).astype(np.float32)
+        c, s, b = ko.quant_codes(S, bits, False, 1.0)
+        assert np.array_equal(c, k) and ko.quant_error(S, bits, False, 1.0) == 0.0
+
+
+def test_quant_uniform_rows_give_step_squared_over_twelve_and_clip_saturates():
+    rng = np.random.default_rng(42)
+    Y = rng.uniform(-1, 1, size=(64, 4096)).astype(np.float32)
+    for bits, asym in ((4, False), (4, True), (6, True), (8, False)):
+        _, s, _ = ko.quant_codes(Y, bits, asym, 1.0)
+        assert ko.quant_error(Y, bits, asym, 1.0) == pytest.approx(float((s.astype(np.float64) ** 2).mean()) / 12,
+                                                                   rel=0.03)
+    # the asymmetric grid has 2^k - 1 steps over the range, the symmetric one 2^k - 2: the asymmetric step is smaller
+    assert ko.quant_error(Y, 4, True) < ko.quant_error(Y, 4, False)
+    # shifted rows: the asymmetric quantizer does not care, the symmetric one wastes its range
+    assert ko.quant_error(Y + 5, 4, True) == pytest.approx(ko.quant_error(Y, 4, True), rel=0.05)
+    assert ko.quant_error(Y + 5, 4, False) > 5 * ko.quant_error(Y, 4, False)
+    # clip: values beyond clip*max saturate at the last level
+    row = np.array([[1.0, -1.0, 0.5, 0.25, 0.0, -0.125, 0.8, 0.6]], dtype=np.float32)
+    c, s, b = ko.quant_codes(row, 4, False, 0.5)
+    assert s[0] == np.float32(0.5 / 7) and c[0, 0] == 7 and c[0, 1] == -7 and c[0, 6] == 7 and c[0, 2] == 7
+    assert c[0, 3] == np.rint(np.float32(0.25) / s[0])
+    c, s, b = ko.quant_codes(row, 4, True, 0.5)
+    assert b[0] == np.float32(-0.5) and s[0] == np.float32(1.0) / np.float32(15.0) and c[0, 0] == 15 and c[0, 1] == 0
+    # a heavy tail: clipping at 0.9 of the maximum lowers the error of a Gaussian row with one large outlier
+    Z = rng.normal(size=(32, 1024)).astype(np.float32); Z[:, 3] = 12.0
+    assert ko.quant_error(Z, 4, False, 0.5) < ko.quant_error(Z, 4, False, 1.0)
+    # constant rows: step 0, codes 0, exact when unclipped
+    cst = np.full((2, 8), 3.0, dtype=np.float32)
+    assert ko.quant_error(cst, 4, True, 1.0) == 0.0 and not ko.quant_codes(cst, 4, True, 1.0)[0].any()
+
+
+def test_rowmax_success_rate():
+    d = 64
+    H = ko.hadamard(d)
+    # one-hot tokens (channel != 0): the Hadamard rotation spreads them, max drops from a to a/sqrt(d): success 1
+    X = np.zeros((10, d)); X[np.arange(10), 1 + np.arange(10)] = 3.0
+    assert ko.rowmax_success(X, H) == 1.0
+    assert ko.rowmax_success(X, np.eye(d)) == 0.0           # strict inequality: equal maxima are no success
+    assert ko.rowmax_success(X, np.eye(d), H) == 0.0 and ko.rowmax_success(X, H, np.eye(d)) == 1.0
+    # constant tokens are concentrated by the Hadamard rotation (all mass to channel 0): success 0
+    assert ko.rowmax_success(np.ones((4, d)), H) == 0.0
+    # a mix: exactly the one-hot half succeeds
+    assert ko.rowmax_success(np.vstack([X, np.ones((10, d))]), H) == 0.5
