@@ -403,6 +403,10 @@ def main():
         q1.record()
         torch.cuda.synchronize()
         out["quant4_error"] = {"mse": mse, "ms": q0.elapsed_time(q1)}
+        # share of tokens whose largest magnitude the fitted rotation lowers: against the un-rotated token and
+        # against the rotation the fit started from
+        out["rowmax_success"] = {"vs_unrotated": ctx.rowmax_success(X, R),
+                                 "vs_init": ctx.rowmax_success(X, R, fresh_R())}
     if shared:
         out["config"].update({"buffers": len(Xs), "rows_per_buffer": int(Xs[0].shape[0]),
                               "rows_per_sample": SHARED_RPS, "batch_samples": SHARED_BATCH,

@@ -291,6 +291,41 @@ kt_status kt_fit_host(kt_ctx* ctx, kt_mat X_host, void* X_dev_staging, float* R_
  * Y is recomputed instead of stored.  Synchronises. */
 kt_status kt_quant4_error(kt_ctx* ctx, kt_mat X, const float* R, double* mse);
 
+/* The general quantizer of the same paragraph, per token (one step and one
+ * shift per row), k = bits in 2..8:
+ *   symmetric:   b = 0,               s = clip * max|y| / (2^(k-1) - 1),
+ *                codes in [-(2^(k-1) - 1), 2^(k-1) - 1];
+ *   asymmetric:  b = clip * min(y),   s = (clip * max(y) - b) / (2^k - 1),
+ *                codes in [0, 2^k - 1]   (Section 4, "Setup": used for the
+ *                KV cache);
+ *   Q(y) = clamp(round_half_even((y - b) / s), lo, hi) * s + b;  s == 0 -> Q(y) = b.
+ * `clip` in (0, 1] shrinks the range towards zero before the step is formed
+ * ("Setup" clips activations; 1 = no clipping, the definition of Section 2).
+ * All decisions in IEEE float32.  {4, 0, 1.0} is kt_quant4_error. */
+typedef struct {
+  int32_t bits;       /* 2..8 */
+  int32_t asymmetric; /* 0 or 1 */
+  float clip;         /* (0, 1] */
+  int32_t reserved;
+} kt_quant_spec;
+
+/* *mse (host) = mean over all N*d entries of (Y - Q(Y))^2, Y = X R recomputed in
+ * two GEMM passes (row range, then error).  KT_ERR_INVALID_ARG for a spec out
+ * of range.  Synchronises. */
+kt_status kt_quant_error(kt_ctx* ctx, kt_mat X, const float* R, const kt_quant_spec* spec, double* mse);
+
+/* Test hook: quantise a given float32 Y (N x d dense, device) with `spec`:
+ * codes (N x d int16), scales s and shifts b (N float32 each), all device.
+ * No workspace needed.  Stream ordered. */
+kt_status kt_quant_codes(kt_ctx* ctx, const float* Y, int64_t N, int64_t d, const kt_quant_spec* spec,
+                         int16_t* codes, float* scales, float* shifts);
+
+/* Success rate of Section 3 (the comparison of per-token maxima): *rate (host) =
+ * the fraction of tokens t with max_j |(X R_a)_tj| < max_j |(X R_b)_tj|.  R_b may
+ * be NULL: the un-rotated token itself (max_j |X_tj|).  Uses the workspace.
+ * Synchronises. */
+kt_status kt_rowmax_success(kt_ctx* ctx, kt_mat X, const float* R_a, const float* R_b, double* rate);
+
 /* Test hook: quantise a given float32 Y (N x d dense, device): codes (N x d
  * int8, device) and scales (N float32, device).  Float32 IEEE divide and
  * round-half-even decide the codes.  No workspace needed.  Stream ordered. */

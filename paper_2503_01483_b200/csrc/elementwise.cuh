@@ -886,6 +886,89 @@ __global__ void k_quant4_codes(const float* __restrict__ Y, int d, int8_t* __res
   }
 }
 
+// The general k-bit quantizer of Section 2 on a dense float32 Y (N x d), one block per row:
+//   symmetric:  s = clip * max|Y_t| / (2^(k-1) - 1), b = 0,            codes in [-(2^(k-1) - 1), 2^(k-1) - 1]
+//   asymmetric: b = clip * min Y_t, s = (clip * max Y_t - b) / (2^k - 1), codes in [0, 2^k - 1]
+//   code = clamp(rint((y - b) / s), lo, hi); s == 0 -> code 0.  All in IEEE float32, ties to even.
+__global__ void k_quant_codes(const float* __restrict__ Y, int d, int asym, float clip, float den, float lo,
+                              float hi, short* __restrict__ codes, float* __restrict__ scales,
+                              float* __restrict__ shifts) {
+  __shared__ float shx[8], shn[8];
+  const long long base = static_cast<long long>(blockIdx.x) * d;
+  float mx = asym ? -INFINITY : 0.f, mn = INFINITY;
+  for (int j = threadIdx.x; j < d; j += 256) {
+    const float y = Y[base + j];
+    mx = fmaxf(mx, asym ? y : fabsf(y));
+    mn = fminf(mn, y);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+  }
+  if ((threadIdx.x & 31) == 0) {
+    shx[threadIdx.x >> 5] = mx;
+    shn[threadIdx.x >> 5] = mn;
+  }
+  __syncthreads();
+  mx = shx[0];
+  mn = shn[0];
+#pragma unroll
+  for (int i = 1; i < 8; ++i) {
+    mx = fmaxf(mx, shx[i]);
+    mn = fminf(mn, shn[i]);
+  }
+  float b = 0.f, range;
+  if (asym) {
+    b = __fmul_rn(clip, mn);
+    range = __fsub_rn(__fmul_rn(clip, mx), b);
+  } else {
+    range = __fmul_rn(clip, mx);
+  }
+  const float s = __fdiv_rn(range, den);
+  if (threadIdx.x == 0) {
+    scales[blockIdx.x] = s;
+    shifts[blockIdx.x] = b;
+  }
+  for (int j = threadIdx.x; j < d; j += 256) {
+    float qv = 0.f;
+    if (s > 0.f) {
+      qv = rintf(__fdiv_rn(__fsub_rn(Y[base + j], b), s));
+      qv = fminf(fmaxf(qv, lo), hi);
+    }
+    codes[base + j] = static_cast<short>(qv);
+  }
+}
+
+// Row abs-max of X itself (N x d, T = float or bf16), as float bits: the un-rotated baseline of the success rate.
+// One block per row.
+template <typename T>
+__global__ void k_row_absmax(const T* __restrict__ X, long long ld, int d, unsigned int* __restrict__ rowmax) {
+  __shared__ float sh[8];
+  const T* x = X + static_cast<long long>(blockIdx.x) * ld;
+  float mx = 0.f;
+  for (int j = threadIdx.x; j < d; j += 256) mx = fmaxf(mx, fabsf(to_f32(x[j])));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = mx;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    mx = sh[0];
+    for (int i = 1; i < 8; ++i) mx = fmaxf(mx, sh[i]);
+    rowmax[blockIdx.x] = __float_as_uint(mx);
+  }
+}
+
+// Per block: how many rows have max_a < max_b (both as bits of non-negative floats).  grid ceil(N/256), block 256.
+__global__ void k_count_less(const unsigned int* __restrict__ a, const unsigned int* __restrict__ b, int N,
+                             double* __restrict__ block_out) {
+  __shared__ double sh[8];
+  const int row = blockIdx.x * 256 + threadIdx.x;
+  const double v = (row < N && a[row] < b[row]) ? 1.0 : 0.0;
+  const double s = block_sum_256(v, sh, threadIdx.x);
+  if (threadIdx.x == 0) block_out[blockIdx.x] = s;
+}
+
 // ---------------------------------------------------------------- initialisers
 // kind 0: identity; kind 1: Sylvester Hadamard (-1)^popcount(i&j) * scale.
 __global__ void k_init_rotation(float* __restrict__ R, int d, int kind, float scale) {

@@ -53,13 +53,28 @@ struct GemmParams {
   const float4* coef;         // kGrad: per row {mu, a, ab, am3}
   __nv_bfloat16* gt;          // kGrad: G transposed, [N][ldg]
   long long ldg;
-  unsigned int* rowmax;       // kAbsMax (out) / kQuantErr (in): per-row max|D| as float bits
+  // kAbsMax (out) / kQuantErr (in).  Symmetric quantizer (rowmin == null): rowmax = per-row max|D| as float bits.
+  // Asymmetric (rowmin != null): rowmax / rowmin = per-row max D / min D as order-preserving keys (ordered_key()).
+  unsigned int* rowmax;
+  unsigned int* rowmin;
   float* qerr;                // kQuantErr: [n_tiles][M] partial squared errors
+  // kQuantErr: step = clip * range / q_den with range = max|D| (symmetric) or max - min (asymmetric, shift =
+  // clip * min); codes are clamped to [q_lo, q_hi]
+  float q_clip, q_den, q_lo, q_hi;
   const unsigned int* gate;   // when not null and *gate < gate_min the kernel does nothing
   unsigned int gate_min;
   const unsigned int* terms_dev;  // when not null, min(terms, *terms_dev) operand pairs are used
   unsigned int* err_word;     // receives the code of a wait that ran out
 };
+
+// Unsigned keys that order like the floats they encode (negative floats reversed, positive ones above them).
+__device__ __forceinline__ unsigned int ordered_key(float x) {
+  const unsigned int b = __float_as_uint(x);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float ordered_value(unsigned int k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
 
 template <int BN>
 struct GemmSmem {
@@ -346,34 +361,62 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
           }
         }
       } else if constexpr (EPI == kAbsMax) {
-        float mx = 0.f;
+        const bool asym = p.rowmin != nullptr;
+        float mx = asym ? -INFINITY : 0.f, mn = INFINITY;
 #pragma unroll 1
         for (int c0 = 0; c0 < BN; c0 += 32) {
           tmem_ld_32x32(t_addr + c0, v);
           tc_wait_ld();
+          if (asym) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, fabsf(__uint_as_float(v[j])));
+            for (int j = 0; j < 32; ++j) {
+              const float y = __uint_as_float(v[j]);
+              mx = fmaxf(mx, y);
+              mn = fminf(mn, y);
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) mx = fmaxf(mx, fabsf(__uint_as_float(v[j])));
+          }
         }
-        // non-negative floats order like their bit patterns; a max is exact, so arrival order does not matter
-        if (row_ok) atomicMax(p.rowmax + row, __float_as_uint(mx));
+        // integer max/min of order-preserving bit patterns are exact: arrival order does not matter
+        // (non-negative floats order like their own bits, which the symmetric case uses directly)
+        if (row_ok) {
+          if (asym) {
+            atomicMax(p.rowmax + row, ordered_key(mx));
+            atomicMin(p.rowmin + row, ordered_key(mn));
+          } else {
+            atomicMax(p.rowmax + row, __float_as_uint(mx));
+          }
+        }
       } else if constexpr (EPI == kQuantErr) {
-        float amax = 0.f;
-        if (row_ok) amax = __uint_as_float(p.rowmax[row]);
-        const float s = __fdiv_rn(amax, 7.0f);
+        // Q(y) = clamp(round((y - b) / s), q_lo, q_hi) * s + b, every operation in IEEE float32
+        float range = 0.f, b = 0.f;
+        if (row_ok) {
+          if (p.rowmin != nullptr) {
+            const float hi = __fmul_rn(p.q_clip, ordered_value(p.rowmax[row]));
+            b = __fmul_rn(p.q_clip, ordered_value(p.rowmin[row]));
+            range = __fsub_rn(hi, b);
+          } else {
+            range = __fmul_rn(p.q_clip, __uint_as_float(p.rowmax[row]));
+          }
+        }
+        const float s = __fdiv_rn(range, p.q_den);
         float e2 = 0.f;
 #pragma unroll 1
         for (int c0 = 0; c0 < BN; c0 += 32) {
           tmem_ld_32x32(t_addr + c0, v);
           tc_wait_ld();
-          if (s > 0.f) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const float y = __uint_as_float(v[j]);
-              float qv = rintf(__fdiv_rn(y, s));
-              qv = fminf(fmaxf(qv, -7.0f), 7.0f);
-              const float e = __fsub_rn(y, __fmul_rn(qv, s));
-              e2 = fmaf(e, e, e2);
+          for (int j = 0; j < 32; ++j) {
+            const float y = __uint_as_float(v[j]);
+            float qv = 0.f;
+            if (s > 0.f) {
+              qv = rintf(__fdiv_rn(__fsub_rn(y, b), s));
+              qv = fminf(fmaxf(qv, p.q_lo), p.q_hi);
             }
+            const float e = __fsub_rn(y, __fadd_rn(__fmul_rn(qv, s), b));
+            e2 = fmaf(e, e, e2);
           }
         }
         if (row_ok) p.qerr[static_cast<long long>(n_tile) * p.M + row] = e2;

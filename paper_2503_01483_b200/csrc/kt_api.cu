@@ -82,7 +82,7 @@ struct WsLayout {
   size_t partial;       // [P][N] float4 partial moment records
   size_t coef, moments; // [N] float4 each
   size_t block_loss, block_deg, norm_blocks;
-  size_t rowmax, qerr;  // quantizer: [N] uint, [P][N] float
+  size_t rowmax, rowmin, qerr;  // quantizer: [N] uint each, [P][N] float
   size_t colpart;       // [d/32][d] float: column sums of squares of R by row slab
   size_t diag;          // [d] float: exact diagonal of R^T R - I
   size_t pvec;          // [2][d] float: the last two vectors of the power iteration on W
@@ -100,7 +100,7 @@ struct WsLayout {
 // cfg == null: the default configuration (no momentum buffer, no normalised copy of a bf16 X).
 // gather_batch > 0: the layout of kt_fit_shared (N = batch * rows per sample): the dense bf16 matrix is the gathered
 // minibatch, and the sample ids of kIdsChunk steps and the buffers' base pointers live in the workspace too.
-static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, const kt_config* cfg = nullptr,
+static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, const kt_config* cfg,
                             int gather_batch = 0) {
   const bool adam = cfg != nullptr && cfg->optimizer == 1;
   const bool xcopy = x_dtype == KT_F32 || (cfg != nullptr && cfg->rmsnorm != 0) || gather_batch > 0;
@@ -139,6 +139,7 @@ static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, const kt_conf
   L.block_deg = take(static_cast<size_t>(L.loss_blocks > 256 ? L.loss_blocks : 256) * 4);
   L.norm_blocks = take(static_cast<size_t>(L.norm_n > 1024 ? L.norm_n : 1024) * 8);
   L.rowmax = take(static_cast<size_t>(N) * 4);
+  L.rowmin = take(static_cast<size_t>(N) * 4);
   L.qerr = take(static_cast<size_t>(L.P) * N * 4);
   L.colpart = take(static_cast<size_t>(d / 32) * d * 4);
   L.diag = take(static_cast<size_t>(d) * 4);
@@ -1193,29 +1194,60 @@ kt_status kt_fit_host(kt_ctx* ctx, kt_mat X_host, void* X_dev_staging, float* R_
   return st;
 }
 
-kt_status kt_quant4_error(kt_ctx* ctx, kt_mat X, const float* R, double* mse) {
+// levels of a k-bit quantizer: symmetric codes in [-(2^(k-1) - 1), 2^(k-1) - 1], asymmetric in [0, 2^k - 1]
+struct QuantLevels {
+  float den, lo, hi;
+};
+static kt_status quant_levels(const kt_quant_spec* spec, QuantLevels* q) {
+  if (!spec) return KT_ERR_INVALID_ARG;
+  if (spec->bits < 2 || spec->bits > 8 || (spec->asymmetric != 0 && spec->asymmetric != 1) ||
+      !(spec->clip > 0.f && spec->clip <= 1.f))
+    return KT_ERR_INVALID_ARG;
+  if (spec->asymmetric) {
+    q->den = static_cast<float>((1 << spec->bits) - 1);
+    q->lo = 0.f;
+    q->hi = q->den;
+  } else {
+    q->den = static_cast<float>((1 << (spec->bits - 1)) - 1);
+    q->lo = -q->den;
+    q->hi = q->den;
+  }
+  return KT_OK;
+}
+
+kt_status kt_quant_error(kt_ctx* ctx, kt_mat X, const float* R, const kt_quant_spec* spec, double* mse) {
   if (!ctx || !R || !mse) return KT_ERR_INVALID_ARG;
+  QuantLevels q;
+  KT_TRY(quant_levels(spec, &q));
   int64_t N64, d64;
   KT_TRY(check_x(X, &N64, &d64));
   if (!aligned16(R)) return KT_ERR_ALIGN;
-  const WsLayout L = make_layout(N64, d64, X.dtype);
+  const WsLayout L = make_layout(N64, d64, X.dtype, &ctx->cfg);
   KT_TRY(check_ws(ctx, L));
   const int N = static_cast<int>(N64), d = static_cast<int>(d64);
   XView xv;
   KT_TRY(ingest_x_forward(ctx, X, L, &xv));
   KT_TRY(cast_rt(ctx, R, d, N, L));
   unsigned int* rowmax = at<unsigned int>(ctx, L.rowmax);
+  unsigned int* rowmin = spec->asymmetric ? at<unsigned int>(ctx, L.rowmin) : nullptr;
   KT_CUDA(cudaMemsetAsync(rowmax, 0, static_cast<size_t>(N) * 4, ctx->stream));
+  if (rowmin) KT_CUDA(cudaMemsetAsync(rowmin, 0xff, static_cast<size_t>(N) * 4, ctx->stream));
   const FwdOperands f = fwd_operands(ctx, xv, d, N, L);
   {
     GemmParams p = blank_params();
     p.rowmax = rowmax;
+    p.rowmin = rowmin;
     KT_TRY(run_gemm<kAbsMax>(ctx, N, d, d, f.terms, f.A, f.B, p, kCatQuant));
   }
   {
     GemmParams p = blank_params();
     p.rowmax = rowmax;
+    p.rowmin = rowmin;
     p.qerr = at<float>(ctx, L.qerr);
+    p.q_clip = spec->clip;
+    p.q_den = q.den;
+    p.q_lo = q.lo;
+    p.q_hi = q.hi;
     KT_TRY(run_gemm<kQuantErr>(ctx, N, d, d, f.terms, f.A, f.B, p, kCatQuant));
   }
   const long long n = static_cast<long long>(L.P) * N;
@@ -1227,6 +1259,65 @@ kt_status kt_quant4_error(kt_ctx* ctx, kt_mat X, const float* R, double* mse) {
   KT_TRY(sync_scalars(ctx));
   *mse = ctx->h_blk->sc.qmse;
   return isfinite(*mse) ? KT_OK : KT_ERR_NONFINITE;
+}
+
+kt_status kt_quant4_error(kt_ctx* ctx, kt_mat X, const float* R, double* mse) {
+  kt_quant_spec spec;
+  spec.bits = 4;
+  spec.asymmetric = 0;
+  spec.clip = 1.0f;
+  spec.reserved = 0;
+  return kt_quant_error(ctx, X, R, &spec, mse);
+}
+
+kt_status kt_quant_codes(kt_ctx* ctx, const float* Y, int64_t N, int64_t d, const kt_quant_spec* spec, int16_t* codes,
+                         float* scales, float* shifts) {
+  if (!ctx || !Y || !codes || !scales || !shifts) return KT_ERR_INVALID_ARG;
+  QuantLevels q;
+  KT_TRY(quant_levels(spec, &q));
+  if (N < 1 || d < 1 || N > 0x7fffffffll || d > 0x7fffffffll) return KT_ERR_SHAPE;
+  k_quant_codes<<<static_cast<unsigned>(N), 256, 0, ctx->stream>>>(Y, static_cast<int>(d), spec->asymmetric,
+                                                                   spec->clip, q.den, q.lo, q.hi, codes, scales,
+                                                                   shifts);
+  KT_LAUNCH_CHECK();
+  return KT_OK;
+}
+
+kt_status kt_rowmax_success(kt_ctx* ctx, kt_mat X, const float* R_a, const float* R_b, double* rate) {
+  if (!ctx || !R_a || !rate) return KT_ERR_INVALID_ARG;
+  int64_t N64, d64;
+  KT_TRY(check_x(X, &N64, &d64));
+  if (!aligned16(R_a) || (R_b && !aligned16(R_b))) return KT_ERR_ALIGN;
+  const WsLayout L = make_layout(N64, d64, X.dtype, &ctx->cfg);
+  KT_TRY(check_ws(ctx, L));
+  const int N = static_cast<int>(N64), d = static_cast<int>(d64);
+  XView xv;
+  KT_TRY(ingest_x_forward(ctx, X, L, &xv));
+  unsigned int* max_a = at<unsigned int>(ctx, L.rowmax);
+  unsigned int* max_b = at<unsigned int>(ctx, L.rowmin);
+  const float* Rs[2] = {R_a, R_b};
+  unsigned int* outs[2] = {max_a, max_b};
+  for (int which = 0; which < 2; ++which) {
+    if (Rs[which] == nullptr) {  // the un-rotated rows themselves
+      k_row_absmax<__nv_bfloat16><<<N, 256, 0, ctx->stream>>>(xv.xb, xv.ldx, d, outs[which]);
+      KT_LAUNCH_CHECK();
+      continue;
+    }
+    KT_TRY(cast_rt(ctx, Rs[which], d, N, L));
+    KT_CUDA(cudaMemsetAsync(outs[which], 0, static_cast<size_t>(N) * 4, ctx->stream));
+    const FwdOperands f = fwd_operands(ctx, xv, d, N, L);
+    GemmParams p = blank_params();
+    p.rowmax = outs[which];
+    KT_TRY(run_gemm<kAbsMax>(ctx, N, d, d, f.terms, f.A, f.B, p, kCatQuant));
+  }
+  k_count_less<<<L.loss_blocks, 256, 0, ctx->stream>>>(max_a, max_b, N, at<double>(ctx, L.block_loss));
+  KT_LAUNCH_CHECK();
+  k_final_sum<<<1, 256, 0, ctx->stream>>>(at<double>(ctx, L.block_loss), L.loss_blocks, 1.0 / N,
+                                          &ctx->d_blk->sc.qmse, nullptr, nullptr, nullptr);
+  KT_LAUNCH_CHECK();
+  KT_TRY(sync_scalars(ctx));
+  *rate = ctx->h_blk->sc.qmse;
+  return KT_OK;
 }
 
 kt_status kt_profile_begin(kt_ctx* ctx) {

@@ -40,6 +40,10 @@ class kt_config(C.Structure):
                 ("reserved", C.c_int32 * 2)]
 
 
+class kt_quant_spec(C.Structure):
+    _fields_ = [("bits", C.c_int32), ("asymmetric", C.c_int32), ("clip", C.c_float), ("reserved", C.c_int32)]
+
+
 class kt_adam_state(C.Structure):
     _fields_ = [("v", C.c_double), ("step", C.c_int32), ("reserved", C.c_int32)]
 
@@ -59,7 +63,7 @@ EXPORTS = ["kt_default_config", "kt_create", "kt_destroy", "kt_status_string", "
            "kt_set_workspace", "kt_init_rotation", "kt_kurtosis_loss", "kt_loss_grad", "kt_row_moments",
            "kt_rotate", "kt_orth_step", "kt_adam_step", "kt_orth_error", "kt_fit", "kt_fit_layers",
            "kt_fit_shared_workspace_bytes", "kt_fit_shared", "kt_fit_host",
-           "kt_quant4_error", "kt_quant4_codes", "kt_profile_begin", "kt_profile_end",
+           "kt_quant4_error", "kt_quant4_codes", "kt_quant_error", "kt_quant_codes", "kt_rowmax_success", "kt_profile_begin", "kt_profile_end",
            "kt_kurtosis_loss_noalloc"]
 
 _lib = None
@@ -101,6 +105,9 @@ def lib():
     L.kt_fit_host.argtypes = [vp, kt_mat, vp, vp, vp, i32, f32, C.POINTER(kt_fit_report)]
     L.kt_quant4_error.argtypes = [vp, kt_mat, vp, dp]
     L.kt_quant4_codes.argtypes = [vp, vp, i64, i64, vp, vp]
+    L.kt_quant_error.argtypes = [vp, kt_mat, vp, C.POINTER(kt_quant_spec), dp]
+    L.kt_quant_codes.argtypes = [vp, vp, i64, i64, C.POINTER(kt_quant_spec), vp, vp, vp]
+    L.kt_rowmax_success.argtypes = [vp, kt_mat, vp, vp, dp]
     L.kt_kurtosis_loss_noalloc.argtypes = [kt_mat, vp, vp, vp]
     L.kt_profile_begin.argtypes = [vp]
     L.kt_profile_end.argtypes = [vp, C.POINTER(kt_profile)]
@@ -310,6 +317,30 @@ class Context:
         m = self._prep(X)
         out = C.c_double()
         _check(lib().kt_quant4_error(self._h, m, R.data_ptr(), C.byref(out)), "kt_quant4_error")
+        return out.value
+
+    def quant_error(self, X, R, bits=4, asymmetric=False, clip=1.0):
+        m = self._prep(X)
+        spec = kt_quant_spec(bits, int(asymmetric), clip, 0)
+        out = C.c_double()
+        _check(lib().kt_quant_error(self._h, m, R.data_ptr(), C.byref(spec), C.byref(out)), "kt_quant_error")
+        return out.value
+
+    def quant_codes(self, Y, bits=4, asymmetric=False, clip=1.0):
+        N, d = Y.shape
+        spec = kt_quant_spec(bits, int(asymmetric), clip, 0)
+        codes = torch.empty((N, d), dtype=torch.int16, device=Y.device)
+        scales = torch.empty((N,), dtype=torch.float32, device=Y.device)
+        shifts = torch.empty((N,), dtype=torch.float32, device=Y.device)
+        _check(lib().kt_quant_codes(self._h, Y.data_ptr(), N, d, C.byref(spec), codes.data_ptr(), scales.data_ptr(),
+                                    shifts.data_ptr()), "kt_quant_codes")
+        return codes, scales, shifts
+
+    def rowmax_success(self, X, R_a, R_b=None):
+        m = self._prep(X)
+        out = C.c_double()
+        _check(lib().kt_rowmax_success(self._h, m, R_a.data_ptr(), R_b.data_ptr() if R_b is not None else None,
+                                       C.byref(out)), "kt_rowmax_success")
         return out.value
 
     def profile_begin(self):
