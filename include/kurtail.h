@@ -116,6 +116,16 @@ typedef struct {
                            loose by up to sqrt(d): more terms and more
                            measurements than needed).  alpha always uses
                            ||W||_F.  Ignored by the d <= 512 one-launch step   */
+  int32_t backward_mode;/* [0]   where the backward pass takes Y from.  1 = a
+                           second pass of the forward GEMM recomputes each Y
+                           tile in tensor memory and nothing of Y is ever
+                           written (2 N d^2 more flops).  0 or 2 = the forward
+                           pass also stores Y as float32 (N*d*4 bytes of
+                           workspace) and an element-wise kernel reads it
+                           back (8 bytes per entry instead of 2 d flops: on a
+                           B200 the cheaper one for d above a few hundred).
+                           The two give bit-identical gradients.  d == 128
+                           with small_d_fused needs neither                    */
   int32_t loss_mode;    /* [0]   0 = one kurtosis per token (row) over its d
                            entries, loss = mean over tokens; 1 = the loss
                            equation of Section 2 taken literally: one kurtosis

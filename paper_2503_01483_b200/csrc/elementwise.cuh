@@ -207,6 +207,50 @@ __global__ void k_moments_finalize(const float4* __restrict__ partial, int P, in
   }
 }
 
+// ------------------------------------------------ backward from a stored Y
+// G^T[j][t] = bf16( a c^3 - ab c - am3 ),  c = Y[t][j] - mu, with the row's coefficients coef[t] = {mu, a, ab, am3}
+// (the same expression, in the same float32 operations, as the GEMM epilogue that recomputes Y).
+// Y is N x d float32 (dense), G^T is d x ldg bf16.  Tiles of 64 tokens x 64 columns through shared memory so that
+// both the reads (along d) and the writes (along tokens) are coalesced.  grid (ceil(N/64), d/64): blocks that run
+// together write neighbouring 128-byte pieces of the same rows of G^T.  block 256.
+__global__ void k_grad_from_y(const float* __restrict__ Y, const float4* __restrict__ coef, int N, int d,
+                              __nv_bfloat16* __restrict__ gt, long long ldg) {
+  __shared__ __nv_bfloat16 tile[64][66];
+  __shared__ float4 cfs[64];
+  const int r0 = blockIdx.x * 64, c0 = blockIdx.y * 64;
+  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;  // ty in 0..3
+  float y[16];
+#pragma unroll
+  for (int q = 0; q < 16; ++q) {
+    const int row = r0 + ty + 4 * q;
+    y[q] = (row < N) ? Y[static_cast<long long>(row) * d + c0 + tx] : 0.f;
+  }
+  if (threadIdx.x < 64)
+    cfs[threadIdx.x] = (r0 + threadIdx.x < N) ? coef[r0 + threadIdx.x] : make_float4(0.f, 0.f, 0.f, 0.f);
+  __syncthreads();
+#pragma unroll
+  for (int q = 0; q < 16; ++q) {
+    const int r = ty + 4 * q;
+    const float4 cf = cfs[r];
+    const float c = y[q] - cf.x;
+    // rows past N: y = 0 and zero coefficients give 0; they are not written anyway
+    tile[tx][r] = __float2bfloat16_rn(fmaf(c, fmaf(cf.y * c, c, -cf.z), -cf.w));
+  }
+  __syncthreads();
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;  // 8 warps, each writes 8 of the 64 output rows
+#pragma unroll
+  for (int q = 0; q < 8; ++q) {
+    const int c = w + 8 * q;
+    const int t = r0 + 2 * lane;
+    __nv_bfloat16* dst = gt + static_cast<long long>(c0 + c) * ldg + t;
+    if (t + 1 < N) {
+      *reinterpret_cast<__nv_bfloat162*>(dst) = *reinterpret_cast<const __nv_bfloat162*>(&tile[c][2 * lane]);
+    } else if (t < N) {
+      dst[0] = tile[c][2 * lane];
+    }
+  }
+}
+
 // ------------------------------------------- flattened (whole-layer) kurtosis
 // The loss of Section 2 taken literally: one kurtosis over the concatenation of all tokens' entries (N*d values).
 // The rows' means and central moments (k_moments_finalize) are merged in two fixed-order passes: the global mean

@@ -47,8 +47,9 @@ struct GemmParams {
   // upper_only != 0 (square symmetric outputs): tiles that lie entirely below the diagonal are skipped
   int upper_only;
   // epilogue operands (which are used depends on EPI)
-  float* out;                 // kStoreF32: M x N, leading dimension ldo
+  float* out;                 // kStoreF32: M x N, leading dimension ldo; kMoments: the same when not null
   long long ldo;
+  int out_sector_aligned;     // out, split_stride*4 and ldo*4 are multiples of 32 bytes: 32-byte stores may be used
   float4* partial;            // kMoments: [n_tiles][M] records {mean, S2, S3, S4}
   const float4* coef;         // kGrad: per row {mu, a, ab, am3}
   __nv_bfloat16* gt;          // kGrad: G transposed, [N][ldg]
@@ -74,6 +75,22 @@ __device__ __forceinline__ unsigned int ordered_key(float x) {
 }
 __device__ __forceinline__ float ordered_value(unsigned int k) {
   return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+// 32 consecutive float32 of one output row (the accumulator chunk a thread holds): 32-byte stores when the
+// destination allows it, 16-byte stores otherwise.
+__device__ __forceinline__ void store_row32(float* dst, const uint32_t* v, bool sector_aligned) {
+  if (sector_aligned) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) st_global_v8(dst + 8 * j, v + 8 * j);
+  } else {
+    float4* d4 = reinterpret_cast<float4*>(dst);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      d4[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
+                          __uint_as_float(v[4 * j + 3]));
+    }
+  }
 }
 
 template <int BN>
@@ -295,15 +312,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
         for (int c0 = 0; c0 < BN; c0 += 32) {
           tmem_ld_32x32(t_addr + c0, v);
           tc_wait_ld();
-          if (row_ok) {
-            float4* dst = reinterpret_cast<float4*>(p.out + static_cast<long long>(unit / plain_tiles) * p.split_stride +
-                                                    static_cast<long long>(row) * p.ldo + n0 + c0);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
-                                   __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
-            }
-          }
+          if (row_ok)
+            store_row32(p.out + static_cast<long long>(unit / plain_tiles) * p.split_stride +
+                            static_cast<long long>(row) * p.ldo + n0 + c0,
+                        v, p.out_sector_aligned != 0);
         }
       } else if constexpr (EPI == kMoments) {
         // pass 1: mean of the BN columns; pass 2: central power sums about it
@@ -328,6 +340,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
         for (int c0 = 0; c0 < BN; c0 += 32) {
           tmem_ld_32x32(t_addr + c0, v);
           tc_wait_ld();
+          // keep the float32 tile for the backward pass (the caller's choice; see kt_config.backward_mode)
+          if (p.out != nullptr && row_ok)
+            store_row32(p.out + static_cast<long long>(row) * p.ldo + n0 + c0, v, p.out_sector_aligned != 0);
           float b2 = 0.f, b3 = 0.f, b4 = 0.f;
 #pragma unroll
           for (int j = 0; j < 32; ++j) {

@@ -79,6 +79,7 @@ struct WsLayout {
   size_t dr;            // d x d float32: gradient inside kt_fit
   size_t xb;            // dense bf16 copy of a float32 X, or of any X after RMSNorm  [N][d]
   size_t xt, gt;        // X^T and G^T as bf16  [d][ldt]
+  size_t ybuf;          // Y = X R as float32 [N][d], kept by the forward pass unless the backward recomputes it
   size_t partial;       // [P][N] float4 partial moment records
   size_t coef, moments; // [N] float4 each
   size_t block_loss, block_deg, norm_blocks;
@@ -104,6 +105,7 @@ static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, const kt_conf
                             int gather_batch = 0) {
   const bool adam = cfg != nullptr && cfg->optimizer == 1;
   const bool xcopy = x_dtype == KT_F32 || (cfg != nullptr && cfg->rmsnorm != 0) || gather_batch > 0;
+  const bool keep_y = cfg == nullptr || cfg->backward_mode != 1;  // Y kept in float32 for the backward pass
   WsLayout L;
   memset(&L, 0, sizeof(L));
   L.bn = (d % 256 == 0) ? 256 : 128;
@@ -131,6 +133,7 @@ static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, const kt_conf
   L.xb = take(xcopy ? static_cast<size_t>(N) * d * 2 : 0);
   L.xt = take(static_cast<size_t>(d) * L.ldt * 2);
   L.gt = take(static_cast<size_t>(d) * L.ldt * 2);
+  L.ybuf = take(keep_y ? static_cast<size_t>(N) * d * 4 : 0);
   L.partial = take(static_cast<size_t>(L.P) * N * 16);
   L.coef = take(static_cast<size_t>(N) * 16);
   L.moments = take(static_cast<size_t>(N) * 16);
@@ -275,6 +278,11 @@ static kt_status run_gemm(kt_ctx* ctx, int M, int N, int K, int terms, const Ope
     p.kb_per_split = (K + kBK - 1) / kBK;
   }
   p.err_word = &ctx->d_blk->sc.err_word;
+  // 32-byte stores need every row start on a 32-byte boundary (the column offsets are multiples of 32 floats)
+  p.out_sector_aligned = (p.out != nullptr && (reinterpret_cast<uintptr_t>(p.out) & 31u) == 0 && (p.ldo & 7) == 0 &&
+                          (p.split_stride & 7) == 0)
+                             ? 1
+                             : 0;
   for (int q = 0; q < terms; ++q) {
     KT_TRY(make_tmap(ctx, &p.tmA[q], A[q].base, K, M, A[q].ld, kBM));
     KT_TRY(make_tmap(ctx, &p.tmB[q], B[q].base, K, N, B[q].ld, bn));
@@ -397,9 +405,15 @@ static FwdOperands fwd_operands(kt_ctx* ctx, const XView& xv, int d, long long N
 }
 
 // moments + loss for the rows of xv; R^T must already be in rt_hi.
-static kt_status forward_loss(kt_ctx* ctx, const XView& xv, int N, int d, const WsLayout& L, double* hist_slot) {
+// keep_y: the epilogue also stores the float32 Y tile into the workspace (for the backward pass).
+static kt_status forward_loss(kt_ctx* ctx, const XView& xv, int N, int d, const WsLayout& L, double* hist_slot,
+                              bool keep_y = false) {
   GemmParams p = blank_params();
   p.partial = at<float4>(ctx, L.partial);
+  if (keep_y) {
+    p.out = at<float>(ctx, L.ybuf);
+    p.ldo = d;
+  }
   const FwdOperands f = fwd_operands(ctx, xv, d, N, L);
   KT_TRY(run_gemm<kMoments>(ctx, N, d, d, f.terms, f.A, f.B, p, kCatForward));
   k_moments_finalize<<<L.loss_blocks, 256, 0, ctx->stream>>>(at<float4>(ctx, L.partial), L.P, N, d, L.bn,
@@ -437,14 +451,25 @@ static kt_status forward_loss(kt_ctx* ctx, const XView& xv, int N, int d, const 
   return KT_OK;
 }
 
-// dR = X^T G, G recomputed from the saved row coefficients.
+// dR = X^T G with G from the saved row coefficients and Y: either the Y tile is recomputed by a second pass of the
+// forward GEMM (nothing of Y ever reaches memory), or the float32 Y the forward pass kept is read back by an
+// element-wise kernel.  Both evaluate the same float32 expression on the same accumulator values: the same bits.
+static bool keep_y_for_backward(const kt_ctx* ctx) { return ctx->cfg.backward_mode != 1; }
+
 static kt_status backward(kt_ctx* ctx, const XView& xv, int N, int d, const WsLayout& L, float* dR) {
-  GemmParams p = blank_params();
-  p.coef = at<float4>(ctx, L.coef);
-  p.gt = at<__nv_bfloat16>(ctx, L.gt);
-  p.ldg = L.ldt;
-  const FwdOperands f = fwd_operands(ctx, xv, d, N, L);
-  KT_TRY(run_gemm<kGrad>(ctx, N, d, d, f.terms, f.A, f.B, p, kCatBackwardA));
+  if (keep_y_for_backward(ctx)) {
+    dim3 grid((N + 63) / 64, d / 64);
+    k_grad_from_y<<<grid, 256, 0, ctx->stream>>>(at<float>(ctx, L.ybuf), at<float4>(ctx, L.coef), N, d,
+                                                 at<__nv_bfloat16>(ctx, L.gt), L.ldt);
+    KT_LAUNCH_CHECK();
+  } else {
+    GemmParams p = blank_params();
+    p.coef = at<float4>(ctx, L.coef);
+    p.gt = at<__nv_bfloat16>(ctx, L.gt);
+    p.ldg = L.ldt;
+    const FwdOperands f = fwd_operands(ctx, xv, d, N, L);
+    KT_TRY(run_gemm<kGrad>(ctx, N, d, d, f.terms, f.A, f.B, p, kCatBackwardA));
+  }
   GemmParams p2 = blank_params();
   const SplitPlan sp = plan_split_k(d, N);
   p2.out = sp.splits > 1 ? at<float>(ctx, L.splitk) : dR;
@@ -467,7 +492,7 @@ static kt_status backward(kt_ctx* ctx, const XView& xv, int N, int d, const WsLa
 static kt_status loss_grad_async(kt_ctx* ctx, const XView& xv, int N, int d, const WsLayout& L, const float* R,
                                  float* dR, double* hist_slot, bool rt_current) {
   if (!rt_current) KT_TRY(cast_rt(ctx, R, d, N, L));
-  KT_TRY(forward_loss(ctx, xv, N, d, L, hist_slot));
+  KT_TRY(forward_loss(ctx, xv, N, d, L, hist_slot, keep_y_for_backward(ctx)));
   KT_TRY(backward(ctx, xv, N, d, L, dR));
   return KT_OK;
 }
@@ -896,6 +921,7 @@ void kt_default_config(kt_config* cfg) {
   cfg->beta2 = 0.99f;
   cfg->adam_eps = 1e-8f;
   cfg->norm_iters = 2;
+  cfg->backward_mode = 0;
   cfg->loss_mode = 0;
   cfg->rmsnorm = 0;
   cfg->rms_eps = 1e-6f;

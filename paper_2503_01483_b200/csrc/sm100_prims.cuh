@@ -181,4 +181,12 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16_f32(int M, int N) {
          (static_cast<uint32_t>(M >> 4) << 24);
 }
 
+// Eight consecutive float32 (32 bytes, 32-byte aligned) in one store: a whole DRAM sector per lane, so that
+// row-per-thread epilogues do not leave half-written sectors for the L2 to fill from memory.
+__device__ __forceinline__ void st_global_v8(float* dst, const uint32_t* v) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(v[0]), "r"(v[1]), "r"(v[2]),
+               "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+               : "memory");
+}
+
 }  // namespace kt
