@@ -5,13 +5,14 @@
 // A_q is M x K and B_q is N x K, both bf16 with k contiguous ("K-major"); the
 // accumulator is float32 in tensor memory.  One CTA per SM walks the output
 // tiles (128 x BN); warp 0 feeds shared memory with TMA, warp 1 issues the MMAs,
-// warps 2..5 drain the accumulator.  Two accumulators alternate, so the epilogue
+// warps 2..9 drain the accumulator (two warps per 32 rows, half the columns each).  Two accumulators alternate, so the epilogue
 // of one tile overlaps the MMAs of the next.  What the epilogue does with a
 // finished tile is selected by `EPI`:
 //
 //   kStoreF32  write D as float32
-//   kMoments   per row: mean and central power sums of the tile's BN columns
-//              (Eq. 3 of the paper, one partial record per column tile)
+//   kMoments   per row: mean and central power sums of BN/2 columns (Eq. 3 of the
+//              paper, one partial record per half column tile); optionally also
+//              stores D as float32
 //   kGrad      G = a c^3 - ab c - am3, c = D - mu  (derivative of the loss
 //              through Eq. 3), written transposed as bf16
 //   kAbsMax    per-row max |D| (first pass of the symmetric quantizer)
@@ -29,7 +30,7 @@ constexpr int kBM = 128;           // rows per tile = tensor-memory lanes
 #endif
 constexpr int kGroupM = KT_GROUP_M;  // row tiles per group of the tile order
 constexpr int kBK = 64;            // k elements per pipeline stage (one 128-byte swizzle row)
-constexpr int kGemmThreads = 192;  // 6 warps
+constexpr int kGemmThreads = 320;  // 10 warps: TMA, MMA, 8 epilogue warps (two per tensor-memory lane quarter)
 constexpr int kMaxTerms = 3;
 
 enum Epi : int { kStoreF32 = 0, kMoments = 1, kGrad = 2, kAbsMax = 3, kQuantErr = 4 };
@@ -50,7 +51,7 @@ struct GemmParams {
   float* out;                 // kStoreF32: M x N, leading dimension ldo; kMoments: the same when not null
   long long ldo;
   int out_sector_aligned;     // out, split_stride*4 and ldo*4 are multiples of 32 bytes: 32-byte stores may be used
-  float4* partial;            // kMoments: [n_tiles][M] records {mean, S2, S3, S4}
+  float4* partial;            // kMoments: [2 * n_tiles][M] records {mean, S2, S3, S4}, one per half tile of columns
   const float4* coef;         // kGrad: per row {mu, a, ab, am3}
   __nv_bfloat16* gt;          // kGrad: G transposed, [N][ldg]
   long long ldg;
@@ -58,7 +59,7 @@ struct GemmParams {
   // Asymmetric (rowmin != null): rowmax / rowmin = per-row max D / min D as order-preserving keys (ordered_key()).
   unsigned int* rowmax;
   unsigned int* rowmin;
-  float* qerr;                // kQuantErr: [n_tiles][M] partial squared errors
+  float* qerr;                // kQuantErr: [2 * n_tiles][M] partial squared errors, one per half tile of columns
   // kQuantErr: step = clip * range / q_den with range = max|D| (symmetric) or max - min (asymmetric, shift =
   // clip * min); codes are clamped to [q_lo, q_hi]
   float q_clip, q_den, q_lo, q_hi;
@@ -180,7 +181,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
       }
       for (int b = 0; b < 2; ++b) {
         mbar_init(acc_full_bar(b), 1);
-        mbar_init(acc_empty_bar(b), 4);
+        mbar_init(acc_empty_bar(b), 8);
       }
       fence_barrier_init();
     }
@@ -284,6 +285,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
   } else {
     // ---------------------------------------------------------------- epilogue
     const int lane_group = warp & 3;  // a warp may touch only tensor-memory lanes 32*(warp%4)..+31
+    // warps 2..5 take the left half of the tile's columns, warps 6..9 the right half: per-row records
+    // (moments, quantisation error) are therefore per half tile, index 2 * n_tile + half
+    constexpr int kHalf = BN / 2;
+    const int half = (warp - 2) >> 2;
+    const int cbeg = half * kHalf, cend = cbeg + kHalf;
     int lt = 0;
     bool ok = true;
     for (int unit = blockIdx.x; unit < total_tiles && ok; unit += gridDim.x) {
@@ -309,7 +315,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
 
       if constexpr (EPI == kStoreF32) {
 #pragma unroll 1
-        for (int c0 = 0; c0 < BN; c0 += 32) {
+        for (int c0 = cbeg; c0 < cend; c0 += 32) {
           tmem_ld_32x32(t_addr + c0, v);
           tc_wait_ld();
           if (row_ok)
@@ -321,7 +327,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
         // pass 1: mean of the BN columns; pass 2: central power sums about it
         float s1 = 0.f;
 #pragma unroll 1
-        for (int c0 = 0; c0 < BN; c0 += 32) {
+        for (int c0 = cbeg; c0 < cend; c0 += 32) {
           tmem_ld_32x32(t_addr + c0, v);
           tc_wait_ld();
           float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
@@ -334,10 +340,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
           }
           s1 += (a0 + a1) + (a2 + a3);
         }
-        const float mean = s1 * (1.0f / BN);
+        const float mean = s1 * (1.0f / kHalf);
         float s2 = 0.f, s3 = 0.f, s4 = 0.f;
 #pragma unroll 1
-        for (int c0 = 0; c0 < BN; c0 += 32) {
+        for (int c0 = cbeg; c0 < cend; c0 += 32) {
           tmem_ld_32x32(t_addr + c0, v);
           tc_wait_ld();
           // keep the float32 tile for the backward pass (the caller's choice; see kt_config.backward_mode)
@@ -356,13 +362,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
           s3 += b3;
           s4 += b4;
         }
-        if (row_ok) p.partial[static_cast<long long>(n_tile) * p.M + row] = make_float4(mean, s2, s3, s4);
+        if (row_ok) p.partial[static_cast<long long>(2 * n_tile + half) * p.M + row] = make_float4(mean, s2, s3, s4);
       } else if constexpr (EPI == kGrad) {
         float4 cf = make_float4(0.f, 0.f, 0.f, 0.f);
         if (row_ok) cf = p.coef[row];
         __nv_bfloat16* gcol = p.gt + static_cast<long long>(n0) * p.ldg + row;
 #pragma unroll 1
-        for (int c0 = 0; c0 < BN; c0 += 32) {
+        for (int c0 = cbeg; c0 < cend; c0 += 32) {
           tmem_ld_32x32(t_addr + c0, v);
           tc_wait_ld();
           if (row_ok) {
@@ -379,7 +385,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
         const bool asym = p.rowmin != nullptr;
         float mx = asym ? -INFINITY : 0.f, mn = INFINITY;
 #pragma unroll 1
-        for (int c0 = 0; c0 < BN; c0 += 32) {
+        for (int c0 = cbeg; c0 < cend; c0 += 32) {
           tmem_ld_32x32(t_addr + c0, v);
           tc_wait_ld();
           if (asym) {
@@ -419,7 +425,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
         const float s = __fdiv_rn(range, p.q_den);
         float e2 = 0.f;
 #pragma unroll 1
-        for (int c0 = 0; c0 < BN; c0 += 32) {
+        for (int c0 = cbeg; c0 < cend; c0 += 32) {
           tmem_ld_32x32(t_addr + c0, v);
           tc_wait_ld();
 #pragma unroll
@@ -434,7 +440,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
             e2 = fmaf(e, e, e2);
           }
         }
-        if (row_ok) p.qerr[static_cast<long long>(n_tile) * p.M + row] = e2;
+        if (row_ok) p.qerr[static_cast<long long>(2 * n_tile + half) * p.M + row] = e2;
       }
 
       // hand the accumulator back to the MMA warp

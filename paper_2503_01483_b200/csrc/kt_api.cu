@@ -108,7 +108,7 @@ static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, const kt_conf
   const bool keep_y = cfg == nullptr || cfg->backward_mode != 1;  // Y kept in float32 for the backward pass
   WsLayout L;
   memset(&L, 0, sizeof(L));
-  L.bn = (d % 256 == 0) ? 256 : 128;
+  L.bn = (d % 256 == 0) ? 128 : 64;  // columns per moment record: half a GEMM column tile
   L.P = static_cast<int>(d / L.bn);
   L.ldt = static_cast<long long>(align_up(static_cast<size_t>(N), 64));
   L.loss_blocks = static_cast<int>((N + 255) / 256);
@@ -1458,7 +1458,7 @@ kt_status kt_kurtosis_loss_noalloc(kt_mat X, const float* R, double* loss_dev, v
   // carve the array: [scalar block][R^T hi][R^T lo][records ...]; sizes are bounded by the maxima above
   WsLayout L;
   memset(&L, 0, sizeof(L));
-  L.bn = (d % 256 == 0) ? 256 : 128;
+  L.bn = (d % 256 == 0) ? 128 : 64;  // columns per moment record: half a GEMM column tile
   L.P = static_cast<int>(d / L.bn);
   L.loss_blocks = static_cast<int>((N + 255) / 256);
   size_t off = align_up(sizeof(DeviceBlock), 256);
