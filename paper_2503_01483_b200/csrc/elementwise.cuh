@@ -579,13 +579,17 @@ __global__ void k_skew_matvec(const __nv_bfloat16* __restrict__ W, int d, const 
 // One block of 1024 threads: ||W||_F, alpha = min(lr, 2q/(||W||_F + eps)), and the decisions that depend on
 // x = alpha ||W||_2 (bounded by alpha ||W||_F; estimated by a short power iteration when pv_prev/pv_last are given):
 //  * n_terms: term k of the series changes R by at most x (x/2)^k (Frobenius bounds the spectral norm, ||R|| = 1);
-//    terms below a quarter unit in the last place of a typical entry (2^-26 / sqrt(d)) are skipped (`gate_terms`);
+//    terms below a quarter unit in the last place of a typical entry (2^-26 / sqrt(d)) are skipped (`gate_terms`),
+//    and so are terms below a quarter of the error the first term already carries because W enters it as bf16
+//    (x 2^-9): (x/2)^k < 2^-11.  What a dropped term would have done for orthogonality (x^2 per step at most) is
+//    in the drift bound below and is repaired by the guard;
 //  * p0_terms: P_0 = W R multiplies alpha directly; with R as a single bf16 term its error is x 2^-9, which is
 //    accepted while that is below 2.5e-6 (a quarter of the default polish threshold), else hi + lo
 //    (`cfg_terms` 1..3 forces a count, 0 = this rule);
 //  * gate_guard: guard_mode 1 = measure R^T R - I in this step, 2 = do not, 0 = only when the drift bound, which
-//    grows by x^2 + x 2^-9 (or x 2^-17 with two terms) + 4e-7 per step (truncation of the series; rounding of R in
-//    P_0; float32 rounding of the update), has reached half the polish threshold.  A measuring step also clears the running maximum.
+//    grows by x^2 + x 2^-9 (or x 2^-17 with two terms) + n_terms 2^-23 per step (truncation of the series; rounding
+//    of R in P_0; float32 rounding of the update: half an ulp per entry and series term, all aligned, through
+//    E = R^T dR + dR^T R with unit columns), has reached half the polish threshold.  A measuring step also clears the running maximum.
 __global__ void k_step_size(const double* __restrict__ block_norm2, int n, float lr, float q, float eps,
                             Scalars* __restrict__ sc, int d, int iters, int cfg_terms, int gate_terms, int guard_mode,
                             float thresh, const float* __restrict__ pv_prev, const float* __restrict__ pv_last) {
@@ -631,7 +635,7 @@ __global__ void k_step_size(const double* __restrict__ block_norm2, int n, float
     double bound = x;
     for (int k = 1; k <= iters; ++k) {
       bound *= 0.5 * x;
-      if (gate_terms && bound < floor_k) break;
+      if (gate_terms && (bound < floor_k || bound < x * ldexp(1.0, -11))) break;
       ++nt;
     }
     sc->n_terms = nt;
@@ -644,7 +648,8 @@ __global__ void k_step_size(const double* __restrict__ block_norm2, int n, float
     } else if (guard_mode == 2) {
       gg = 0u;
     } else {
-      const float drift = sc->drift + static_cast<float>(x * x + x * ldexp(1.0, p0t == 1u ? -9 : -17)) + 4e-7f;
+      const float drift = sc->drift + static_cast<float>(x * x + x * ldexp(1.0, p0t == 1u ? -9 : -17) +
+                                                        nt * ldexp(1.0, -23));
       sc->drift = drift;
       gg = (thresh <= 0.f || drift >= 0.5f * thresh) ? 1u : 0u;
     }
