@@ -200,6 +200,9 @@ def main():
     ap.add_argument("--forward-terms", type=int, default=0, help="kt_config.forward_terms (0 = automatic)")
     ap.add_argument("--optimizer", default="sgd", choices=["sgd", "adam"],
                     help="kt_config.optimizer: Cayley SGD (the headline configuration) or Cayley Adam")
+    ap.add_argument("--backward", default="stored", choices=["stored", "recompute"],
+                    help="kt_config.backward_mode: read back the float32 Y the forward pass kept (default) or "
+                         "recompute Y in a second GEMM pass")
     ap.add_argument("--loss-mode", default="token", choices=["token", "layer"],
                     help="kt_config.loss_mode: one kurtosis per token (headline) or one over the whole layer")
     ap.add_argument("--rmsnorm", action="store_true", help="kt_config.rmsnorm: row-normalise X first")
@@ -248,7 +251,8 @@ def main():
     N = SHARED_RPS * SHARED_BATCH if shared else X.shape[0]
     lr = cfg["lr"]
     ctx = kurtail.Context(dev, forward_terms=args.forward_terms, optimizer=1 if args.optimizer == "adam" else 0,
-                          loss_mode=1 if args.loss_mode == "layer" else 0, rmsnorm=1 if args.rmsnorm else 0)
+                          loss_mode=1 if args.loss_mode == "layer" else 0, rmsnorm=1 if args.rmsnorm else 0,
+                          backward_mode=1 if args.backward == "recompute" else 0)
 
     def fresh_R():
         if cfg["init"] == "hadamard":
@@ -363,15 +367,17 @@ def main():
         achieved = flops_per_launch / (t_tok / max(n_launch, 1) * 1e-3) / 1e12 if t_tok > 0 else None
         peak = peaks["tflops_sustained"]
         traffic = None
-        if args.workload == "llama2_7b_attn":
-            # mean DRAM bytes per launch of the three kernels: ncu capture at N = 16384 (same d); the part that
-            # grows with N (everything but the 33.5 MB of R^T read by forward and backward-A) is scaled by N / 16384
-            var_mb = (167.8 + 7.3 - 33.5) + (174.8 + 116.5 - 33.5) + (683.8 + 62.2)
-            traffic = (var_mb * (N / 16384.0) + 2 * 33.5) / 3.0 * 1e6
+        if args.workload == "llama2_7b_attn" and not tok[1]["launches"]:
+            # mean DRAM bytes per launch of the two token GEMMs (forward with its float32 Y store, backward-B): ncu
+            # capture at N = 16384 (same d); the part that grows with N (everything but the 33.5 MB of R^T read by
+            # the forward pass) is scaled by N / 16384
+            var_mb = (376.0 + 248.6 - 33.5) + (627.8 + 61.5)
+            traffic = (var_mb * (N / 16384.0) + 33.5) / 2.0 * 1e6
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                     "frac": (achieved / peak) if achieved else None, "traffic": traffic,
                     "frac_of_burst_peak": (achieved / peaks["tflops_burst"]) if achieved else None,
-                    "kernel": "gemm_tn_kernel (forward+moments, backward-A, backward-B): 2*N*d^2 flops per launch",
+                    "kernel": "gemm_tn_kernel (forward + moments, backward-B; backward-A too when it recomputes Y): "
+                              "2*N*d^2 flops per launch",
                     "peak_source": "%s bf16 GEMM, sustained (kernel timed inside a long step)" % peaks["source"],
                     "per_role_ms_per_launch": per_role, "share_of_step": share}
 
@@ -382,6 +388,7 @@ def main():
         "data": "synthetic",
         "config": {"workload": args.workload, "N": N, "d": d, "R_init": cfg["init"], "lr": lr,
                    "optimizer": "cayley_" + args.optimizer, "loss_mode": args.loss_mode, "rmsnorm": bool(args.rmsnorm),
+                   "backward": args.backward,
                    "l2": "inputs (%.0f MiB of X per step) exceed the 126 MB L2" % (N * d * 2 / 2**20)
                    if N * d * 2 > 126e6 else "inputs fit in L2; no flush (small case)",
                    "parallelism": "one independent layer per GPU" if world > 1 else "single GPU",
