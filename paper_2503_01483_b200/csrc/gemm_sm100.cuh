@@ -324,38 +324,45 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
                         v, p.out_sector_aligned != 0);
         }
       } else if constexpr (EPI == kMoments) {
-        // pass 1: mean of the BN columns; pass 2: central power sums about it
+        // The thread's half row (kHalf columns) is read into registers in one go and the accumulator goes back to the
+        // MMA warp at once: the arithmetic and the stores below no longer sit between two tiles' MMAs.
+        constexpr int kChunks = kHalf / 32;
+        uint32_t vv[kChunks][32];
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c) tmem_ld_32x32(t_addr + cbeg + 32 * c, vv[c]);
+        tc_wait_ld();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acc_empty_bar(buf));
+        // pass 1: mean of the kHalf columns; pass 2: central power sums about it
         float s1 = 0.f;
-#pragma unroll 1
-        for (int c0 = cbeg; c0 < cend; c0 += 32) {
-          tmem_ld_32x32(t_addr + c0, v);
-          tc_wait_ld();
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c) {
           float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
-            a0 += __uint_as_float(v[j]);
-            a1 += __uint_as_float(v[j + 1]);
-            a2 += __uint_as_float(v[j + 2]);
-            a3 += __uint_as_float(v[j + 3]);
+            a0 += __uint_as_float(vv[c][j]);
+            a1 += __uint_as_float(vv[c][j + 1]);
+            a2 += __uint_as_float(vv[c][j + 2]);
+            a3 += __uint_as_float(vv[c][j + 3]);
           }
           s1 += (a0 + a1) + (a2 + a3);
         }
         const float mean = s1 * (1.0f / kHalf);
         float s2 = 0.f, s3 = 0.f, s4 = 0.f;
-#pragma unroll 1
-        for (int c0 = cbeg; c0 < cend; c0 += 32) {
-          tmem_ld_32x32(t_addr + c0, v);
-          tc_wait_ld();
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c) {
           // keep the float32 tile for the backward pass (the caller's choice; see kt_config.backward_mode)
           if (p.out != nullptr && row_ok)
-            store_row32(p.out + static_cast<long long>(row) * p.ldo + n0 + c0, v, p.out_sector_aligned != 0);
+            store_row32(p.out + static_cast<long long>(row) * p.ldo + n0 + cbeg + 32 * c, vv[c],
+                        p.out_sector_aligned != 0);
           float b2 = 0.f, b3 = 0.f, b4 = 0.f;
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
-            const float c = __uint_as_float(v[j]) - mean;
-            const float c2 = c * c;
+            const float cc = __uint_as_float(vv[c][j]) - mean;
+            const float c2 = cc * cc;
             b2 += c2;
-            b3 = fmaf(c2, c, b3);
+            b3 = fmaf(c2, cc, b3);
             b4 = fmaf(c2, c2, b4);
           }
           s2 += b2;
@@ -443,10 +450,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
         if (row_ok) p.qerr[static_cast<long long>(2 * n_tile + half) * p.M + row] = e2;
       }
 
-      // hand the accumulator back to the MMA warp
-      tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(acc_empty_bar(buf));
+      // hand the accumulator back to the MMA warp (kMoments did so as soon as it had the tile in registers)
+      if constexpr (EPI != kMoments) {
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acc_empty_bar(buf));
+      }
       ++lt;
     }
   }
