@@ -126,6 +126,10 @@ typedef struct {
                            B200 the cheaper one for d above a few hundred).
                            The two give bit-identical gradients.  d == 128
                            with small_d_fused needs neither                    */
+  int32_t cta_pairs;    /* [1]   1 = GEMMs with 256-wide column tiles run on
+                           pairs of CTAs (thread-block clusters of two, one
+                           MMA over both SMs' tensor cores, each CTA loading
+                           half of the second operand); 0 = one CTA per tile  */
   int32_t loss_mode;    /* [0]   0 = one kurtosis per token (row) over its d
                            entries, loss = mean over tokens; 1 = the loss
                            equation of Section 2 taken literally: one kurtosis

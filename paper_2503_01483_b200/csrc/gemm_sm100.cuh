@@ -94,22 +94,31 @@ __device__ __forceinline__ void store_row32(float* dst, const uint32_t* v, bool 
   }
 }
 
-template <int BN>
+// CTAS = 2: a pair of CTAs works on a 256 x BN tile; each CTA stages its 128 rows of A and BN/2 rows of B.
+template <int BN, int CTAS = 1>
 struct GemmSmem {
-  static constexpr int kStages = (BN == 256) ? 4 : 6;
+  static constexpr int kBRows = BN / CTAS;  // rows of B this CTA loads per k-block
+  static constexpr int kStages = (kBRows == 256) ? 4 : 6;
   static constexpr int kABytes = kBM * kBK * 2;
-  static constexpr int kBBytes = BN * kBK * 2;
+  static constexpr int kBBytes = kBRows * kBK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kBarBytes = 256;
   static constexpr int kTotal = 1024 /*alignment slack*/ + kStages * kStageBytes + kBarBytes;
 };
 
-template <int BN, int EPI>
+template <int BN, int EPI, int CTAS = 1>
 __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_constant__ GemmParams p) {
-  using S = GemmSmem<BN>;
+  using S = GemmSmem<BN, CTAS>;
   constexpr int kStages = S::kStages;
+  constexpr int kTileM = kBM * CTAS;      // rows of an output tile (of the pair's, when CTAS = 2)
+  constexpr int kGroup = kGroupM / CTAS;  // row tiles per group of the tile order
   constexpr uint32_t kTmemCols = 2 * BN;  // two accumulators: 256 or 512 columns
-  constexpr uint32_t kIdesc = umma_idesc_bf16_f32(kBM, BN);
+  constexpr uint32_t kIdesc = umma_idesc_bf16_f32(kTileM, BN);
+  // CTAS = 2 (launched as clusters of two): rank 0 of a pair is the leader: it issues the MMAs for both and owns the
+  // barriers that count loads (full) and drained accumulators (acc_empty); both CTAs own stage (empty) and
+  // accumulator-ready (acc_full) barriers, which the leader's commits reach in both at once.
+  const uint32_t rank = (CTAS == 2) ? cluster_ctarank() : 0u;
+  const int first_unit = blockIdx.x / CTAS, unit_step = gridDim.x / CTAS;
 
   if (p.gate != nullptr && *p.gate < p.gate_min) return;  // uniform over the grid
   int n_terms = p.terms;
@@ -146,18 +155,18 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
   // A and CTAs/kGroupM column panels of B instead of a few row panels and all of B (which, once B no longer fits
   // in L2, streamed the whole of B from memory for every two or three row tiles).
   auto tile_mn = [&](int tile, int& mt, int& nt) {
-    const int per_group = kGroupM * p.n_tiles;
+    const int per_group = kGroup * p.n_tiles;
     const int g = tile / per_group, r = tile - g * per_group;
-    const int rem = p.m_tiles - g * kGroupM;
-    const int gm = rem < kGroupM ? rem : kGroupM;
+    const int rem = p.m_tiles - g * kGroup;
+    const int gm = rem < kGroup ? rem : kGroup;
     nt = r / gm;
-    mt = g * kGroupM + (r - nt * gm);
+    mt = g * kGroup + (r - nt * gm);
   };
   auto skipped = [&](int tile) {
     if (p.upper_only == 0) return false;
     int mt, nt;
     tile_mn(tile, mt, nt);
-    return (nt + 1) * BN <= mt * kBM;
+    return (nt + 1) * BN <= mt * kTileM;
   };
   auto unit_kb0 = [&](int u) { return (u / plain_tiles) * p.kb_per_split; };
   auto unit_iters = [&](int u) {
@@ -181,16 +190,22 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
       }
       for (int b = 0; b < 2; ++b) {
         mbar_init(acc_full_bar(b), 1);
-        mbar_init(acc_empty_bar(b), 8);
+        mbar_init(acc_empty_bar(b), 8 * CTAS);  // every epilogue warp of every CTA of the tile
       }
       fence_barrier_init();
     }
     __syncwarp();
-    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
-    tmem_relinquish();
+    if constexpr (CTAS == 2) {
+      tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+      tmem_relinquish_pair();
+    } else {
+      tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+      tmem_relinquish();
+    }
   }
   tc_fence_before_sync();
   __syncthreads();
+  if constexpr (CTAS == 2) cluster_sync_all();  // the partner's barriers exist before anything reaches them
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -202,13 +217,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
       uint32_t issued_mask = 0;  // stages that have had a load issued
       uint32_t last_parity = 0;  // parity of the last load issued, per stage
       bool ok = true;
-      for (int unit = blockIdx.x; unit < total_tiles && ok; unit += gridDim.x) {
+      for (int unit = first_unit; unit < total_tiles && ok; unit += unit_step) {
         const int tile = unit % plain_tiles;
         if (skipped(tile)) continue;
         int m_tile, n_tile;
         tile_mn(tile, m_tile, n_tile);
-        const int m0 = m_tile * kBM;
-        const int n0 = n_tile * BN;
+        const int m0 = m_tile * kTileM + static_cast<int>(rank) * kBM;         // this CTA's rows of A
+        const int n0 = n_tile * BN + static_cast<int>(rank) * S::kBRows;        // this CTA's rows of B
         const int kb0 = unit_kb0(unit);
         const int iters = unit_iters(unit);
         for (int it = 0; it < iters; ++it) {
@@ -219,9 +234,17 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
             ok = false;
             break;
           }
-          mbar_arrive_expect_tx(full_bar(stage), S::kStageBytes);
-          tma_load_2d(smem_a + stage * S::kABytes, &p.tmA[q], kb * kBK, m0, full_bar(stage));
-          tma_load_2d(smem_b + stage * S::kBBytes, &p.tmB[q], kb * kBK, n0, full_bar(stage));
+          if constexpr (CTAS == 2) {
+            // both CTAs' bytes are counted on the leader's barrier; only the leader announces them
+            if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * S::kStageBytes);
+            const uint32_t lead_full = cluster_map_shared(full_bar(stage), 0);
+            tma_load_2d_pair(smem_a + stage * S::kABytes, &p.tmA[q], kb * kBK, m0, lead_full);
+            tma_load_2d_pair(smem_b + stage * S::kBBytes, &p.tmB[q], kb * kBK, n0, lead_full);
+          } else {
+            mbar_arrive_expect_tx(full_bar(stage), S::kStageBytes);
+            tma_load_2d(smem_a + stage * S::kABytes, &p.tmA[q], kb * kBK, m0, full_bar(stage));
+            tma_load_2d(smem_b + stage * S::kBBytes, &p.tmB[q], kb * kBK, n0, full_bar(stage));
+          }
           issued_mask |= 1u << stage;
           last_parity = (last_parity & ~(1u << stage)) | (phase << stage);
           if (++stage == kStages) {
@@ -230,7 +253,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
           }
         }
       }
-      if (!ok) {
+      if (!ok && rank == 0) {
         // leave no copy in flight behind: wait (bounded) for every load issued
         for (int s = 0; s < kStages; ++s) {
           if (!(issued_mask & (1u << s))) continue;
@@ -242,13 +265,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
       }
     }
   } else if (warp == 1) {
-    // -------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
+    // -------------------------------------------------------------- MMA issuer (of a pair: the leader only)
+    if (lane == 0 && rank == 0) {
       int stage = 0;
       uint32_t phase = 0;
       int lt = 0;
       bool ok = true;
-      for (int unit = blockIdx.x; unit < total_tiles && ok; unit += gridDim.x) {
+      for (int unit = first_unit; unit < total_tiles && ok; unit += unit_step) {
         if (skipped(unit % plain_tiles)) continue;
         const int iters = unit_iters(unit);
         const int buf = lt & 1;
@@ -270,15 +293,21 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
 #pragma unroll
           for (int kk = 0; kk < kBK / 16; ++kk) {
             // 16 k-elements = 32 bytes further along the swizzled row: +2 in address>>4 units
-            tc_mma_bf16(d_tmem, a_desc + 2u * kk, b_desc + 2u * kk, kIdesc, (it > 0 || kk > 0) ? 1u : 0u);
+            if constexpr (CTAS == 2)
+              tc_mma_bf16_pair(d_tmem, a_desc + 2u * kk, b_desc + 2u * kk, kIdesc, (it > 0 || kk > 0) ? 1u : 0u);
+            else
+              tc_mma_bf16(d_tmem, a_desc + 2u * kk, b_desc + 2u * kk, kIdesc, (it > 0 || kk > 0) ? 1u : 0u);
           }
-          tc_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
+          // frees the stage (in both CTAs of a pair) once these MMAs have read it
+          if constexpr (CTAS == 2) tc_commit_pair(empty_bar(stage), 3); else tc_commit(empty_bar(stage));
           if (++stage == kStages) {
             stage = 0;
             phase ^= 1u;
           }
         }
-        if (ok) tc_commit(acc_full_bar(buf));  // accumulator complete
+        if (ok) {  // accumulator complete
+          if constexpr (CTAS == 2) tc_commit_pair(acc_full_bar(buf), 3); else tc_commit(acc_full_bar(buf));
+        }
         ++lt;
       }
     }
@@ -290,14 +319,19 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
     constexpr int kHalf = BN / 2;
     const int half = (warp - 2) >> 2;
     const int cbeg = half * kHalf, cend = cbeg + kHalf;
+    // the leader counts drained accumulators: the partner's warps arrive on the leader's barrier
+    auto release_acc = [&](int b) {
+      if constexpr (CTAS == 2) mbar_arrive_cluster(cluster_map_shared(acc_empty_bar(b), 0));
+      else mbar_arrive(acc_empty_bar(b));
+    };
     int lt = 0;
     bool ok = true;
-    for (int unit = blockIdx.x; unit < total_tiles && ok; unit += gridDim.x) {
+    for (int unit = first_unit; unit < total_tiles && ok; unit += unit_step) {
       const int tile = unit % plain_tiles;
       if (skipped(tile)) continue;
       int m_tile, n_tile;
       tile_mn(tile, m_tile, n_tile);
-      const int row = m_tile * kBM + lane_group * 32 + lane;
+      const int row = m_tile * kTileM + static_cast<int>(rank) * kBM + lane_group * 32 + lane;
       const int n0 = n_tile * BN;
       const int buf = lt & 1;
       const uint32_t acc_phase = (lt >> 1) & 1;
@@ -333,7 +367,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
         tc_wait_ld();
         tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) mbar_arrive(acc_empty_bar(buf));
+        if (lane == 0) release_acc(buf);
         // pass 1: mean of the kHalf columns; pass 2: central power sums about it
         float s1 = 0.f;
 #pragma unroll
@@ -454,7 +488,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
       if constexpr (EPI != kMoments) {
         tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) mbar_arrive(acc_empty_bar(buf));
+        if (lane == 0) release_acc(buf);
       }
       ++lt;
     }
@@ -463,10 +497,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
   // ------------------------------------------------------------------ teardown
   tc_fence_before_sync();
   __syncthreads();
+  if constexpr (CTAS == 2) cluster_sync_all();  // neither CTA frees tensor memory or leaves while its partner still works
   if (warp == 1) {
     __syncwarp();
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, kTmemCols);
+    if constexpr (CTAS == 2) tmem_dealloc_pair(tmem_base, kTmemCols); else tmem_dealloc(tmem_base, kTmemCols);
   }
   if (threadIdx.x == 0 && *abort_flag != 0 && p.err_word != nullptr) atomicMax(p.err_word, *abort_flag);
 }

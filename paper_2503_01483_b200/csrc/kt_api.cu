@@ -236,19 +236,38 @@ static kt_status make_tmap(const kt_ctx* ctx, CUtensorMap* tm, const void* base,
   return r == CUDA_SUCCESS ? KT_OK : KT_ERR_CUDA;
 }
 
-template <int BN, int EPI>
+template <int BN, int EPI, int CTAS>
 static kt_status launch_gemm_inst(kt_ctx* ctx, const GemmParams& p, int cat) {
   static bool attr_done[16] = {false};
-  const int smem = GemmSmem<BN>::kTotal;
+  const int smem = GemmSmem<BN, CTAS>::kTotal;
   if (!attr_done[ctx->device & 15]) {
-    KT_CUDA(cudaFuncSetAttribute(gemm_tn_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    KT_CUDA(cudaFuncSetAttribute(gemm_tn_kernel<BN, EPI, CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     attr_done[ctx->device & 15] = true;
   }
-  const int tiles = p.m_tiles * p.n_tiles * p.k_splits;
-  const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+  // one CTA (or one pair of CTAs) per work unit, at most one CTA per SM
+  const int units = p.m_tiles * p.n_tiles * p.k_splits;
+  const int slots = ctx->sm_count / CTAS;
+  const int grid = (units < slots ? units : slots) * CTAS;
   const bool rec = ctx->prof_on && ctx->prof_used < kProfPairs;
   if (rec) KT_CUDA(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], ctx->stream));
-  gemm_tn_kernel<BN, EPI><<<grid, kGemmThreads, smem, ctx->stream>>>(p);
+  if (CTAS == 1) {
+    gemm_tn_kernel<BN, EPI, CTAS><<<grid, kGemmThreads, smem, ctx->stream>>>(p);
+  } else {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = ctx->stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = CTAS;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    KT_CUDA(cudaLaunchKernelEx(&cfg, gemm_tn_kernel<BN, EPI, CTAS>, p));
+  }
   KT_LAUNCH_CHECK();
   if (rec) {
     KT_CUDA(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used + 1], ctx->stream));
@@ -267,11 +286,13 @@ template <int EPI>
 static kt_status run_gemm(kt_ctx* ctx, int M, int N, int K, int terms, const Operand* A, const Operand* B,
                           GemmParams& p, int cat) {
   const int bn = (N % 256 == 0) ? 256 : 128;
+  // 256-wide tiles with more than one row tile run on pairs of CTAs (256 x 256 tiles, each CTA loading half of B)
+  const int ctas = (bn == 256 && M > kBM && ctx->cfg.cta_pairs != 0 && ctx->sm_count % 2 == 0) ? 2 : 1;
   p.terms = terms;
   p.M = M;
   p.N = N;
   p.K = K;
-  p.m_tiles = (M + kBM - 1) / kBM;
+  p.m_tiles = (M + kBM * ctas - 1) / (kBM * ctas);
   p.n_tiles = N / bn;
   if (p.k_splits < 1) {
     p.k_splits = 1;
@@ -285,10 +306,11 @@ static kt_status run_gemm(kt_ctx* ctx, int M, int N, int K, int terms, const Ope
                              : 0;
   for (int q = 0; q < terms; ++q) {
     KT_TRY(make_tmap(ctx, &p.tmA[q], A[q].base, K, M, A[q].ld, kBM));
-    KT_TRY(make_tmap(ctx, &p.tmB[q], B[q].base, K, N, B[q].ld, bn));
+    KT_TRY(make_tmap(ctx, &p.tmB[q], B[q].base, K, N, B[q].ld, bn / ctas));
   }
-  if (bn == 256) return launch_gemm_inst<256, EPI>(ctx, p, cat);
-  return launch_gemm_inst<128, EPI>(ctx, p, cat);
+  if (ctas == 2) return launch_gemm_inst<256, EPI, 2>(ctx, p, cat);
+  if (bn == 256) return launch_gemm_inst<256, EPI, 1>(ctx, p, cat);
+  return launch_gemm_inst<128, EPI, 1>(ctx, p, cat);
 }
 
 static GemmParams blank_params() {
@@ -922,6 +944,7 @@ void kt_default_config(kt_config* cfg) {
   cfg->adam_eps = 1e-8f;
   cfg->norm_iters = 2;
   cfg->backward_mode = 0;
+  cfg->cta_pairs = 1;
   cfg->loss_mode = 0;
   cfg->rmsnorm = 0;
   cfg->rms_eps = 1e-6f;
