@@ -371,7 +371,7 @@ def main():
             # mean DRAM bytes per launch of the two token GEMMs (forward with its float32 Y store, backward-B): ncu
             # capture at N = 16384 (same d); the part that grows with N (everything but the 33.5 MB of R^T read by
             # the forward pass) is scaled by N / 16384
-            var_mb = (376.0 + 248.6 - 33.5) + (627.8 + 61.5)
+            var_mb = (392.9 + 246.7 - 33.5) + (628.4 + 61.5)
             traffic = (var_mb * (N / 16384.0) + 33.5) / 2.0 * 1e6
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                     "frac": (achieved / peak) if achieved else None, "traffic": traffic,
