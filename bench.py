@@ -181,7 +181,7 @@ def run_reference(args, wl_name, d, N_full):
     print(json.dumps({
         "impl": "reference", "metric": METRIC + " at d=%d" % d, "value": val, "unit": "tokens/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_step * 1e3,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "higher_is_better": True, "scaling": "strong" if row_sharded else "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": wl_name, "N": N_full, "d": d},
         "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -200,6 +200,9 @@ def main():
     ap.add_argument("--forward-terms", type=int, default=0, help="kt_config.forward_terms (0 = automatic)")
     ap.add_argument("--optimizer", default="sgd", choices=["sgd", "adam"],
                     help="kt_config.optimizer: Cayley SGD (the headline configuration) or Cayley Adam")
+    ap.add_argument("--shard", default="layers", choices=["layers", "rows"],
+                    help="with --gpus N > 1: one independent layer per GPU (weak scaling, no collective), or the rows "
+                         "of one X sharded over the GPUs with an all-reduce of dR per step (strong scaling)")
     ap.add_argument("--backward", default="stored", choices=["stored", "recompute"],
                     help="kt_config.backward_mode: read back the float32 Y the forward pass kept (default) or "
                          "recompute Y in a second GEMM pass")
@@ -245,7 +248,13 @@ def main():
     cfg = synth.config(wl_cfg, **kw)
     Xs = cfg["X"] if isinstance(cfg["X"], list) else [cfg["X"]]   # all layer buffers stay resident in HBM
     X = Xs[0]
-    if world > 1:
+    row_sharded = world > 1 and args.shard == "rows" and not sweep and not shared
+    N_all = X.shape[0]
+    if row_sharded:
+        # every rank generated the same X: keep this rank's block of rows (multiples of 128 except the last)
+        per = (N_all // world + 127) // 128 * 128
+        X = X[rank * per:min((rank + 1) * per, N_all)].contiguous()
+    elif world > 1:
         # different data per rank: re-draw with a rank-dependent seed by rolling rows
         X = torch.roll(X, shifts=rank * 977, dims=0).contiguous()
     N = SHARED_RPS * SHARED_BATCH if shared else X.shape[0]
@@ -272,6 +281,8 @@ def main():
         w = max(args.warmup, 1)
         ctx.fit_shared(Xs, SHARED_RPS, order[:w * SHARED_BATCH], SHARED_BATCH, R, w, lr)
         order = order[w * SHARED_BATCH:]
+    elif row_sharded:
+        dist_util.fit_row_sharded(ctx, X, R, max(args.warmup, 1), lr, dist, N_all)
     else:
         ctx.fit(X, R, max(args.warmup, 1), lr)          # warm-up steps (also sizes the workspace)
     torch.cuda.synchronize()
@@ -294,6 +305,10 @@ def main():
         rep = reps[-1]
     elif shared:
         rep = ctx.fit_shared(Xs, SHARED_RPS, order, SHARED_BATCH, R, args.steps, lr)
+    elif row_sharded:
+        hist = dist_util.fit_row_sharded(ctx, X, R, args.steps, lr, dist, N_all)
+        rep = dict(loss_first=hist[0], loss_last=hist[-1], orth_err=ctx.orth_error(R), alpha_last=None,
+                   w_norm_last=None, w_op_last=None, series_terms_last=None, p0_terms_last=None, guards_run=None)
     else:
         rep = ctx.fit(X, R, args.steps, lr)
     ev1.record()
@@ -306,11 +321,11 @@ def main():
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
     n_layers = len(Xs) if sweep else 1
     ms_per_step = ms / (args.steps * n_layers)
-    value = world * N * args.steps * n_layers / (ms * 1e-3)
+    value = (N_all if row_sharded else world * N) * args.steps * n_layers / (ms * 1e-3)
 
     # ---- end to end through kt_fit_host: pinned host X and R in, R out, copies inside the timed region
     e2e = None
-    if not args.no_e2e and not sweep and not shared:
+    if not args.no_e2e and not sweep and not shared and not row_sharded:
         Xh = X.cpu().pin_memory()
         Rh = torch.from_numpy(R0_host.copy()).pin_memory()
         stage = torch.empty_like(X)
@@ -391,7 +406,8 @@ def main():
                    "backward": args.backward,
                    "l2": "inputs (%.0f MiB of X per step) exceed the 126 MB L2" % (N * d * 2 / 2**20)
                    if N * d * 2 > 126e6 else "inputs fit in L2; no flush (small case)",
-                   "parallelism": "one independent layer per GPU" if world > 1 else "single GPU",
+                   "parallelism": ("rows of one X over the GPUs, all-reduce of dR per step" if row_sharded else
+                                   "one independent layer per GPU") if world > 1 else "single GPU",
                    **({"layers": n_layers, "steps_per_layer": args.steps, "resident_gib": n_layers * N * d * 2 / 2**30,
                        "sweep_seconds": ms * 1e-3} if sweep else {})},
         "algorithmic_tflops": (4.0 * N * d * d) * world / (ms_per_step * 1e-3) / 1e12,

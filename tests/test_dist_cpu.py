@@ -54,3 +54,61 @@ def test_single_rank_is_a_no_op():
     assert dist_util.max_over_ranks(None, 3.5) == 3.5
     assert dist_util.layers_of_rank(7, 0, 1) == list(range(7))
     assert sorted(sum((dist_util.layers_of_rank(80, r, 8) for r in range(8)), [])) == list(range(80))
+
+
+class _OracleCtx:
+    """Stands in for the library's Context on the CPU: same two calls, computed by the float64 oracle."""
+
+    def loss_grad(self, X, R):
+        from oracle import kurtail_oracle as ko
+        L, dR = ko.loss_grad(X.numpy(), R.numpy())
+        return L, torch.from_numpy(dR)
+
+    def orth_step(self, R, dR, lr):
+        from oracle import kurtail_oracle as ko
+        Rn, _, _ = ko.orth_step(R.numpy(), dR.numpy(), lr)
+        R.copy_(torch.from_numpy(Rn))
+        return R
+
+
+def _problem():
+    g = torch.Generator().manual_seed(5)
+    X = torch.randn((48, 8), generator=g, dtype=torch.float64)
+    X[:, 3] *= 25.0
+    return X, torch.eye(8, dtype=torch.float64)
+
+
+def _shard_worker(rank, world, port, out):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    dist = dist_util.init("gloo")
+    X, R = _problem()
+    rows = [slice(0, 16), slice(16, 48)][rank]          # unequal shards: the weights matter
+    losses = dist_util.fit_row_sharded(_OracleCtx(), X[rows], R, 5, 1e-2, dist, X.shape[0])
+    out.put((rank, losses, R.numpy().tolist()))
+    dist_util.barrier(dist)
+    dist_util.finalize(dist)
+
+
+def test_row_sharded_fit_equals_the_full_batch_fit():
+    import numpy as np
+    from oracle import kurtail_oracle as ko
+    world = 2
+    port = _free_port()
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_shard_worker, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = sorted(out.get(timeout=120) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    X, R0 = _problem()
+    R_ref, losses_ref = ko.fit(X.numpy(), R0.numpy(), 5, 1e-2)
+    assert res[0][2] == res[1][2]                                    # replicas bit-identical
+    assert np.abs(np.array(res[0][2]) - R_ref).max() < 1e-12
+    assert np.allclose(res[0][1], losses_ref, rtol=1e-12) and res[0][1] == res[1][1]
+    # one rank alone: the plain loop
+    X, R = _problem()
+    assert np.allclose(dist_util.fit_row_sharded(_OracleCtx(), X, R, 5, 1e-2, None, X.shape[0]), losses_ref, rtol=1e-12)
