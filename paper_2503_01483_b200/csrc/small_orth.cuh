@@ -43,14 +43,16 @@ struct SmallOrthParams {
 };
 
 // out[r] = sum_k arow[r][k] * B[k][j] for this thread's column j and the CTA's ROWS rows.
+// (B may have been written by other CTAs earlier in this launch: it is read with L2-only loads, never through the
+// non-coherent path.)
 template <int ROWS>
-__device__ __forceinline__ void rows_times_matrix(const float (*arow)[512], const float* __restrict__ B, int d, int j,
+__device__ __forceinline__ void rows_times_matrix(const float (*arow)[512], const float* B, int d, int j,
                                                   float (&out)[ROWS]) {
 #pragma unroll
   for (int r = 0; r < ROWS; ++r) out[r] = 0.f;
 #pragma unroll 8
   for (int k = 0; k < d; ++k) {
-    const float b = B[static_cast<long long>(k) * d + j];
+    const float b = __ldcg(B + static_cast<long long>(k) * d + j);
 #pragma unroll
     for (int r = 0; r < ROWS; ++r) out[r] = fmaf(arow[r][k], b, out[r]);
   }
