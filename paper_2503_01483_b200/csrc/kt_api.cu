@@ -105,7 +105,10 @@ static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, const kt_conf
                             int gather_batch = 0) {
   const bool adam = cfg != nullptr && cfg->optimizer == 1;
   const bool xcopy = x_dtype == KT_F32 || (cfg != nullptr && cfg->rmsnorm != 0) || gather_batch > 0;
-  const bool keep_y = cfg == nullptr || cfg->backward_mode != 1;  // Y kept in float32 for the backward pass
+  // Y kept in float32 for the backward pass, unless the backward recomputes it or the single-pass kernel (d = 128,
+  // per-token loss) does forward and backward together
+  const bool single_pass = d == kFsD && (cfg == nullptr || (cfg->small_d_fused != 0 && cfg->loss_mode == 0));
+  const bool keep_y = (cfg == nullptr || cfg->backward_mode != 1) && !single_pass;
   WsLayout L;
   memset(&L, 0, sizeof(L));
   L.bn = (d % 256 == 0) ? 128 : 64;  // columns per moment record: half a GEMM column tile
