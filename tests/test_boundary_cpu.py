@@ -76,3 +76,19 @@ def test_create_without_gpu_fails_cleanly(L):
     h = C.c_void_p()
     st = L.kt_create(C.byref(h), None, None)
     assert st in (5, 6) and not h.value
+
+
+def test_bench_reference_arm_prints_the_contract_line():
+    # the CPU arm of the benchmark (the oracle, timed on the host) on the small workload
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    res = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--impl", "reference", "--workload", "tiny",
+                          "--steps", "1", "--warmup", "0"], capture_output=True, text=True, timeout=600, cwd=root)
+    assert res.returncode == 0, res.stderr[-2000:]
+    line = json.loads(res.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["unit"] == "tokens/s" and line["value"] > 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
+    assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
+    assert line["config"]["workload"] == "tiny" and line["higher_is_better"] is True
