@@ -182,6 +182,27 @@ def test_backward_from_stored_y_equals_recomputed_backward(N, d, init):
     reco.close()
 
 
+@pytest.mark.parametrize("N,d", [(1000, 256), (129, 512), (128 * 40 + 9, 1024), (300, 4096)])
+def test_cta_pairs_give_the_same_bits_as_single_ctas(N, d):
+    # 256-wide tiles run on pairs of CTAs by default (one MMA over both SMs); the accumulation order over k is the
+    # same as with one CTA per tile, so every result must be bit-identical
+    X = make_x(N, d, seed=46)
+    pair = kurtail.Context(DEV)
+    solo = kurtail.Context(DEV, cta_pairs=0)
+    R = rand_orth(d, seed=4)
+    assert torch.equal(pair.rotate(X, R), solo.rotate(X, R))
+    la, da = pair.loss_grad(X, R)
+    lb, db = solo.loss_grad(X, R)
+    assert la == lb and torch.equal(da, db)
+    assert pair.quant4_error(X, R) == solo.quant4_error(X, R)
+    Ra, Rb = R.clone(), R.clone()
+    pair.fit(X, Ra, 3, 1e-2)
+    solo.fit(X, Rb, 3, 1e-2)
+    assert torch.equal(Ra, Rb)
+    pair.close()
+    solo.close()
+
+
 def test_loss_grad_tiny_config_float32(ctx):
     cfg = synth.config("tiny", device=DEV)
     X = cfg["X"]
