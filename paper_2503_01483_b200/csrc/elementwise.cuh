@@ -31,7 +31,8 @@ struct Scalars {
   double adam_v;            // Cayley Adam: running mean of ||dR||_F^2
   double adam_r;            // Cayley Adam: (1 - beta1^k) sqrt(v / (1 - beta2^k) + eps) of the current step
   float wop;                // size of W as an operator used by the current step's choices
-  unsigned int pad;
+  unsigned int need_op;     // 1 = the Frobenius norm alone would cost this step extra work: estimate ||W||_2
+  double wnorm2;            // ||W||_F^2 of the current step
 };
 
 constexpr float kDegenerateRel = 1e-6f;
@@ -545,7 +546,8 @@ __device__ __forceinline__ float start_sign(int j) {
   return ((h >> 13) & 1u) ? 1.f : -1.f;
 }
 __global__ void k_skew_matvec(const __nv_bfloat16* __restrict__ W, int d, const float* __restrict__ v,
-                              float* __restrict__ y) {
+                              float* __restrict__ y, const Scalars* __restrict__ sc) {
+  if (sc->need_op == 0u) return;  // the step's choices are already the cheapest with ||W||_F: no estimate needed
   const int lane = threadIdx.x & 31;
   const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
   const __nv_bfloat16* w = W + static_cast<long long>(row) * d;
@@ -576,6 +578,30 @@ __global__ void k_skew_matvec(const __nv_bfloat16* __restrict__ W, int d, const 
   if (lane == 0) y[row] = acc;
 }
 
+// One block of 1024 threads, before the power iteration: ||W||_F^2 in fixed order, and whether the estimate of
+// ||W||_2 can change anything this step.  With x_F = alpha ||W||_F: if already x_F / 2 < 2^-11 (one series term) and
+// x_F 2^-9 < 2.5e-6 (one bf16 term of R), the step is as cheap as it gets and the matrix-vector products are skipped
+// (the drift bound then uses x_F, which only makes the next measurement come a little sooner).
+__global__ void k_w_norm(const double* __restrict__ block_norm2, int n, float lr, float q, float eps, int iters,
+                         Scalars* __restrict__ sc) {
+  __shared__ double sh[32];
+  double s = 0.0;
+  for (int i = threadIdx.x; i < n; i += 1024) s += block_norm2[i];
+  s = warp_sum(s);
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    s = 0.0;
+    for (int w = 0; w < 32; ++w) s += sh[w];
+    sc->wnorm2 = s;
+    const double nrm = sqrt(s);
+    const double cap = 2.0 * static_cast<double>(q) / (nrm + static_cast<double>(eps));
+    const double a = (static_cast<double>(lr) < cap) ? static_cast<double>(lr) : cap;
+    const double x = a * nrm;
+    sc->need_op = ((iters >= 1 && 0.5 * x >= ldexp(1.0, -11)) || x * ldexp(1.0, -9) >= 2.5e-6) ? 1u : 0u;
+  }
+}
+
 // One block of 1024 threads: ||W||_F, alpha = min(lr, 2q/(||W||_F + eps)), and the decisions that depend on
 // x = alpha ||W||_2 (bounded by alpha ||W||_F; estimated by a short power iteration when pv_prev/pv_last are given):
 //  * n_terms: term k of the series changes R by at most x (x/2)^k (Frobenius bounds the spectral norm, ||R|| = 1);
@@ -599,8 +625,8 @@ __global__ void k_step_size(const double* __restrict__ block_norm2, int n, float
   for (int what = 0; what < 3; ++what) {
     double s = 0.0;
     if (what == 0) {
-      for (int i = threadIdx.x; i < n; i += 1024) s += block_norm2[i];
-    } else if (pv_prev) {
+      for (int i = threadIdx.x; i < n; i += 1024) s += block_norm2[i];  // n == 0: k_w_norm has summed already
+    } else if (pv_prev && sc->need_op != 0u) {
       const float* v = (what == 1) ? pv_prev : pv_last;
       for (int i = threadIdx.x; i < d; i += 1024) s += static_cast<double>(v[i]) * v[i];
     }
@@ -615,7 +641,7 @@ __global__ void k_step_size(const double* __restrict__ block_norm2, int n, float
     __syncthreads();
   }
   if (threadIdx.x == 0) {
-    const double nrm = sqrt(tot[0]);
+    const double nrm = sqrt(n > 0 ? tot[0] : sc->wnorm2);
     const double cap = 2.0 * static_cast<double>(q) / (nrm + static_cast<double>(eps));
     const double a = (static_cast<double>(lr) < cap) ? static_cast<double>(lr) : cap;
     sc->alpha = static_cast<float>(a);
@@ -624,7 +650,7 @@ __global__ void k_step_size(const double* __restrict__ block_norm2, int n, float
     // power iteration ran, pv_last = W pv_prev, and ||pv_last|| / ||pv_prev|| <= ||W||_2 is its estimate from
     // below; twice that (the iteration is short), capped by the Frobenius norm, stands in for ||W||_2.
     double wop = nrm;
-    if (pv_prev && tot[1] > 0.0) {
+    if (pv_prev && sc->need_op != 0u && tot[1] > 0.0) {
       const double est = 2.0 * sqrt(tot[2] / tot[1]);
       if (est < wop) wop = est;
     }

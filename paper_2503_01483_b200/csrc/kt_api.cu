@@ -729,17 +729,20 @@ static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, 
   const float* pv_last = nullptr;
   const int n_mv = c.norm_iters > 0 ? 2 * (c.norm_iters > 16 ? 16 : c.norm_iters) : 0;
   if (n_mv > 0) {
+    // (the products return at once when ||W||_F alone already gives the cheapest step: see k_w_norm)
+    k_w_norm<<<1, 1024, 0, ctx->stream>>>(at<double>(ctx, L.norm_blocks), L.norm_n, lr, c.q, c.eps, s, sc);
+    KT_LAUNCH_CHECK();
     float* pv[2] = {at<float>(ctx, L.pvec), at<float>(ctx, L.pvec) + d};
     for (int i = 0; i < n_mv; ++i) {
-      k_skew_matvec<<<d / 8, 256, 0, ctx->stream>>>(w_hi, d, i == 0 ? nullptr : pv[(i + 1) & 1], pv[i & 1]);
+      k_skew_matvec<<<d / 8, 256, 0, ctx->stream>>>(w_hi, d, i == 0 ? nullptr : pv[(i + 1) & 1], pv[i & 1], sc);
       KT_LAUNCH_CHECK();
     }
     pv_prev = pv[n_mv & 1];        // written by application n_mv - 2
     pv_last = pv[(n_mv + 1) & 1];  // written by application n_mv - 1
   }
-  k_step_size<<<1, 1024, 0, ctx->stream>>>(at<double>(ctx, L.norm_blocks), L.norm_n, lr, c.q, c.eps, sc, d, s,
-                                          cfg_terms, cfg_terms == 0 ? 1 : 0, guard_mode, c.polish_thresh, pv_prev,
-                                          pv_last);
+  k_step_size<<<1, 1024, 0, ctx->stream>>>(at<double>(ctx, L.norm_blocks), n_mv > 0 ? 0 : L.norm_n, lr, c.q, c.eps, sc,
+                                          d, s, cfg_terms, cfg_terms == 0 ? 1 : 0, guard_mode, c.polish_thresh,
+                                          pv_prev, pv_last);
   KT_LAUNCH_CHECK();
 
   // P_0 = W R with R^T as a bf16 split (it multiplies alpha directly; the device picks one or two terms);
