@@ -424,8 +424,9 @@ __global__ void k_block_sums_f32(const float* __restrict__ v, long long n, doubl
 
 // out[i] = sum over s of part[s * stride + i], s ascending (fixed order).  n a multiple of 4.
 // grid ceil(n/4/256), block 256.
+// out_hi != null: also out_hi[i] = bf16(out[i]) (the form the Cayley step's first product reads).
 __global__ void k_sum_splits(const float* __restrict__ part, int splits, long long stride, long long n,
-                             float* __restrict__ out) {
+                             float* __restrict__ out, __nv_bfloat16* __restrict__ out_hi) {
   const long long i4 = (static_cast<long long>(blockIdx.x) * 256 + threadIdx.x) * 4;
   if (i4 >= n) return;
   float4 acc = *reinterpret_cast<const float4*>(part + i4);
@@ -437,6 +438,13 @@ __global__ void k_sum_splits(const float* __restrict__ part, int splits, long lo
     acc.w += v.w;
   }
   *reinterpret_cast<float4*>(out + i4) = acc;
+  if (out_hi != nullptr) {
+    __nv_bfloat162 lo2 = __floats2bfloat162_rn(acc.x, acc.y), hi2 = __floats2bfloat162_rn(acc.z, acc.w);
+    uint2 pk;
+    pk.x = *reinterpret_cast<unsigned int*>(&lo2);
+    pk.y = *reinterpret_cast<unsigned int*>(&hi2);
+    *reinterpret_cast<uint2*>(out_hi + i4) = pk;
+  }
 }
 
 // --------------------------------------------------------------- Cayley Adam

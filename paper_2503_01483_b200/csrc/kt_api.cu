@@ -481,7 +481,9 @@ static kt_status forward_loss(kt_ctx* ctx, const XView& xv, int N, int d, const 
 // element-wise kernel.  Both evaluate the same float32 expression on the same accumulator values: the same bits.
 static bool keep_y_for_backward(const kt_ctx* ctx) { return ctx->cfg.backward_mode != 1; }
 
-static kt_status backward(kt_ctx* ctx, const XView& xv, int N, int d, const WsLayout& L, float* dR) {
+// dr_hi != null: the split-K sum also leaves bf16(dR) there (only when the sum runs; see dr_hi_from_backward()).
+static kt_status backward(kt_ctx* ctx, const XView& xv, int N, int d, const WsLayout& L, float* dR,
+                          __nv_bfloat16* dr_hi = nullptr) {
   if (keep_y_for_backward(ctx)) {
     dim3 grid((N + 63) / 64, d / 64);
     k_grad_from_y<<<grid, 256, 0, ctx->stream>>>(at<float>(ctx, L.ybuf), at<float4>(ctx, L.coef), N, d,
@@ -508,17 +510,17 @@ static kt_status backward(kt_ctx* ctx, const XView& xv, int N, int d, const WsLa
   if (sp.splits > 1) {
     const long long n = static_cast<long long>(d) * d;
     k_sum_splits<<<static_cast<unsigned>((n / 4 + 255) / 256), 256, 0, ctx->stream>>>(at<float>(ctx, L.splitk),
-                                                                                       sp.splits, n, n, dR);
+                                                                                       sp.splits, n, n, dR, dr_hi);
     KT_LAUNCH_CHECK();
   }
   return KT_OK;
 }
 
 static kt_status loss_grad_async(kt_ctx* ctx, const XView& xv, int N, int d, const WsLayout& L, const float* R,
-                                 float* dR, double* hist_slot, bool rt_current) {
+                                 float* dR, double* hist_slot, bool rt_current, __nv_bfloat16* dr_hi = nullptr) {
   if (!rt_current) KT_TRY(cast_rt(ctx, R, d, N, L));
   KT_TRY(forward_loss(ctx, xv, N, d, L, hist_slot, keep_y_for_backward(ctx)));
-  KT_TRY(backward(ctx, xv, N, d, L, dR));
+  KT_TRY(backward(ctx, xv, N, d, L, dR, dr_hi));
   return KT_OK;
 }
 
@@ -567,7 +569,8 @@ static kt_status fused_loss_grad_async(kt_ctx* ctx, const XView& xv, int N, cons
     ctx->prof_cat[ctx->prof_used++] = static_cast<unsigned char>(kCatFused);
   }
   const long long n = static_cast<long long>(d) * d;
-  k_sum_splits<<<static_cast<unsigned>((n / 4 + 255) / 256), 256, 0, ctx->stream>>>(p.dr_partial, grid, n, n, dR);
+  k_sum_splits<<<static_cast<unsigned>((n / 4 + 255) / 256), 256, 0, ctx->stream>>>(p.dr_partial, grid, n, n, dR,
+                                                                                     nullptr);
   KT_LAUNCH_CHECK();
   k_final_sum<<<1, 256, 0, ctx->stream>>>(p.loss_partial, grid, 1.0 / N, &ctx->d_blk->sc.loss, hist_slot,
                                           p.deg_partial, &ctx->d_blk->sc.deg_rows);
@@ -678,7 +681,8 @@ static kt_status small_orth_step_async(kt_ctx* ctx, float* R, const float* dR, i
 // its drift bound (see k_step_size).
 // adam_m != null: Cayley Adam (momentum buffer; v and the step count live in the device scalar block).
 static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, float lr, const WsLayout& L,
-                                 int guard_mode, bool forms_current, bool adaptive = false, float* adam_m = nullptr) {
+                                 int guard_mode, bool forms_current, bool adaptive = false, float* adam_m = nullptr,
+                                 bool dr_hi_ready = false) {
   if (!adam_m && use_small_orth(ctx, d)) return small_orth_step_async(ctx, R, dR, d, lr, L, guard_mode != 2);
   const kt_config& c = ctx->cfg;
   Scalars* sc = &ctx->d_blk->sc;
@@ -704,7 +708,7 @@ static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, 
     k_adam_scalars<<<1, 1024, 0, ctx->stream>>>(at<double>(ctx, L.norm_blocks), L.norm_n, c.beta1, c.beta2, c.adam_eps,
                                                 sc);
     KT_LAUNCH_CHECK();
-  } else {
+  } else if (!dr_hi_ready) {  // (inside kt_fit the split-K sum of the gradient has already left bf16(dR) in z_hi)
     k_split_bf16<false><<<tgrid, tblock, 0, ctx->stream>>>(dR, d, z_hi /* dR hi: free until P^T is written */,
                                                            nullptr, d);
     KT_LAUNCH_CHECK();
@@ -836,6 +840,10 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
     if (fused) KT_TRY(ingest_x_forward(ctx, X, L, &xv)); else KT_TRY(ingest_x_full(ctx, X, L, &xv));
   }
   float* dR = at<float>(ctx, L.dr);
+  // the Cayley step's first product reads bf16(dR): when the gradient ends in a split-K sum, that sum writes it too
+  __nv_bfloat16* dr_hi = (!fused && !adam && !use_small_orth(ctx, d) && plan_split_k(d, N).splits > 1)
+                             ? at<__nv_bfloat16>(ctx, L.z_hi)
+                             : nullptr;
   const int ge = ctx->cfg.guard_every < 1 ? 1 : ctx->cfg.guard_every;
   double first = 0.0, last = 0.0;
   int done = 0;
@@ -882,7 +890,7 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
     if (fused)
       KT_TRY(fused_loss_grad_async(ctx, xv, N, L, R, dR, &ctx->d_blk->hist[slot], k > 0));
     else
-      KT_TRY(loss_grad_async(ctx, xv, N, d, L, R, dR, &ctx->d_blk->hist[slot], k > 0));
+      KT_TRY(loss_grad_async(ctx, xv, N, d, L, R, dR, &ctx->d_blk->hist[slot], k > 0, dr_hi));
     // guard: a fixed cadence when guard_every >= 1; otherwise measured on the first and the last step and in between
     // whenever the device's drift bound asks for it
     int guard_mode;
@@ -890,7 +898,8 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
       guard_mode = (((k + 1) % ge == 0) || (k + 1 == steps)) ? 1 : 2;
     else
       guard_mode = (k == 0 || k + 1 == steps) ? 1 : 0;
-    KT_TRY(orth_step_async(ctx, R, dR, d, lr, L, guard_mode, k > 0, ctx->cfg.guard_every < 1, adam_m));
+    KT_TRY(orth_step_async(ctx, R, dR, d, lr, L, guard_mode, k > 0, ctx->cfg.guard_every < 1, adam_m,
+                           dr_hi != nullptr));
     done = k + 1;
   }
   if (steps > 0) {
