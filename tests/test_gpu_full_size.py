@@ -154,3 +154,24 @@ def test_layer_sweep_driver_resident_buffers(ctx):
     for r, R in zip(reps, Rs):
         assert r["steps_done"] == 2 and np.isfinite(r["loss_last"])
         assert ctx.orth_error(R) <= 1e-4
+
+
+def test_full_size_launch_variants_agree_bitwise():
+    # At the headline size: the backward that reads the stored Y against the one that recomputes it, and GEMMs on
+    # pairs of CTAs against one CTA per tile.  All three evaluate the same float32 operations in the same order.
+    cfg = synth.config("llama2_7b_attn", device=DEV)
+    X = cfg["X"]
+    base = kurtail.Context(DEV)
+    R = base.init_rotation(4096, "hadamard")
+    l0, d0 = base.loss_grad(X, R)
+    R0 = R.clone()
+    base.fit(X, R0, 2, 1e-2)
+    base.close()
+    for kw in (dict(backward_mode=1), dict(cta_pairs=0)):
+        c = kurtail.Context(DEV, **kw)
+        l1, d1 = c.loss_grad(X, R)
+        assert l1 == l0 and torch.equal(d1, d0), kw
+        R1 = R.clone()
+        c.fit(X, R1, 2, 1e-2)
+        assert torch.equal(R1, R0), kw
+        c.close()
