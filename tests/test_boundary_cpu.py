@@ -44,6 +44,28 @@ def test_default_config(L):
     cfg = kurtail.default_config()
     assert cfg.kappa_target == pytest.approx(1.8)
     assert cfg.cayley_iters == 2 and cfg.q == 0.5 and cfg.retract_terms == 0 and cfg.guard_every == 0 and cfg.forward_terms == 0
+    # the fields at the end of the struct come out right only if the binding's layout is the header's
+    assert cfg.optimizer == 0 and cfg.beta1 == pytest.approx(0.9) and cfg.beta2 == pytest.approx(0.99)
+    assert cfg.norm_iters == 2 and cfg.backward_mode == 0 and cfg.cta_pairs == 1
+    assert cfg.loss_mode == 0 and cfg.rmsnorm == 0 and cfg.rms_eps == pytest.approx(1e-6)
+
+
+def _struct_fields(name):
+    with open(os.path.join(ROOT, "include", "kurtail.h")) as f:
+        text = re.sub(r"/\*.*?\*/", "", f.read(), flags=re.S)
+    body = re.search(r"typedef struct \{([^}]*)\} %s;" % name, text).group(1)
+    out = []
+    for decl in body.split(";"):
+        decl = decl.strip()
+        if decl:
+            for part in decl.split(","):
+                out.append(re.sub(r"\[.*\]", "", part.strip().split()[-1]).lstrip("*"))
+    return out
+
+
+@pytest.mark.parametrize("name", ["kt_config", "kt_fit_report", "kt_quant_spec", "kt_adam_state", "kt_profile", "kt_mat"])
+def test_binding_structs_list_the_header_fields_in_order(name):
+    assert [f[0] for f in getattr(kurtail, name)._fields_] == _struct_fields(name)
 
 
 def test_workspace_bytes_host_only(L):
