@@ -175,3 +175,20 @@ def test_full_size_launch_variants_agree_bitwise():
         c.fit(X, R1, 2, 1e-2)
         assert torch.equal(R1, R0), kw
         c.close()
+
+
+def test_more_than_two_to_the_32_entries():
+    # N * d = (2^20 + 77) * 4096 > 2^32 entries (an 8.6 GB X, a 17 GB float32 Y): every row index has to be carried in
+    # 64 bits; a ragged last tile on top.  Checked on sampled rows (first, last, random) and through the gradient's
+    # size-independent properties.
+    N, d = (1 << 20) + 77, 4096
+    X = synth.activations(N, d, dist="student_t", nu=3.0, n_outliers=16, outlier_scale=100.0, seed=11,
+                          dtype=torch.bfloat16, device=DEV)
+    c = kurtail.Context(DEV)
+    R = c.init_rotation(d, "hadamard")
+    mom = _sampled_rows_match_oracle(c, X, R, n_sample=32, seed=3)
+    _loss_is_mean_of_row_terms(c, X, R, mom)
+    _gradient_properties(c, X, R, blocks=3)
+    c.close()
+    del X
+    torch.cuda.empty_cache()
