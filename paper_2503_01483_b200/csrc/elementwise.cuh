@@ -369,26 +369,66 @@ __global__ void k_gather_samples(const void* const* __restrict__ bases, long lon
 }
 
 // ------------------------------------------------------- RMSNorm of the rows
-// xb[t][:] = bf16( X[t][:] / sqrt(mean_j X[t][j]^2 + eps) ) -- the RMSNorm (unit gain) that follows the rotation in
+// Eight consecutive elements of a row as float32 (16-byte loads; the row starts on a 16-byte boundary).
+__device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&v)[8]) {
+  const uint4 raw = *reinterpret_cast<const uint4*>(p);
+  const __nv_bfloat162* pr = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float2 f = __bfloat1622float2(pr[e]);
+    v[2 * e] = f.x;
+    v[2 * e + 1] = f.y;
+  }
+}
+__device__ __forceinline__ void load8(const float* p, float (&v)[8]) {
+  const float4 a = *reinterpret_cast<const float4*>(p);
+  const float4 b = *reinterpret_cast<const float4*>(p + 4);
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+  v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+
+// xb[t][:] = bf16( x_t / sqrt(mean_j x_t[j]^2 + eps) ) -- the RMSNorm (unit gain) that follows the rotation in
 // the paper's small network (Section 3, "Learning the Rotations"); an orthogonal R keeps every row's norm, so it
-// can be applied to X once.  One block of 256 threads per row; T = float or bf16; xb dense N x d.  xb may be X
-// itself (bf16, ld == d): a thread writes only elements it has read, after the row's sum is complete.
+// can be applied to X once.  Row t is X[t] (bases == null), or, for a rotation shared by several buffers, row t of
+// the minibatch `ids` gathered straight from the buffers (see k_gather_samples for the numbering), which saves the
+// separate gathering pass.  One block of 256 threads per row; T = float or bf16; xb dense N x d; d a multiple
+// of 8.  xb may be X itself (bf16, ld == d): a thread writes only elements it has read, after the row's sum is
+// complete.
 template <typename T>
-__global__ void k_rmsnorm_rows(const T* X, long long ld, int d, float eps, __nv_bfloat16* xb) {
+__global__ void k_rmsnorm_rows(const T* X, long long ld, int d, float eps, __nv_bfloat16* xb,
+                               const void* const* bases, int samples_per_buf, int rps, const int* ids) {
   __shared__ double sh[8];
   __shared__ float scale_sh;
-  const T* x = X + static_cast<long long>(blockIdx.x) * ld;
+  const T* x;
+  if (bases != nullptr) {
+    const int b = blockIdx.x / rps, r = blockIdx.x - b * rps;
+    const int id = ids[b];
+    const int buf = id / samples_per_buf, smp = id - buf * samples_per_buf;
+    x = static_cast<const T*>(bases[buf]) + (static_cast<long long>(smp) * rps + r) * ld;
+  } else {
+    x = X + static_cast<long long>(blockIdx.x) * ld;
+  }
   float part = 0.f;  // at most d/256 terms per thread in float32, the 256 partials in float64
-  for (int j = threadIdx.x; j < d; j += 256) {
-    const float v = to_f32(x[j]);
-    part = fmaf(v, v, part);
+  for (int j = threadIdx.x * 8; j < d; j += 256 * 8) {
+    float v[8];
+    load8(x + j, v);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) part = fmaf(v[e], v[e], part);
   }
   double acc = block_sum_256(static_cast<double>(part), sh, threadIdx.x);
   if (threadIdx.x == 0) scale_sh = static_cast<float>(1.0 / sqrt(acc / d + static_cast<double>(eps)));
   __syncthreads();
   const float sc = scale_sh;
   __nv_bfloat16* o = xb + static_cast<long long>(blockIdx.x) * d;
-  for (int j = threadIdx.x; j < d; j += 256) o[j] = __float2bfloat16_rn(to_f32(x[j]) * sc);
+  for (int j = threadIdx.x * 8; j < d; j += 256 * 8) {
+    float v[8];
+    load8(x + j, v);
+    uint4 out;
+    __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&out);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) po[e] = __floats2bfloat162_rn(v[2 * e] * sc, v[2 * e + 1] * sc);
+    *reinterpret_cast<uint4*>(o + j) = out;
+  }
 }
 
 // One block: *dst = scale * sum(vals[0..n)) (also to *dst2 when not null);

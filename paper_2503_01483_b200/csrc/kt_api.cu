@@ -341,10 +341,10 @@ static kt_status rmsnorm_x(kt_ctx* ctx, const kt_mat& X, const WsLayout& L, XVie
   const unsigned rows = static_cast<unsigned>(X.rows);
   if (X.dtype == KT_BF16)
     k_rmsnorm_rows<__nv_bfloat16><<<rows, 256, 0, ctx->stream>>>(static_cast<const __nv_bfloat16*>(X.data), X.ld, d,
-                                                                 ctx->cfg.rms_eps, xb);
+                                                                 ctx->cfg.rms_eps, xb, nullptr, 0, 0, nullptr);
   else
     k_rmsnorm_rows<float><<<rows, 256, 0, ctx->stream>>>(static_cast<const float*>(X.data), X.ld, d, ctx->cfg.rms_eps,
-                                                         xb);
+                                                         xb, nullptr, 0, 0, nullptr);
   KT_LAUNCH_CHECK();
   v->xb = xb;
   v->ldx = d;
@@ -871,20 +871,29 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
       const void* const* bases = at<const void*>(ctx, L.gather_bases);
       const int* ids = at<int>(ctx, L.gather_ids) + static_cast<size_t>(cslot) * sh->batch;
       const int rps = static_cast<int>(sh->rps);
-      if (X.dtype == KT_BF16)
+      const bool norm = ctx->cfg.rmsnorm != 0;
+      if (norm) {
+        // gather and RMSNorm in one pass: the normalised rows go straight from the buffers into the dense matrix
+        if (X.dtype == KT_BF16)
+          k_rmsnorm_rows<__nv_bfloat16><<<N, 256, 0, ctx->stream>>>(nullptr, X.ld, d, ctx->cfg.rms_eps, xb, bases, spb,
+                                                                    rps, ids);
+        else
+          k_rmsnorm_rows<float><<<N, 256, 0, ctx->stream>>>(nullptr, X.ld, d, ctx->cfg.rms_eps, xb, bases, spb, rps,
+                                                            ids);
+      } else if (X.dtype == KT_BF16) {
         k_gather_samples<__nv_bfloat16><<<N, 256, 0, ctx->stream>>>(bases, X.ld, spb, rps, ids, d, xb);
-      else
+      } else {
         k_gather_samples<float><<<N, 256, 0, ctx->stream>>>(bases, X.ld, spb, rps, ids, d, xb);
+      }
       KT_LAUNCH_CHECK();
-      kt_mat Xb;
-      Xb.data = xb;
-      Xb.dtype = KT_BF16;
-      Xb.reserved = 0;
-      Xb.rows = N;
-      Xb.cols = d;
-      Xb.ld = d;
-      // (with rmsnorm the rows are normalised in place: each block reads its whole row before it writes it)
-      if (fused) KT_TRY(ingest_x_forward(ctx, Xb, L, &xv)); else KT_TRY(ingest_x_full(ctx, Xb, L, &xv));
+      xv.xb = xb;
+      xv.ldx = d;
+      if (!fused) {  // the token GEMM of the backward pass reads the transpose
+        dim3 pgrid(d / 64, (N + 63) / 64), pblock(32, 8);
+        k_prepare_x<__nv_bfloat16><<<pgrid, pblock, 0, ctx->stream>>>(xb, d, N, d, at<__nv_bfloat16>(ctx, L.xt), L.ldt,
+                                                                      nullptr);
+        KT_LAUNCH_CHECK();
+      }
     }
     // from the second step on, the previous step left the bf16 forms of R in the workspace
     if (fused)
