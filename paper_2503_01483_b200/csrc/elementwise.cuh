@@ -138,6 +138,39 @@ __global__ void k_prepare_x(const T* __restrict__ X, long long ld, int N, int d,
   }
 }
 
+// The same transpose for a bf16 X with no dense copy asked for, in tiles of 64 tokens x 128 channels with 16-byte
+// loads (four in flight per thread).  d a multiple of 128.  grid (d/128, ceil(N/64)), block 256.
+__global__ void k_transpose_x_bf16(const __nv_bfloat16* __restrict__ X, long long ld, int N, int d,
+                                   __nv_bfloat16* __restrict__ xt, long long ldt) {
+  __shared__ __nv_bfloat16 tile[64][130];
+  const int c0 = blockIdx.x * 128, r0 = blockIdx.y * 64;
+  const int rr = threadIdx.x >> 4, cc = (threadIdx.x & 15) * 8;  // 16 rows per pass, 8 channels per thread
+  uint4 v[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int row = r0 + rr + 16 * q;
+    v[q] = (row < N) ? *reinterpret_cast<const uint4*>(X + static_cast<long long>(row) * ld + c0 + cc)
+                     : make_uint4(0u, 0u, 0u, 0u);
+  }
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    unsigned int* dst = reinterpret_cast<unsigned int*>(&tile[rr + 16 * q][cc]);
+    dst[0] = v[q].x;
+    dst[1] = v[q].y;
+    dst[2] = v[q].z;
+    dst[3] = v[q].w;
+  }
+  __syncthreads();
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+#pragma unroll 4
+  for (int c = w; c < 128; c += 8) {
+    __nv_bfloat162 pr;
+    pr.x = tile[2 * lane][c];
+    pr.y = tile[2 * lane + 1][c];
+    *reinterpret_cast<__nv_bfloat162*>(xt + static_cast<long long>(c0 + c) * ldt + r0 + 2 * lane) = pr;
+  }
+}
+
 // float32 X (N x d, ld) -> dense bf16 Xb (N x d).  grid ceil(N*d/2/256), block 256.
 __global__ void k_cast_x(const float* __restrict__ X, long long ld, long long N, int d,
                          __nv_bfloat16* __restrict__ xb) {

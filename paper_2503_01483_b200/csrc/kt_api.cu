@@ -369,6 +369,14 @@ static kt_status ingest_x_forward(kt_ctx* ctx, const kt_mat& X, const WsLayout& 
   return KT_OK;
 }
 
+// X^T of a bf16 X (no dense copy needed): the wide-load transpose.
+static kt_status transpose_x_bf16(kt_ctx* ctx, const __nv_bfloat16* X, long long ld, int N, int d, const WsLayout& L) {
+  dim3 grid(d / 128, (N + 63) / 64);
+  k_transpose_x_bf16<<<grid, 256, 0, ctx->stream>>>(X, ld, N, d, at<__nv_bfloat16>(ctx, L.xt), L.ldt);
+  KT_LAUNCH_CHECK();
+  return KT_OK;
+}
+
 // view for loss + gradient: also builds X^T (the token dimension becomes contiguous)
 static kt_status ingest_x_full(kt_ctx* ctx, const kt_mat& X, const WsLayout& L, XView* v) {
   const int N = static_cast<int>(X.rows), d = static_cast<int>(X.cols);
@@ -376,12 +384,9 @@ static kt_status ingest_x_full(kt_ctx* ctx, const kt_mat& X, const WsLayout& L, 
   __nv_bfloat16* xt = at<__nv_bfloat16>(ctx, L.xt);
   if (ctx->cfg.rmsnorm != 0) {
     KT_TRY(rmsnorm_x(ctx, X, L, v));
-    k_prepare_x<__nv_bfloat16><<<grid, block, 0, ctx->stream>>>(v->xb, v->ldx, N, d, xt, L.ldt, nullptr);
-    KT_LAUNCH_CHECK();
+    KT_TRY(transpose_x_bf16(ctx, v->xb, v->ldx, N, d, L));
   } else if (X.dtype == KT_BF16) {
-    k_prepare_x<__nv_bfloat16><<<grid, block, 0, ctx->stream>>>(static_cast<const __nv_bfloat16*>(X.data), X.ld, N, d,
-                                                                xt, L.ldt, nullptr);
-    KT_LAUNCH_CHECK();
+    KT_TRY(transpose_x_bf16(ctx, static_cast<const __nv_bfloat16*>(X.data), X.ld, N, d, L));
     v->xb = static_cast<const __nv_bfloat16*>(X.data);
     v->ldx = X.ld;
   } else {
@@ -889,10 +894,7 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
       xv.xb = xb;
       xv.ldx = d;
       if (!fused) {  // the token GEMM of the backward pass reads the transpose
-        dim3 pgrid(d / 64, (N + 63) / 64), pblock(32, 8);
-        k_prepare_x<__nv_bfloat16><<<pgrid, pblock, 0, ctx->stream>>>(xb, d, N, d, at<__nv_bfloat16>(ctx, L.xt), L.ldt,
-                                                                      nullptr);
-        KT_LAUNCH_CHECK();
+        KT_TRY(transpose_x_bf16(ctx, xb, d, N, d, L));
       }
     }
     // from the second step on, the previous step left the bf16 forms of R in the workspace
