@@ -213,7 +213,7 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
 // 2-D tile load into this CTA's shared memory whose byte count is credited to `cluster_bar`, a barrier given by its
-// shared::cluster address (the leader's).  No multicast: each CTA loads its own tile.
+// shared::cluster address (the leader's).  Each CTA loads its own tile: nothing is sent to more than one CTA.
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst_smem, const void* tmap, int x, int y,
                                                  uint32_t cluster_bar) {
   asm volatile(
