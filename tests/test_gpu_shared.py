@@ -57,12 +57,15 @@ def test_shared_fit_equals_fit_on_gathered_batches(d, dtype):
     c.close()
 
 
-@pytest.mark.parametrize("flat,rms,adam", [(False, False, False), (True, True, True), (True, False, False),
-                                           (False, True, True)])
-def test_shared_fit_follows_the_oracle(flat, rms, adam):
+@pytest.mark.parametrize("flat,rms,adam,dtype", [(False, False, False, torch.bfloat16),
+                                                 (True, True, True, torch.bfloat16),
+                                                 (True, False, False, torch.bfloat16),
+                                                 (False, True, True, torch.bfloat16),
+                                                 (True, True, False, torch.float32)])
+def test_shared_fit_follows_the_oracle(flat, rms, adam, dtype):
     d, rps, spb, nb, batch, steps = 256, 128, 4, 3, 3, 3
     c = kurtail.Context(DEV, loss_mode=int(flat), rmsnorm=int(rms), optimizer=int(adam))
-    Xs = buffers(nb, rps * spb, d)
+    Xs = buffers(nb, rps * spb, d, dtype)
     Xs[1] *= 4.0                                     # buffers of different scale, as layers are
     order = shuffle(nb * spb, batch, steps, seed=2)
     R0 = synth.random_orthogonal(d, seed=21, device=DEV).contiguous()
