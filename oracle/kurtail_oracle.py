@@ -207,11 +207,13 @@ def cayley_exact(R, W, alpha):
     return np.linalg.solve(I + 0.5 * alpha * W, (I - 0.5 * alpha * W) @ np.asarray(R, dtype=np.float64))
 
 
-def cayley_stepwise(R, W, alpha, iters=2):
+def cayley_stepwise(R, W, alpha, iters=2, start=None):
     """The same map by the fixed-point iteration the Cayley-SGD algorithm uses:
-    Y0 = R - a W R;  Yi = R - a/2 W (R + Y(i-1)),  i = 1..iters."""
+    Y0 = R - a W R;  Yi = R - a/2 W (R + Y(i-1)),  i = 1..iters.
+    `start` replaces Y0 (the iteration contracts towards the Cayley transform
+    from any start; the cited Cayley-Adam listing starts it from R - a M)."""
     R = np.asarray(R, dtype=np.float64)
-    Y = R - alpha * (W @ R)
+    Y = R - alpha * (W @ R) if start is None else np.asarray(start, dtype=np.float64)
     for _ in range(iters):
         Y = R - 0.5 * alpha * (W @ (R + Y))
     return Y
@@ -299,12 +301,10 @@ def gather_samples(X_bufs, rows_per_sample, ids):
 
 
 def fit_shared(X_bufs, rows_per_sample, order, batch, R, steps, lr, flat=False, rmsnorm=False, adam=False,
-               rms_eps=1e-6, kappa_target=KAPPA_UNIFORM, polish_thresh=0.0, round_batch=None):
+               rms_eps=1e-6, kappa_target=KAPPA_UNIFORM, polish_thresh=0.0):
     """steps x (gather the step's minibatch; [RMSNorm its rows]; loss and
     gradient, per token or over the whole minibatch; Cayley SGD or Cayley Adam
     step).  `order` holds steps*batch sample ids: the shuffle is an input.
-    `round_batch`, if given, is applied to the normalised minibatch (the tests
-    pass the bfloat16 rounding the library applies to its stored copy).
     Returns (R_final, [loss per step])."""
     R = np.asarray(R, dtype=np.float64).copy()
     d = R.shape[0]
@@ -315,8 +315,6 @@ def fit_shared(X_bufs, rows_per_sample, order, batch, R, steps, lr, flat=False, 
         Xk = gather_samples(X_bufs, rows_per_sample, order[k * batch:(k + 1) * batch])
         if rmsnorm:
             Xk = rmsnorm_rows(Xk, rms_eps)
-            if round_batch is not None:
-                Xk = round_batch(Xk)
         L, dR = lg(Xk, R, kappa_target)
         losses.append(L)
         if adam:

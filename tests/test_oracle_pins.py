@@ -339,6 +339,45 @@ def test_cayley_adam_second_moment_and_momentum_recurrences_d2():
         R = Rn
 
 
+def test_cayley_adam_start_of_the_fixed_point_iteration_does_not_move_its_limit():
+    # The publication cited for Cayley Adam starts the fixed-point iteration from R - alpha M (M = r W R after the
+    # re-projection), cayley_adam_step starts it from R - alpha W R.  The map Y -> R - alpha/2 W (R + Y) contracts with
+    # factor ||alpha W / 2||_2 towards the exact Cayley transform whatever the start, so the two differ from it by
+    #   (alpha ||W||_2 / 2)^s ||Y0 - Y*||:  O((alpha ||W|| / 2)^(s+1)) for R - alpha W R, and the same times |1 - r|
+    # more for R - alpha M.  Checked for several s against cayley_exact.
+    rng = np.random.default_rng(17)
+    d = 9
+    R = scipy.stats.ortho_group.rvs(d, random_state=12)
+    A = rng.normal(size=(d, d))
+    W = 0.5 * (A - A.T)
+    W /= np.linalg.norm(W, 2)                      # ||W||_2 = 1
+    alpha = 0.2
+    c = alpha / 2.0                                # contraction factor
+    exact = ko.cayley_exact(R, W, alpha)
+    assert ko.orthogonality_error(exact) < 1e-13
+    for r in (0.05, 1.0, 3.0):                     # r = (1 - beta1^k) sqrt(v_hat + eps) takes any positive value
+        M = r * (W @ R)
+        e_prev = None
+        for s in range(0, 6):
+            own = ko.cayley_stepwise(R, W, alpha, s)
+            cited = ko.cayley_stepwise(R, W, alpha, s, start=R - alpha * M)
+            e_own = np.linalg.norm(own - exact, 2)
+            e_cit = np.linalg.norm(cited - exact, 2)
+            d0_own = np.linalg.norm((R - alpha * (W @ R)) - exact, 2)
+            d0_cit = np.linalg.norm((R - alpha * M) - exact, 2)
+            assert e_own <= c ** s * d0_own * (1 + 1e-9) + 1e-15
+            assert e_cit <= c ** s * d0_cit * (1 + 1e-9) + 1e-15
+            assert d0_own <= 2.5 * c ** 1 * alpha + 1e-15          # Y0 - Y* = O(alpha^2 ||W||^2 / 2)
+            if e_prev is not None:
+                assert e_cit <= c * e_prev * (1 + 1e-9) + 1e-15   # geometric, whatever the start
+            e_prev = e_cit
+        # with the two iterations the library runs, both starts sit within (alpha/2)^2 (1 + |1 - r|) alpha of the limit
+        two_own = np.linalg.norm(ko.cayley_stepwise(R, W, alpha, 2) - exact, 2)
+        two_cit = np.linalg.norm(ko.cayley_stepwise(R, W, alpha, 2, start=R - alpha * M) - exact, 2)
+        assert two_own <= c ** 3 * 2.5 * alpha
+        assert two_cit <= c ** 2 * alpha * (abs(1 - r) + 2.5 * c)
+
+
 # ---------------- flattened (whole-layer) kurtosis and the RMSNorm ----------------
 def test_flat_kurtosis_library_and_closed_forms():
     rng = np.random.default_rng(21)
