@@ -50,10 +50,16 @@ typedef enum {
   KT_ERR_CUDA = 6,        /* a CUDA runtime/driver call failed              */
   KT_ERR_NONFINITE = 7,   /* the loss came out NaN/Inf (outputs are written)*/
   KT_ERR_TIMEOUT = 8,     /* a bounded device-side wait ran out             */
-  KT_ERR_TOO_LARGE = 9    /* kt_kurtosis_loss_noalloc: N or d above its maximum */
+  KT_ERR_TOO_LARGE = 9,   /* kt_kurtosis_loss_noalloc: N or d above its maximum */
+  KT_ERR_COOPERATIVE = 10,/* the one-launch orthogonal step (d <= 512) needs 128
+                             CTAs resident at once and the device cannot hold
+                             them: set kt_config.small_d_orth = 0            */
+  KT_ERR_REDUCE = 11      /* kt_fit_sharded: the caller's reduce hook failed   */
 } kt_status;
 
-typedef enum { KT_BF16 = 0, KT_F32 = 1 } kt_dtype;
+/* Element types.  X is KT_BF16 or KT_F32; KT_F64 only names the type of a buffer
+ * handed to a kt_reduce_fn. */
+typedef enum { KT_BF16 = 0, KT_F32 = 1, KT_F64 = 2 } kt_dtype;
 
 /* A row-major matrix: rows x cols elements of `dtype`, leading dimension `ld`
  * elements. */
@@ -137,13 +143,22 @@ typedef struct {
                            layer, loss = |kappa - kappa_target| (zero rows are
                            then part of the distribution; d == 128 uses the
                            general path)                                        */
-  int32_t rmsnorm;      /* [0]   1 = every call that takes X first replaces it by
-                           its row-normalised bf16 copy x / sqrt(mean(x^2) +
-                           rms_eps) in the workspace: the unit-gain RMSNorm of
-                           the small network of Section 3, "Learning the
-                           Rotations", which commutes with an orthogonal R     */
-  float rms_eps;        /* [1e-6] */
-  int32_t reserved[2];
+  int32_t rmsnorm;      /* [0]   1 = the unit-gain RMSNorm of the small network of
+                           Section 3, "Learning the Rotations", follows the
+                           rotation: row t of X R is multiplied by
+                           1 / sqrt(mean(x_t^2) + rms_eps) (an orthogonal R
+                           keeps the norm of a row, so the factor is taken
+                           from X, once per call; it is applied to the
+                           float32 accumulator, X is neither copied nor
+                           rounded again, and the gradient is the one with
+                           respect to R of the normalised output with the
+                           factor held fixed).  The per-token loss does not
+                           depend on it; the whole-layer loss, kt_rotate and
+                           the quantisation errors do                          */
+  float rms_eps;        /* [1e-6] (0 is allowed: all-zero rows then get factor 0) */
+  int32_t wait_limit_ms;/* [4000] bound of every device-side wait, in
+                           milliseconds (<= 0: the default)                    */
+  int32_t reserved;
 } kt_config;
 
 /* Filled by kt_fit / kt_fit_layers (host memory). */
@@ -262,6 +277,28 @@ kt_status kt_orth_error(kt_ctx* ctx, const float* R, int64_t d, double* err);
  * middle of a step R may hold a partially applied step. */
 kt_status kt_fit(kt_ctx* ctx, kt_mat X, float* R, int32_t steps, float lr, kt_fit_report* report);
 
+/* kt_fit for one shard of the rows of a batch that is spread over several
+ * processes or GPUs (one rotation over many tokens: Section 3, "Learning the
+ * Rotations").  X_local holds this shard's rows; rows_total is the number of
+ * rows of all shards together (the loss is the mean over all of them).  Every
+ * step the library calls `reduce` from the host thread, while it enqueues the
+ * step, for each device buffer that has to be summed over the shards:
+ *   per-token loss:   the loss (1 x KT_F64), then dR (d*d x KT_F32);
+ *   whole-layer loss: the batch mean (1 x KT_F64), its three central sums
+ *                     (3 x KT_F64), then dR.
+ * The hook must enqueue an in-place sum all-reduce of `count` elements of type
+ * `dtype` (a kt_dtype) at dev_ptr on `cuda_stream` (the context's stream) --
+ * e.g. ncclAllReduce -- and return 0; it must not synchronise the stream.  A
+ * non-zero return ends the fit with KT_ERR_REDUCE.  Every shard then holds the
+ * same gradient and takes the same orthogonal step, so the replicas of R stay
+ * bit-identical without being exchanged, and nothing synchronises with the
+ * host inside the loop.  reduce == NULL stands for a single shard; with
+ * rows_total == X_local.rows the call is then kt_fit, bit for bit.  The
+ * report's degenerate_rows counts this shard's rows only. */
+typedef int32_t (*kt_reduce_fn)(void* user, void* dev_ptr, int64_t count, int32_t dtype, void* cuda_stream);
+kt_status kt_fit_sharded(kt_ctx* ctx, kt_mat X_local, float* R, int64_t rows_total, kt_reduce_fn reduce, void* user,
+                         int32_t steps, float lr, kt_fit_report* report);
+
 /* Layer-wise driver (Section 3, "Training Cost": activations are stored per
  * layer, then one rotation is optimised at a time).  X_layers[l] and
  * R_layers[l] for l in [first_layer, L) are fitted one after another on the
@@ -289,6 +326,14 @@ kt_status kt_fit_shared_workspace_bytes(const kt_ctx* ctx, int64_t rows_per_samp
 kt_status kt_fit_shared(kt_ctx* ctx, const kt_mat* X_bufs, int32_t n_bufs, int64_t rows_per_sample,
                         const int32_t* order, int32_t batch, float* R, int32_t steps, float lr,
                         kt_fit_report* report);
+
+/* kt_fit_shared for one shard of every minibatch: this process gathers `batch`
+ * samples per step from its own buffers (its own `order`), the other shards
+ * theirs; rows_total = rows of a whole minibatch over all shards.  `reduce` as
+ * in kt_fit_sharded. */
+kt_status kt_fit_shared_sharded(kt_ctx* ctx, const kt_mat* X_bufs, int32_t n_bufs, int64_t rows_per_sample,
+                                const int32_t* order, int32_t batch, float* R, int64_t rows_total,
+                                kt_reduce_fn reduce, void* user, int32_t steps, float lr, kt_fit_report* report);
 
 /* kt_fit with HOST buffers: copies X_host (N x d, pinned or pageable host
  * memory) into X_dev_staging (device, N*ld elements), R_host (d x d float32)
@@ -367,6 +412,13 @@ kt_status kt_quant4_codes(kt_ctx* ctx, const float* Y, int64_t N, int64_t d, int
  *   loss_dev DEVICE pointer to one double (8-byte aligned) that receives the
  *            loss.  The call is stream ordered on `cuda_stream` and does not
  *            synchronise; read the value after synchronising that stream.
+ *            Since the call never reads anything back, it cannot return
+ *            KT_ERR_TIMEOUT or KT_ERR_NONFINITE: if one of its kernels gave up
+ *            a bounded wait, *loss_dev is NaN, and a non-finite loss is simply
+ *            stored.  Treat a NaN there as a failed call.
+ *   X, R and loss_dev must be device (or managed) memory of the CURRENT
+ *   device, whose copy of the array is the one used; KT_ERR_INVALID_ARG
+ *   otherwise.
  *
  * The first call on each device looks up the device address of the built-in
  * array and a driver entry point, with that device current.  Make that first
@@ -379,6 +431,16 @@ kt_status kt_quant4_codes(kt_ctx* ctx, const float* Y, int64_t N, int64_t d, int
 #define KT_NOALLOC_MAX_N 16384
 #define KT_NOALLOC_MAX_D 1024
 kt_status kt_kurtosis_loss_noalloc(kt_mat X, const float* R, double* loss_dev, void* cuda_stream);
+
+/* --- error-path test hook ------------------------------------------------- */
+
+/* Enqueues a one-warp kernel that waits, through the same bounded wait every
+ * kernel of this library uses, on a barrier that nothing ever signals, with a
+ * limit of limit_ms (1..1000) milliseconds.  The wait runs out, the kernel
+ * returns normally and records it: the next synchronising call on this context
+ * returns KT_ERR_TIMEOUT (and clears the record); the call after that works
+ * again.  Nothing traps or faults.  Stream ordered. */
+kt_status kt_test_wait_timeout(kt_ctx* ctx, int32_t limit_ms);
 
 /* --- measurement ---------------------------------------------------------- */
 

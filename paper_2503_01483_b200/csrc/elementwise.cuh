@@ -193,9 +193,13 @@ __global__ void k_cast_x(const float* __restrict__ X, long long ld, long long N,
 //   G = a c^3 - ab c - am3,  a = sgn(kappa-kappa_t) 4/(N d m2^2), ab = a m4/m2, am3 = a m3.
 // A row with m2 <= 1e-6 * (m2 + mean^2), or all zero, contributes nothing.
 // grid ceil(N/256), block 256.
+// n_mean: the number of tokens the loss is a mean over (N, or more when these rows are one shard of the batch).
+// row_scale != null: the rows were multiplied by it in the GEMM epilogue; the coefficients then carry the factor
+// too, so that G is the derivative with respect to the unscaled X R.
 __global__ void k_moments_finalize(const float4* __restrict__ partial, int P, int N, int d, int bn, float kappa_t,
                                    float4* __restrict__ moments, float4* __restrict__ coef,
-                                   double* __restrict__ block_loss, unsigned int* __restrict__ block_deg) {
+                                   double* __restrict__ block_loss, unsigned int* __restrict__ block_deg,
+                                   double n_mean, const float* __restrict__ row_scale) {
   __shared__ double sh[8];
   const int row = blockIdx.x * 256 + threadIdx.x;
   double term = 0.0, deg = 0.0;
@@ -221,7 +225,8 @@ __global__ void k_moments_finalize(const float4* __restrict__ partial, int P, in
       const double diff = kappa - static_cast<double>(kappa_t);
       term = fabs(diff);
       const double sgn = (diff > 0.0) ? 1.0 : ((diff < 0.0) ? -1.0 : 0.0);
-      const double a = sgn * 4.0 / (static_cast<double>(N) * d * m2 * m2);
+      const double rs = row_scale ? static_cast<double>(row_scale[row]) : 1.0;
+      const double a = rs * sgn * 4.0 / (n_mean * d * m2 * m2);
       cf.y = static_cast<float>(a);
       cf.z = static_cast<float>(a * m4 / m2);
       cf.w = static_cast<float>(a * m3);
@@ -325,8 +330,9 @@ __global__ void k_flat_central(const float4* __restrict__ moments, int N, const 
 // One block of 256 threads: global m2, m3, m4, kappa, the loss |kappa - kappa_t| and the coefficients of
 // dL/dY = a c^3 - ab c - am3 with c = Y - mean and a = sgn 4/(N d m2^2) (one kurtosis over n = N d values).
 // A layer with (numerically) no variance gives loss 0, zero coefficients and deg_rows = N.
+// N: rows the moments are a mean over (all shards' rows when the batch is sharded and b2..b4 hold the reduced sums).
 __global__ void k_flat_finalize(const double* __restrict__ b2, const double* __restrict__ b3,
-                                const double* __restrict__ b4, int nb, int N, int d, float kappa_t,
+                                const double* __restrict__ b4, int nb, long long N, int d, float kappa_t,
                                 const double* __restrict__ mean, Scalars* __restrict__ sc,
                                 double* __restrict__ hist_slot, float4* __restrict__ coef_global) {
   __shared__ double sh[8];
@@ -347,7 +353,7 @@ __global__ void k_flat_finalize(const double* __restrict__ b2, const double* __r
     double loss = 0.0;
     unsigned int deg = 0u;
     if (ms == 0.0 || m2 <= static_cast<double>(kDegenerateRel) * ms) {
-      deg = static_cast<unsigned int>(N);
+      deg = static_cast<unsigned int>(N > 0xffffffffll ? 0xffffffffll : N);
     } else {
       const double kappa = m4 / (m2 * m2);
       const double diff = kappa - static_cast<double>(kappa_t);
@@ -365,10 +371,20 @@ __global__ void k_flat_finalize(const double* __restrict__ b2, const double* __r
   }
 }
 
-// Every row gets the layer's coefficients.  grid ceil(N/256), block 256.
-__global__ void k_flat_fill(const float4* __restrict__ coef_global, int N, float4* __restrict__ coef) {
+// Every row gets the layer's coefficients (times the row's RMSNorm factor when the rows were scaled by one: G is
+// the derivative with respect to the unscaled X R).  grid ceil(N/256), block 256.
+__global__ void k_flat_fill(const float4* __restrict__ coef_global, int N, float4* __restrict__ coef,
+                            const float* __restrict__ row_scale) {
   const int row = blockIdx.x * 256 + threadIdx.x;
-  if (row < N) coef[row] = *coef_global;
+  if (row >= N) return;
+  float4 c = *coef_global;
+  if (row_scale) {
+    const float rs = row_scale[row];
+    c.y *= rs;
+    c.z *= rs;
+    c.w *= rs;
+  }
+  coef[row] = c;
 }
 
 // ------------------------------------------------ minibatch of stored samples
@@ -420,18 +436,19 @@ __device__ __forceinline__ void load8(const float* p, float (&v)[8]) {
   v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
 }
 
-// xb[t][:] = bf16( x_t / sqrt(mean_j x_t[j]^2 + eps) ) -- the RMSNorm (unit gain) that follows the rotation in
-// the paper's small network (Section 3, "Learning the Rotations"); an orthogonal R keeps every row's norm, so it
-// can be applied to X once.  Row t is X[t] (bases == null), or, for a rotation shared by several buffers, row t of
-// the minibatch `ids` gathered straight from the buffers (see k_gather_samples for the numbering), which saves the
-// separate gathering pass.  One block of 256 threads per row; T = float or bf16; xb dense N x d; d a multiple
-// of 8.  xb may be X itself (bf16, ld == d): a thread writes only elements it has read, after the row's sum is
-// complete.
+// rowscale[t] = 1 / sqrt(mean_j x_t[j]^2 + eps): the factor of the unit-gain RMSNorm that follows the rotation in
+// the paper's small network (Section 3, "Learning the Rotations").  An orthogonal R keeps every row's norm, so the
+// factor of row t of X R is that of row t of X; the GEMM epilogues apply it to the float32 accumulator, and X
+// itself is never rescaled or re-rounded.  A row whose mean square plus eps is zero gets the factor 0.
+// Row t is X[t] (bases == null), or, for a rotation shared by several buffers, row t of the minibatch `ids`
+// gathered from the buffers (see k_gather_samples for the numbering).  xb != null: the row is also copied, as it
+// is but rounded to bf16, to row t of the dense matrix xb (the gathered minibatch; the bf16 form of a float32 X).
+// One block of 256 threads per row; T = float or bf16; d a multiple of 8.
 template <typename T>
-__global__ void k_rmsnorm_rows(const T* X, long long ld, int d, float eps, __nv_bfloat16* xb,
-                               const void* const* bases, int samples_per_buf, int rps, const int* ids) {
+__global__ void k_row_scale(const T* X, long long ld, int d, float eps, float* __restrict__ rowscale,
+                            __nv_bfloat16* xb, const void* const* bases, int samples_per_buf, int rps,
+                            const int* ids) {
   __shared__ double sh[8];
-  __shared__ float scale_sh;
   const T* x;
   if (bases != nullptr) {
     const int b = blockIdx.x / rps, r = blockIdx.x - b * rps;
@@ -441,34 +458,35 @@ __global__ void k_rmsnorm_rows(const T* X, long long ld, int d, float eps, __nv_
   } else {
     x = X + static_cast<long long>(blockIdx.x) * ld;
   }
+  __nv_bfloat16* o = xb ? xb + static_cast<long long>(blockIdx.x) * d : nullptr;
   float part = 0.f;  // at most d/256 terms per thread in float32, the 256 partials in float64
   for (int j = threadIdx.x * 8; j < d; j += 256 * 8) {
     float v[8];
     load8(x + j, v);
 #pragma unroll
     for (int e = 0; e < 8; ++e) part = fmaf(v[e], v[e], part);
-  }
-  double acc = block_sum_256(static_cast<double>(part), sh, threadIdx.x);
-  if (threadIdx.x == 0) scale_sh = static_cast<float>(1.0 / sqrt(acc / d + static_cast<double>(eps)));
-  __syncthreads();
-  const float sc = scale_sh;
-  __nv_bfloat16* o = xb + static_cast<long long>(blockIdx.x) * d;
-  for (int j = threadIdx.x * 8; j < d; j += 256 * 8) {
-    float v[8];
-    load8(x + j, v);
-    uint4 out;
-    __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&out);
+    if (o) {
+      uint4 out;
+      __nv_bfloat162* po = reinterpret_cast<__nv_bfloat162*>(&out);
 #pragma unroll
-    for (int e = 0; e < 4; ++e) po[e] = __floats2bfloat162_rn(v[2 * e] * sc, v[2 * e + 1] * sc);
-    *reinterpret_cast<uint4*>(o + j) = out;
+      for (int e = 0; e < 4; ++e) po[e] = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
+      *reinterpret_cast<uint4*>(o + j) = out;
+    }
+  }
+  const double acc = block_sum_256(static_cast<double>(part), sh, threadIdx.x);
+  if (threadIdx.x == 0) {
+    const double ms = acc / d + static_cast<double>(eps);
+    rowscale[blockIdx.x] = ms > 0.0 ? static_cast<float>(1.0 / sqrt(ms)) : 0.f;
   }
 }
 
 // One block: *dst = scale * sum(vals[0..n)) (also to *dst2 when not null);
 // *count_dst = sum(counts) when counts != null.
+// err_word != null: when *err_word is not zero (a bounded wait of an earlier kernel of this call ran out, so the
+// sums are not to be trusted) *dst2 receives NaN instead.
 __global__ void k_final_sum(const double* __restrict__ vals, int n, double scale, double* __restrict__ dst,
                             double* __restrict__ dst2, const unsigned int* __restrict__ counts,
-                            unsigned int* __restrict__ count_dst) {
+                            unsigned int* __restrict__ count_dst, const unsigned int* __restrict__ err_word = nullptr) {
   __shared__ double sh[8];
   double s = 0.0, c = 0.0;
   for (int i = threadIdx.x; i < n; i += 256) {
@@ -479,7 +497,7 @@ __global__ void k_final_sum(const double* __restrict__ vals, int n, double scale
   c = block_sum_256(c, sh, threadIdx.x);
   if (threadIdx.x == 0) {
     *dst = s * scale;
-    if (dst2) *dst2 = s * scale;
+    if (dst2) *dst2 = (err_word != nullptr && *err_word != 0u) ? __longlong_as_double(0x7ff8000000000000ll) : s * scale;
     if (count_dst) *count_dst = static_cast<unsigned int>(c);
   }
 }

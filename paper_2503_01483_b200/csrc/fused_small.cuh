@@ -32,21 +32,20 @@ struct FusedCfg {
   static constexpr int kGBufs = (TERMS == 1) ? 2 : 1;
   static constexpr int kSmem = 1024 + TERMS * kFsTile /*R^T*/ + kFsXStages * kFsTile + kGBufs * kFsTile /*G*/ + 256;
 };
-// Rows whose variance is below this are skipped like zero-variance rows: the coefficients of dL/dY are formed in
-// float32 (float64 is an order of magnitude slower on this part) and 1/m2^2 must stay finite.
-constexpr float kFsMinVariance = 1e-18f;
 
 struct FusedParams {
   CUtensorMap tmX;    // X  [N][128] bf16, box 128 rows x 64
   CUtensorMap tmRhi;  // R^T hi [128][128] bf16, box 128 x 64
   CUtensorMap tmRlo;  // R^T lo
   int N;
+  double n_mean;      // tokens the loss is a mean over (N, or all shards' rows in a sharded fit)
   int tiles;          // ceil(N / 128)
   float kappa_t;
   float* dr_partial;        // [gridDim.x][128][128]
   double* loss_partial;     // [gridDim.x]
   unsigned int* deg_partial;// [gridDim.x]
   unsigned int* err_word;
+  unsigned long long wait_limit_ns;  // bound of every device-side wait of this launch
 };
 
 // Shared-memory descriptor for an "MN-major" bf16 operand stored as rows of 64 elements (128 bytes,
@@ -151,7 +150,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
       for (int n = 0; n < my_tiles; ++n) {
         const int s = n % kFsXStages;
         const uint32_t ph = (n / kFsXStages) & 1;
-        if (!mbar_wait_bounded(x_empty(s), ph ^ 1u, abort_flag, 11u)) {
+        if (!mbar_wait_bounded(x_empty(s), ph ^ 1u, abort_flag, 11u, p.wait_limit_ns)) {
           ok = false;
           break;
         }
@@ -176,7 +175,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
     if (lane == 0 && my_tiles > 0) {
-      bool ok = mbar_wait_bounded(r_full, 0u, abort_flag, 12u);
+      bool ok = mbar_wait_bounded(r_full, 0u, abort_flag, 12u, p.wait_limit_ns);
       const uint32_t acc_dr = tmem_base + kColDr;
       // MMA1 runs two tiles ahead of MMA2, so the tensor pipe has work while a tile is in the epilogue
       for (int n = 0; n <= my_tiles + 1 && ok; ++n) {
@@ -184,8 +183,8 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
           // Y(n) = X(n) R
           const int s = n % kFsXStages;
           const int b = n & 1;
-          if (!mbar_wait_bounded(x_full(s), (n / kFsXStages) & 1, abort_flag, 13u) ||
-              !mbar_wait_bounded(y_empty(b), ((n >> 1) & 1) ^ 1u, abort_flag, 14u)) {
+          if (!mbar_wait_bounded(x_full(s), (n / kFsXStages) & 1, abort_flag, 13u, p.wait_limit_ns) ||
+              !mbar_wait_bounded(y_empty(b), ((n >> 1) & 1) ^ 1u, abort_flag, 14u, p.wait_limit_ns)) {
             ok = false;
             break;
           }
@@ -212,7 +211,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
           // dR += X(m)^T G(m): contraction over the tile's 128 tokens, 16 per MMA = two 8-row groups
           const int m = n - 2;
           const int s = m % kFsXStages;
-          if (!mbar_wait_bounded(g_full(m & 1), (m >> 1) & 1, abort_flag, 15u)) {
+          if (!mbar_wait_bounded(g_full(m & 1), (m >> 1) & 1, abort_flag, 15u, p.wait_limit_ns)) {
             ok = false;
             break;
           }
@@ -238,13 +237,13 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
     const int grp = (warp - 2) >> 2;    // = tile parity = Y accumulator = G buffer
     const int trow = lg * 32 + lane;    // token within the tile (and row of dR at the end)
     const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(lg * 32) << 16);
-    const float kscale = static_cast<float>(4.0 / (static_cast<double>(p.N) * 128.0));
+    const float kscale = static_cast<float>(4.0 / (p.n_mean * 128.0));
     double loss_acc = 0.0;
     unsigned int deg_acc = 0;
     bool ok = true;
     for (int n = grp; n < my_tiles && ok; n += 2) {
       const uint32_t par = (n >> 1) & 1;
-      const bool got = mbar_wait_bounded(y_full(grp), par, abort_flag, 16u);
+      const bool got = mbar_wait_bounded(y_full(grp), par, abort_flag, 16u, p.wait_limit_ns);
       if (!__all_sync(0xffffffffu, got)) {
         ok = false;
         break;
@@ -260,35 +259,54 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(y_empty(grp));
+      const int row = (static_cast<int>(blockIdx.x) + n * static_cast<int>(gridDim.x)) * 128 + trow;
 
       // Eq. 3 on the row: mean, then central power sums about it.  Two-wide arithmetic (packed f32x2
       // add/mul/fma): this epilogue is bound by instruction issue and latency, not by memory.
-      float mean;
+      // The kurtosis does not depend on the scale of the row, and neither must its evaluation: the first pass also
+      // takes the row's mean square, and everything after it works on the row times pw, the power of two nearest to
+      // 1/rms, so that no power sum leaves float32's range whatever the scale of X.
+      float mean, pw;
       {
-        float2 a0 = make_float2(0.f, 0.f), a1 = a0, a2 = a0, a3 = a0;
+        float2 a0 = make_float2(0.f, 0.f), a1 = a0, a2 = a0, a3 = a0, q0 = a0, q1 = a0, q2 = a0, q3 = a0;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
 #pragma unroll
           for (int j = 0; j < 32; j += 8) {
-            a0 = __fadd2_rn(a0, make_float2(__uint_as_float(v[c][j]), __uint_as_float(v[c][j + 1])));
-            a1 = __fadd2_rn(a1, make_float2(__uint_as_float(v[c][j + 2]), __uint_as_float(v[c][j + 3])));
-            a2 = __fadd2_rn(a2, make_float2(__uint_as_float(v[c][j + 4]), __uint_as_float(v[c][j + 5])));
-            a3 = __fadd2_rn(a3, make_float2(__uint_as_float(v[c][j + 6]), __uint_as_float(v[c][j + 7])));
+            const float2 x0 = make_float2(__uint_as_float(v[c][j]), __uint_as_float(v[c][j + 1]));
+            const float2 x1 = make_float2(__uint_as_float(v[c][j + 2]), __uint_as_float(v[c][j + 3]));
+            const float2 x2 = make_float2(__uint_as_float(v[c][j + 4]), __uint_as_float(v[c][j + 5]));
+            const float2 x3 = make_float2(__uint_as_float(v[c][j + 6]), __uint_as_float(v[c][j + 7]));
+            a0 = __fadd2_rn(a0, x0);
+            a1 = __fadd2_rn(a1, x1);
+            a2 = __fadd2_rn(a2, x2);
+            a3 = __fadd2_rn(a3, x3);
+            q0 = __ffma2_rn(x0, x0, q0);
+            q1 = __ffma2_rn(x1, x1, q1);
+            q2 = __ffma2_rn(x2, x2, q2);
+            q3 = __ffma2_rn(x3, x3, q3);
           }
         }
         a0 = __fadd2_rn(__fadd2_rn(a0, a1), __fadd2_rn(a2, a3));
+        q0 = __fadd2_rn(__fadd2_rn(q0, q1), __fadd2_rn(q2, q3));
         mean = (a0.x + a0.y) * (1.0f / 128.0f);
+        const float msq = (q0.x + q0.y) * (1.0f / 128.0f);
+        // pw = 2^-floor(e/2), e the binary exponent of the mean square (an all-zero row gives 2^63: harmless)
+        const int e = static_cast<int>((__float_as_uint(msq) >> 23) & 0xffu) - 127;
+        pw = __uint_as_float(static_cast<uint32_t>(127 - (e >> 1)) << 23);
       }
+      const float nmp = -mean * pw;  // the scaled row is v * pw + nmp
       float s2, s3, s4;
       {
-        const float2 nm = make_float2(-mean, -mean);
+        const float2 pw2 = make_float2(pw, pw), nm = make_float2(nmp, nmp);
         float2 b2 = make_float2(0.f, 0.f), b3 = b2, b4 = b2, e2 = b2, e3 = b2, e4 = b2;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
-            const float2 c0 = __fadd2_rn(make_float2(__uint_as_float(v[c][j]), __uint_as_float(v[c][j + 1])), nm);
-            const float2 c1 = __fadd2_rn(make_float2(__uint_as_float(v[c][j + 2]), __uint_as_float(v[c][j + 3])), nm);
+            const float2 c0 = __ffma2_rn(make_float2(__uint_as_float(v[c][j]), __uint_as_float(v[c][j + 1])), pw2, nm);
+            const float2 c1 =
+                __ffma2_rn(make_float2(__uint_as_float(v[c][j + 2]), __uint_as_float(v[c][j + 3])), pw2, nm);
             const float2 q0 = __fmul2_rn(c0, c0), q1 = __fmul2_rn(c1, c1);
             b2 = __fadd2_rn(b2, q0);
             e2 = __fadd2_rn(e2, q1);
@@ -305,32 +323,32 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
         s3 = b3.x + b3.y;
         s4 = b4.x + b4.y;
       }
-      // kappa, the loss term and the coefficients of dL/dY (same rules as the general path, in float32)
-      const int row = (static_cast<int>(blockIdx.x) + n * static_cast<int>(gridDim.x)) * 128 + trow;
+      // kappa, the loss term and the coefficients of dL/dY (same rules as the general path, in float32).  m2, m3, m4
+      // are moments of the scaled row (rms about 1); G for the unscaled row is pw times the scaled row's.
       const float m2 = s2 * (1.0f / 128.0f), m3 = s3 * (1.0f / 128.0f), m4 = s4 * (1.0f / 128.0f);
-      const float ms = fmaf(mean, mean, m2);
-      const bool degenerate = (ms == 0.f) || (m2 <= 1e-6f * ms) || (m2 < kFsMinVariance);
+      const float ms = fmaf(nmp, nmp, m2);
+      const bool degenerate = (ms == 0.f) || (m2 <= 1e-6f * ms);
       float ca = 0.f, cab = 0.f, cam3 = 0.f;
       if (!degenerate) {
         const float r = __frcp_rn(m2);
         const float kappa = (m4 * r) * r;
         const float diff = kappa - p.kappa_t;
         const float sgn = (diff > 0.f) ? 1.0f : ((diff < 0.f) ? -1.0f : 0.0f);
-        ca = ((sgn * kscale) * r) * r;
+        ca = (((sgn * kscale) * pw) * r) * r;
         cab = ca * (m4 * r);
         cam3 = ca * m3;
         if (row < p.N) loss_acc += static_cast<double>(fabsf(diff));
       } else if (row < p.N) {
         ++deg_acc;
       }
-      const float2 nmean2 = make_float2(-mean, -mean), ca2 = make_float2(ca, ca), ncab2 = make_float2(-cab, -cab),
-                   ncam32 = make_float2(-cam3, -cam3);
+      const float2 pwg = make_float2(pw, pw), nmean2 = make_float2(nmp, nmp), ca2 = make_float2(ca, ca),
+                   ncab2 = make_float2(-cab, -cab), ncam32 = make_float2(-cam3, -cam3);
 
       // G = a c^3 - ab c - am3 as bf16, token-major, into the swizzled tile MMA2 reads
       // with one G tile it is free once MMA2 of the previous tile (the other group's) has read it; with two,
       // once MMA2 of this group's previous tile has
       const int gw = (kGBufs == 2) ? n - 2 : n - 1;
-      const bool free_g = (gw < 0) || mbar_wait_bounded(g_empty(gw & 1), (gw >> 1) & 1, abort_flag, 17u);
+      const bool free_g = (gw < 0) || mbar_wait_bounded(g_empty(gw & 1), (gw >> 1) & 1, abort_flag, 17u, p.wait_limit_ns);
       if (!__all_sync(0xffffffffu, free_g)) {
         ok = false;
         break;
@@ -343,8 +361,8 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
           uint32_t pk[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            const float2 cc = __fadd2_rn(make_float2(__uint_as_float(v[c][j8 * 8 + 2 * e]),
-                                                     __uint_as_float(v[c][j8 * 8 + 2 * e + 1])), nmean2);
+            const float2 cc = __ffma2_rn(make_float2(__uint_as_float(v[c][j8 * 8 + 2 * e]),
+                                                     __uint_as_float(v[c][j8 * 8 + 2 * e + 1])), pwg, nmean2);
             const float2 g = __ffma2_rn(cc, __ffma2_rn(__fmul2_rn(ca2, cc), cc, ncab2), ncam32);
             __nv_bfloat162 h = __floats2bfloat162_rn(g.x, g.y);
             pk[e] = *reinterpret_cast<uint32_t*>(&h);
@@ -379,7 +397,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
     // partial dR of this CTA: each warp writes its 32 rows x 64 columns (group 0 the left half)
     float* dst = p.dr_partial + (static_cast<long long>(blockIdx.x) * 128 + trow) * 128 + grp * 64;
     if (my_tiles > 0 && ok) {
-      const bool got = mbar_wait_bounded(dr_full, 0u, abort_flag, 18u);
+      const bool got = mbar_wait_bounded(dr_full, 0u, abort_flag, 18u, p.wait_limit_ns);
       if (__all_sync(0xffffffffu, got)) {
         tc_fence_after_sync();
         uint32_t w[32];

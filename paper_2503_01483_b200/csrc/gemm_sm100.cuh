@@ -67,6 +67,10 @@ struct GemmParams {
   unsigned int gate_min;
   const unsigned int* terms_dev;  // when not null, min(terms, *terms_dev) operand pairs are used
   unsigned int* err_word;     // receives the code of a wait that ran out
+  unsigned long long wait_limit_ns;  // bound of every device-side wait of this launch
+  // when not null: row m of D is multiplied by row_scale[m] before the epilogue sees it (the RMSNorm that follows
+  // the rotation in the paper's small network, applied to the float32 accumulator)
+  const float* row_scale;
 };
 
 // Unsigned keys that order like the floats they encode (negative floats reversed, positive ones above them).
@@ -230,7 +234,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
           const int kbl = it / n_terms;
           const int q = it - kbl * n_terms;
           const int kb = kb0 + kbl;
-          if (!mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, 1u)) {
+          if (!mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, 1u, p.wait_limit_ns)) {
             ok = false;
             break;
           }
@@ -276,14 +280,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
         const int iters = unit_iters(unit);
         const int buf = lt & 1;
         const uint32_t acc_phase = (lt >> 1) & 1;
-        if (!mbar_wait_bounded(acc_empty_bar(buf), acc_phase ^ 1u, abort_flag, 2u)) {
+        if (!mbar_wait_bounded(acc_empty_bar(buf), acc_phase ^ 1u, abort_flag, 2u, p.wait_limit_ns)) {
           ok = false;
           break;
         }
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * BN);
         for (int it = 0; it < iters; ++it) {
-          if (!mbar_wait_bounded(full_bar(stage), phase, abort_flag, 3u)) {
+          if (!mbar_wait_bounded(full_bar(stage), phase, abort_flag, 3u, p.wait_limit_ns)) {
             ok = false;
             break;
           }
@@ -336,7 +340,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
       const int buf = lt & 1;
       const uint32_t acc_phase = (lt >> 1) & 1;
       // the tensor-memory loads below are warp-collective: the whole warp goes on or the whole warp leaves
-      const bool got = mbar_wait_bounded(acc_full_bar(buf), acc_phase, abort_flag, 4u);
+      const bool got = mbar_wait_bounded(acc_full_bar(buf), acc_phase, abort_flag, 4u, p.wait_limit_ns);
       if (!__all_sync(0xffffffffu, got)) {
         ok = false;
         break;
@@ -345,6 +349,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
       const uint32_t t_addr =
           tmem_base + (static_cast<uint32_t>(lane_group * 32) << 16) + static_cast<uint32_t>(buf * BN);
       const bool row_ok = row < p.M;
+      const bool scaled = p.row_scale != nullptr;  // uniform over the grid
+      const float rs = (scaled && row_ok) ? p.row_scale[row] : 1.0f;
+      auto scale32 = [&](uint32_t (&a)[32]) {
+        if (scaled) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) a[j] = __float_as_uint(__uint_as_float(a[j]) * rs);
+        }
+      };
       uint32_t v[32];
 
       if constexpr (EPI == kStoreF32) {
@@ -352,6 +364,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
         for (int c0 = cbeg; c0 < cend; c0 += 32) {
           tmem_ld_32x32(t_addr + c0, v);
           tc_wait_ld();
+          scale32(v);
           if (row_ok)
             store_row32(p.out + static_cast<long long>(unit / plain_tiles) * p.split_stride +
                             static_cast<long long>(row) * p.ldo + n0 + c0,
@@ -368,6 +381,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
         tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) release_acc(buf);
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c) scale32(vv[c]);
         // pass 1: mean of the kHalf columns; pass 2: central power sums about it
         float s1 = 0.f;
 #pragma unroll
@@ -412,6 +427,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
         for (int c0 = cbeg; c0 < cend; c0 += 32) {
           tmem_ld_32x32(t_addr + c0, v);
           tc_wait_ld();
+          scale32(v);
           if (row_ok) {
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
@@ -429,6 +445,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
         for (int c0 = cbeg; c0 < cend; c0 += 32) {
           tmem_ld_32x32(t_addr + c0, v);
           tc_wait_ld();
+          scale32(v);
           if (asym) {
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
@@ -469,6 +486,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
         for (int c0 = cbeg; c0 < cend; c0 += 32) {
           tmem_ld_32x32(t_addr + c0, v);
           tc_wait_ld();
+          scale32(v);
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
             const float y = __uint_as_float(v[j]);
@@ -504,6 +522,23 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
     if constexpr (CTAS == 2) tmem_dealloc_pair(tmem_base, kTmemCols); else tmem_dealloc(tmem_base, kTmemCols);
   }
   if (threadIdx.x == 0 && *abort_flag != 0 && p.err_word != nullptr) atomicMax(p.err_word, *abort_flag);
+}
+
+// Test hook: one thread waits, through the same bounded wait as every kernel of this library, on a barrier that
+// nobody ever arrives on.  The wait gives up after limit_ns, the kernel returns normally, and *err_word receives
+// the waiting role's code (99): exactly what a stalled pipeline would leave behind.
+__global__ void k_wait_probe(unsigned long long limit_ns, unsigned int* err_word) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ uint32_t abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    fence_barrier_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) (void)mbar_wait_bounded(smem_u32(&bar), 0u, &abort_flag, 99u, limit_ns);
+  __syncthreads();
+  if (threadIdx.x == 0 && abort_flag != 0 && err_word != nullptr) atomicMax(err_word, abort_flag);
 }
 
 }  // namespace kt

@@ -47,15 +47,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Wait with a bound.  Gives up after kWaitLimitNs of wall time, or as soon as
-// another thread of the CTA has raised *abort_flag; on giving up it raises the
-// flag itself (with `where`, a code naming the waiting role) and returns false,
-// so that every role leaves its loop and the CTA reaches its teardown.  No wait
-// in this library can spin for ever.
-constexpr uint64_t kWaitLimitNs = 4000000000ull;  // 4 s: far above any legitimate wait
+// Wait with a bound.  Gives up after `limit_ns` of wall time (kernels take it from
+// their parameters; kDefaultWaitLimitNs unless the caller configured another), or
+// as soon as another thread of the CTA has raised *abort_flag; on giving up it
+// raises the flag itself (with `where`, a code naming the waiting role) and
+// returns false, so that every role leaves its loop and the CTA reaches its
+// teardown.  No wait in this library can spin for ever.
+constexpr uint64_t kDefaultWaitLimitNs = 4000000000ull;  // 4 s: far above any legitimate wait
 
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                                  uint32_t where) {
+                                                  uint32_t where, uint64_t limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   uint32_t spins = 0;
@@ -63,7 +64,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 63u) == 0) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) {
+      if (global_timer_ns() - t0 > limit_ns) {
         *abort_flag = where;
         return false;
       }

@@ -3,8 +3,9 @@
 Two ways to use several GPUs.  Layers are independent problems (each has its own rotation): sharded over
 ranks they exchange no data on the compute path, and the process group is used only for the start barrier,
 for the maximum of the per-rank times and for summing the work done.  One rotation over many tokens is the
-other: the rows of X are sharded (`fit_row_sharded`), every rank computes the loss and gradient of its rows,
-and one sum all-reduce per step of dR (d x d float32) and of the loss makes the step identical on all ranks.
+other: the rows of X are sharded (`fit_row_sharded` -> kt_fit_sharded), every rank computes the loss and gradient of
+its rows, and the library calls back, while it enqueues a step, for one sum all-reduce of dR (d x d float32) and of
+the loss, which makes the step identical on all ranks.
 Works with NCCL (GPU) and gloo (CPU tests).
 """
 from __future__ import annotations
@@ -69,26 +70,49 @@ def whole_job_throughput(dist, units_this_rank, seconds_this_rank, device="cpu")
     return total / t, t
 
 
-def fit_row_sharded(ctx, X_local, R, steps, lr, dist, rows_total):
-    """`steps` x (loss and gradient of this rank's rows; all-reduce; step on the orthogonal group).
+class _DeviceBuffer:
+    """A raw device pointer dressed up for torch.as_tensor (no copy)."""
 
-    The loss is a mean over all `rows_total` tokens (per-token mode), so the full-batch gradient is the sum over
-    ranks of (rows of the rank / rows_total) x the rank's own gradient: one SUM all-reduce of dR and one of the
-    loss per step.  Every rank then takes the same step from the same dR, so the replicas of R stay bit-identical
-    without ever being exchanged.  `ctx` needs loss_grad(X, R) -> (loss, dR) and orth_step(R, dR, lr) (the
-    library's Context); returns the per-step full-batch losses."""
-    w = float(X_local.shape[0]) / float(rows_total)
-    losses = []
-    for _ in range(steps):
-        loss, dR = ctx.loss_grad(X_local, R)
-        dR.mul_(w)
-        lt = torch.tensor([loss * w], dtype=torch.float64, device=dR.device)
-        if dist is not None:
-            dist.all_reduce(dR, op=dist.ReduceOp.SUM)
-            dist.all_reduce(lt, op=dist.ReduceOp.SUM)
-        ctx.orth_step(R, dR, lr)
-        losses.append(float(lt.item()))
-    return losses
+    def __init__(self, ptr, count, typestr):
+        self.__cuda_array_interface__ = {"shape": (count,), "typestr": typestr, "data": (ptr, False), "version": 2}
+
+
+def all_reduce_hook(dist, device):
+    """The `reduce` callable of Context.fit_sharded: an in-place SUM all-reduce, through torch.distributed, of the
+    buffer the library hands over (NCCL for device memory: the collective is ordered after the work already enqueued
+    on torch's current stream, which must be the context's stream, and nothing waits on the host; gloo for the CPU
+    tests).  Returns None when there is one process only."""
+    if dist is None:
+        return None
+    import ctypes as C
+    dev = torch.device(device)
+    views = {}
+
+    def reduce(ptr, count, dtype, stream):
+        key = (ptr, count, dtype)
+        t = views.get(key)
+        if t is None:
+            if dev.type == "cuda":
+                t = torch.as_tensor(_DeviceBuffer(ptr, count, "<f4" if dtype == 1 else "<f8"), device=dev)
+            else:
+                ctype = C.c_float if dtype == 1 else C.c_double
+                t = torch.frombuffer((ctype * count).from_address(ptr),
+                                     dtype=torch.float32 if dtype == 1 else torch.float64)
+            views[key] = t
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        return 0
+
+    return reduce
+
+
+def fit_row_sharded(ctx, X_local, R, steps, lr, dist, rows_total):
+    """One rotation over a batch whose rows are spread over the ranks: `ctx.fit_sharded` (kt_fit_sharded) on this
+    rank's rows with the all-reduce hook above.  The loss is a mean over all `rows_total` tokens; per step the
+    library sums the loss and dR (d x d float32) over the ranks -- and, for the whole-layer loss, the batch's mean
+    and central sums -- on its stream, without a host round trip, and every rank then takes the same step, so the
+    replicas of R stay bit-identical without ever being exchanged.  Returns the per-step losses of the whole batch."""
+    rep = ctx.fit_sharded(X_local, R, rows_total, all_reduce_hook(dist, R.device), steps, lr, history=True)
+    return rep["loss_history"]
 
 
 def finalize(dist):

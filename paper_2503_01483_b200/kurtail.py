@@ -15,9 +15,10 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libkurtail.so")
 
-KT_BF16, KT_F32 = 0, 1
+KT_BF16, KT_F32, KT_F64 = 0, 1, 2
 STATUS = {0: "KT_OK", 1: "KT_ERR_INVALID_ARG", 2: "KT_ERR_SHAPE", 3: "KT_ERR_ALIGN", 4: "KT_ERR_WORKSPACE",
-          5: "KT_ERR_ARCH", 6: "KT_ERR_CUDA", 7: "KT_ERR_NONFINITE", 8: "KT_ERR_TIMEOUT", 9: "KT_ERR_TOO_LARGE"}
+          5: "KT_ERR_ARCH", 6: "KT_ERR_CUDA", 7: "KT_ERR_NONFINITE", 8: "KT_ERR_TIMEOUT", 9: "KT_ERR_TOO_LARGE",
+          10: "KT_ERR_COOPERATIVE", 11: "KT_ERR_REDUCE"}
 
 
 class KtError(RuntimeError):
@@ -37,7 +38,7 @@ class kt_config(C.Structure):
                 ("forward_terms", C.c_int32), ("small_d_fused", C.c_int32), ("small_d_orth", C.c_int32),
                 ("optimizer", C.c_int32), ("beta1", C.c_float), ("beta2", C.c_float), ("adam_eps", C.c_float),
                 ("norm_iters", C.c_int32), ("backward_mode", C.c_int32), ("cta_pairs", C.c_int32), ("loss_mode", C.c_int32), ("rmsnorm", C.c_int32), ("rms_eps", C.c_float),
-                ("reserved", C.c_int32 * 2)]
+                ("wait_limit_ms", C.c_int32), ("reserved", C.c_int32)]
 
 
 class kt_quant_spec(C.Structure):
@@ -62,9 +63,13 @@ class kt_profile(C.Structure):
 EXPORTS = ["kt_default_config", "kt_create", "kt_destroy", "kt_status_string", "kt_workspace_bytes",
            "kt_set_workspace", "kt_init_rotation", "kt_kurtosis_loss", "kt_loss_grad", "kt_row_moments",
            "kt_rotate", "kt_orth_step", "kt_adam_step", "kt_orth_error", "kt_fit", "kt_fit_layers",
-           "kt_fit_shared_workspace_bytes", "kt_fit_shared", "kt_fit_host",
+           "kt_fit_shared_workspace_bytes", "kt_fit_shared", "kt_fit_host", "kt_fit_sharded", "kt_fit_shared_sharded",
+           "kt_test_wait_timeout",
            "kt_quant4_error", "kt_quant4_codes", "kt_quant_error", "kt_quant_codes", "kt_rowmax_success", "kt_profile_begin", "kt_profile_end",
            "kt_kurtosis_loss_noalloc"]
+
+# int32 reduce(void* user, void* dev_ptr, int64 count, int32 dtype, void* cuda_stream)
+REDUCE_FN = C.CFUNCTYPE(C.c_int32, C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p)
 
 _lib = None
 
@@ -103,6 +108,10 @@ def lib():
     L.kt_fit_shared.argtypes = [vp, C.POINTER(kt_mat), i32, i64, C.POINTER(i32), i32, vp, i32, f32,
                                 C.POINTER(kt_fit_report)]
     L.kt_fit_host.argtypes = [vp, kt_mat, vp, vp, vp, i32, f32, C.POINTER(kt_fit_report)]
+    L.kt_fit_sharded.argtypes = [vp, kt_mat, vp, i64, REDUCE_FN, vp, i32, f32, C.POINTER(kt_fit_report)]
+    L.kt_fit_shared_sharded.argtypes = [vp, C.POINTER(kt_mat), i32, i64, C.POINTER(i32), i32, vp, i64, REDUCE_FN, vp,
+                                        i32, f32, C.POINTER(kt_fit_report)]
+    L.kt_test_wait_timeout.argtypes = [vp, i32]
     L.kt_quant4_error.argtypes = [vp, kt_mat, vp, dp]
     L.kt_quant4_codes.argtypes = [vp, vp, i64, i64, vp, vp]
     L.kt_quant_error.argtypes = [vp, kt_mat, vp, C.POINTER(kt_quant_spec), dp]
@@ -158,8 +167,9 @@ def kurtosis_loss_noalloc(X, R, loss_dev, stream=None):
     `loss_dev` is a caller-owned float64 device tensor of one element; the call is stream
     ordered (synchronise before reading it).  Raises KtError(9) above N 16384 / d 1024."""
     sp = C.c_void_p(stream.cuda_stream if stream is not None else 0)
-    _check(lib().kt_kurtosis_loss_noalloc(as_mat(X), R.data_ptr(), loss_dev.data_ptr(), sp),
-           "kt_kurtosis_loss_noalloc")
+    with torch.cuda.device(X.device):     # the call works on the current device's copy of the built-in array
+        _check(lib().kt_kurtosis_loss_noalloc(as_mat(X), R.data_ptr(), loss_dev.data_ptr(), sp),
+               "kt_kurtosis_loss_noalloc")
 
 
 class Context:
@@ -287,15 +297,7 @@ class Context:
         """kt_fit_shared: one R for the equally shaped buffers Xs; `order` is a sequence of steps*batch sample ids."""
         nb = len(Xs)
         mats = (kt_mat * nb)(*[as_mat(X) for X in Xs])
-        need = C.c_size_t()
-        _check(lib().kt_fit_shared_workspace_bytes(self._h, rows_per_sample, batch, mats[0].cols, C.byref(need)),
-               "kt_fit_shared_workspace_bytes")
-        if need.value > self._ws_bytes:
-            self._ws = None
-            self._ws = torch.empty(need.value + 256, dtype=torch.uint8, device=self.device)
-            base = (self._ws.data_ptr() + 255) // 256 * 256
-            _check(lib().kt_set_workspace(self._h, C.c_void_p(base), need.value), "kt_set_workspace")
-            self._ws_bytes = need.value
+        self._shared_workspace(rows_per_sample, batch, mats[0].cols)
         ids = (C.c_int32 * (steps * batch))(*[int(v) for v in order[:steps * batch]])
         rep = kt_fit_report()
         hist = (C.c_double * steps)() if history and steps > 0 else None
@@ -304,6 +306,50 @@ class Context:
         _check(lib().kt_fit_shared(self._h, mats, nb, rows_per_sample, ids, batch, R.data_ptr(), steps, lr,
                                    C.byref(rep)), "kt_fit_shared")
         return _rep_dict(rep, hist)
+
+    def _shared_workspace(self, rows_per_sample, batch, d):
+        need = C.c_size_t()
+        _check(lib().kt_fit_shared_workspace_bytes(self._h, rows_per_sample, batch, d, C.byref(need)),
+               "kt_fit_shared_workspace_bytes")
+        if need.value > self._ws_bytes:
+            self._ws = None
+            self._ws = torch.empty(need.value + 256, dtype=torch.uint8, device=self.device)
+            base = (self._ws.data_ptr() + 255) // 256 * 256
+            _check(lib().kt_set_workspace(self._h, C.c_void_p(base), need.value), "kt_set_workspace")
+            self._ws_bytes = need.value
+
+    def fit_sharded(self, X_local, R, rows_total, reduce, steps, lr, history=False):
+        """kt_fit_sharded.  `reduce` is None (a single shard) or a Python callable
+        reduce(dev_ptr, count, dtype, cuda_stream) -> 0 that enqueues an in-place sum all-reduce."""
+        m = self._prep(X_local)
+        rep = kt_fit_report()
+        hist = (C.c_double * max(steps, 1))() if history else None
+        if history:
+            rep.loss_history = C.cast(hist, C.POINTER(C.c_double))
+        cb = REDUCE_FN(lambda user, ptr, count, dtype, stream: int(reduce(ptr, count, dtype, stream))) \
+            if reduce is not None else C.cast(None, REDUCE_FN)
+        _check(lib().kt_fit_sharded(self._h, m, R.data_ptr(), rows_total, cb, None, steps, lr, C.byref(rep)),
+               "kt_fit_sharded")
+        return _rep_dict(rep, hist[:steps] if history else None)
+
+    def fit_shared_sharded(self, Xs, rows_per_sample, order, batch, R, rows_total, reduce, steps, lr, history=False):
+        """kt_fit_shared_sharded: this process's share (`batch` samples per step, its own `order`) of every minibatch."""
+        nb = len(Xs)
+        mats = (kt_mat * nb)(*[as_mat(X) for X in Xs])
+        self._shared_workspace(rows_per_sample, batch, mats[0].cols)
+        ids = (C.c_int32 * (steps * batch))(*[int(v) for v in order[:steps * batch]])
+        rep = kt_fit_report()
+        hist = (C.c_double * steps)() if history and steps > 0 else None
+        if hist is not None:
+            rep.loss_history = C.cast(hist, C.POINTER(C.c_double))
+        cb = REDUCE_FN(lambda user, ptr, count, dtype, stream: int(reduce(ptr, count, dtype, stream))) \
+            if reduce is not None else C.cast(None, REDUCE_FN)
+        _check(lib().kt_fit_shared_sharded(self._h, mats, nb, rows_per_sample, ids, batch, R.data_ptr(), rows_total,
+                                           cb, None, steps, lr, C.byref(rep)), "kt_fit_shared_sharded")
+        return _rep_dict(rep, hist)
+
+    def test_wait_timeout(self, limit_ms):
+        _check(lib().kt_test_wait_timeout(self._h, limit_ms), "kt_test_wait_timeout")
 
     def fit_host(self, X_host, X_staging, R_host, R_dev, steps, lr):
         m = as_mat(X_host)

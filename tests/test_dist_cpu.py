@@ -57,18 +57,25 @@ def test_single_rank_is_a_no_op():
 
 
 class _OracleCtx:
-    """Stands in for the library's Context on the CPU: same two calls, computed by the float64 oracle."""
+    """Stands in for the library's Context on the CPU: fit_sharded with the library's sequence of reductions per
+    step (the loss, then dR, each already weighted by this shard's share of the rows), computed by the float64
+    oracle and summed through the very hook the GPU path hands to kt_fit_sharded."""
 
-    def loss_grad(self, X, R):
+    def fit_sharded(self, X, R, rows_total, reduce, steps, lr, history=False):
         from oracle import kurtail_oracle as ko
-        L, dR = ko.loss_grad(X.numpy(), R.numpy())
-        return L, torch.from_numpy(dR)
-
-    def orth_step(self, R, dR, lr):
-        from oracle import kurtail_oracle as ko
-        Rn, _, _ = ko.orth_step(R.numpy(), dR.numpy(), lr)
-        R.copy_(torch.from_numpy(Rn))
-        return R
+        w = X.shape[0] / float(rows_total)
+        losses = []
+        for _ in range(steps):
+            L, dR = ko.loss_grad(X.numpy(), R.numpy())
+            loss_t = torch.tensor([L * w], dtype=torch.float64)
+            dR_t = torch.from_numpy(dR * w).contiguous()
+            if reduce is not None:
+                assert reduce(loss_t.data_ptr(), 1, 2, None) == 0
+                assert reduce(dR_t.data_ptr(), dR_t.numel(), 2, None) == 0
+            Rn, _, _ = ko.orth_step(R.numpy(), dR_t.numpy(), lr)
+            R.copy_(torch.from_numpy(Rn))
+            losses.append(float(loss_t.item()))
+        return dict(loss_history=losses)
 
 
 def _problem():
@@ -112,3 +119,37 @@ def test_row_sharded_fit_equals_the_full_batch_fit():
     # one rank alone: the plain loop
     X, R = _problem()
     assert np.allclose(dist_util.fit_row_sharded(_OracleCtx(), X, R, 5, 1e-2, None, X.shape[0]), losses_ref, rtol=1e-12)
+
+
+def _hook_worker(rank, world, port, out):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    dist = dist_util.init("gloo")
+    hook = dist_util.all_reduce_hook(dist, "cpu")
+    a = torch.full((6,), float(rank + 1), dtype=torch.float32)
+    b = torch.tensor([0.5 + rank], dtype=torch.float64)
+    for _ in range(2):                                   # the second call reuses the cached view of the buffer
+        assert hook(a.data_ptr(), a.numel(), 1, None) == 0
+    assert hook(b.data_ptr(), 1, 2, None) == 0
+    out.put((rank, a.tolist(), b.tolist()))
+    dist_util.barrier(dist)
+    dist_util.finalize(dist)
+
+
+def test_all_reduce_hook_sums_raw_buffers_in_place():
+    # the hook receives what kt_fit_sharded hands it: an address, a count and a type code (1 float32, 2 float64)
+    world = 2
+    port = _free_port()
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_hook_worker, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = sorted(out.get(timeout=120) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    # first reduction: 1 + 2 = 3 on both ranks; second: 3 + 3 = 6
+    assert res[0][1] == res[1][1] == [6.0] * 6
+    assert res[0][2] == res[1][2] == [2.0]
+    assert dist_util.all_reduce_hook(None, "cpu") is None
