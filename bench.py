@@ -9,12 +9,16 @@ initialised to the normalised Hadamard matrix).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
 
-Prints ONE JSON line.  With --impl reference the float64 CPU checker is timed on
-the host cores on a bounded sample of the same workload.
+Prints ONE JSON line.  The timed region is a fit of K steps, repeated back to back
+until it has lasted --min-seconds (so that clocks settle and the clock record
+holds many samples); ms_per_step is the mean over the repeats.  With --impl
+reference the float64 CPU checker is timed on the host cores on a bounded sample
+of the same workload.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import subprocess
@@ -42,6 +46,9 @@ WORKLOADS = {
     "llama2_7b_r1_shared": ("llama2_7b_r1_shared", 4096, 65536),
 }
 SHARED_RPS, SHARED_BATCH = 2048, 32
+NOMINAL_BF16_TFLOPS = 2250.0
+KERNEL_SOURCES = {"gemm_tn_kernel": ("gemm_sm100.cuh", "sm100_prims.cuh"),
+                  "fused_small_kernel": ("fused_small.cuh", "sm100_prims.cuh")}
 
 
 def measured_peaks():
@@ -54,6 +61,38 @@ def measured_peaks():
     return dict(tflops_sustained=1400.0, tflops_burst=1590.0, hbm_gbs=6650.0, source="fallback")
 
 
+def kernel_source_hash(kernel):
+    """Fingerprint of the files a kernel is compiled from: DRAM counters taken from an older kernel are not quoted."""
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES[kernel]:
+        with open(os.path.join(ROOT, "paper_2503_01483_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(kernel, role):
+    """DRAM bytes (read + written) per token of one launch, from the ncu capture summarised under profiles/.
+
+    profiles/dram_traffic.txt holds one line per captured launch:
+        kernel role rows d bytes_read bytes_write fixed_bytes source_hash
+    (fixed_bytes: the part that does not grow with the rows, e.g. the d x d operand).  Returns
+    (bytes per row, fixed bytes) or None when there is no line for this kernel and role, or when the kernel's
+    source has changed since the counters were taken."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    if not os.path.exists(path):
+        return None
+    want = kernel_source_hash(kernel)
+    with open(path) as f:
+        for line in f:
+            parts = line.split()
+            if len(parts) != 8 or parts[0].startswith("#"):
+                continue
+            k, r, rows, _d, rd, wr, fixed, src = parts
+            if k == kernel and r == role and src == want:
+                return (float(rd) + float(wr) - float(fixed)) / float(rows), float(fixed)
+    return None
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
 
@@ -61,15 +100,16 @@ class ClockSampler:
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index):
+    def __init__(self, index, period_ms=20):
         self.index = index
+        self.period_ms = period_ms
         self.rows = []
         self.proc = None
 
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", str(self.period_ms)],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.th = threading.Thread(target=self._read, daemon=True)
             self.th.start()
@@ -83,13 +123,13 @@ class ClockSampler:
     def stop(self, t0, t1):
         if self.proc is None:
             return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
-        time.sleep(0.15)
+        time.sleep(0.1)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=2)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], None, set()
+        sm, mx, power, reasons = [], None, [], set()
         for t, line in self.rows:
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 7:
@@ -98,28 +138,21 @@ class ClockSampler:
                 clk = float(parts[0]); mx = float(parts[1])
             except ValueError:
                 continue
-            if t0 <= t <= t1 + 0.1:
+            if t0 <= t <= t1:
                 sm.append(clk)
+                try:
+                    power.append(float(parts[2]))
+                except ValueError:
+                    pass
                 for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
                                      parts[3:7]):
                     if val.lower().startswith("active"):
                         reasons.add(name)
         sm.sort()
         med = sm[len(sm) // 2] if sm else None
-        return dict(sm_mhz=med, sm_max_mhz=mx, samples=len(sm), reasons=sorted(reasons))
-
-
-def oracle_step_time(X64, R64, lr, repeats=1):
-    """Seconds for the oracle's loss+gradient on the sample rows, and for its orthogonal step."""
-    from oracle import kurtail_oracle as ko
-    t0 = time.perf_counter()
-    for _ in range(repeats):
-        _, dR = ko.loss_grad(X64, R64)
-    t_lg = (time.perf_counter() - t0) / repeats
-    t0 = time.perf_counter()
-    ko.orth_step(R64, dR, lr)
-    t_orth = time.perf_counter() - t0
-    return t_lg, t_orth
+        return dict(sm_mhz=med, sm_max_mhz=mx, sm_mhz_min=sm[0] if sm else None, sm_mhz_p90=sm[int(len(sm) * 0.9)] if sm
+                    else None, power_w_max=max(power) if power else None, samples=len(sm),
+                    sample_period_ms=self.period_ms, reasons=sorted(reasons))
 
 
 def threads_in_use():
@@ -133,24 +166,58 @@ def threads_in_use():
     return len(os.sched_getaffinity(0))
 
 
-def cpu_baseline(sample_X, R_init, N_full, lr):
-    """The oracle as it stands, on the host cores, on a bounded row sample (rows are independent,
-    so loss+gradient time scales with N; the orthogonal step does not depend on N)."""
+def oracle_step_time(X64, R64, lr):
+    """Seconds for the oracle's loss+gradient on the sample rows, and for its orthogonal step."""
+    from oracle import kurtail_oracle as ko
+    t0 = time.perf_counter()
+    _, dR = ko.loss_grad(X64, R64)
+    t_lg = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    ko.orth_step(R64, dR, lr)
+    t_orth = time.perf_counter() - t0
+    return t_lg, t_orth
+
+
+def cpu_baseline(sample_X, R_init, N_full, lr, d):
+    """The oracle as it stands, on the host cores, on a bounded row sample (rows are independent, so the time of
+    loss+gradient scales with N; the orthogonal step does not depend on N).  Timed on all cores numpy uses, and once
+    more on one thread (loss+gradient on a quarter of the sample; the d^3 step only when it stays within seconds)."""
     import numpy as np
     X64 = sample_X.astype(np.float64)
     R64 = R_init.astype(np.float64)
     n_s = X64.shape[0]
     t_lg, t_orth = oracle_step_time(X64, R64, lr)
     t_full = t_lg * (N_full / n_s) + t_orth
-    return dict(value=N_full / t_full, unit="tokens/s", cores=threads_in_use(), kind="oracle",
-                sample="float64 loss+gradient on %d of %d rows at full d (%.2f s) scaled to N, plus one full "
-                       "orthogonal step (%.2f s)" % (n_s, N_full, t_lg, t_orth))
+    out = dict(value=N_full / t_full, unit="tokens/s", cores=threads_in_use(), kind="oracle",
+               sample="float64 loss+gradient on %d of %d rows at full d (%.2f s) scaled to N, plus one full "
+                      "orthogonal step (%.2f s)" % (n_s, N_full, t_lg, t_orth))
+    try:
+        from threadpoolctl import threadpool_limits
+        from oracle import kurtail_oracle as ko
+        n1 = max(16, n_s // 4)
+        with threadpool_limits(limits=1):
+            t0 = time.perf_counter()
+            _, dR = ko.loss_grad(X64[:n1], R64)
+            t1 = time.perf_counter() - t0
+            # 14 d^3 float64 flops for the step's matrix products at ~10 GFLOP/s on one core
+            if 14.0 * d ** 3 / 1e10 < 15.0:
+                t0 = time.perf_counter()
+                ko.orth_step(R64, dR, lr)
+                t1o = time.perf_counter() - t0
+                note = "one full orthogonal step (%.2f s)" % t1o
+            else:
+                t1o = t_orth * out["cores"]
+                note = "the orthogonal step's all-core time x cores (%.1f s; too long to run on one thread here)" % t1o
+        out["single_thread"] = dict(value=N_full / (t1 * (N_full / n1) + t1o), unit="tokens/s", cores=1,
+                                    sample="loss+gradient on %d rows (%.2f s) scaled to N, plus %s" % (n1, t1, note))
+    except Exception as e:  # threadpoolctl missing: the all-core figure stands alone
+        out["single_thread"] = dict(value=None, note="not measured: %s" % type(e).__name__)
+    return out
 
 
 def run_reference(args, wl_name, d, N_full):
     """--impl reference: the CPU oracle, as it stands, on a bounded sample per step."""
     import numpy as np
-    import torch
     from paper_2503_01483_b200 import synth
     from oracle import kurtail_oracle as ko
     rank = int(os.environ.get("RANK", "0"))
@@ -158,7 +225,8 @@ def run_reference(args, wl_name, d, N_full):
         return
     n_s = min(N_full, max(64, int(2.0e10 / (4.0 * d * d))))   # ~2e10 f64 flops of GEMM per step
     cfg = synth.config(WORKLOADS[wl_name][0], device="cpu", rows=n_s if wl_name != "kv_heads" else n_s // 32 * 32,
-                       **({"layers": 1} if wl_name == "llama3_70b_layer" else {}))
+                       **({"layers": 1} if WORKLOADS[wl_name][0] in ("llama3_70b_sweep", "llama2_7b_r1_shared")
+                          else {}))
     X = cfg["X"][0] if isinstance(cfg["X"], list) else cfg["X"]
     X64 = X.float().numpy().astype(np.float64)
     n_s = X64.shape[0]
@@ -188,6 +256,25 @@ def run_reference(args, wl_name, d, N_full):
     }))
 
 
+def executed_flops_per_step(N, d, rep, fwd_terms, recompute, steps, fused):
+    """Tensor-core flops one step really issues: the token GEMMs with every bf16 term of R and the recomputation,
+    and the d x d products the device did not gate off (from the last step's choices and the fit's guard count)."""
+    nd2 = 2.0 * N * d * d
+    tok = nd2 * fwd_terms + nd2 + (nd2 * fwd_terms if recompute else 0.0)
+    if fused:
+        return tok, None
+    d3 = 2.0 * float(d) ** 3
+    st = rep.get("series_terms_last") or 0
+    p0 = rep.get("p0_terms_last") or 0
+    guards = rep.get("guards_run") or 0
+    square = None
+    if st:
+        # A = dR R^T (1 term), P0 = W R (p0 terms), the further series terms, and per measuring step the 3-term
+        # R^T R on the upper tiles (a little over half of the output) -- the polish product only runs when needed
+        square = d3 * (1 + p0 + (st - 1)) + d3 * 3 * 0.53 * guards / max(steps, 1)
+    return tok, square
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -202,13 +289,19 @@ def main():
                     help="kt_config.optimizer: Cayley SGD (the headline configuration) or Cayley Adam")
     ap.add_argument("--shard", default="layers", choices=["layers", "rows"],
                     help="with --gpus N > 1: one independent layer per GPU (weak scaling, no collective), or the rows "
-                         "of one X sharded over the GPUs with an all-reduce of dR per step (strong scaling)")
+                         "of one X sharded over the GPUs (kt_fit_sharded: an all-reduce of dR and of the loss per "
+                         "step, enqueued by the library through its reduce hook; strong scaling)")
     ap.add_argument("--backward", default="stored", choices=["stored", "recompute"],
-                    help="kt_config.backward_mode: read back the float32 Y the forward pass kept (default) or "
-                         "recompute Y in a second GEMM pass")
+                    help="kt_config.backward_mode: read back the Y the forward pass kept (default) or recompute Y in "
+                         "a second GEMM pass, so that Y never reaches memory")
     ap.add_argument("--loss-mode", default="token", choices=["token", "layer"],
                     help="kt_config.loss_mode: one kurtosis per token (headline) or one over the whole layer")
-    ap.add_argument("--rmsnorm", action="store_true", help="kt_config.rmsnorm: row-normalise X first")
+    ap.add_argument("--rmsnorm", action="store_true", help="kt_config.rmsnorm: RMSNorm after the rotation")
+    ap.add_argument("--lr", type=float, default=0.0, help="override the workload's learning rate")
+    ap.add_argument("--min-seconds", type=float, default=2.0,
+                    help="repeat the timed K-step fit until the timed region has lasted this long (0: once)")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the short side measurements (other modes and workloads) added to the line")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -238,7 +331,7 @@ def main():
 
     # each rank fits its own layer buffer (layers are independent: no data-path collective)
     sweep = args.workload == "llama3_70b_sweep"
-    kw = dict(device=dev, rows=N_full if wl_cfg != "kv_heads" else N_full)
+    kw = dict(device=dev, rows=N_full)
     if wl_cfg == "llama3_70b_sweep":
         kw["layers"] = args.layers if sweep else 1
     shared = args.workload == "llama2_7b_r1_shared"
@@ -248,80 +341,105 @@ def main():
     cfg = synth.config(wl_cfg, **kw)
     Xs = cfg["X"] if isinstance(cfg["X"], list) else [cfg["X"]]   # all layer buffers stay resident in HBM
     X = Xs[0]
-    row_sharded = world > 1 and args.shard == "rows" and not sweep and not shared
+    row_sharded = world > 1 and args.shard == "rows" and not sweep
     N_all = X.shape[0]
-    if row_sharded:
+    if shared and world > 1:
+        # every rank holds its own block of the stored buffers and gathers its share of every minibatch
+        Xs = Xs[rank::world]
+        X = Xs[0]
+    elif row_sharded:
         # every rank generated the same X: keep this rank's block of rows (multiples of 128 except the last)
         per = (N_all // world + 127) // 128 * 128
         X = X[rank * per:min((rank + 1) * per, N_all)].contiguous()
     elif world > 1:
         # different data per rank: re-draw with a rank-dependent seed by rolling rows
         X = torch.roll(X, shifts=rank * 977, dims=0).contiguous()
-    N = SHARED_RPS * SHARED_BATCH if shared else X.shape[0]
-    lr = cfg["lr"]
-    ctx = kurtail.Context(dev, forward_terms=args.forward_terms, optimizer=1 if args.optimizer == "adam" else 0,
-                          loss_mode=1 if args.loss_mode == "layer" else 0, rmsnorm=1 if args.rmsnorm else 0,
-                          backward_mode=1 if args.backward == "recompute" else 0)
+    batch_local = SHARED_BATCH // world if (shared and row_sharded) else SHARED_BATCH
+    N = SHARED_RPS * batch_local if shared else X.shape[0]
+    lr = args.lr if args.lr > 0 else cfg["lr"]
+    ctx_kw = dict(forward_terms=args.forward_terms, optimizer=1 if args.optimizer == "adam" else 0,
+                  loss_mode=1 if args.loss_mode == "layer" else 0, rmsnorm=1 if args.rmsnorm else 0,
+                  backward_mode=1 if args.backward == "recompute" else 0)
+    ctx = kurtail.Context(dev, **ctx_kw)
+    fwd_terms = args.forward_terms if args.forward_terms in (1, 2) else (2 if d <= 512 else 1)
 
-    def fresh_R():
-        if cfg["init"] == "hadamard":
-            return ctx.init_rotation(d, "hadamard")
-        if cfg["init"] == "random_orthogonal":
-            return synth.random_orthogonal(d, seed=3, device=dev).contiguous()
-        return ctx.init_rotation(d, "identity")
+    def fresh_R(c=ctx, dd=d, init=cfg["init"]):
+        if init == "hadamard":
+            return c.init_rotation(dd, "hadamard")
+        if init == "random_orthogonal":
+            return synth.random_orthogonal(dd, seed=3, device=dev).contiguous()
+        return c.init_rotation(dd, "identity")
 
     R = fresh_R()
     R0_host = R.cpu().numpy()
+    hook = dist_util.all_reduce_hook(dist, dev) if row_sharded else None
+    order = None
     if shared:
-        # the shuffle: epochs of a seeded permutation of all stored samples, cut into minibatches
+        # the shuffle: epochs of a seeded permutation of this rank's stored samples, cut into minibatches
         n_samples = len(Xs) * (Xs[0].shape[0] // SHARED_RPS)
         rng = np.random.default_rng(1234 + rank)
-        need = (max(args.warmup, 1) + args.steps) * SHARED_BATCH
-        order = np.concatenate([rng.permutation(n_samples) for _ in range(need // n_samples + 1)])[:need].tolist()
-        w = max(args.warmup, 1)
-        ctx.fit_shared(Xs, SHARED_RPS, order[:w * SHARED_BATCH], SHARED_BATCH, R, w, lr)
-        order = order[w * SHARED_BATCH:]
-    elif row_sharded:
-        dist_util.fit_row_sharded(ctx, X, R, max(args.warmup, 1), lr, dist, N_all)
-    else:
-        ctx.fit(X, R, max(args.warmup, 1), lr)          # warm-up steps (also sizes the workspace)
+
+        def draw(steps):
+            need = steps * batch_local
+            return np.concatenate([rng.permutation(n_samples) for _ in range(need // n_samples + 1)])[:need].tolist()
+
+    def one_fit(steps):
+        """A fit of `steps` steps on this rank's data, continuing from the current R; returns the report."""
+        if sweep:
+            return ctx.fit_layers(Xs, sweep_Rs, steps, lr)[-1]
+        if shared and row_sharded:
+            return ctx.fit_shared_sharded(Xs, SHARED_RPS, draw(steps), batch_local, R, SHARED_RPS * SHARED_BATCH, hook,
+                                          steps, lr)
+        if shared:
+            return ctx.fit_shared(Xs, SHARED_RPS, draw(steps), batch_local, R, steps, lr)
+        if row_sharded:
+            return ctx.fit_sharded(X, R, N_all, hook, steps, lr)
+        return ctx.fit(X, R, steps, lr)
+
+    sweep_Rs = [R]
+    one_fit(max(args.warmup, 1))          # warm-up steps (also sizes the workspace)
+    if sweep:
+        sweep_Rs = [R] + [fresh_R() for _ in Xs[1:]]
     torch.cuda.synchronize()
 
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-        time.sleep(0.3)
+        time.sleep(0.2)
     dist_util.barrier(dist)
     torch.cuda.synchronize()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ctx.profile_begin()
     t_wall0 = time.time()
-    ev0.record()
-    if sweep:
-        Rs = [R] + [fresh_R() for _ in Xs[1:]]
-        torch.cuda.synchronize()
+    times_ms, reps = [], []
+    # every rank runs the same number of repeats: rank 0's clock decides, the others follow its count
+    while True:
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ev0.record()
-        reps = ctx.fit_layers(Xs, Rs, args.steps, lr)
-        rep = reps[-1]
-    elif shared:
-        rep = ctx.fit_shared(Xs, SHARED_RPS, order, SHARED_BATCH, R, args.steps, lr)
-    elif row_sharded:
-        hist = dist_util.fit_row_sharded(ctx, X, R, args.steps, lr, dist, N_all)
-        rep = dict(loss_first=hist[0], loss_last=hist[-1], orth_err=ctx.orth_error(R), alpha_last=None,
-                   w_norm_last=None, w_op_last=None, series_terms_last=None, p0_terms_last=None, guards_run=None)
-    else:
-        rep = ctx.fit(X, R, args.steps, lr)
-    ev1.record()
-    torch.cuda.synchronize()
+        rep = one_fit(args.steps)
+        ev1.record()
+        torch.cuda.synchronize()
+        ms_r = dist_util.max_over_ranks(dist, ev0.elapsed_time(ev1), dev)
+        times_ms.append(ms_r)
+        reps.append(rep)
+        go_on = 1.0 if (sum(times_ms) < args.min_seconds * 1e3 and len(times_ms) < 1000 and not sweep) else 0.0
+        if dist is not None:
+            t = torch.tensor([go_on], device=dev)
+            dist.broadcast(t, src=0)
+            go_on = float(t.item())
+        if go_on == 0.0:
+            break
     t_wall1 = time.time()
     prof = ctx.profile_end()
-    ms = ev0.elapsed_time(ev1)
-    ms = dist_util.max_over_ranks(dist, ms, dev)
     dist_util.barrier(dist)
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
     n_layers = len(Xs) if sweep else 1
+    repeats = len(times_ms)
+    ms = sum(times_ms) / repeats                     # mean device time of one K-step fit (max over ranks each)
     ms_per_step = ms / (args.steps * n_layers)
-    value = (N_all if row_sharded else world * N) * args.steps * n_layers / (ms * 1e-3)
+    tokens_per_step = N_all if (row_sharded and not shared) else (SHARED_RPS * SHARED_BATCH if (shared and row_sharded)
+                                                                   else world * N)
+    value = tokens_per_step * args.steps * n_layers / (ms * 1e-3)
+    rep = reps[-1]
 
     # ---- end to end through kt_fit_host: pinned host X and R in, R out, copies inside the timed region
     e2e = None
@@ -356,20 +474,21 @@ def main():
     g = prof["gemm"]
     per_role = {k: (g[k]["ms"] / g[k]["launches"] if g[k]["launches"] else None) for k in g}
     # every step launches exactly one forward (or one single-pass) kernel: the steps the event window covered
-    # (it holds 8192 launches; the 80-layer sweep overruns it, and then the split describes the steps it holds)
+    # (it holds 8192 launches; long runs overrun it, and then the split describes the steps it holds)
     steps_seen = max(g["fused"]["launches"] or g["forward"]["launches"], 1)
     share = {k: g[k]["ms"] / steps_seen / ms_per_step for k in g}
-    if g["fused"]["launches"] > 0:
+    timed_s = sum(times_ms) * 1e-3
+    capped = bool(clocks and "sw_power_cap" in (clocks.get("reasons") or []))
+    fused = g["fused"]["launches"] > 0
+    if fused:
         # d = 128: the single-pass kernel reads X once; HBM bound.  Algorithmic bytes per launch = N * d * 2.
         t_f = g["fused"]["ms"] / g["fused"]["launches"] * 1e-3
         alg_bytes = 2.0 * N * d
         achieved = alg_bytes / t_f / 1e9
         peak = peaks["hbm_gbs"]
-        # DRAM bytes per launch: ncu capture at 1 048 576 rows (268.4 MB algorithmic; read + written 272.8 MB with
-        # R as two bf16 terms, the default, and 272.0 MB with one), scaled by N
-        traffic = alg_bytes * ((272.0 if args.forward_terms == 1 else 272.8) / 268.435)
+        tr = recorded_traffic("fused_small_kernel", "terms%d" % fwd_terms)
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                    "traffic": traffic,
+                    "traffic": (tr[0] * N + tr[1]) if tr else None, "algorithmic_bytes": alg_bytes,
                     "kernel": "fused_small_kernel (loss + gradient in one pass over X): N*d*2 bytes per launch",
                     "peak_source": "%s copy bandwidth" % peaks["source"],
                     "per_role_ms_per_launch": per_role, "share_of_step": share}
@@ -380,39 +499,57 @@ def main():
         t_tok = sum(x["ms"] for x in tok)
         flops_per_launch = 2.0 * N * d * d
         achieved = flops_per_launch / (t_tok / max(n_launch, 1) * 1e-3) / 1e12 if t_tok > 0 else None
-        peak = peaks["tflops_sustained"]
+        # which measured cuBLAS figure the run compares with: the burst one for a short region that never met the
+        # power cap, the sustained one for a region of a second or more or one whose clock record shows the cap
+        use_burst = (not capped) and timed_s < 1.0
+        peak = peaks["tflops_burst"] if use_burst else peaks["tflops_sustained"]
+        trs = [recorded_traffic("gemm_tn_kernel", r) for r in
+               (("forward_stored" if args.backward == "stored" else "forward"), "backward_b")]
         traffic = None
-        if args.workload == "llama2_7b_attn" and not tok[1]["launches"]:
-            # mean DRAM bytes per launch of the two token GEMMs (forward with its float32 Y store, backward-B): ncu
-            # capture at N = 16384 (same d); the part that grows with N (everything but the 33.5 MB of R^T read by
-            # the forward pass) is scaled by N / 16384
-            var_mb = (392.9 + 246.7 - 33.5) + (628.4 + 61.5)
-            traffic = (var_mb * (N / 16384.0) + 33.5) / 2.0 * 1e6
+        if all(trs):
+            traffic = sum(t[0] * N + t[1] for t in trs) / 2.0        # mean of the two token GEMMs, per launch
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                     "frac": (achieved / peak) if achieved else None, "traffic": traffic,
+                    "algorithmic_bytes": 2.0 * N * d,
+                    "frac_of_sustained_peak": (achieved / peaks["tflops_sustained"]) if achieved else None,
                     "frac_of_burst_peak": (achieved / peaks["tflops_burst"]) if achieved else None,
-                    "frac_of_nominal_peak": (achieved / 2250.0) if achieved else None,
+                    "frac_of_nominal_peak": (achieved / NOMINAL_BF16_TFLOPS) if achieved else None,
                     "kernel": "gemm_tn_kernel (forward + moments, backward-B; backward-A too when it recomputes Y): "
                               "2*N*d^2 flops per launch",
-                    "peak_source": "%s bf16 GEMM, sustained (kernel timed inside a long step)" % peaks["source"],
+                    "peak_source": "%s cuBLAS bf16 GEMM, %s" % (
+                        peaks["source"], "burst (timed region %.2f s, no power-cap sample)" % timed_s if use_burst else
+                        "sustained (timed region %.2f s%s)" % (timed_s, ", sw_power_cap seen" if capped else "")),
                     "per_role_ms_per_launch": per_role, "share_of_step": share}
 
+    tok_exec, sq_exec = executed_flops_per_step(N, d, rep, fwd_terms, args.backward == "recompute", args.steps, fused)
+    s_iters = 2
+    alg_flops = 4.0 * N * d * d + 2.0 * float(d) ** 3 * (2 + s_iters)
     out = {
         "metric": METRIC + " at d=%d" % d, "value": value, "unit": "tokens/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "steps_per_s": 1e3 / ms_per_step,
+        "repeats": repeats, "timed_region_s": timed_s,
+        "ms_per_step_min": min(times_ms) / (args.steps * n_layers),
+        "ms_per_step_max": max(times_ms) / (args.steps * n_layers),
         "higher_is_better": True, "scaling": "strong" if row_sharded else "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": args.workload, "N": N, "d": d, "R_init": cfg["init"], "lr": lr,
                    "optimizer": "cayley_" + args.optimizer, "loss_mode": args.loss_mode, "rmsnorm": bool(args.rmsnorm),
-                   "backward": args.backward,
+                   "backward": args.backward + (" (Y kept between the forward and the backward pass)"
+                                                if args.backward == "stored" else " (Y never written)"),
                    "l2": "inputs (%.0f MiB of X per step) exceed the 126 MB L2" % (N * d * 2 / 2**20)
                    if N * d * 2 > 126e6 else "inputs fit in L2; no flush (small case)",
-                   "parallelism": ("rows of one X over the GPUs, all-reduce of dR per step" if row_sharded else
-                                   "one independent layer per GPU") if world > 1 else "single GPU",
+                   "parallelism": ("rows of one batch over the GPUs, kt_fit_sharded: all-reduce of dR and loss per "
+                                   "step" if row_sharded else "one independent layer per GPU") if world > 1
+                   else "single GPU",
                    **({"layers": n_layers, "steps_per_layer": args.steps, "resident_gib": n_layers * N * d * 2 / 2**30,
                        "sweep_seconds": ms * 1e-3} if sweep else {})},
-        "algorithmic_tflops": (4.0 * N * d * d) * world / (ms_per_step * 1e-3) / 1e12,
-        "loss_first": rep["loss_first"], "loss_last": rep["loss_last"], "orth_err": rep["orth_err"],
+        # useful work: the two token GEMMs and the step's d x d products as the method states them (s = 2 iterations)
+        "algorithmic_tflops": alg_flops * (1 if row_sharded else world) / (ms_per_step * 1e-3) / 1e12,
+        # what the tensor cores really issued: every bf16 term, the recomputation, the products the device kept
+        "executed_tflops": ((tok_exec + (sq_exec or 0.0)) * (1 if row_sharded else world) / (ms_per_step * 1e-3) / 1e12),
+        "executed_flops_per_step": {"token_gemms": tok_exec, "square_products": sq_exec},
+        "kcycles_per_step": (ms_per_step * clocks["sm_mhz"]) if clocks and clocks.get("sm_mhz") else None,
+        "loss_first": reps[0]["loss_first"], "loss_last": rep["loss_last"], "orth_err": rep["orth_err"],
         "alpha_last": rep["alpha_last"], "w_norm_last": rep["w_norm_last"],
         "step_choices": {k: rep[k] for k in ("w_op_last", "series_terms_last", "p0_terms_last", "guards_run")},
         "gpu_launches": prof["launches_total"], "clocks": clocks, "roofline": roofline, "e2e": e2e,
@@ -433,12 +570,73 @@ def main():
                                  "vs_init": ctx.rowmax_success(X, R, fresh_R())}
     if shared:
         out["config"].update({"buffers": len(Xs), "rows_per_buffer": int(Xs[0].shape[0]),
-                              "rows_per_sample": SHARED_RPS, "batch_samples": SHARED_BATCH,
+                              "rows_per_sample": SHARED_RPS, "batch_samples": batch_local,
                               "resident_gib": len(Xs) * Xs[0].shape[0] * d * 2 / 2**30})
     if not args.no_cpu_baseline and world == 1 and not shared:
         n_s = min(N, max(64, int(2.0e10 / (4.0 * d * d))))
         sample = X[:n_s].float().cpu().numpy()
-        out["cpu_baseline"] = cpu_baseline(sample, R0_host, N, lr)
+        out["cpu_baseline"] = cpu_baseline(sample, R0_host, N, lr, d)
+
+    # ---- short side measurements, so that one line carries the other modes and workloads too
+    if world == 1 and not args.no_extras and args.workload == "llama2_7b_attn" and not args.rows:
+        extras = {}
+
+        def short_fit(c, Xw, Rw, steps, lr_w, warm=3):
+            c.fit(Xw, Rw, warm, lr_w)
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            c.profile_begin()
+            a.record()
+            r = c.fit(Xw, Rw, steps, lr_w)
+            b.record()
+            torch.cuda.synchronize()
+            pr = c.profile_end()
+            return a.elapsed_time(b) / steps, r, pr
+
+        for name, kwx in (("backward_recompute", dict(backward_mode=1)), ("optimizer_adam", dict(optimizer=1)),
+                          ("lr_10_full_series", dict())):
+            c2 = kurtail.Context(dev, **kwx)
+            ms_x, r_x, _ = short_fit(c2, X, fresh_R(c2), 20, 10.0 if name == "lr_10_full_series" else lr)
+            extras[name] = {"ms_per_step": ms_x, "tokens_per_s": N / (ms_x * 1e-3), "steps": 20,
+                            "series_terms_last": r_x["series_terms_last"], "p0_terms_last": r_x["p0_terms_last"],
+                            "guards_run": r_x["guards_run"], "orth_err": r_x["orth_err"]}
+            c2.close()
+        ctx.close()
+        del X, Xs, R
+        torch.cuda.empty_cache()
+        for wl, steps_w in (("kv_heads", 50), ("llama3_70b_layer", 10), ("llama3_8b_down", 6)):
+            wcfg_name, dw, Nw = WORKLOADS[wl]
+            kww = dict(device=dev, rows=Nw)
+            if wcfg_name == "llama3_70b_sweep":
+                kww["layers"] = 1
+            wc = synth.config(wcfg_name, **kww)
+            Xw = wc["X"][0] if isinstance(wc["X"], list) else wc["X"]
+            c2 = kurtail.Context(dev)
+            # (the random orthogonal start of the widest workload is a float64 QR of minutes on the host: the side
+            # measurement starts from a float32 QR made on the device)
+            if wc["init"] == "random_orthogonal":
+                gq = torch.Generator(device=dev).manual_seed(3)
+                Rw = torch.linalg.qr(torch.randn((dw, dw), device=dev, generator=gq))[0].contiguous()
+            else:
+                Rw = fresh_R(c2, dw, wc["init"])
+            ms_x, r_x, pr = short_fit(c2, Xw, Rw, steps_w, wc["lr"])
+            gg = pr["gemm"]
+            ex = {"ms_per_step": ms_x, "tokens_per_s": Nw / (ms_x * 1e-3), "steps": steps_w, "N": Nw, "d": dw,
+                  "orth_err": r_x["orth_err"]}
+            if gg["fused"]["launches"]:
+                t_f = gg["fused"]["ms"] / gg["fused"]["launches"] * 1e-3
+                ex["single_pass_kernel_us"] = t_f * 1e6
+                ex["hbm_frac_of_measured"] = 2.0 * Nw * dw / t_f / 1e9 / peaks["hbm_gbs"]
+            else:
+                tk = [gg[k] for k in ("forward", "backward_b")]
+                t_l = sum(x["ms"] for x in tk) / max(sum(x["launches"] for x in tk), 1) * 1e-3
+                ex["token_gemm_tflops"] = 2.0 * Nw * dw * dw / t_l / 1e12
+                ex["square_share_of_step"] = gg["square"]["ms"] / steps_w / ms_x
+            extras[wl] = ex
+            c2.close()
+            del Xw, Rw, wc
+            torch.cuda.empty_cache()
+        out["extras"] = extras
     print(json.dumps(out))
     dist_util.finalize(dist)
 
