@@ -99,7 +99,11 @@ typedef struct {
                            twice the MMA work); 0 = automatic: 2 when d <= 512
                            (with few channels the rounding error of R is
                            systematic over tokens and one term can miss the
-                           1e-3 loss tolerance), else 1                         */
+                           1e-3 loss tolerance), else 1.  The single-pass
+                           d == 128 kernel of kt_loss_grad / kt_fit uses one
+                           term in the automatic mode too and corrects the loss
+                           to first order, L(R) = L(bf16 R) + <dR, R - bf16 R>,
+                           from the gradient the same pass yields                */
   int32_t small_d_fused;/* [1]   d == 128: kt_loss_grad / kt_fit use the single-pass
                            kernel (X read once per evaluation); 0 = the general
                            three-GEMM path                                      */

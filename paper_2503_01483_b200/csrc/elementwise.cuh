@@ -33,6 +33,8 @@ struct Scalars {
   float wop;                // size of W as an operator used by the current step's choices
   unsigned int need_op;     // 1 = the Frobenius norm alone would cost this step extra work: estimate ||W||_2
   double wnorm2;            // ||W||_F^2 of the current step
+  unsigned int finish_count;  // blocks of k_fused_finish that are done (back to 0 when the kernel ends)
+  unsigned int pad_;
 };
 
 constexpr float kDegenerateRel = 1e-6f;

@@ -24,6 +24,10 @@ namespace kt {
 constexpr int kFsD = 128;          // channels = rows of a token tile
 constexpr int kFsThreads = 320;    // warp 0: TMA, warp 1: MMA, warps 2..5 and 6..9: two epilogue groups
 constexpr int kFsXStages = 4;
+#ifndef KT_FS_PREFETCH
+#define KT_FS_PREFETCH 8
+#endif
+constexpr int kFsPrefetch = KT_FS_PREFETCH;  // X tiles requested into L2 ahead of their shared-memory load
 constexpr int kFsHalf = 128 * 64 * 2;      // bytes of one 128-row x 64-element swizzled block
 constexpr int kFsTile = 2 * kFsHalf;       // one 128 x 128 bf16 tile
 // TERMS = 1: R^T hi only, which leaves room for a second G tile; TERMS = 2: R^T hi + lo and one G tile.
@@ -147,7 +151,19 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
       }
       bool ok = true;
       uint32_t issued = 0, last_parity = 0;
+      // X tiles are asked into L2 kFsPrefetch tiles before their shared-memory stage is free: the stage's own load
+      // then costs an L2 round trip instead of one to memory, and the stage is held for that much less time
+      for (int n = 0; n < kFsPrefetch && n < my_tiles; ++n) {
+        const int row0 = (static_cast<int>(blockIdx.x) + n * static_cast<int>(gridDim.x)) * 128;
+        tma_prefetch_2d(&p.tmX, 0, row0);
+        tma_prefetch_2d(&p.tmX, 64, row0);
+      }
       for (int n = 0; n < my_tiles; ++n) {
+        if (n + kFsPrefetch < my_tiles) {
+          const int rowp = (static_cast<int>(blockIdx.x) + (n + kFsPrefetch) * static_cast<int>(gridDim.x)) * 128;
+          tma_prefetch_2d(&p.tmX, 0, rowp);
+          tma_prefetch_2d(&p.tmX, 64, rowp);
+        }
         const int s = n % kFsXStages;
         const uint32_t ph = (n / kFsXStages) & 1;
         if (!mbar_wait_bounded(x_empty(s), ph ^ 1u, abort_flag, 11u, p.wait_limit_ns)) {
@@ -307,6 +323,11 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
             const float2 c0 = __ffma2_rn(make_float2(__uint_as_float(v[c][j]), __uint_as_float(v[c][j + 1])), pw2, nm);
             const float2 c1 =
                 __ffma2_rn(make_float2(__uint_as_float(v[c][j + 2]), __uint_as_float(v[c][j + 3])), pw2, nm);
+            // the centred, scaled row replaces the raw one in the registers: the gradient pass starts from it
+            v[c][j] = __float_as_uint(c0.x);
+            v[c][j + 1] = __float_as_uint(c0.y);
+            v[c][j + 2] = __float_as_uint(c1.x);
+            v[c][j + 3] = __float_as_uint(c1.y);
             const float2 q0 = __fmul2_rn(c0, c0), q1 = __fmul2_rn(c1, c1);
             b2 = __fadd2_rn(b2, q0);
             e2 = __fadd2_rn(e2, q1);
@@ -341,8 +362,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
       } else if (row < p.N) {
         ++deg_acc;
       }
-      const float2 pwg = make_float2(pw, pw), nmean2 = make_float2(nmp, nmp), ca2 = make_float2(ca, ca),
-                   ncab2 = make_float2(-cab, -cab), ncam32 = make_float2(-cam3, -cam3);
+      const float2 ca2 = make_float2(ca, ca), ncab2 = make_float2(-cab, -cab), ncam32 = make_float2(-cam3, -cam3);
 
       // G = a c^3 - ab c - am3 as bf16, token-major, into the swizzled tile MMA2 reads
       // with one G tile it is free once MMA2 of the previous tile (the other group's) has read it; with two,
@@ -361,8 +381,8 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
           uint32_t pk[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            const float2 cc = __ffma2_rn(make_float2(__uint_as_float(v[c][j8 * 8 + 2 * e]),
-                                                     __uint_as_float(v[c][j8 * 8 + 2 * e + 1])), pwg, nmean2);
+            const float2 cc = make_float2(__uint_as_float(v[c][j8 * 8 + 2 * e]),
+                                          __uint_as_float(v[c][j8 * 8 + 2 * e + 1]));
             const float2 g = __ffma2_rn(cc, __ffma2_rn(__fmul2_rn(ca2, cc), cc, ncab2), ncam32);
             __nv_bfloat162 h = __floats2bfloat162_rn(g.x, g.y);
             pk[e] = *reinterpret_cast<uint32_t*>(&h);

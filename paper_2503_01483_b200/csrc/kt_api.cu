@@ -642,8 +642,10 @@ static bool use_fused(const kt_ctx* ctx, int d) {
   return d == kFsD && ctx->cfg.small_d_fused != 0 && ctx->cfg.loss_mode == 0;
 }
 
-static kt_status fused_loss_grad_async(kt_ctx* ctx, const XView& xv, int N, const WsLayout& L, const float* R,
-                                       float* dR, double* hist_slot, bool rt_current) {
+// The single-pass kernel alone: leaves per-CTA partials of dR, of the loss and of the skipped-row count in the
+// workspace, described by *fp (to be summed by k_fused_finish or by the first phase of small_orth_kernel).
+static kt_status fused_launch(kt_ctx* ctx, const XView& xv, int N, const WsLayout& L, const float* R,
+                              double* hist_slot, bool rt_current, FusedPartials* fp) {
   const int d = kFsD;
   if (!rt_current) KT_TRY(cast_rt(ctx, R, d, N, L));
   {
@@ -660,7 +662,11 @@ static kt_status fused_loss_grad_async(kt_ctx* ctx, const XView& xv, int N, cons
   }
   FusedParams p;
   memset(&p, 0, sizeof(p));
-  const int terms = forward_terms(ctx, d, N);
+  // R enters the single-pass kernel as one bf16 term unless two are asked for explicitly: the loss, whose error
+  // under a rounded R is systematic at this size (see forward_terms()), is corrected to first order from the
+  // gradient the same pass yields (first_order_term), which costs nothing next to a second term's MMAs
+  const int terms = ctx->cfg.forward_terms == 2 ? 2 : 1;
+  const bool correct_loss = ctx->cfg.forward_terms == 0;
   p.N = N;
   p.n_mean = mean_rows(ctx, N);
   p.tiles = (N + 127) / 128;
@@ -686,15 +692,26 @@ static kt_status fused_loss_grad_async(kt_ctx* ctx, const XView& xv, int N, cons
     KT_CUDA(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used + 1], ctx->stream));
     ctx->prof_cat[ctx->prof_used++] = static_cast<unsigned char>(kCatFused);
   }
-  const long long n = static_cast<long long>(d) * d;
-  k_sum_splits<<<static_cast<unsigned>((n / 4 + 255) / 256), 256, 0, ctx->stream>>>(p.dr_partial, grid, n, n, dR,
-                                                                                     nullptr);
-  KT_LAUNCH_CHECK();
-  k_final_sum<<<1, 256, 0, ctx->stream>>>(p.loss_partial, grid, 1.0 / p.n_mean, &ctx->d_blk->sc.loss, hist_slot,
-                                          p.deg_partial, &ctx->d_blk->sc.deg_rows);
+  fp->dr_part = p.dr_partial;
+  fp->parts = grid;
+  fp->loss_part = p.loss_partial;
+  fp->deg_part = p.deg_partial;
+  fp->loss_scale = 1.0 / p.n_mean;
+  fp->correct = correct_loss ? 1 : 0;
+  fp->rowdot = at<double>(ctx, L.norm_blocks);
+  fp->hist_slot = hist_slot;
+  return KT_OK;
+}
+
+// d = 128: loss and gradient in one pass over X, then the fixed-order sums over the CTAs' partials.
+static kt_status fused_loss_grad_async(kt_ctx* ctx, const XView& xv, int N, const WsLayout& L, const float* R,
+                                       float* dR, double* hist_slot, bool rt_current) {
+  FusedPartials fp;
+  KT_TRY(fused_launch(ctx, xv, N, L, R, hist_slot, rt_current, &fp));
+  k_fused_finish<<<kFsD, 128, 0, ctx->stream>>>(fp, R, dR, &ctx->d_blk->sc);
   KT_LAUNCH_CHECK();
   if (hist_slot != nullptr) KT_TRY(reduce_shards(ctx, hist_slot, 1, KT_F64));
-  KT_TRY(reduce_shards(ctx, dR, n, KT_F32));
+  KT_TRY(reduce_shards(ctx, dR, static_cast<int64_t>(kFsD) * kFsD, KT_F32));
   return KT_OK;
 }
 
@@ -755,8 +772,11 @@ static kt_status guard(kt_ctx* ctx, const float* R_in, float* R, int d, const Ws
 // d <= 512: the whole step and its guard in one cooperative launch (float32 on the CUDA cores).
 static bool use_small_orth(const kt_ctx* ctx, int d) { return d <= 512 && ctx->cfg.small_d_orth != 0; }
 
+// run_guard: 1 = measure R^T R - I in this step, 0 = do not, 2 = when the device's drift bound asks for it (and
+// then polish already at a quarter of the threshold, as the general path does inside kt_fit).
+// parts != null (d == 128): dR is summed inside the launch from the single-pass kernel's partials.
 static kt_status small_orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, float lr, const WsLayout& L,
-                                       bool run_guard) {
+                                       int run_guard, bool adaptive, const FusedPartials* parts = nullptr) {
   const kt_config& c = ctx->cfg;
   SmallOrthParams p;
   memset(&p, 0, sizeof(p));
@@ -766,11 +786,16 @@ static kt_status small_orth_step_async(kt_ctx* ctx, float* R, const float* dR, i
   p.dR = dR;
   p.d = d;
   p.iters = c.cayley_iters < 0 ? 0 : c.cayley_iters;
-  p.run_guard = run_guard ? 1 : 0;
+  p.run_guard = run_guard;
   p.lr = lr;
   p.q = c.q;
   p.eps = c.eps;
   p.thresh = c.polish_thresh;
+  p.polish_at = (adaptive && c.polish_thresh > 0.f) ? 0.25f * c.polish_thresh : c.polish_thresh;
+  if (parts != nullptr) {
+    p.use_parts = 1;
+    p.fp = *parts;
+  }
   p.Rt = sm;
   p.A = sm + dd;
   p.W = sm + 2 * dd;
@@ -812,7 +837,8 @@ static kt_status small_orth_step_async(kt_ctx* ctx, float* R, const float* dR, i
 static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, float lr, const WsLayout& L,
                                  int guard_mode, bool forms_current, bool adaptive = false, float* adam_m = nullptr,
                                  bool dr_hi_ready = false) {
-  if (!adam_m && use_small_orth(ctx, d)) return small_orth_step_async(ctx, R, dR, d, lr, L, guard_mode != 2);
+  if (!adam_m && use_small_orth(ctx, d))
+    return small_orth_step_async(ctx, R, dR, d, lr, L, guard_mode == 1 ? 1 : (guard_mode == 2 ? 0 : 2), adaptive);
   const kt_config& c = ctx->cfg;
   Scalars* sc = &ctx->d_blk->sc;
   const uint64_t ld = static_cast<uint64_t>(d);
@@ -1028,7 +1054,12 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
       }
     }
     // from the second step on, the previous step left the bf16 forms of R in the workspace
-    if (fused)
+    // d = 128 with the one-launch orthogonal step: that launch also sums the single-pass kernel's partials
+    const bool fold = fused && !adam && use_small_orth(ctx, d) && ctx->reduce_fn == nullptr;
+    FusedPartials parts;
+    if (fold)
+      KT_TRY(fused_launch(ctx, xv, N, L, R, &ctx->d_blk->hist[slot], k > 0, &parts));
+    else if (fused)
       KT_TRY(fused_loss_grad_async(ctx, xv, N, L, R, dR, &ctx->d_blk->hist[slot], k > 0));
     else
       KT_TRY(loss_grad_async(ctx, xv, N, d, L, R, dR, &ctx->d_blk->hist[slot], k > 0, dr_hi));
@@ -1039,8 +1070,12 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
       guard_mode = (((k + 1) % ge == 0) || (k + 1 == steps)) ? 1 : 2;
     else
       guard_mode = (k == 0 || k + 1 == steps) ? 1 : 0;
-    KT_TRY(orth_step_async(ctx, R, dR, d, lr, L, guard_mode, k > 0, ctx->cfg.guard_every < 1, adam_m,
-                           dr_hi != nullptr));
+    if (fold)
+      KT_TRY(small_orth_step_async(ctx, R, dR, d, lr, L, guard_mode == 1 ? 1 : (guard_mode == 2 ? 0 : 2),
+                                   ctx->cfg.guard_every < 1, &parts));
+    else
+      KT_TRY(orth_step_async(ctx, R, dR, d, lr, L, guard_mode, k > 0, ctx->cfg.guard_every < 1, adam_m,
+                             dr_hi != nullptr));
     done = k + 1;
   }
   if (steps > 0) {

@@ -20,14 +20,108 @@ namespace cg = cooperative_groups;
 
 constexpr int kSoGrid = 128;      // CTAs; each owns d / 128 consecutive rows
 constexpr int kSoMaxRows = 4;     // d <= 512
+constexpr int kSoD128 = 128 * 128;
+
+// What the single-pass d = 128 loss+gradient kernel leaves behind: one partial dR, loss and count of skipped rows
+// per CTA.  Summing them (fixed order) is done either by k_fused_finish or, inside kt_fit, by the first phase of
+// small_orth_kernel, which has exactly one thread per entry of dR; both use the functions below, so both give the
+// same bits.
+struct FusedPartials {
+  const float* dr_part;           // [parts][128 * 128]
+  int parts;                      // <= 256
+  const double* loss_part;        // [parts]
+  const unsigned int* deg_part;   // [parts]
+  double loss_scale;              // 1 / (tokens the loss is a mean over)
+  int correct;                    // 1: add the first-order term <dR, R - bf16(R)> to the loss
+  double* rowdot;                 // [128] scratch: that term, row by row
+  double* hist_slot;              // receives the loss too when not null
+};
+
+// Entry idx of dR: the partials in ascending order.
+__device__ __forceinline__ float sum_dr_parts(const FusedPartials& f, int idx) {
+  float acc = __ldcg(f.dr_part + idx);
+#pragma unroll 8
+  for (int s = 1; s < f.parts; ++s) acc += __ldcg(f.dr_part + static_cast<long long>(s) * kSoD128 + idx);
+  return acc;
+}
+
+// First-order correction of a loss that was evaluated at bf16(R) instead of R:
+//   L(R) = L(bf16 R) + <dL/dR, R - bf16 R> + O(|R - bf16 R|^2),
+// dR being the gradient at bf16(R) from the same pass.  The remainder R - bf16(R) is exact in float32 and about
+// 2^-9 of R, so what is neglected is about 2^-18 of the loss's variation over R.  This is one entry's term.
+__device__ __forceinline__ double first_order_term(float dr, float r) {
+  return static_cast<double>(dr) * static_cast<double>(r - __bfloat162float(__float2bfloat16_rn(r)));
+}
+
+// Sum over a block of 128 threads in a fixed order (shuffle tree, then the four warps in order); valid in thread 0.
+__device__ __forceinline__ double row_sum_128(double v, double* sh4) {
+  v = warp_sum(v);
+  if ((threadIdx.x & 31) == 0) sh4[threadIdx.x >> 5] = v;
+  __syncthreads();
+  double r = 0.0;
+  if (threadIdx.x == 0) r = ((sh4[0] + sh4[1]) + sh4[2]) + sh4[3];
+  __syncthreads();
+  return r;
+}
+
+// One block of 128 threads, after every row's term is in f.rowdot: the loss of the pass and the count of skipped
+// rows into the scalar block (values staged through shared memory, then added by one thread in index order).
+__device__ __forceinline__ void finish_fused_loss(const FusedPartials& f, Scalars* sc, double* shl /*256*/,
+                                                  double* shr /*128*/, unsigned int* shd /*256*/) {
+  for (int i = threadIdx.x; i < 256; i += 128) {
+    shl[i] = i < f.parts ? __ldcg(f.loss_part + i) : 0.0;
+    shd[i] = i < f.parts ? __ldcg(f.deg_part + i) : 0u;
+  }
+  shr[threadIdx.x] = f.correct ? __ldcg(f.rowdot + threadIdx.x) : 0.0;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double s = 0.0, corr = 0.0;
+    unsigned int dg = 0;
+    for (int i = 0; i < f.parts; ++i) {
+      s += shl[i];
+      dg += shd[i];
+    }
+    for (int i = 0; i < 128; ++i) corr += shr[i];
+    const double loss = s * f.loss_scale + corr;
+    sc->loss = loss;
+    sc->deg_rows = dg;
+    if (f.hist_slot) *f.hist_slot = loss;
+  }
+  __syncthreads();
+}
+
+// dR, the loss and the skipped-row count from the partials of the single-pass kernel.  grid 128, block 128: one
+// thread per entry of dR, one block per row; the block that finishes last adds up the loss.
+__global__ void __launch_bounds__(128) k_fused_finish(const FusedPartials f, const float* __restrict__ R,
+                                                      float* __restrict__ dR, Scalars* sc) {
+  __shared__ double sh4[4];
+  __shared__ double shl[256], shr[128];
+  __shared__ unsigned int shd[256];
+  __shared__ unsigned int is_last;
+  const int idx = blockIdx.x * 128 + threadIdx.x;
+  const float acc = sum_dr_parts(f, idx);
+  dR[idx] = acc;
+  const double row = row_sum_128(f.correct ? first_order_term(acc, R[idx]) : 0.0, sh4);
+  if (threadIdx.x == 0) {
+    f.rowdot[blockIdx.x] = row;
+    __threadfence();
+    is_last = (atomicAdd(&sc->finish_count, 1u) == gridDim.x - 1u) ? 1u : 0u;
+  }
+  __syncthreads();
+  if (is_last == 0u) return;
+  __threadfence();
+  finish_fused_loss(f, sc, shl, shr, shd);
+  if (threadIdx.x == 0) sc->finish_count = 0u;  // ready for the next call
+}
 
 struct SmallOrthParams {
   float* R;            // d x d, in/out
   const float* dR;     // d x d
   int d;
   int iters;           // s: series terms 0..s
-  int run_guard;
+  int run_guard;       // 1: measure R^T R - I, 0: do not, 2: when the device's drift bound reaches thresh / 2
   float lr, q, eps, thresh;
+  float polish_at;     // the polish runs when the measured error exceeds this (<= thresh)
   // scratch, all d x d float32 unless noted
   float* Rt;           // R^T (then R_new^T)
   float* A;            // dR R^T, later E
@@ -40,6 +134,9 @@ struct SmallOrthParams {
   __nv_bfloat16* r_hi; // bf16 forms of the new R for the next loss evaluation
   __nv_bfloat16* rt_hi;
   __nv_bfloat16* rt_lo;
+  // d == 128 inside kt_fit: dR is not read from p.dR but summed here from the single-pass kernel's partials
+  int use_parts;
+  FusedPartials fp;
 };
 
 // out[r] = sum_k arow[r][k] * B[k][j] for this thread's column j and the CTA's ROWS rows.
@@ -82,11 +179,31 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
     rcur[r] = p.R[static_cast<long long>(i0 + r) * d + j];
     p.Rt[static_cast<long long>(j) * d + i0 + r] = rcur[r];
   }
+  const float drift_in = p.sc->drift;  // (written only by the end of an earlier launch)
+  float dr_own = 0.f;
+  if (ROWS == 1 && p.use_parts) {
+    // this CTA's row of dR from the single-pass kernel's partials, and its term of the loss correction
+    __shared__ double sh4[4];
+    dr_own = sum_dr_parts(p.fp, i0 * d + j);
+    const double row = row_sum_128(p.fp.correct ? first_order_term(dr_own, rcur[0]) : 0.0, sh4);
+    if (threadIdx.x == 0) p.fp.rowdot[blockIdx.x] = row;
+  }
   grid.sync();
+  if (ROWS == 1 && p.use_parts && blockIdx.x == 0) {
+    __shared__ double shl[256], shr[128];
+    __shared__ unsigned int shdg[256];
+    finish_fused_loss(p.fp, p.sc, shl, shr, shdg);
+  }
 
   // A = dR R^T:  A[i][j] = sum_k dR[i][k] Rt[k][j]
   float acc[ROWS];
-  load_rows(p.dR);
+  if (ROWS == 1 && p.use_parts) {
+    __syncthreads();
+    arow[0][j] = dr_own;
+    __syncthreads();
+  } else {
+    load_rows(p.dR);
+  }
   rows_times_matrix<ROWS>(arow, p.Rt, d, j, acc);
 #pragma unroll
   for (int r = 0; r < ROWS; ++r) p.A[static_cast<long long>(i0 + r) * d + j] = acc[r];
@@ -112,20 +229,31 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
   }
   grid.sync();
   float alpha;
+  bool do_guard;   // the same in every CTA
+  float drift;     // bound on the orthogonality error accumulated since the last measurement
   {
     double s = 0.0;
-    for (int c = 0; c < kSoGrid; ++c) s += p.norm_part[c];
+    for (int c = 0; c < kSoGrid; ++c) s += __ldcg(p.norm_part + c);
     const double nrm = sqrt(s);
     const double cap = 2.0 * static_cast<double>(p.q) / (nrm + static_cast<double>(p.eps));
     const double a = (static_cast<double>(p.lr) < cap) ? static_cast<double>(p.lr) : cap;
     alpha = static_cast<float>(a);
+    // run_guard 1: measure R^T R - I in this step; 0: do not; 2: only when the drift bound asks for it.  Every
+    // product here is float32, so a step adds the truncation of the series, 2 x (x/2)^(s+1) with x = alpha ||W||_F
+    // (the remainder of the Neumann series, twice through E = R^T dR + dR^T R), and float32 rounding of the update.
+    const double x = a * nrm;
+    double trunc = 2.0 * x;
+    for (int k = 0; k <= p.iters; ++k) trunc *= 0.5 * x;
+    drift = drift_in + static_cast<float>(trunc + (p.iters + 2) * ldexp(1.0, -23));
+    do_guard = p.run_guard == 1 || (p.run_guard == 2 && (p.thresh <= 0.f || drift >= 0.5f * p.thresh));
     if (blockIdx.x == 0 && threadIdx.x == 0) {
       p.sc->alpha = alpha;
       p.sc->wnorm = static_cast<float>(nrm);
       p.sc->wop = static_cast<float>(nrm);  // this path evaluates every term in float32 and decides nothing
       p.sc->n_terms = static_cast<unsigned int>(p.iters + 1);
       p.sc->p0_terms = 0u;
-      if (p.run_guard) p.sc->guards += 1u;
+      if (do_guard) p.sc->guards += 1u;
+      else p.sc->drift = drift;
     }
   }
 
@@ -158,7 +286,7 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
   }
 
   float max_e = 0.f;
-  if (p.run_guard) {
+  if (do_guard) {
     grid.sync();
     // E = R^T R - I:  E[i][j] = sum_k Rt[i][k] R[k][j]
     load_rows(p.Rt);
@@ -180,8 +308,8 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
       p.max_part[blockIdx.x] = mx;
     }
     grid.sync();
-    for (int c = 0; c < kSoGrid; ++c) max_e = fmaxf(max_e, p.max_part[c]);
-    if (max_e > p.thresh) {  // same value in every CTA: the branch is grid-uniform
+    for (int c = 0; c < kSoGrid; ++c) max_e = fmaxf(max_e, __ldcg(p.max_part + c));
+    if (max_e > p.polish_at) {  // same value in every CTA: the branch is grid-uniform
       // R <- R - R E / 2; each CTA reads only its own rows of R and all of E
       load_rows(p.R);
       rows_times_matrix<ROWS>(arow, p.A, d, j, acc);
@@ -193,7 +321,8 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) {
       p.sc->max_e_bits = __float_as_uint(max_e);
-      p.sc->gate = (max_e > p.thresh) ? 1u : 0u;
+      p.sc->gate = (max_e > p.polish_at) ? 1u : 0u;
+      p.sc->drift = (max_e > p.polish_at) ? 0.f : max_e;  // the bound restarts from what was just measured
     }
   }
 

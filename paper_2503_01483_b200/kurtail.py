@@ -13,7 +13,8 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libkurtail.so")
+# KURTAIL_LIB names another build of the same library (e.g. one compiled with other nvcc flags) to load instead
+LIB_PATH = os.environ.get("KURTAIL_LIB") or os.path.join(_HERE, "libkurtail.so")
 
 KT_BF16, KT_F32, KT_F64 = 0, 1, 2
 STATUS = {0: "KT_OK", 1: "KT_ERR_INVALID_ARG", 2: "KT_ERR_SHAPE", 3: "KT_ERR_ALIGN", 4: "KT_ERR_WORKSPACE",

@@ -245,9 +245,17 @@ def test_single_pass_kernel_d128(ctx, N):
     # the general three-GEMM path computes the same thing
     gen = kurtail.Context(DEV, small_d_fused=0)
     loss_g, dR_g = gen.loss_grad(X, R)
-    assert abs(loss - loss_g) <= 1e-6 * abs(loss_g)
-    assert np.linalg.norm(f64(dR) - f64(dR_g)) / np.linalg.norm(f64(dR_g)) <= 5e-3
+    # (the general path uses R as two bf16 terms; the single-pass kernel uses one and corrects the loss to first
+    # order with its own gradient: what is left is second order in the rounding of R)
+    assert abs(loss - loss_g) <= 1e-4 * abs(loss_g)
+    assert np.linalg.norm(f64(dR) - f64(dR_g)) / np.linalg.norm(f64(dR_g)) <= 8e-3
     gen.close()
+    # two bf16 terms of R in the single-pass kernel itself (no correction): the general path's loss to float32 noise
+    two = kurtail.Context(DEV, forward_terms=2)
+    loss_2, dR_2 = two.loss_grad(X, R)
+    assert abs(loss_2 - loss_g) <= 1e-6 * abs(loss_g)
+    assert np.linalg.norm(f64(dR_2) - dR_ref) / np.linalg.norm(dR_ref) <= 1e-2
+    two.close()
     # fixed-order reductions: a second evaluation is bit-identical
     loss2, dR2 = ctx.loss_grad(X, R)
     assert loss2 == loss and torch.equal(dR2, dR)
