@@ -445,11 +445,13 @@ __device__ __forceinline__ void load8(const float* p, float (&v)[8]) {
 // Row t is X[t] (bases == null), or, for a rotation shared by several buffers, row t of the minibatch `ids`
 // gathered from the buffers (see k_gather_samples for the numbering).  xb != null: the row is also copied, as it
 // is but rounded to bf16, to row t of the dense matrix xb (the gathered minibatch; the bf16 form of a float32 X).
+// mean_square != 0: rowscale[t] receives mean_j x_t[j]^2 itself instead of the factor (the single-pass d = 128
+// kernel's measure of a row's size).
 // One block of 256 threads per row; T = float or bf16; d a multiple of 8.
 template <typename T>
 __global__ void k_row_scale(const T* X, long long ld, int d, float eps, float* __restrict__ rowscale,
                             __nv_bfloat16* xb, const void* const* bases, int samples_per_buf, int rps,
-                            const int* ids) {
+                            const int* ids, int mean_square = 0) {
   __shared__ double sh[8];
   const T* x;
   if (bases != nullptr) {
@@ -478,7 +480,8 @@ __global__ void k_row_scale(const T* X, long long ld, int d, float eps, float* _
   const double acc = block_sum_256(static_cast<double>(part), sh, threadIdx.x);
   if (threadIdx.x == 0) {
     const double ms = acc / d + static_cast<double>(eps);
-    rowscale[blockIdx.x] = ms > 0.0 ? static_cast<float>(1.0 / sqrt(ms)) : 0.f;
+    if (mean_square) rowscale[blockIdx.x] = static_cast<float>(acc / d);
+    else rowscale[blockIdx.x] = ms > 0.0 ? static_cast<float>(1.0 / sqrt(ms)) : 0.f;
   }
 }
 

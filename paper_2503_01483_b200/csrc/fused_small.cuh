@@ -5,17 +5,29 @@
 // tokens through the complete chain without leaving the SM:
 //
 //   TMA:  X tile (128 tokens x 128 channels, bf16)                     -> shared memory
-//   MMA1: Y = X R (R^T resident in shared memory, hi [+ lo])           -> tensor memory
-//   epilogue (two groups of 4 warps that take alternate tiles, one row per thread): mean, m2, m3, m4
-//             (Eq. 3), kappa, loss term, then
-//             G = a c^3 - ab c - am3 as bf16                           -> shared memory
-//   MMA2: dR += X^T G  (both operands read token-major straight from the tiles above,
+//   MMA1: C = X Rc (Rc = R with each row's mean taken off, so that C is Y = X R minus its row means;
+//             Rc^T resident in shared memory, hi [+ lo])               -> tensor memory
+//   epilogue (two groups of 4 warps that take alternate tiles, one row per thread): m2, m4 (Eq. 3),
+//             kappa, loss term, then
+//             G = a c^3 - ab c as bf16 (the gradient with respect to C) -> shared memory
+//   MMA2: dRc += X^T G (both operands read token-major straight from the tiles above,
 //             "MN-major" shared-memory descriptors)                    -> one persistent accumulator
 //
 // X is read from HBM exactly once per evaluation; Y and G never leave the SM.  Each CTA ends by
 // writing its partial dR (128 x 128 float32) and partial loss; a fixed-order sum over CTAs follows.
+//
+// Operand encoding.  The kernel does not read the caller's bf16 X but a copy made once per X (k_encode_rows_128):
+// every row multiplied by the power of two that brings its largest entry into [1, 2), as float16.  A bf16 value
+// has 8 significant bits and float16 holds 11, so the copy is exact (entries more than 2^14 below the row's
+// largest one lose bits: less than 2^-25 of the row's size).  Neither the kurtosis of a row nor dL/dR depends on
+// the row's scale, so nothing else changes -- except that R can now enter as float16 too, with 2^-12 instead of
+// 2^-9 relative rounding at the same tensor-core cost (the systematic error this size is sensitive to, see
+// kt_config.forward_terms), that the power sums can never leave float32's range whatever the scale of X, and that
+// G fits float16.  The row's mean square (of the encoded row) comes with the copy.
 #pragma once
 #include <cuda.h>
+
+#include <cuda_fp16.h>
 
 #include "sm100_prims.cuh"
 
@@ -38,9 +50,9 @@ struct FusedCfg {
 };
 
 struct FusedParams {
-  CUtensorMap tmX;    // X  [N][128] bf16, box 128 rows x 64
-  CUtensorMap tmRhi;  // R^T hi [128][128] bf16, box 128 x 64
-  CUtensorMap tmRlo;  // R^T lo
+  CUtensorMap tmX;    // encoded X [N][128] float16, box 128 rows x 64
+  CUtensorMap tmRhi;  // Rc^T as float16 [128][128], box 128 x 64
+  CUtensorMap tmRlo;  // its rounding remainder as float16 (TERMS == 2)
   int N;
   double n_mean;      // tokens the loss is a mean over (N, or all shards' rows in a sharded fit)
   int tiles;          // ceil(N / 128)
@@ -50,6 +62,7 @@ struct FusedParams {
   unsigned int* deg_partial;// [gridDim.x]
   unsigned int* err_word;
   unsigned long long wait_limit_ns;  // bound of every device-side wait of this launch
+  const float* row_ms;      // [N] mean square of every encoded row of X (for the rule that skips rows without spread)
 };
 
 // Shared-memory descriptor for an "MN-major" bf16 operand stored as rows of 64 elements (128 bytes,
@@ -70,8 +83,9 @@ __device__ __forceinline__ uint64_t umma_desc_mnmajor_sw128(uint32_t smem_addr, 
 template <int TERMS>
 __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid_constant__ FusedParams p) {
   constexpr int kGBufs = FusedCfg<TERMS>::kGBufs;
-  constexpr uint32_t kIdescK = umma_idesc_bf16_f32(128, 128);                            // both K-major
-  constexpr uint32_t kIdescMN = umma_idesc_bf16_f32(128, 128) | (1u << 15) | (1u << 16);  // both MN-major
+  // every operand of this kernel is float16 (see the note on the encoding of X at the top of this file)
+  constexpr uint32_t kIdescK = umma_idesc_f16_f32(128, 128);                            // both K-major
+  constexpr uint32_t kIdescMN = umma_idesc_f16_f32(128, 128) | (1u << 15) | (1u << 16);  // both MN-major
   // tensor memory: Y accumulators at columns 0 (even tiles) and 128 (odd tiles), dR accumulator at 256
   constexpr uint32_t kTmemCols = 512;
   constexpr uint32_t kColDr = 256;
@@ -253,12 +267,14 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
     const int grp = (warp - 2) >> 2;    // = tile parity = Y accumulator = G buffer
     const int trow = lg * 32 + lane;    // token within the tile (and row of dR at the end)
     const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(lg * 32) << 16);
-    const float kscale = static_cast<float>(4.0 / (p.n_mean * 128.0));
     double loss_acc = 0.0;
     unsigned int deg_acc = 0;
     bool ok = true;
     for (int n = grp; n < my_tiles && ok; n += 2) {
       const uint32_t par = (n >> 1) & 1;
+      // (asked for before the wait for the accumulator, so that the load's latency is not on the tile's path)
+      const int row = (static_cast<int>(blockIdx.x) + n * static_cast<int>(gridDim.x)) * 128 + trow;
+      const float msx = (row < p.N) ? __ldg(p.row_ms + row) : 0.f;
       const bool got = mbar_wait_bounded(y_full(grp), par, abort_flag, 16u, p.wait_limit_ns);
       if (!__all_sync(0xffffffffu, got)) {
         ok = false;
@@ -275,96 +291,58 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(y_empty(grp));
-      const int row = (static_cast<int>(blockIdx.x) + n * static_cast<int>(gridDim.x)) * 128 + trow;
 
-      // Eq. 3 on the row: mean, then central power sums about it.  Two-wide arithmetic (packed f32x2
-      // add/mul/fma): this epilogue is bound by instruction issue and latency, not by memory.
-      // The kurtosis does not depend on the scale of the row, and neither must its evaluation: the first pass also
-      // takes the row's mean square, and everything after it works on the row times pw, the power of two nearest to
-      // 1/rms, so that no power sum leaves float32's range whatever the scale of X.
-      float mean, pw;
-      {
-        float2 a0 = make_float2(0.f, 0.f), a1 = a0, a2 = a0, a3 = a0, q0 = a0, q1 = a0, q2 = a0, q3 = a0;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-#pragma unroll
-          for (int j = 0; j < 32; j += 8) {
-            const float2 x0 = make_float2(__uint_as_float(v[c][j]), __uint_as_float(v[c][j + 1]));
-            const float2 x1 = make_float2(__uint_as_float(v[c][j + 2]), __uint_as_float(v[c][j + 3]));
-            const float2 x2 = make_float2(__uint_as_float(v[c][j + 4]), __uint_as_float(v[c][j + 5]));
-            const float2 x3 = make_float2(__uint_as_float(v[c][j + 6]), __uint_as_float(v[c][j + 7]));
-            a0 = __fadd2_rn(a0, x0);
-            a1 = __fadd2_rn(a1, x1);
-            a2 = __fadd2_rn(a2, x2);
-            a3 = __fadd2_rn(a3, x3);
-            q0 = __ffma2_rn(x0, x0, q0);
-            q1 = __ffma2_rn(x1, x1, q1);
-            q2 = __ffma2_rn(x2, x2, q2);
-            q3 = __ffma2_rn(x3, x3, q3);
-          }
-        }
-        a0 = __fadd2_rn(__fadd2_rn(a0, a1), __fadd2_rn(a2, a3));
-        q0 = __fadd2_rn(__fadd2_rn(q0, q1), __fadd2_rn(q2, q3));
-        mean = (a0.x + a0.y) * (1.0f / 128.0f);
-        const float msq = (q0.x + q0.y) * (1.0f / 128.0f);
-        // pw = 2^-floor(e/2), e the binary exponent of the mean square (an all-zero row gives 2^63: harmless)
-        const int e = static_cast<int>((__float_as_uint(msq) >> 23) & 0xffu) - 127;
-        pw = __uint_as_float(static_cast<uint32_t>(127 - (e >> 1)) << 23);
-      }
-      const float nmp = -mean * pw;  // the scaled row is v * pw + nmp
-      float s2, s3, s4;
-      {
-        const float2 pw2 = make_float2(pw, pw), nm = make_float2(nmp, nmp);
-        float2 b2 = make_float2(0.f, 0.f), b3 = b2, b4 = b2, e2 = b2, e3 = b2, e4 = b2;
+      // Eq. 3 on the row.  The second operand of MMA1 is Rc^T (R with every row's mean taken off), so the row that
+      // comes out of tensor memory is already the centred row c = y - mean(y): its second and fourth power sums are
+      // the central moments, and the gradient has no term through the mean.  Two-wide arithmetic (packed f32x2
+      // mul/add/fma): this epilogue is bound by the float32 pipe, three operations per entry here and three below.
+      float s2, s4;
+      auto power_sums = [&]() {
+        float2 b2 = make_float2(0.f, 0.f), e2 = b2, b4 = b2, e4 = b2;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
-            const float2 c0 = __ffma2_rn(make_float2(__uint_as_float(v[c][j]), __uint_as_float(v[c][j + 1])), pw2, nm);
-            const float2 c1 =
-                __ffma2_rn(make_float2(__uint_as_float(v[c][j + 2]), __uint_as_float(v[c][j + 3])), pw2, nm);
-            // the centred, scaled row replaces the raw one in the registers: the gradient pass starts from it
-            v[c][j] = __float_as_uint(c0.x);
-            v[c][j + 1] = __float_as_uint(c0.y);
-            v[c][j + 2] = __float_as_uint(c1.x);
-            v[c][j + 3] = __float_as_uint(c1.y);
+            const float2 c0 = make_float2(__uint_as_float(v[c][j]), __uint_as_float(v[c][j + 1]));
+            const float2 c1 = make_float2(__uint_as_float(v[c][j + 2]), __uint_as_float(v[c][j + 3]));
             const float2 q0 = __fmul2_rn(c0, c0), q1 = __fmul2_rn(c1, c1);
             b2 = __fadd2_rn(b2, q0);
             e2 = __fadd2_rn(e2, q1);
-            b3 = __ffma2_rn(q0, c0, b3);
-            e3 = __ffma2_rn(q1, c1, e3);
             b4 = __ffma2_rn(q0, q0, b4);
             e4 = __ffma2_rn(q1, q1, e4);
           }
         }
         b2 = __fadd2_rn(b2, e2);
-        b3 = __fadd2_rn(b3, e3);
         b4 = __fadd2_rn(b4, e4);
         s2 = b2.x + b2.y;
-        s3 = b3.x + b3.y;
         s4 = b4.x + b4.y;
-      }
-      // kappa, the loss term and the coefficients of dL/dY (same rules as the general path, in float32).  m2, m3, m4
-      // are moments of the scaled row (rms about 1); G for the unscaled row is pw times the scaled row's.
-      const float m2 = s2 * (1.0f / 128.0f), m3 = s3 * (1.0f / 128.0f), m4 = s4 * (1.0f / 128.0f);
-      const float ms = fmaf(nmp, nmp, m2);
-      const bool degenerate = (ms == 0.f) || (m2 <= 1e-6f * ms);
-      float ca = 0.f, cab = 0.f, cam3 = 0.f;
-      if (!degenerate) {
+      };
+      power_sums();
+      // kappa, the loss term and the coefficients of dL/dc = a c^3 - ab c (in float32), up to the constant factor
+      // 4 / (tokens * 128), which is applied once to the summed gradient instead of to every entry (that also keeps
+      // G inside float16's range: |c| <= 11.3 sigma and sigma >= 0.09 for a row whose largest entry is in [1, 2)).
+      // A row without spread is one whose variance is below 1e-6 of its mean square INCLUDING the mean, which the
+      // centred row no longer shows: that mean square is the one of the encoded row of X (an orthogonal R keeps it),
+      // handed in per row.  A NaN there (a non-finite entry of X) goes into the loss.
+      const float m2 = s2 * (1.0f / 128.0f), m4 = s4 * (1.0f / 128.0f);
+      const bool degenerate = !(msx > 0.f) || (m2 <= 1e-6f * msx);
+      float ca = 0.f, cab = 0.f;
+      if (msx != msx || s4 != s4) {
+        if (row < p.N) loss_acc += static_cast<double>(__uint_as_float(0x7fc00000u));
+      } else if (!degenerate) {
         const float r = __frcp_rn(m2);
         const float kappa = (m4 * r) * r;
         const float diff = kappa - p.kappa_t;
         const float sgn = (diff > 0.f) ? 1.0f : ((diff < 0.f) ? -1.0f : 0.0f);
-        ca = (((sgn * kscale) * pw) * r) * r;
+        ca = (sgn * r) * r;
         cab = ca * (m4 * r);
-        cam3 = ca * m3;
         if (row < p.N) loss_acc += static_cast<double>(fabsf(diff));
       } else if (row < p.N) {
         ++deg_acc;
       }
-      const float2 ca2 = make_float2(ca, ca), ncab2 = make_float2(-cab, -cab), ncam32 = make_float2(-cam3, -cam3);
+      const float2 ca2 = make_float2(ca, ca), ncab2 = make_float2(-cab, -cab);
 
-      // G = a c^3 - ab c - am3 as bf16, token-major, into the swizzled tile MMA2 reads
+      // G = a c^3 - ab c as float16, token-major, into the swizzled tile MMA2 reads
       // with one G tile it is free once MMA2 of the previous tile (the other group's) has read it; with two,
       // once MMA2 of this group's previous tile has
       const int gw = (kGBufs == 2) ? n - 2 : n - 1;
@@ -383,8 +361,8 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
           for (int e = 0; e < 4; ++e) {
             const float2 cc = make_float2(__uint_as_float(v[c][j8 * 8 + 2 * e]),
                                           __uint_as_float(v[c][j8 * 8 + 2 * e + 1]));
-            const float2 g = __ffma2_rn(cc, __ffma2_rn(__fmul2_rn(ca2, cc), cc, ncab2), ncam32);
-            __nv_bfloat162 h = __floats2bfloat162_rn(g.x, g.y);
+            const float2 g = __fmul2_rn(cc, __ffma2_rn(__fmul2_rn(ca2, cc), cc, ncab2));
+            __half2 h = __floats2half2_rn(g.x, g.y);
             pk[e] = *reinterpret_cast<uint32_t*>(&h);
           }
           const int chunk = c * 4 + j8;  // 16-byte chunk 0..15 of the 256-byte row

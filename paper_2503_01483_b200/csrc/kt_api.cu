@@ -93,7 +93,8 @@ struct WsLayout {
   size_t gather_ids;    // kt_fit_shared: [kIdsChunk][batch] int sample ids
   size_t gather_bases;  // kt_fit_shared: [kMaxSharedBufs] buffer base pointers
   size_t flat;          // flattened-kurtosis mode: the global coefficients, the global mean, 3 x [blocks] doubles
-  size_t rowscale;      // [N] float: RMSNorm factor of every row (when kt_config.rmsnorm is on)
+  size_t rowscale;      // [N] float: RMSNorm factor of every row (kt_config.rmsnorm), or, for the single-pass
+                        // d = 128 kernel, the mean square of every row of X
   size_t total;
   long long ldt;
   int P, bn, loss_blocks, norm_n;
@@ -105,7 +106,9 @@ struct WsLayout {
 static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, const kt_config* cfg,
                             int gather_batch = 0) {
   const bool adam = cfg != nullptr && cfg->optimizer == 1;
-  const bool xcopy = x_dtype == KT_F32 || gather_batch > 0;
+  // (d = 128: the single-pass kernel reads its own float16 encoding of X, whatever X's type)
+  const bool xcopy = x_dtype == KT_F32 || gather_batch > 0 ||
+                     (d == kFsD && (cfg == nullptr || (cfg->small_d_fused != 0 && cfg->loss_mode == 0)));
   // Y kept in float32 for the backward pass, unless the backward recomputes it or the single-pass kernel (d = 128,
   // per-token loss) does forward and backward together
   const bool single_pass = d == kFsD && (cfg == nullptr || (cfg->small_d_fused != 0 && cfg->loss_mode == 0));
@@ -162,7 +165,8 @@ static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, const kt_conf
   L.gather_ids = take(gather_batch > 0 ? static_cast<size_t>(kIdsChunk) * gather_batch * 4 : 0);
   L.gather_bases = take(gather_batch > 0 ? static_cast<size_t>(kMaxSharedBufs) * 8 : 0);
   L.flat = take(static_cast<size_t>(L.loss_blocks) * 8 * 3 + 64);
-  L.rowscale = take((cfg != nullptr && cfg->rmsnorm != 0) ? static_cast<size_t>(N) * 4 : 0);
+  // (d = 128: the single-pass kernel's per-row mean square of X lives here too)
+  L.rowscale = take(((cfg != nullptr && cfg->rmsnorm != 0) || d == kFsD) ? static_cast<size_t>(N) * 4 : 0);
   L.total = off;
   return L;
 }
@@ -404,7 +408,12 @@ struct XView {
   const __nv_bfloat16* xb;  // bf16 rows
   long long ldx;
   const float* row_scale;   // RMSNorm factor of every row (kt_config.rmsnorm), or null
+  const float* row_ms;      // single-pass d = 128 kernel: mean square of every row of X
 };
+
+// The single-pass d = 128 kernel's own encoding of X (row-normalised float16, see k_encode_rows_128) and each encoded
+// row's mean square: one pass over X, needed once per X.
+static kt_status fused_encode(kt_ctx* ctx, const kt_mat& X, const WsLayout& L, XView* v);
 
 // RMSNorm mode: the factor 1/sqrt(mean(x^2) + eps) of every row, applied later to the float32 accumulator rows of
 // X R (an orthogonal R keeps the norm of a row); a float32 X is rounded to its bf16 copy in the same pass.
@@ -642,12 +651,36 @@ static bool use_fused(const kt_ctx* ctx, int d) {
   return d == kFsD && ctx->cfg.small_d_fused != 0 && ctx->cfg.loss_mode == 0;
 }
 
+static kt_status fused_encode(kt_ctx* ctx, const kt_mat& X, const WsLayout& L, XView* v) {
+  const int N = static_cast<int>(X.rows);
+  float* ms = at<float>(ctx, L.rowscale);
+  __half* x16 = at<__half>(ctx, L.xb);
+  const unsigned grid = static_cast<unsigned>((N + 15) / 16);
+  if (X.dtype == KT_BF16)
+    k_encode_rows_128<__nv_bfloat16><<<grid, 256, 0, ctx->stream>>>(static_cast<const __nv_bfloat16*>(X.data), X.ld, N,
+                                                                    x16, ms, nullptr, 0, 0, nullptr);
+  else
+    k_encode_rows_128<float><<<grid, 256, 0, ctx->stream>>>(static_cast<const float*>(X.data), X.ld, N, x16, ms,
+                                                            nullptr, 0, 0, nullptr);
+  KT_LAUNCH_CHECK();
+  v->xb = reinterpret_cast<const __nv_bfloat16*>(x16);   // 16-bit words: float16 here
+  v->ldx = kFsD;
+  v->row_scale = nullptr;
+  v->row_ms = ms;
+  return KT_OK;
+}
+
 // The single-pass kernel alone: leaves per-CTA partials of dR, of the loss and of the skipped-row count in the
 // workspace, described by *fp (to be summed by k_fused_finish or by the first phase of small_orth_kernel).
 static kt_status fused_launch(kt_ctx* ctx, const XView& xv, int N, const WsLayout& L, const float* R,
                               double* hist_slot, bool rt_current, FusedPartials* fp) {
   const int d = kFsD;
-  if (!rt_current) KT_TRY(cast_rt(ctx, R, d, N, L));
+  if (!rt_current) {
+    // the kernel's second operand is Rc^T, R with every row's mean taken off (see first_order_term)
+    k_center_split_128<<<kFsD, 128, 0, ctx->stream>>>(R, at<__nv_bfloat16>(ctx, L.rt_hi),
+                                                      at<__nv_bfloat16>(ctx, L.rt_lo));
+    KT_LAUNCH_CHECK();
+  }
   {
     static bool attr_done[kMaxDevices] = {false};
     std::lock_guard<std::mutex> lock(g_setup_mutex);
@@ -676,6 +709,7 @@ static kt_status fused_launch(kt_ctx* ctx, const XView& xv, int N, const WsLayou
   p.loss_partial = at<double>(ctx, L.block_loss);
   p.deg_partial = at<unsigned int>(ctx, L.block_deg);
   p.err_word = &ctx->d_blk->sc.err_word;
+  p.row_ms = xv.row_ms;
   KT_TRY(make_tmap(ctx, &p.tmX, xv.xb, d, N, xv.ldx, 128));
   KT_TRY(make_tmap(ctx, &p.tmRhi, at<__nv_bfloat16>(ctx, L.rt_hi), d, d, d, 128));
   KT_TRY(make_tmap(ctx, &p.tmRlo, at<__nv_bfloat16>(ctx, L.rt_lo), d, d, d, 128));
@@ -697,6 +731,7 @@ static kt_status fused_launch(kt_ctx* ctx, const XView& xv, int N, const WsLayou
   fp->loss_part = p.loss_partial;
   fp->deg_part = p.deg_partial;
   fp->loss_scale = 1.0 / p.n_mean;
+  fp->dr_scale = static_cast<float>(4.0 / (p.n_mean * 128.0));
   fp->correct = correct_loss ? 1 : 0;
   fp->rowdot = at<double>(ctx, L.norm_blocks);
   fp->hist_slot = hist_slot;
@@ -993,7 +1028,11 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
   memset(&xv, 0, sizeof(xv));
   const bool fused = use_fused(ctx, d);
   if (!sh) {
-    if (fused) KT_TRY(ingest_x_forward(ctx, X, L, &xv, false)); else KT_TRY(ingest_x_full(ctx, X, L, &xv));
+    if (fused) {
+      KT_TRY(fused_encode(ctx, X, L, &xv));
+    } else {
+      KT_TRY(ingest_x_full(ctx, X, L, &xv));
+    }
   }
   float* dR = at<float>(ctx, L.dr);
   // the Cayley step's first product reads bf16(dR): when the gradient ends in a split-K sum, that sum writes it too
@@ -1031,7 +1070,17 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
       const int rps = static_cast<int>(sh->rps);
       const bool norm = ctx->cfg.rmsnorm != 0 && !fused;
       xv.row_scale = nullptr;
-      if (norm) {
+      if (fused) {
+        // gather straight into the single-pass kernel's encoding (row-normalised float16 and the rows' mean squares)
+        float* ms = at<float>(ctx, L.rowscale);
+        __half* x16 = reinterpret_cast<__half*>(xb);
+        const unsigned eg = static_cast<unsigned>((N + 15) / 16);
+        if (X.dtype == KT_BF16)
+          k_encode_rows_128<__nv_bfloat16><<<eg, 256, 0, ctx->stream>>>(nullptr, X.ld, N, x16, ms, bases, spb, rps, ids);
+        else
+          k_encode_rows_128<float><<<eg, 256, 0, ctx->stream>>>(nullptr, X.ld, N, x16, ms, bases, spb, rps, ids);
+        xv.row_ms = ms;
+      } else if (norm) {
         // gather and RMSNorm factors in one pass over the samples' rows
         float* rsc = at<float>(ctx, L.rowscale);
         if (X.dtype == KT_BF16)
@@ -1057,10 +1106,12 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
     // d = 128 with the one-launch orthogonal step: that launch also sums the single-pass kernel's partials
     const bool fold = fused && !adam && use_small_orth(ctx, d) && ctx->reduce_fn == nullptr;
     FusedPartials parts;
+    // (that launch also leaves the bf16 forms of the new Rc^T; any other step leaves those of R^T, so the
+    // single-pass kernel's operand is then made afresh)
     if (fold)
       KT_TRY(fused_launch(ctx, xv, N, L, R, &ctx->d_blk->hist[slot], k > 0, &parts));
     else if (fused)
-      KT_TRY(fused_loss_grad_async(ctx, xv, N, L, R, dR, &ctx->d_blk->hist[slot], k > 0));
+      KT_TRY(fused_loss_grad_async(ctx, xv, N, L, R, dR, &ctx->d_blk->hist[slot], false));
     else
       KT_TRY(loss_grad_async(ctx, xv, N, d, L, R, dR, &ctx->d_blk->hist[slot], k > 0, dr_hi));
     // guard: a fixed cadence when guard_every >= 1; otherwise measured on the first and the last step and in between
@@ -1074,7 +1125,8 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
       KT_TRY(small_orth_step_async(ctx, R, dR, d, lr, L, guard_mode == 1 ? 1 : (guard_mode == 2 ? 0 : 2),
                                    ctx->cfg.guard_every < 1, &parts));
     else
-      KT_TRY(orth_step_async(ctx, R, dR, d, lr, L, guard_mode, k > 0, ctx->cfg.guard_every < 1, adam_m,
+      // (the single-pass kernel has put the forms of Rc^T where the step expects those of R^T: not current then)
+      KT_TRY(orth_step_async(ctx, R, dR, d, lr, L, guard_mode, k > 0 && !fused, ctx->cfg.guard_every < 1, adam_m,
                              dr_hi != nullptr));
     done = k + 1;
   }
@@ -1305,7 +1357,7 @@ kt_status kt_loss_grad(kt_ctx* ctx, kt_mat X, const float* R, float* dR, double*
   KT_TRY(check_ws(ctx, L));
   XView xv;
   if (use_fused(ctx, static_cast<int>(d))) {
-    KT_TRY(ingest_x_forward(ctx, X, L, &xv, false));
+    KT_TRY(fused_encode(ctx, X, L, &xv));
     KT_TRY(fused_loss_grad_async(ctx, xv, static_cast<int>(N), L, R, dR, nullptr, false));
   } else {
     KT_TRY(ingest_x_full(ctx, X, L, &xv));

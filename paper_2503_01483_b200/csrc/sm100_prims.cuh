@@ -189,6 +189,11 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16_f32(int M, int N) {
          (static_cast<uint32_t>(M >> 4) << 24);
 }
 
+// The same with float16 A and B (format code 0 in both fields).
+__host__ __device__ constexpr uint32_t umma_idesc_f16_f32(int M, int N) {
+  return (1u << 4) | (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(M >> 4) << 24);
+}
+
 // Eight consecutive float32 (32 bytes, 32-byte aligned) in one store: a whole DRAM sector per lane, so that
 // row-per-thread epilogues do not leave half-written sectors for the L2 to fill from memory.
 __device__ __forceinline__ void st_global_v8(float* dst, const uint32_t* v) {

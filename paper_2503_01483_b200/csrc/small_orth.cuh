@@ -10,6 +10,7 @@
 #pragma once
 #include <cooperative_groups.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
 #include "elementwise.cuh"
@@ -32,25 +33,143 @@ struct FusedPartials {
   const double* loss_part;        // [parts]
   const unsigned int* deg_part;   // [parts]
   double loss_scale;              // 1 / (tokens the loss is a mean over)
+  float dr_scale;                 // 4 / (tokens * 128): the constant factor of dL/dc the kernel leaves out
   int correct;                    // 1: add the first-order term <dR, R - bf16(R)> to the loss
   double* rowdot;                 // [128] scratch: that term, row by row
   double* hist_slot;              // receives the loss too when not null
 };
 
-// Entry idx of dR: the partials in ascending order.
+// Entry idx of dR: the partials added in ascending order (loads issued 32 at a time, so that their latency is paid
+// five times, not once per partial).
 __device__ __forceinline__ float sum_dr_parts(const FusedPartials& f, int idx) {
-  float acc = __ldcg(f.dr_part + idx);
-#pragma unroll 8
-  for (int s = 1; s < f.parts; ++s) acc += __ldcg(f.dr_part + static_cast<long long>(s) * kSoD128 + idx);
-  return acc;
+  float acc = 0.f;
+  for (int s0 = 0; s0 < f.parts; s0 += 32) {
+    float t[32];
+#pragma unroll
+    for (int u = 0; u < 32; ++u)
+      t[u] = (s0 + u < f.parts) ? __ldcg(f.dr_part + static_cast<long long>(s0 + u) * kSoD128 + idx) : 0.f;
+#pragma unroll
+    for (int u = 0; u < 32; ++u) acc = (s0 + u == 0) ? t[u] : ((s0 + u < f.parts) ? acc + t[u] : acc);
+  }
+  return acc * f.dr_scale;
 }
 
-// First-order correction of a loss that was evaluated at bf16(R) instead of R:
-//   L(R) = L(bf16 R) + <dL/dR, R - bf16 R> + O(|R - bf16 R|^2),
-// dR being the gradient at bf16(R) from the same pass.  The remainder R - bf16(R) is exact in float32 and about
-// 2^-9 of R, so what is neglected is about 2^-18 of the loss's variation over R.  This is one entry's term.
-__device__ __forceinline__ double first_order_term(float dr, float r) {
-  return static_cast<double>(dr) * static_cast<double>(r - __bfloat162float(__float2bfloat16_rn(r)));
+// The single-pass kernel's copy of X (128 columns): row t times the power of two that brings its largest entry into
+// [1, 2), as float16, and ms[t] = the mean square of that encoded row.  bf16 has 8 significant bits, float16 11: the
+// copy is exact but for entries more than 2^14 below the row's largest (they lose bits worth < 2^-25 of the row's
+// size).  A float32 X is rounded to bf16 first, as everywhere.  An all-zero row stays zero; a row with a NaN or Inf
+// becomes all NaN (and so does the loss).  Row t is X[t] (bases == null) or row t of the minibatch `ids` gathered
+// from several buffers (see k_gather_samples for the numbering).  Sixteen lanes per row, eight entries per lane;
+// grid ceil(N / 16), block 256.
+template <typename T>
+__global__ void k_encode_rows_128(const T* __restrict__ X, long long ld, int N, __half* __restrict__ x16,
+                                  float* __restrict__ ms, const void* const* __restrict__ bases, int samples_per_buf,
+                                  int rps, const int* __restrict__ ids) {
+  const int row = blockIdx.x * 16 + (threadIdx.x >> 4);
+  const int part = threadIdx.x & 15;
+  const bool live = row < N;
+  float v[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) v[e] = 0.f;
+  if (live) {
+    const T* x;
+    if (bases != nullptr) {
+      const int b = row / rps, r = row - b * rps;
+      const int id = ids[b];
+      const int buf = id / samples_per_buf, smp = id - buf * samples_per_buf;
+      x = static_cast<const T*>(bases[buf]) + (static_cast<long long>(smp) * rps + r) * ld;
+    } else {
+      x = X + static_cast<long long>(row) * ld;
+    }
+    load8(x + part * 8, v);
+    if (sizeof(T) == 4) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = __bfloat162float(__float2bfloat16_rn(v[e]));
+    }
+  }
+  float amax = 0.f;
+  bool bad = false;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    amax = fmaxf(amax, fabsf(v[e]));
+    bad |= !(fabsf(v[e]) <= 3.4e38f);   // NaN or Inf
+  }
+#pragma unroll
+  for (int o = 8; o > 0; o >>= 1) {     // within the row's 16 lanes
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    bad |= (__shfl_xor_sync(0xffffffffu, bad ? 1 : 0, o) != 0);
+  }
+  float scale = 1.0f;
+  if (amax > 0.f) {
+    int e = static_cast<int>((__float_as_uint(amax) >> 23) & 0xffu) - 127;   // amax in [2^e, 2^(e+1)); subnormal: -127
+    e = e < -126 ? -126 : e;
+    scale = __uint_as_float(static_cast<uint32_t>(127 - e) << 23);           // 2^-e, e in [-126, 127]
+  }
+  float acc = 0.f;
+  uint4 out;
+  __half2* po = reinterpret_cast<__half2*>(&out);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float a = bad ? __uint_as_float(0x7fc00000u) : v[2 * e] * scale;
+    const float b = bad ? __uint_as_float(0x7fc00000u) : v[2 * e + 1] * scale;
+    po[e] = __floats2half2_rn(a, b);
+    const float2 f = __half22float2(po[e]);
+    acc = fmaf(f.x, f.x, acc);
+    acc = fmaf(f.y, f.y, acc);
+  }
+#pragma unroll
+  for (int o = 8; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (live) {
+    *reinterpret_cast<uint4*>(x16 + static_cast<long long>(row) * 128 + part * 8) = out;
+    if (part == 0) ms[row] = acc * (1.0f / 128.0f);
+  }
+}
+
+// Mean over a block of 128 threads (one row), in a fixed order, returned to every thread.
+__device__ __forceinline__ float row_mean_128(float v, double* sh4) {
+  const double w = warp_sum(static_cast<double>(v));
+  if ((threadIdx.x & 31) == 0) sh4[threadIdx.x >> 5] = w;
+  __syncthreads();
+  const float m = static_cast<float>((((sh4[0] + sh4[1]) + sh4[2]) + sh4[3]) * (1.0 / 128.0));
+  __syncthreads();
+  return m;
+}
+
+// The single-pass kernel multiplies X not by R but by Rc = R (I - 1 1^T / d), R with the mean of each row taken off:
+// every row of X Rc is the row of X R minus its own mean, so the kernel gets the centred row of Eq. 3 straight out of
+// the tensor cores and needs neither the mean nor the mean's part of the gradient.  The chain rule through the
+// centring is a projection of the result, dL/dR = (dL/dRc) (I - 1 1^T / d): the mean of each row of the raw gradient
+// is taken off again (both by the sums below).
+//
+// First-order correction of a loss that was evaluated at f16(Rc), Rc rounded to float16, instead of Rc:
+//   L = f(Rc) = f(f16 Rc) + <df, Rc - f16 Rc> + O(|Rc - f16 Rc|^2),
+// df being the raw gradient at f16(Rc) from the same pass.  The remainder Rc - f16(Rc) is exact in float32 and
+// about 2^-12 of Rc, so what is neglected is about 2^-24 of the loss's variation over R.  This is one entry's term.
+__device__ __forceinline__ double first_order_term(float dr_raw, float rc) {
+  return static_cast<double>(dr_raw) * static_cast<double>(rc - __half2float(__float2half_rn(rc)));
+}
+
+// float16 forms of one entry of Rc: the rounded value and the remainder (as the bit patterns the operand buffers,
+// which are declared as 16-bit words, receive).
+__device__ __forceinline__ void split_f16(float rc, __nv_bfloat16& hi, __nv_bfloat16& lo) {
+  const __half h = __float2half_rn(rc);
+  const __half l = __float2half_rn(rc - __half2float(h));
+  hi = *reinterpret_cast<const __nv_bfloat16*>(&h);
+  lo = *reinterpret_cast<const __nv_bfloat16*>(&l);
+}
+
+// float16 forms of Rc^T (hi, and lo = the rounding remainder) for the single-pass kernel: one block of 128 threads
+// per row of R.  grid 128.
+__global__ void __launch_bounds__(128) k_center_split_128(const float* __restrict__ R, __nv_bfloat16* __restrict__ rt_hi,
+                                                          __nv_bfloat16* __restrict__ rt_lo) {
+  __shared__ double sh4[4];
+  const int i = blockIdx.x, j = threadIdx.x;
+  const float r = R[i * 128 + j];
+  const float rc = r - row_mean_128(r, sh4);
+  __nv_bfloat16 h, l;
+  split_f16(rc, h, l);
+  rt_hi[j * 128 + i] = h;
+  rt_lo[j * 128 + i] = l;
 }
 
 // Sum over a block of 128 threads in a fixed order (shuffle tree, then the four warps in order); valid in thread 0.
@@ -99,9 +218,11 @@ __global__ void __launch_bounds__(128) k_fused_finish(const FusedPartials f, con
   __shared__ unsigned int shd[256];
   __shared__ unsigned int is_last;
   const int idx = blockIdx.x * 128 + threadIdx.x;
-  const float acc = sum_dr_parts(f, idx);
-  dR[idx] = acc;
-  const double row = row_sum_128(f.correct ? first_order_term(acc, R[idx]) : 0.0, sh4);
+  const float acc = sum_dr_parts(f, idx);                 // raw gradient with respect to Rc
+  const float r = R[idx];
+  const float rc = r - row_mean_128(r, sh4);
+  dR[idx] = acc - row_mean_128(acc, sh4);                 // projected: the gradient with respect to R
+  const double row = row_sum_128(f.correct ? first_order_term(acc, rc) : 0.0, sh4);
   if (threadIdx.x == 0) {
     f.rowdot[blockIdx.x] = row;
     __threadfence();
@@ -184,8 +305,10 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
   if (ROWS == 1 && p.use_parts) {
     // this CTA's row of dR from the single-pass kernel's partials, and its term of the loss correction
     __shared__ double sh4[4];
-    dr_own = sum_dr_parts(p.fp, i0 * d + j);
-    const double row = row_sum_128(p.fp.correct ? first_order_term(dr_own, rcur[0]) : 0.0, sh4);
+    const float raw = sum_dr_parts(p.fp, i0 * d + j);     // raw gradient with respect to Rc (see first_order_term)
+    const float rc = rcur[0] - row_mean_128(rcur[0], sh4);
+    dr_own = raw - row_mean_128(raw, sh4);
+    const double row = row_sum_128(p.fp.correct ? first_order_term(raw, rc) : 0.0, sh4);
     if (threadIdx.x == 0) p.fp.rowdot[blockIdx.x] = row;
   }
   grid.sync();
@@ -326,14 +449,24 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
     }
   }
 
-  // bf16 forms of the new R for the next evaluation of the loss
-#pragma unroll
-  for (int r = 0; r < ROWS; ++r) {
+  // bf16 forms of the new R for the next evaluation of the loss (for the single-pass d = 128 kernel: of Rc)
+  if (ROWS == 1 && p.use_parts) {
+    __shared__ double sh4b[4];
+    const float rc = rcur[0] - row_mean_128(rcur[0], sh4b);
     __nv_bfloat16 h, l;
-    split_bf16(rcur[r], h, l);
-    p.r_hi[static_cast<long long>(i0 + r) * d + j] = h;
-    p.rt_hi[static_cast<long long>(j) * d + i0 + r] = h;
-    p.rt_lo[static_cast<long long>(j) * d + i0 + r] = l;
+    split_f16(rc, h, l);
+    p.r_hi[static_cast<long long>(i0) * d + j] = __float2bfloat16_rn(rcur[0]);
+    p.rt_hi[static_cast<long long>(j) * d + i0] = h;
+    p.rt_lo[static_cast<long long>(j) * d + i0] = l;
+  } else {
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) {
+      __nv_bfloat16 h, l;
+      split_bf16(rcur[r], h, l);
+      p.r_hi[static_cast<long long>(i0 + r) * d + j] = h;
+      p.rt_hi[static_cast<long long>(j) * d + i0 + r] = h;
+      p.rt_lo[static_cast<long long>(j) * d + i0 + r] = l;
+    }
   }
 }
 

@@ -253,7 +253,7 @@ def test_single_pass_kernel_d128(ctx, N):
     # two bf16 terms of R in the single-pass kernel itself (no correction): the general path's loss to float32 noise
     two = kurtail.Context(DEV, forward_terms=2)
     loss_2, dR_2 = two.loss_grad(X, R)
-    assert abs(loss_2 - loss_g) <= 1e-6 * abs(loss_g)
+    assert abs(loss_2 - loss_g) <= 1e-5 * abs(loss_g)
     assert np.linalg.norm(f64(dR_2) - dR_ref) / np.linalg.norm(dR_ref) <= 1e-2
     two.close()
     # fixed-order reductions: a second evaluation is bit-identical
