@@ -207,44 +207,18 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
     if (lane == 0 && my_tiles > 0) {
       bool ok = mbar_wait_bounded(r_full, 0u, abort_flag, 12u, p.wait_limit_ns);
       const uint32_t acc_dr = tmem_base + kColDr;
-      // MMA1 runs two tiles ahead of MMA2, so the tensor pipe has work while a tile is in the epilogue
-      for (int n = 0; n <= my_tiles + 1 && ok; ++n) {
-        if (n < my_tiles) {
-          // Y(n) = X(n) R
-          const int s = n % kFsXStages;
-          const int b = n & 1;
-          if (!mbar_wait_bounded(x_full(s), (n / kFsXStages) & 1, abort_flag, 13u, p.wait_limit_ns) ||
-              !mbar_wait_bounded(y_empty(b), ((n >> 1) & 1) ^ 1u, abort_flag, 14u, p.wait_limit_ns)) {
-            ok = false;
-            break;
-          }
-          tc_fence_after_sync();
-          const uint32_t acc_y = tmem_base + static_cast<uint32_t>(b * 128);
-          uint32_t first = 1;
-#pragma unroll
-          for (int q = 0; q < TERMS; ++q) {
-            const uint32_t rb = (q == 0) ? s_rhi : s_rlo;
-#pragma unroll
-            for (int kb = 0; kb < 2; ++kb) {
-              const uint64_t a_desc = umma_desc_kmajor_sw128(s_x + s * kFsTile + kb * kFsHalf, 1024);
-              const uint64_t b_desc = umma_desc_kmajor_sw128(rb + kb * kFsHalf, 1024);
-#pragma unroll
-              for (int kk = 0; kk < 4; ++kk) {
-                tc_mma_bf16(acc_y, a_desc + 2u * kk, b_desc + 2u * kk, kIdescK, first ? 0u : 1u);
-                first = 0;
-              }
-            }
-          }
-          tc_commit(y_full(b));
-        }
-        if (n >= 2) {
+      // Two instruction streams share this thread: MMA1 of tile n1 can go as soon as the tile is in shared memory and
+      // its Y accumulator has been read out, MMA2 of tile n2 as soon as the epilogue has written that tile's G.
+      // Whichever is ready is issued (MMA2 first: it frees a shared-memory stage); neither waits for the other's turn.
+      int n1 = 0, n2 = 0;
+      uint64_t idle_since = 0;
+      uint32_t spins = 0;
+      while (n2 < my_tiles && ok) {
+        bool progressed = false;
+        if (n2 < n1 && mbar_test_wait(g_full(n2 & 1), (n2 >> 1) & 1)) {
           // dR += X(m)^T G(m): contraction over the tile's 128 tokens, 16 per MMA = two 8-row groups
-          const int m = n - 2;
+          const int m = n2;
           const int s = m % kFsXStages;
-          if (!mbar_wait_bounded(g_full(m & 1), (m >> 1) & 1, abort_flag, 15u, p.wait_limit_ns)) {
-            ok = false;
-            break;
-          }
           tc_fence_after_sync();
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
@@ -253,8 +227,51 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
                 umma_desc_mnmajor_sw128(s_g + (kGBufs == 2 ? (m & 1) * kFsTile : 0) + ks * 2048, kFsHalf, 1024);
             tc_mma_bf16(acc_dr, a_desc, b_desc, kIdescMN, (m > 0 || ks > 0) ? 1u : 0u);
           }
-          tc_commit(x_empty(s));   // the X tile is free once these MMAs have read it
+          tc_commit(x_empty(s));      // the X tile is free once these MMAs have read it
           tc_commit(g_empty(m & 1));  // and so is the G tile
+          ++n2;
+          progressed = true;
+        }
+        if (n1 < my_tiles) {
+          // Y(n) = X(n) Rc
+          const int n = n1;
+          const int s = n % kFsXStages;
+          const int b = n & 1;
+          if (mbar_test_wait(x_full(s), (n / kFsXStages) & 1) && mbar_test_wait(y_empty(b), ((n >> 1) & 1) ^ 1u)) {
+            tc_fence_after_sync();
+            const uint32_t acc_y = tmem_base + static_cast<uint32_t>(b * 128);
+            uint32_t first = 1;
+#pragma unroll
+            for (int q = 0; q < TERMS; ++q) {
+              const uint32_t rb = (q == 0) ? s_rhi : s_rlo;
+#pragma unroll
+              for (int kb = 0; kb < 2; ++kb) {
+                const uint64_t a_desc = umma_desc_kmajor_sw128(s_x + s * kFsTile + kb * kFsHalf, 1024);
+                const uint64_t b_desc = umma_desc_kmajor_sw128(rb + kb * kFsHalf, 1024);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                  tc_mma_bf16(acc_y, a_desc + 2u * kk, b_desc + 2u * kk, kIdescK, first ? 0u : 1u);
+                  first = 0;
+                }
+              }
+            }
+            tc_commit(y_full(b));
+            ++n1;
+            progressed = true;
+          }
+        }
+        // bounded like every other wait: no progress for the limit's length ends the kernel with an error code
+        if (progressed) {
+          spins = 0;
+        } else if ((++spins & 63u) == 0) {
+          if (*abort_flag) {
+            ok = false;
+          } else if (spins == 64u) {
+            idle_since = global_timer_ns();
+          } else if (global_timer_ns() - idle_since > p.wait_limit_ns) {
+            *abort_flag = 13u;
+            ok = false;
+          }
         }
       }
       if (ok) tc_commit(dr_full);

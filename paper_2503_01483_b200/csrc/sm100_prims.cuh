@@ -47,6 +47,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
+// The same question without any waiting: try_wait may park the thread for a while when the phase is not complete,
+// test_wait answers at once (for a thread that polls several barriers in turn).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
 // Wait with a bound.  Gives up after `limit_ns` of wall time (kernels take it from
 // their parameters; kDefaultWaitLimitNs unless the caller configured another), or
 // as soon as another thread of the CTA has raised *abort_flag; on giving up it
