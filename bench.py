@@ -291,9 +291,9 @@ def main():
                     help="with --gpus N > 1: one independent layer per GPU (weak scaling, no collective), or the rows "
                          "of one X sharded over the GPUs (kt_fit_sharded: an all-reduce of dR and of the loss per "
                          "step, enqueued by the library through its reduce hook; strong scaling)")
-    ap.add_argument("--backward", default="stored", choices=["stored", "recompute"],
-                    help="kt_config.backward_mode: read back the Y the forward pass kept (default) or recompute Y in "
-                         "a second GEMM pass, so that Y never reaches memory")
+    ap.add_argument("--backward", default="stored", choices=["stored", "stored_f32", "recompute"],
+                    help="kt_config.backward_mode: read back the Y the forward pass kept as float16 (default) or as "
+                         "float32, or recompute Y in a second GEMM pass, so that Y never reaches memory")
     ap.add_argument("--loss-mode", default="token", choices=["token", "layer"],
                     help="kt_config.loss_mode: one kurtosis per token (headline) or one over the whole layer")
     ap.add_argument("--rmsnorm", action="store_true", help="kt_config.rmsnorm: RMSNorm after the rotation")
@@ -359,7 +359,7 @@ def main():
     lr = args.lr if args.lr > 0 else cfg["lr"]
     ctx_kw = dict(forward_terms=args.forward_terms, optimizer=1 if args.optimizer == "adam" else 0,
                   loss_mode=1 if args.loss_mode == "layer" else 0, rmsnorm=1 if args.rmsnorm else 0,
-                  backward_mode=1 if args.backward == "recompute" else 0)
+                  backward_mode={"stored": 0, "recompute": 1, "stored_f32": 2}[args.backward])
     ctx = kurtail.Context(dev, **ctx_kw)
     fwd_terms = args.forward_terms if args.forward_terms in (1, 2) else (2 if d <= 512 else 1)
 
@@ -504,7 +504,8 @@ def main():
         use_burst = (not capped) and timed_s < 1.0
         peak = peaks["tflops_burst"] if use_burst else peaks["tflops_sustained"]
         trs = [recorded_traffic("gemm_tn_kernel", r) for r in
-               (("forward_stored" if args.backward == "stored" else "forward"), "backward_b")]
+               ({"stored": "forward_stored", "stored_f32": "forward_stored_f32", "recompute": "forward"}[args.backward],
+                "backward_b")]
         traffic = None
         if all(trs):
             traffic = sum(t[0] * N + t[1] for t in trs) / 2.0        # mean of the two token GEMMs, per launch
@@ -534,8 +535,9 @@ def main():
         "data": "synthetic",
         "config": {"workload": args.workload, "N": N, "d": d, "R_init": cfg["init"], "lr": lr,
                    "optimizer": "cayley_" + args.optimizer, "loss_mode": args.loss_mode, "rmsnorm": bool(args.rmsnorm),
-                   "backward": args.backward + (" (Y kept between the forward and the backward pass)"
-                                                if args.backward == "stored" else " (Y never written)"),
+                   "backward": args.backward + {"stored": " (Y kept as float16 between the forward and the backward pass)",
+                                                "stored_f32": " (Y kept as float32 between the two passes)",
+                                                "recompute": " (Y never written)"}[args.backward],
                    "l2": "inputs (%.0f MiB of X per step) exceed the 126 MB L2" % (N * d * 2 / 2**20)
                    if N * d * 2 > 126e6 else "inputs fit in L2; no flush (small case)",
                    "parallelism": ("rows of one batch over the GPUs, kt_fit_sharded: all-reduce of dR and loss per "
@@ -593,7 +595,8 @@ def main():
             pr = c.profile_end()
             return a.elapsed_time(b) / steps, r, pr
 
-        for name, kwx in (("backward_recompute", dict(backward_mode=1)), ("optimizer_adam", dict(optimizer=1)),
+        for name, kwx in (("backward_recompute", dict(backward_mode=1)), ("backward_stored_f32", dict(backward_mode=2)),
+                          ("optimizer_adam", dict(optimizer=1)),
                           ("lr_10_full_series", dict())):
             c2 = kurtail.Context(dev, **kwx)
             ms_x, r_x, _ = short_fit(c2, X, fresh_R(c2), 20, 10.0 if name == "lr_10_full_series" else lr)

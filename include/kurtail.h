@@ -129,13 +129,23 @@ typedef struct {
   int32_t backward_mode;/* [0]   where the backward pass takes Y from.  1 = a
                            second pass of the forward GEMM recomputes each Y
                            tile in tensor memory and nothing of Y is ever
-                           written (2 N d^2 more flops).  0 or 2 = the forward
-                           pass also stores Y as float32 (N*d*4 bytes of
-                           workspace) and an element-wise kernel reads it
-                           back (8 bytes per entry instead of 2 d flops: on a
-                           B200 the cheaper one for d above a few hundred).
-                           The two give bit-identical gradients.  d == 128
-                           with small_d_fused needs neither                    */
+                           written (2 N d^2 more flops).  0 = the forward pass
+                           also stores Y as float16 (N*d*2 bytes of workspace;
+                           every run of 128 entries of a row, 64 when d is not
+                           a multiple of 256, carries its own power-of-two
+                           factor, taken from the run's mean and sum of
+                           squares, so the scale of X does not matter) and an
+                           element-wise kernel reads it back: 4 bytes of
+                           memory traffic per entry instead of 2 d flops, on a
+                           B200 the cheaper side for d above a few hundred.
+                           The loss and the row moments come from the float32
+                           accumulators in every mode; the gradient of mode 0
+                           differs from mode 1's by the rounding of Y to 11
+                           significant bits (one or two parts in a thousand of
+                           its norm).
+                           2 = Y is stored as float32 (N*d*4 bytes): gradients
+                           bit-identical to mode 1.  d == 128 with
+                           small_d_fused needs none of this                    */
   int32_t cta_pairs;    /* [1]   1 = GEMMs with 256-wide column tiles run on
                            pairs of CTAs (thread-block clusters of two, one
                            MMA over both SMs' tensor cores, each CTA loading

@@ -35,7 +35,10 @@ namespace kt {
 
 constexpr int kFsD = 128;          // channels = rows of a token tile
 constexpr int kFsThreads = 320;    // warp 0: TMA, warp 1: MMA, warps 2..5 and 6..9: two epilogue groups
-constexpr int kFsXStages = 4;
+#ifndef KT_FS_STAGES
+#define KT_FS_STAGES 4
+#endif
+constexpr int kFsXStages = KT_FS_STAGES;   // X tiles in shared memory (4 is what fits beside R^T and the G tiles)
 #ifndef KT_FS_PREFETCH
 #define KT_FS_PREFETCH 8
 #endif

@@ -12,13 +12,14 @@
 //   kStoreF32  write D as float32
 //   kMoments   per row: mean and central power sums of BN/2 columns (Eq. 3 of the
 //              paper, one partial record per half column tile); optionally also
-//              stores D as float32
+//              stores D as float32, or as float16 with a power-of-two factor per half row
 //   kGrad      G = a c^3 - ab c - am3, c = D - mu  (derivative of the loss
 //              through Eq. 3), written transposed as bf16
 //   kAbsMax    per-row max |D| (first pass of the symmetric quantizer)
 //   kQuantErr  per-row sum of (D - Q(D))^2 for the 4-bit symmetric quantizer
 #pragma once
 #include <cuda.h>
+#include <cuda_fp16.h>
 
 #include "sm100_prims.cuh"
 
@@ -71,6 +72,11 @@ struct GemmParams {
   // when not null: row m of D is multiplied by row_scale[m] before the epilogue sees it (the RMSNorm that follows
   // the rotation in the paper's small network, applied to the float32 accumulator)
   const float* row_scale;
+  // kMoments, when not null: D is kept as float16 (for the backward pass) instead of float32.  Every half row of a
+  // tile (the BN/2 columns one thread holds) is multiplied by its own power of two 2^(140 - e), chosen from the half
+  // row's mean and sum of squares so that no entry can exceed 2^14; e goes to out16_exp[2 * n_tile + half][row].
+  __half* out16;
+  unsigned char* out16_exp;
 };
 
 // Unsigned keys that order like the floats they encode (negative floats reversed, positive ones above them).
@@ -419,6 +425,30 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
           s4 += b4;
         }
         if (row_ok) p.partial[static_cast<long long>(2 * n_tile + half) * p.M + row] = make_float4(mean, s2, s3, s4);
+        if (p.out16 != nullptr && row_ok) {
+          // float16 copy of the half row for the backward pass.  |y| <= |mean| + |c| and c^2 <= sum of c^2:
+          // with e the biased exponent of that bound (< 2^(e - 126)), 2^(140 - e) brings every entry below 2^14.
+          // e is kept in [14, 254] so that both the factor and its inverse 2^(e - 140) are normal float32 numbers.
+          const float bound = fabsf(mean) + sqrtf(s2);
+          unsigned int e = (__float_as_uint(bound) >> 23) & 0xffu;
+          e = e < 14u ? 14u : (e > 254u ? 254u : e);
+          const float mul = __uint_as_float((267u - e) << 23);
+          p.out16_exp[static_cast<long long>(2 * n_tile + half) * p.M + row] = static_cast<unsigned char>(e);
+          __half* dst = p.out16 + static_cast<long long>(row) * p.ldo + n0 + cbeg;
+#pragma unroll
+          for (int c = 0; c < kChunks; ++c) {
+            uint32_t h[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const __half2 hh = __floats2half2_rn(__uint_as_float(vv[c][2 * j]) * mul,
+                                                   __uint_as_float(vv[c][2 * j + 1]) * mul);
+              h[j] = *reinterpret_cast<const uint32_t*>(&hh);
+            }
+            // (column offsets are multiples of 32 entries and the row pitch of 128 entries: 32-byte aligned)
+            st_global_v8(reinterpret_cast<float*>(dst + 32 * c), h);
+            st_global_v8(reinterpret_cast<float*>(dst + 32 * c + 16), h + 8);
+          }
+        }
       } else if constexpr (EPI == kGrad) {
         float4 cf = make_float4(0.f, 0.f, 0.f, 0.f);
         if (row_ok) cf = p.coef[row];

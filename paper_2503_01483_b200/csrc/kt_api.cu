@@ -79,7 +79,9 @@ struct WsLayout {
   size_t dr;            // d x d float32: gradient inside kt_fit
   size_t xb;            // dense bf16 copy of a float32 X, or of any X after RMSNorm  [N][d]
   size_t xt, gt;        // X^T and G^T as bf16  [d][ldt]
-  size_t ybuf;          // Y = X R as float32 [N][d], kept by the forward pass unless the backward recomputes it
+  size_t ybuf;          // Y = X R [N][d], kept by the forward pass unless the backward recomputes it: float16 with
+                        // a power-of-two factor per half tile row (backward_mode 0) or float32 (backward_mode 2)
+  size_t yexp;          // [P][N] bytes: the exponents of those factors
   size_t partial;       // [P][N] float4 partial moment records
   size_t coef, moments; // [N] float4 each
   size_t block_loss, block_deg, norm_blocks;
@@ -109,10 +111,11 @@ static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, const kt_conf
   // (d = 128: the single-pass kernel reads its own float16 encoding of X, whatever X's type)
   const bool xcopy = x_dtype == KT_F32 || gather_batch > 0 ||
                      (d == kFsD && (cfg == nullptr || (cfg->small_d_fused != 0 && cfg->loss_mode == 0)));
-  // Y kept in float32 for the backward pass, unless the backward recomputes it or the single-pass kernel (d = 128,
-  // per-token loss) does forward and backward together
+  // Y kept for the backward pass, unless the backward recomputes it or the single-pass kernel (d = 128, per-token
+  // loss) does forward and backward together
   const bool single_pass = d == kFsD && (cfg == nullptr || (cfg->small_d_fused != 0 && cfg->loss_mode == 0));
   const bool keep_y = (cfg == nullptr || cfg->backward_mode != 1) && !single_pass;
+  const bool y_f32 = cfg != nullptr && cfg->backward_mode == 2;
   WsLayout L;
   memset(&L, 0, sizeof(L));
   L.bn = (d % 256 == 0) ? 128 : 64;  // columns per moment record: half a GEMM column tile
@@ -140,7 +143,8 @@ static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, const kt_conf
   L.xb = take(xcopy ? static_cast<size_t>(N) * d * 2 : 0);
   L.xt = take(static_cast<size_t>(d) * L.ldt * 2);
   L.gt = take(static_cast<size_t>(d) * L.ldt * 2);
-  L.ybuf = take(keep_y ? static_cast<size_t>(N) * d * 4 : 0);
+  L.ybuf = take(keep_y ? static_cast<size_t>(N) * d * (y_f32 ? 4 : 2) : 0);
+  L.yexp = take((keep_y && !y_f32) ? static_cast<size_t>(L.P) * N : 0);
   L.partial = take(static_cast<size_t>(L.P) * N * 16);
   L.coef = take(static_cast<size_t>(N) * 16);
   L.moments = take(static_cast<size_t>(N) * 16);
@@ -526,16 +530,22 @@ static FwdOperands fwd_operands(kt_ctx* ctx, const XView& xv, int d, long long N
   return f;
 }
 
+static bool y_stored_f32(const kt_ctx* ctx) { return ctx->cfg.backward_mode == 2; }
+
 // moments + loss for the rows of xv; R^T must already be in rt_hi.
-// keep_y: the epilogue also stores the float32 Y tile into the workspace (for the backward pass).
+// keep_y: the epilogue also stores the Y tile into the workspace (for the backward pass), as float32 or float16.
 // err_to_nan: *hist_slot receives NaN when a device-side wait of this call ran out (for callers that never read
 // the status word on the host).
 static kt_status forward_loss(kt_ctx* ctx, const XView& xv, int N, int d, const WsLayout& L, double* hist_slot,
                               bool keep_y = false, bool err_to_nan = false) {
   GemmParams p = blank_params();
   p.partial = at<float4>(ctx, L.partial);
-  if (keep_y) {
+  if (keep_y && y_stored_f32(ctx)) {
     p.out = at<float>(ctx, L.ybuf);
+    p.ldo = d;
+  } else if (keep_y) {
+    p.out16 = at<__half>(ctx, L.ybuf);
+    p.out16_exp = at<unsigned char>(ctx, L.yexp);
     p.ldo = d;
   }
   p.row_scale = xv.row_scale;
@@ -596,17 +606,24 @@ static kt_status forward_loss(kt_ctx* ctx, const XView& xv, int N, int d, const 
 }
 
 // dR = X^T G with G from the saved row coefficients and Y: either the Y tile is recomputed by a second pass of the
-// forward GEMM (nothing of Y ever reaches memory), or the float32 Y the forward pass kept is read back by an
-// element-wise kernel.  Both evaluate the same float32 expression on the same accumulator values: the same bits.
+// forward GEMM (nothing of Y ever reaches memory), or the Y the forward pass kept is read back by an element-wise
+// kernel.  A float32 Y (backward_mode 2) gives the recomputing pass's bits: the same float32 expression on the same
+// accumulator values.  The float16 Y (the default) is those values rounded to 11 significant bits.
 static bool keep_y_for_backward(const kt_ctx* ctx) { return ctx->cfg.backward_mode != 1; }
 
 // dr_hi != null: the split-K sum also leaves bf16(dR) there (only when the sum runs; see dr_hi_from_backward()).
 static kt_status backward(kt_ctx* ctx, const XView& xv, int N, int d, const WsLayout& L, float* dR,
                           __nv_bfloat16* dr_hi = nullptr) {
-  if (keep_y_for_backward(ctx)) {
+  if (keep_y_for_backward(ctx) && y_stored_f32(ctx)) {
     dim3 grid((N + 63) / 64, d / 64);
     k_grad_from_y<<<grid, 256, 0, ctx->stream>>>(at<float>(ctx, L.ybuf), at<float4>(ctx, L.coef), N, d,
                                                  at<__nv_bfloat16>(ctx, L.gt), L.ldt);
+    KT_LAUNCH_CHECK();
+  } else if (keep_y_for_backward(ctx)) {
+    dim3 grid((N + 63) / 64, d / 64);
+    k_grad_from_y16<<<grid, 256, 0, ctx->stream>>>(at<__half>(ctx, L.ybuf), at<unsigned char>(ctx, L.yexp), L.bn,
+                                                   at<float4>(ctx, L.coef), N, d, at<__nv_bfloat16>(ctx, L.gt),
+                                                   L.ldt);
     KT_LAUNCH_CHECK();
   } else {
     GemmParams p = blank_params();

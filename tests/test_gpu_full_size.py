@@ -157,17 +157,18 @@ def test_layer_sweep_driver_resident_buffers(ctx):
 
 
 def test_full_size_launch_variants_agree_bitwise():
-    # At the headline size: the backward that reads the stored Y against the one that recomputes it, and GEMMs on
-    # pairs of CTAs against one CTA per tile.  All three evaluate the same float32 operations in the same order.
+    # At the headline size: the backward that reads a float32 Y kept by the forward pass against the one that
+    # recomputes it, and GEMMs on pairs of CTAs against one CTA per tile.  All three evaluate the same float32
+    # operations in the same order.
     cfg = synth.config("llama2_7b_attn", device=DEV)
     X = cfg["X"]
-    base = kurtail.Context(DEV)
+    base = kurtail.Context(DEV, backward_mode=2)
     R = base.init_rotation(4096, "hadamard")
     l0, d0 = base.loss_grad(X, R)
     R0 = R.clone()
     base.fit(X, R0, 2, 1e-2)
     base.close()
-    for kw in (dict(backward_mode=1), dict(cta_pairs=0)):
+    for kw in (dict(backward_mode=1), dict(backward_mode=2, cta_pairs=0)):
         c = kurtail.Context(DEV, **kw)
         l1, d1 = c.loss_grad(X, R)
         assert l1 == l0 and torch.equal(d1, d0), kw

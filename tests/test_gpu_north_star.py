@@ -58,11 +58,17 @@ def test_gradient_matches_oracle_at_full_width(ctx, workload, rows, init):
     L_ref, dR_ref = ko.loss_grad(f64(X), f64(R))
     assert abs(loss - L_ref) <= 1e-3 * abs(L_ref)
     assert rel_fro(f64(dR), dR_ref) <= 1e-2
-    # the mode that never writes Y (a second GEMM pass recomputes it): same bits
+    # the mode that never writes Y (a second GEMM pass recomputes it) is held to the same bar, and equals the
+    # mode that keeps Y in float32 bit for bit (the default keeps it in float16)
     c2 = kurtail.Context(DEV, backward_mode=1)
     l2, dR2 = c2.loss_grad(X, R)
-    assert l2 == loss and torch.equal(dR2, dR)
     c2.close()
+    assert l2 == loss
+    assert rel_fro(f64(dR2), dR_ref) <= 1e-2
+    c3 = kurtail.Context(DEV, backward_mode=2)
+    l3, dR3 = c3.loss_grad(X, R)
+    c3.close()
+    assert l3 == loss and torch.equal(dR3, dR2)
 
 
 # ------------------------------------------------------- one orthogonal step
