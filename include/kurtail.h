@@ -86,7 +86,10 @@ typedef struct {
                            the retraction: 1..3 forces a count; 0 = chosen on
                            the device per step (one term while alpha*||W||_F *
                            2^-9 < 2.5e-6, else hi + lo), and series terms that
-                           fall below float32 resolution are skipped           */
+                           fall below float32 resolution are skipped (the
+                           one-launch step for d <= 512, whose products are
+                           float32, skips those terms by the same rule and
+                           evaluates them all when a count is forced)          */
   int32_t guard_every;  /* [0]   kt_fit: k >= 1 measures R^T R - I every k-th step
                            (and after the last one); 0 = on the first and the
                            last step and in between whenever a device-side

@@ -39,10 +39,6 @@ constexpr int kFsThreads = 320;    // warp 0: TMA, warp 1: MMA, warps 2..5 and 6
 #define KT_FS_STAGES 4
 #endif
 constexpr int kFsXStages = KT_FS_STAGES;   // X tiles in shared memory (4 is what fits beside R^T and the G tiles)
-#ifndef KT_FS_PREFETCH
-#define KT_FS_PREFETCH 8
-#endif
-constexpr int kFsPrefetch = KT_FS_PREFETCH;  // X tiles requested into L2 ahead of their shared-memory load
 constexpr int kFsHalf = 128 * 64 * 2;      // bytes of one 128-row x 64-element swizzled block
 constexpr int kFsTile = 2 * kFsHalf;       // one 128 x 128 bf16 tile
 // TERMS = 1: R^T hi only, which leaves room for a second G tile; TERMS = 2: R^T hi + lo and one G tile.
@@ -168,19 +164,9 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
       }
       bool ok = true;
       uint32_t issued = 0, last_parity = 0;
-      // X tiles are asked into L2 kFsPrefetch tiles before their shared-memory stage is free: the stage's own load
-      // then costs an L2 round trip instead of one to memory, and the stage is held for that much less time
-      for (int n = 0; n < kFsPrefetch && n < my_tiles; ++n) {
-        const int row0 = (static_cast<int>(blockIdx.x) + n * static_cast<int>(gridDim.x)) * 128;
-        tma_prefetch_2d(&p.tmX, 0, row0);
-        tma_prefetch_2d(&p.tmX, 64, row0);
-      }
+      // (asking for the tiles into L2 ahead of their shared-memory load was measured and costs time: the loads alone
+      // already run at 0.85 of the copy bandwidth, and the extra requests only add to the memory system's queues)
       for (int n = 0; n < my_tiles; ++n) {
-        if (n + kFsPrefetch < my_tiles) {
-          const int rowp = (static_cast<int>(blockIdx.x) + (n + kFsPrefetch) * static_cast<int>(gridDim.x)) * 128;
-          tma_prefetch_2d(&p.tmX, 0, rowp);
-          tma_prefetch_2d(&p.tmX, 64, rowp);
-        }
         const int s = n % kFsXStages;
         const uint32_t ph = (n / kFsXStages) & 1;
         if (!mbar_wait_bounded(x_empty(s), ph ^ 1u, abort_flag, 11u, p.wait_limit_ns)) {

@@ -838,6 +838,7 @@ static kt_status small_orth_step_async(kt_ctx* ctx, float* R, const float* dR, i
   p.dR = dR;
   p.d = d;
   p.iters = c.cayley_iters < 0 ? 0 : c.cayley_iters;
+  p.gate_terms = c.retract_terms <= 0 ? 1 : 0;
   p.run_guard = run_guard;
   p.lr = lr;
   p.q = c.q;

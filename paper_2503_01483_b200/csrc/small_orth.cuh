@@ -240,6 +240,7 @@ struct SmallOrthParams {
   const float* dR;     // d x d
   int d;
   int iters;           // s: series terms 0..s
+  int gate_terms;      // 1: series terms that cannot change the float32 R are not evaluated
   int run_guard;       // 1: measure R^T R - I, 0: do not, 2: when the device's drift bound reaches thresh / 2
   float lr, q, eps, thresh;
   float polish_at;     // the polish runs when the measured error exceeds this (<= thresh)
@@ -354,6 +355,7 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
   float alpha;
   bool do_guard;   // the same in every CTA
   float drift;     // bound on the orthogonality error accumulated since the last measurement
+  int n_terms;     // series terms evaluated (the same in every CTA: the grid-wide barriers below depend on it)
   {
     double s = 0.0;
     for (int c = 0; c < kSoGrid; ++c) s += __ldcg(p.norm_part + c);
@@ -365,15 +367,28 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
     // product here is float32, so a step adds the truncation of the series, 2 x (x/2)^(s+1) with x = alpha ||W||_F
     // (the remainder of the Neumann series, twice through E = R^T dR + dR^T R), and float32 rounding of the update.
     const double x = a * nrm;
+    // Term k of the series is at most x (x/2)^k in norm; below 2^-26 / sqrt(d), a quarter ulp of a typical entry of
+    // R, it cannot change the float32 R and is not evaluated (what it would have done for orthogonality is part
+    // of the drift bound: the truncation below is taken at the last evaluated term).
+    n_terms = 1;
+    {
+      const double floor_k = ldexp(1.0, -26) / sqrt(static_cast<double>(d));
+      double bound = x;
+      for (int k = 1; k <= p.iters; ++k) {
+        bound *= 0.5 * x;
+        if (p.gate_terms && bound < floor_k) break;
+        ++n_terms;
+      }
+    }
     double trunc = 2.0 * x;
-    for (int k = 0; k <= p.iters; ++k) trunc *= 0.5 * x;
-    drift = drift_in + static_cast<float>(trunc + (p.iters + 2) * ldexp(1.0, -23));
+    for (int k = 0; k < n_terms; ++k) trunc *= 0.5 * x;
+    drift = drift_in + static_cast<float>(trunc + (n_terms + 1) * ldexp(1.0, -23));
     do_guard = p.run_guard == 1 || (p.run_guard == 2 && (p.thresh <= 0.f || drift >= 0.5f * p.thresh));
     if (blockIdx.x == 0 && threadIdx.x == 0) {
       p.sc->alpha = alpha;
       p.sc->wnorm = static_cast<float>(nrm);
-      p.sc->wop = static_cast<float>(nrm);  // this path evaluates every term in float32 and decides nothing
-      p.sc->n_terms = static_cast<unsigned int>(p.iters + 1);
+      p.sc->wop = static_cast<float>(nrm);  // (every product here is float32: the Frobenius norm is all it needs)
+      p.sc->n_terms = static_cast<unsigned int>(n_terms);
       p.sc->p0_terms = 0u;
       if (do_guard) p.sc->guards += 1u;
       else p.sc->drift = drift;
@@ -386,15 +401,15 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
     const float* src = p.R;
     float* dst = p.P0;
     float ck = -alpha;
-    for (int k = 0; k <= p.iters; ++k) {
+    for (int k = 0; k < n_terms; ++k) {
       rows_times_matrix<ROWS>(arow, src, d, j, acc);
 #pragma unroll
       for (int r = 0; r < ROWS; ++r) {
         rcur[r] = fmaf(ck, acc[r], rcur[r]);
-        if (k < p.iters) dst[static_cast<long long>(i0 + r) * d + j] = acc[r];
+        if (k + 1 < n_terms) dst[static_cast<long long>(i0 + r) * d + j] = acc[r];
       }
       ck *= -0.5f * alpha;
-      if (k < p.iters) {
+      if (k + 1 < n_terms) {
         grid.sync();  // all rows of P_k written; (R itself is not read after the first product)
         src = dst;
         dst = (dst == p.P0) ? p.P1 : p.P0;
