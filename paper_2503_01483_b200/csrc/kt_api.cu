@@ -90,7 +90,7 @@ struct WsLayout {
   size_t diag;          // [d] float: exact diagonal of R^T R - I
   size_t pvec;          // [2][d] float: the last two vectors of the power iteration on W
   size_t splitk;        // [splits][d][d] float: partial dR of the split-K backward-B (when splits > 1)
-  size_t small;         // d <= 512: scratch of the one-launch orthogonal step (5 d x d floats + per-CTA partials)
+  size_t small;         // d <= 512: scratch of the one-launch orthogonal step (6 d x d floats + per-CTA partials)
   size_t adam_m;        // d x d float32: momentum of Cayley Adam inside kt_fit (only when asked for)
   size_t gather_ids;    // kt_fit_shared: [kIdsChunk][batch] int sample ids
   size_t gather_bases;  // kt_fit_shared: [kMaxSharedBufs] buffer base pointers
@@ -164,7 +164,7 @@ static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, const kt_conf
     if (d == kFsD && parts < 256) parts = 256;  // per-CTA partial dR of the fused d = 128 kernel
     L.splitk = take(static_cast<size_t>(parts) * dd * 4);
   }
-  L.small = take(d <= 512 ? 5 * dd * 4 + 4096 : 0);
+  L.small = take(d <= 512 ? 6 * dd * 4 + 4096 : 0);
   L.adam_m = take(adam ? dd * 4 : 0);
   L.gather_ids = take(gather_batch > 0 ? static_cast<size_t>(kIdsChunk) * gather_batch * 4 : 0);
   L.gather_bases = take(gather_batch > 0 ? static_cast<size_t>(kMaxSharedBufs) * 8 : 0);
@@ -854,7 +854,8 @@ static kt_status small_orth_step_async(kt_ctx* ctx, float* R, const float* dR, i
   p.W = sm + 2 * dd;
   p.P0 = sm + 3 * dd;
   p.P1 = sm + 4 * dd;
-  p.norm_part = reinterpret_cast<double*>(sm + 5 * dd);
+  p.Rs = sm + 5 * dd;
+  p.norm_part = reinterpret_cast<double*>(sm + 6 * dd);
   p.max_part = reinterpret_cast<float*>(p.norm_part + kSoGrid);
   p.sc = &ctx->d_blk->sc;
   p.r_hi = at<__nv_bfloat16>(ctx, L.r_hi);
@@ -868,11 +869,22 @@ static kt_status small_orth_step_async(kt_ctx* ctx, float* R, const float* dR, i
     case 3: fn = reinterpret_cast<const void*>(small_orth_kernel<3>); break;
     default: fn = reinterpret_cast<const void*>(small_orth_kernel<4>); break;
   }
+  // d == 128: the products stage their second operand (d x d float32) in dynamic shared memory
+  const size_t stage_bytes = d == 128 ? dd * sizeof(float) : 0;
+  if (stage_bytes > 0) {
+    static bool attr_done[kMaxDevices] = {false};
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    const bool cached = ctx->device >= 0 && ctx->device < kMaxDevices;
+    if (!cached || !attr_done[ctx->device]) {
+      KT_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(stage_bytes)));
+      if (cached) attr_done[ctx->device] = true;
+    }
+  }
   // the grid-wide barriers need all kSoGrid CTAs resident at once
   int per_sm = 0;
-  KT_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, d, 0));
+  KT_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, d, stage_bytes));
   if (per_sm * ctx->sm_count < kSoGrid) return KT_ERR_COOPERATIVE;
-  const cudaError_t le = cudaLaunchCooperativeKernel(fn, dim3(kSoGrid), dim3(d), args, 0, ctx->stream);
+  const cudaError_t le = cudaLaunchCooperativeKernel(fn, dim3(kSoGrid), dim3(d), args, stage_bytes, ctx->stream);
   if (le == cudaErrorCooperativeLaunchTooLarge) {
     (void)cudaGetLastError();
     return KT_ERR_COOPERATIVE;

@@ -246,6 +246,8 @@ struct SmallOrthParams {
   float polish_at;     // the polish runs when the measured error exceeds this (<= thresh)
   // scratch, all d x d float32 unless noted
   float* Rt;           // R^T (then R_new^T)
+  float* Rs;           // copy of R as it was on entry: what the products read, so that R can be updated in place
+                       // without waiting for the other CTAs to finish with it
   float* A;            // dR R^T, later E
   float* W;
   float* P0;           // ping
@@ -277,9 +279,35 @@ __device__ __forceinline__ void rows_times_matrix(const float (*arow)[512], cons
   }
 }
 
+// The same with the whole of B (d x d) copied into shared memory first (16-byte L2-only loads, many in flight per
+// thread) instead of one load per multiply-add: at d = 128 the d dependent-latency loads of the plain version are
+// most of a product's time.  Same operations in the same order: the same bits.  Every thread of the block calls it.
+template <int ROWS>
+__device__ __forceinline__ void rows_times_staged_matrix(const float (*arow)[512], const float* B, int d, int j,
+                                                         float (&out)[ROWS], float* bs) {
+  const float4* B4 = reinterpret_cast<const float4*>(B);
+  float4* bs4 = reinterpret_cast<float4*>(bs);
+  const int n4 = d * d / 4;
+  __syncthreads();  // the previous product has finished with bs
+#pragma unroll 16
+  for (int i = threadIdx.x; i < n4; i += blockDim.x) bs4[i] = __ldcg(B4 + i);
+  __syncthreads();
+#pragma unroll
+  for (int r = 0; r < ROWS; ++r) out[r] = 0.f;
+#pragma unroll 8
+  for (int k = 0; k < d; ++k) {
+    const float b = bs[k * d + j];
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) out[r] = fmaf(arow[r][k], b, out[r]);
+  }
+}
+
+// Dynamic shared memory: d * d floats when d == 128 (the staged products above), none otherwise.
 template <int ROWS>
 __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParams p) {
   cg::grid_group grid = cg::this_grid();
+  extern __shared__ float4 stage4[];
+  float* const bs = reinterpret_cast<float*>(stage4);
   __shared__ float arow[ROWS][512];
   __shared__ double shd[16];
   __shared__ float shf[16];
@@ -288,6 +316,10 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
   const int i0 = blockIdx.x * ROWS;        // first row owned by this CTA
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
 
+  auto product = [&](const float* B, float (&out)[ROWS]) {   // out[r] = sum_k arow[r][k] B[k][j]
+    if (ROWS == 1 && d == 128) rows_times_staged_matrix<ROWS>(arow, B, d, j, out, bs);
+    else rows_times_matrix<ROWS>(arow, B, d, j, out);
+  };
   auto load_rows = [&](const float* M) {   // arow[r][:] = M[i0 + r][:]
     __syncthreads();
 #pragma unroll
@@ -300,6 +332,7 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
   for (int r = 0; r < ROWS; ++r) {
     rcur[r] = p.R[static_cast<long long>(i0 + r) * d + j];
     p.Rt[static_cast<long long>(j) * d + i0 + r] = rcur[r];
+    p.Rs[static_cast<long long>(i0 + r) * d + j] = rcur[r];
   }
   const float drift_in = p.sc->drift;  // (written only by the end of an earlier launch)
   float dr_own = 0.f;
@@ -328,7 +361,7 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
   } else {
     load_rows(p.dR);
   }
-  rows_times_matrix<ROWS>(arow, p.Rt, d, j, acc);
+  product(p.Rt, acc);
 #pragma unroll
   for (int r = 0; r < ROWS; ++r) p.A[static_cast<long long>(i0 + r) * d + j] = acc[r];
   grid.sync();
@@ -398,11 +431,11 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
   // R_new = R - alpha sum_k (-alpha/2)^k P_k,  P_0 = W R,  P_{k+1} = W P_k
   load_rows(p.W);
   {
-    const float* src = p.R;
+    const float* src = p.Rs;
     float* dst = p.P0;
     float ck = -alpha;
     for (int k = 0; k < n_terms; ++k) {
-      rows_times_matrix<ROWS>(arow, src, d, j, acc);
+      product(src, acc);
 #pragma unroll
       for (int r = 0; r < ROWS; ++r) {
         rcur[r] = fmaf(ck, acc[r], rcur[r]);
@@ -410,13 +443,13 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
       }
       ck *= -0.5f * alpha;
       if (k + 1 < n_terms) {
-        grid.sync();  // all rows of P_k written; (R itself is not read after the first product)
+        grid.sync();  // all rows of P_k written
         src = dst;
         dst = (dst == p.P0) ? p.P1 : p.P0;
       }
     }
   }
-  grid.sync();  // every CTA has finished reading R
+  // (no CTA reads R or R^T between the first barrier and the guard's: the products above read the copy)
 #pragma unroll
   for (int r = 0; r < ROWS; ++r) {
     p.R[static_cast<long long>(i0 + r) * d + j] = rcur[r];
@@ -428,7 +461,7 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
     grid.sync();
     // E = R^T R - I:  E[i][j] = sum_k Rt[i][k] R[k][j]
     load_rows(p.Rt);
-    rows_times_matrix<ROWS>(arow, p.R, d, j, acc);
+    product(p.R, acc);
     float mx = 0.f;
 #pragma unroll
     for (int r = 0; r < ROWS; ++r) {
@@ -450,7 +483,7 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
     if (max_e > p.polish_at) {  // same value in every CTA: the branch is grid-uniform
       // R <- R - R E / 2; each CTA reads only its own rows of R and all of E
       load_rows(p.R);
-      rows_times_matrix<ROWS>(arow, p.A, d, j, acc);
+      product(p.A, acc);
 #pragma unroll
       for (int r = 0; r < ROWS; ++r) {
         rcur[r] = fmaf(-0.5f, acc[r], rcur[r]);
