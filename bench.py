@@ -361,7 +361,8 @@ def main():
                   loss_mode=1 if args.loss_mode == "layer" else 0, rmsnorm=1 if args.rmsnorm else 0,
                   backward_mode={"stored": 0, "recompute": 1, "stored_f32": 2}[args.backward])
     ctx = kurtail.Context(dev, **ctx_kw)
-    fwd_terms = args.forward_terms if args.forward_terms in (1, 2) else (2 if d <= 512 else 1)
+    # (automatic: two bf16 terms of R for d <= 512, except that the single-pass d = 128 kernel takes one float16 term)
+    fwd_terms = args.forward_terms if args.forward_terms in (1, 2) else (2 if 128 < d <= 512 else 1)
 
     def fresh_R(c=ctx, dd=d, init=cfg["init"]):
         if init == "hadamard":

@@ -294,21 +294,22 @@ __global__ void k_grad_from_y(const float* __restrict__ Y, const float4* __restr
 
 // The same from the float16 Y (kt_config.backward_mode 0): Y16[t][j] = float16(Y[t][j] * 2^(140 - e)) with one
 // exponent byte e per row and run of `bn` columns, yexp[j / bn][t] (written by the forward GEMM's epilogue).
-// 16-byte loads: eight threads read the 64 columns of a row, the block's 256 threads 32 rows at a time.
+// Tiles of 128 tokens x 64 columns.  16-byte loads: eight threads read the 64 columns of a row, the block's 256
+// threads 32 rows at a time, four such loads in flight per thread.  grid (ceil(N/128), d/64), block 256.
 __global__ void k_grad_from_y16(const __half* __restrict__ Y, const unsigned char* __restrict__ yexp, int bn,
                                 const float4* __restrict__ coef, int N, int d, __nv_bfloat16* __restrict__ gt,
                                 long long ldg) {
   // [column][token]; columns 32..63 are shifted by two words so that the eight column groups a warp writes at once
   // fall into different banks
-  __shared__ __nv_bfloat16 tile[64][70];
-  const int r0 = blockIdx.x * 64, c0 = blockIdx.y * 64;
-  const int seg = threadIdx.x & 7, rr = threadIdx.x >> 3;  // 8 columns at c0 + 8 * seg of rows rr and rr + 32
+  __shared__ __nv_bfloat16 tile[64][134];
+  const int r0 = blockIdx.x * 128, c0 = blockIdx.y * 64;
+  const int seg = threadIdx.x & 7, rr = threadIdx.x >> 3;  // 8 columns at c0 + 8 * seg of rows rr + 32 q
   const unsigned char* ex = yexp + static_cast<long long>(c0 / bn) * N;
-  uint4 raw[2];
-  float4 cf[2];
-  float inv[2];
+  uint4 raw[4];
+  float4 cf[4];
+  float inv[4];
 #pragma unroll
-  for (int q = 0; q < 2; ++q) {
+  for (int q = 0; q < 4; ++q) {
     const int row = r0 + rr + 32 * q;
     const bool in = row < N;
     raw[q] = in ? *reinterpret_cast<const uint4*>(Y + static_cast<long long>(row) * d + c0 + 8 * seg)
@@ -318,14 +319,14 @@ __global__ void k_grad_from_y16(const __half* __restrict__ Y, const unsigned cha
     inv[q] = in ? __uint_as_float((static_cast<unsigned int>(ex[row]) - 13u) << 23) : 0.f;
   }
 #pragma unroll
-  for (int q = 0; q < 2; ++q) {
+  for (int q = 0; q < 4; ++q) {
     const uint32_t w[4] = {raw[q].x, raw[q].y, raw[q].z, raw[q].w};
+    const int tr = rr + 32 * q + 4 * (seg >> 2);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const float2 y2 = __half22float2(*reinterpret_cast<const __half2*>(&w[j]));
       const float ca = y2.x * inv[q] - cf[q].x, cb = y2.y * inv[q] - cf[q].x;
       // rows past N: y = 0 and zero coefficients give 0; they are not written anyway
-      const int tr = rr + 32 * q + 4 * (seg >> 2);
       tile[8 * seg + 2 * j][tr] = __float2bfloat16_rn(fmaf(ca, fmaf(cf[q].y * ca, ca, -cf[q].z), -cf[q].w));
       tile[8 * seg + 2 * j + 1][tr] = __float2bfloat16_rn(fmaf(cb, fmaf(cf[q].y * cb, cb, -cf[q].z), -cf[q].w));
     }
@@ -335,13 +336,17 @@ __global__ void k_grad_from_y16(const __half* __restrict__ Y, const unsigned cha
 #pragma unroll
   for (int q = 0; q < 8; ++q) {
     const int c = w + 8 * q;
-    const int t = r0 + 2 * lane;
-    __nv_bfloat16* dst = gt + static_cast<long long>(c0 + c) * ldg + t;
-    if (t + 1 < N) {
-      *reinterpret_cast<__nv_bfloat162*>(dst) =
-          *reinterpret_cast<const __nv_bfloat162*>(&tile[c][2 * lane + 4 * (c >> 5)]);
-    } else if (t < N) {
-      dst[0] = tile[c][2 * lane + 4 * (c >> 5)];
+    __nv_bfloat16* dst_row = gt + static_cast<long long>(c0 + c) * ldg;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {   // two runs of 64 tokens: 128 contiguous bytes per warp and store
+      const int tl = 64 * h + 2 * lane;
+      const int t = r0 + tl;
+      if (t + 1 < N) {
+        *reinterpret_cast<__nv_bfloat162*>(dst_row + t) =
+            *reinterpret_cast<const __nv_bfloat162*>(&tile[c][tl + 4 * (c >> 5)]);
+      } else if (t < N) {
+        dst_row[t] = tile[c][tl + 4 * (c >> 5)];
+      }
     }
   }
 }

@@ -620,7 +620,7 @@ static kt_status backward(kt_ctx* ctx, const XView& xv, int N, int d, const WsLa
                                                  at<__nv_bfloat16>(ctx, L.gt), L.ldt);
     KT_LAUNCH_CHECK();
   } else if (keep_y_for_backward(ctx)) {
-    dim3 grid((N + 63) / 64, d / 64);
+    dim3 grid((N + 127) / 128, d / 64);
     k_grad_from_y16<<<grid, 256, 0, ctx->stream>>>(at<__half>(ctx, L.ybuf), at<unsigned char>(ctx, L.yexp), L.bn,
                                                    at<float4>(ctx, L.coef), N, d, at<__nv_bfloat16>(ctx, L.gt),
                                                    L.ldt);

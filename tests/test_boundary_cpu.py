@@ -114,3 +114,26 @@ def test_bench_reference_arm_prints_the_contract_line():
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
     assert line["config"]["workload"] == "tiny" and line["higher_is_better"] is True
+
+
+def test_bench_quotes_dram_counters_only_for_the_kernel_they_were_taken_from(tmp_path, monkeypatch):
+    # profiles/dram_traffic.txt carries a fingerprint of the kernel's source files with every line: counters taken
+    # from an older kernel are not quoted (the bench line then says traffic: null)
+    import importlib.util
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    spec = importlib.util.spec_from_file_location("bench_mod", os.path.join(root, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    now = bench.kernel_source_hash("gemm_tn_kernel")
+    fake_root = tmp_path
+    (fake_root / "profiles").mkdir()
+    (fake_root / "paper_2503_01483_b200").symlink_to(os.path.join(root, "paper_2503_01483_b200"))
+    (fake_root / "profiles" / "dram_traffic.txt").write_text(
+        "# kernel role rows d bytes_read bytes_write fixed_bytes source_hash\n"
+        "gemm_tn_kernel backward_b 1000 4096 5000000 1000000 2000000 %s\n"
+        "gemm_tn_kernel forward 1000 4096 5000000 1000000 2000000 0123456789abcdef\n" % now)
+    monkeypatch.setattr(bench, "ROOT", str(fake_root))
+    per_row, fixed = bench.recorded_traffic("gemm_tn_kernel", "backward_b")
+    assert per_row == pytest.approx(4000.0) and fixed == 2000000.0
+    assert bench.recorded_traffic("gemm_tn_kernel", "forward") is None        # stale fingerprint
+    assert bench.recorded_traffic("fused_small_kernel", "terms1") is None     # no line at all
