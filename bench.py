@@ -398,9 +398,11 @@ def main():
         return ctx.fit(X, R, steps, lr)
 
     sweep_Rs = [R]
-    one_fit(max(args.warmup, 1))          # warm-up steps (also sizes the workspace)
     if sweep:
+        ctx.fit(X, fresh_R(), max(args.warmup, 1), lr)   # warm-up steps on the first layer (also sizes the workspace)
         sweep_Rs = [R] + [fresh_R() for _ in Xs[1:]]
+    else:
+        one_fit(max(args.warmup, 1))      # warm-up steps (also sizes the workspace)
     torch.cuda.synchronize()
 
     sampler = ClockSampler(local_rank)

@@ -257,7 +257,11 @@ kt_status kt_rotate(kt_ctx* ctx, kt_mat X, const float* R, float* Y);
  * Y_s = R - alpha sum_{k<=s} (-alpha/2)^k W^k (W R).  Built from d x d
  * tensor-core products only.  R is updated in place, one series term per
  * kernel; dR is read only.  Uses the workspace (sized for any N >= 1 and this
- * d).  Stream ordered. */
+ * d).  Stream ordered.
+ * d <= 512 with kt_config.small_d_orth (the default): the whole step is one
+ * cooperative launch of 128 CTAs in float32 on the CUDA cores instead; all
+ * 128 CTAs must be resident at once (a device with at least 128 free SMs),
+ * else the call returns KT_ERR_COOPERATIVE and R is untouched. */
 kt_status kt_orth_step(kt_ctx* ctx, float* R, const float* dR, int64_t d, float lr);
 
 /* Cayley Adam (Section 3, "Optimization in the Orthogonal Space", names it as

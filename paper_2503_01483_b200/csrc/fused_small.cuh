@@ -34,18 +34,18 @@
 namespace kt {
 
 constexpr int kFsD = 128;          // channels = rows of a token tile
-constexpr int kFsThreads = 320;    // warp 0: TMA, warp 1: MMA, warps 2..5 and 6..9: two epilogue groups
-#ifndef KT_FS_STAGES
-#define KT_FS_STAGES 4
-#endif
-constexpr int kFsXStages = KT_FS_STAGES;   // X tiles in shared memory (4 is what fits beside R^T and the G tiles)
+constexpr int kFsThreads = 352;    // warp 0: TMA, warp 1: MMA1, warps 2..5 and 6..9: two epilogue groups, warp 10: MMA2
+constexpr int kFsMma2Warp = 10;
 constexpr int kFsHalf = 128 * 64 * 2;      // bytes of one 128-row x 64-element swizzled block
 constexpr int kFsTile = 2 * kFsHalf;       // one 128 x 128 bf16 tile
-// TERMS = 1: R^T hi only, which leaves room for a second G tile; TERMS = 2: R^T hi + lo and one G tile.
+// Shared memory: R^T (hi, and lo when TERMS == 2), four X stages, and the G tiles: one per epilogue group with
+// one term, a single one with two.  (Measured with one term: five X stages and a single G tile are 8 % slower
+// than four and two, because a group's G stores then wait for MMA2 of the other group's tile.)
 template <int TERMS>
 struct FusedCfg {
+  static constexpr int kStages = 4;
   static constexpr int kGBufs = (TERMS == 1) ? 2 : 1;
-  static constexpr int kSmem = 1024 + TERMS * kFsTile /*R^T*/ + kFsXStages * kFsTile + kGBufs * kFsTile /*G*/ + 256;
+  static constexpr int kSmem = 1024 + TERMS * kFsTile /*R^T*/ + kStages * kFsTile + kGBufs * kFsTile /*G*/ + 384;
 };
 
 struct FusedParams {
@@ -82,6 +82,7 @@ __device__ __forceinline__ uint64_t umma_desc_mnmajor_sw128(uint32_t smem_addr, 
 template <int TERMS>
 __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid_constant__ FusedParams p) {
   constexpr int kGBufs = FusedCfg<TERMS>::kGBufs;
+  constexpr int kFsXStages = FusedCfg<TERMS>::kStages;
   // every operand of this kernel is float16 (see the note on the encoding of X at the top of this file)
   constexpr uint32_t kIdescK = umma_idesc_f16_f32(128, 128);                            // both K-major
   constexpr uint32_t kIdescMN = umma_idesc_f16_f32(128, 128) | (1u << 15) | (1u << 16);  // both MN-major
@@ -107,10 +108,11 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
   const uint32_t r_full = bars + 8u * (2 * kFsXStages + 8);
   const uint32_t dr_full = bars + 8u * (2 * kFsXStages + 9);
   uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gbase + (bars - base) + 152);
+  // (the barriers take 8 * (2 * kFsXStages + 10) <= 160 bytes)
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gbase + (bars - base) + 160);
   volatile uint32_t* abort_flag = tmem_slot + 1;
-  double* sh_loss = reinterpret_cast<double*>(gbase + (bars - base) + 160);             // 8 doubles
-  unsigned int* sh_deg = reinterpret_cast<unsigned int*>(gbase + (bars - base) + 224);  // 8 words
+  double* sh_loss = reinterpret_cast<double*>(gbase + (bars - base) + 168);             // 8 doubles
+  unsigned int* sh_deg = reinterpret_cast<unsigned int*>(gbase + (bars - base) + 232);  // 8 words
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -169,7 +171,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
       for (int n = 0; n < my_tiles; ++n) {
         const int s = n % kFsXStages;
         const uint32_t ph = (n / kFsXStages) & 1;
-        if (!mbar_wait_bounded(x_empty(s), ph ^ 1u, abort_flag, 11u, p.wait_limit_ns)) {
+        if (!mbar_poll_bounded(x_empty(s), ph ^ 1u, abort_flag, 11u, p.wait_limit_ns)) {
           ok = false;
           break;
         }
@@ -192,76 +194,64 @@ __global__ void __launch_bounds__(kFsThreads, 1) fused_small_kernel(const __grid
       }
     }
   } else if (warp == 1) {
-    // -------------------------------------------------------------- MMA issuer
+    // -------------------------------------------------------------- MMA issuer, first stream
+    // MMA1 stream: Y(n) = X(n) Rc as soon as tile n is in shared memory and its Y accumulator has been read out.
+    // (MMA2 has a warp of its own, below: one thread feeding both streams is blocked in the issue of one while the
+    // other's barrier completes -- measured: 680 cycles from "G written" to the first MMA2, with the tile's
+    // shared-memory stage held all the while.)
     if (lane == 0 && my_tiles > 0) {
       bool ok = mbar_wait_bounded(r_full, 0u, abort_flag, 12u, p.wait_limit_ns);
-      const uint32_t acc_dr = tmem_base + kColDr;
-      // Two instruction streams share this thread: MMA1 of tile n1 can go as soon as the tile is in shared memory and
-      // its Y accumulator has been read out, MMA2 of tile n2 as soon as the epilogue has written that tile's G.
-      // Whichever is ready is issued (MMA2 first: it frees a shared-memory stage); neither waits for the other's turn.
-      int n1 = 0, n2 = 0;
-      uint64_t idle_since = 0;
-      uint32_t spins = 0;
-      while (n2 < my_tiles && ok) {
-        bool progressed = false;
-        if (n2 < n1 && mbar_test_wait(g_full(n2 & 1), (n2 >> 1) & 1)) {
-          // dR += X(m)^T G(m): contraction over the tile's 128 tokens, 16 per MMA = two 8-row groups
-          const int m = n2;
-          const int s = m % kFsXStages;
-          tc_fence_after_sync();
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            const uint64_t a_desc = umma_desc_mnmajor_sw128(s_x + s * kFsTile + ks * 2048, kFsHalf, 1024);
-            const uint64_t b_desc =
-                umma_desc_mnmajor_sw128(s_g + (kGBufs == 2 ? (m & 1) * kFsTile : 0) + ks * 2048, kFsHalf, 1024);
-            tc_mma_bf16(acc_dr, a_desc, b_desc, kIdescMN, (m > 0 || ks > 0) ? 1u : 0u);
-          }
-          tc_commit(x_empty(s));      // the X tile is free once these MMAs have read it
-          tc_commit(g_empty(m & 1));  // and so is the G tile
-          ++n2;
-          progressed = true;
+      for (int n = 0; n < my_tiles && ok; ++n) {
+        const int s = n % kFsXStages;
+        const int b = n & 1;
+        if (!mbar_poll_bounded(y_empty(b), ((n >> 1) & 1) ^ 1u, abort_flag, 13u, p.wait_limit_ns) ||
+            !mbar_poll_bounded(x_full(s), (n / kFsXStages) & 1, abort_flag, 13u, p.wait_limit_ns)) {
+          ok = false;
+          break;
         }
-        if (n1 < my_tiles) {
-          // Y(n) = X(n) Rc
-          const int n = n1;
-          const int s = n % kFsXStages;
-          const int b = n & 1;
-          if (mbar_test_wait(x_full(s), (n / kFsXStages) & 1) && mbar_test_wait(y_empty(b), ((n >> 1) & 1) ^ 1u)) {
-            tc_fence_after_sync();
-            const uint32_t acc_y = tmem_base + static_cast<uint32_t>(b * 128);
-            uint32_t first = 1;
+        tc_fence_after_sync();
+        const uint32_t acc_y = tmem_base + static_cast<uint32_t>(b * 128);
+        uint32_t first = 1;
 #pragma unroll
-            for (int q = 0; q < TERMS; ++q) {
-              const uint32_t rb = (q == 0) ? s_rhi : s_rlo;
+        for (int q = 0; q < TERMS; ++q) {
+          const uint32_t rb = (q == 0) ? s_rhi : s_rlo;
 #pragma unroll
-              for (int kb = 0; kb < 2; ++kb) {
-                const uint64_t a_desc = umma_desc_kmajor_sw128(s_x + s * kFsTile + kb * kFsHalf, 1024);
-                const uint64_t b_desc = umma_desc_kmajor_sw128(rb + kb * kFsHalf, 1024);
+          for (int kb = 0; kb < 2; ++kb) {
+            const uint64_t a_desc = umma_desc_kmajor_sw128(s_x + s * kFsTile + kb * kFsHalf, 1024);
+            const uint64_t b_desc = umma_desc_kmajor_sw128(rb + kb * kFsHalf, 1024);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                  tc_mma_bf16(acc_y, a_desc + 2u * kk, b_desc + 2u * kk, kIdescK, first ? 0u : 1u);
-                  first = 0;
-                }
-              }
+            for (int kk = 0; kk < 4; ++kk) {
+              tc_mma_bf16(acc_y, a_desc + 2u * kk, b_desc + 2u * kk, kIdescK, first ? 0u : 1u);
+              first = 0;
             }
-            tc_commit(y_full(b));
-            ++n1;
-            progressed = true;
           }
         }
-        // bounded like every other wait: no progress for the limit's length ends the kernel with an error code
-        if (progressed) {
-          spins = 0;
-        } else if ((++spins & 63u) == 0) {
-          if (*abort_flag) {
-            ok = false;
-          } else if (spins == 64u) {
-            idle_since = global_timer_ns();
-          } else if (global_timer_ns() - idle_since > p.wait_limit_ns) {
-            *abort_flag = 13u;
-            ok = false;
-          }
+        tc_commit(y_full(b));
+      }
+    }
+  } else if (warp == kFsMma2Warp) {
+    // -------------------------------------------------------------- MMA issuer, second stream
+    // dR += X(m)^T G(m) as soon as the epilogue has written that tile's G: contraction over the tile's 128 tokens,
+    // 16 per MMA = two 8-row groups.
+    if (lane == 0 && my_tiles > 0) {
+      const uint32_t acc_dr = tmem_base + kColDr;
+      bool ok = true;
+      for (int m = 0; m < my_tiles && ok; ++m) {
+        const int s = m % kFsXStages;
+        if (!mbar_poll_bounded(g_full(m & 1), (m >> 1) & 1, abort_flag, 14u, p.wait_limit_ns)) {
+          ok = false;
+          break;
         }
+        tc_fence_after_sync();
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint64_t a_desc = umma_desc_mnmajor_sw128(s_x + s * kFsTile + ks * 2048, kFsHalf, 1024);
+          const uint64_t b_desc =
+              umma_desc_mnmajor_sw128(s_g + (kGBufs == 2 ? (m & 1) * kFsTile : 0) + ks * 2048, kFsHalf, 1024);
+          tc_mma_bf16(acc_dr, a_desc, b_desc, kIdescMN, (m > 0 || ks > 0) ? 1u : 0u);
+        }
+        tc_commit(x_empty(s));      // the X tile is free once these MMAs have read it
+        tc_commit(g_empty(m & 1));  // and so is the G tile
       }
       if (ok) tc_commit(dr_full);
     }

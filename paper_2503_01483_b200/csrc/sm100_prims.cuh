@@ -47,22 +47,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// The same question without any waiting: try_wait may park the thread for a while when the phase is not complete,
-// test_wait answers at once (for a thread that polls several barriers in turn).
-__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n"
-      ".reg .pred p;\n"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n"
-      "}\n"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-
 // Wait with a bound.  Gives up after `limit_ns` of wall time (kernels take it from
 // their parameters; kDefaultWaitLimitNs unless the caller configured another), or
 // as soon as another thread of the CTA has raised *abort_flag; on giving up it
@@ -79,6 +63,40 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 63u) == 0) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > limit_ns) {
+        *abort_flag = where;
+        return false;
+      }
+    }
+  }
+}
+
+// The same wait by polling: mbarrier.try_wait may suspend the thread for a while when the phase is not complete,
+// and waking it up again is then on the critical path; test_wait answers at once.  For the single threads that
+// feed a pipeline (TMA producer, MMA issuers), which have nothing else to do and no warp to share a scheduler slot
+// with.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_poll_bounded(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                                  uint32_t where, uint64_t limit_ns) {
+  if (mbar_test_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  uint32_t spins = 0;
+  while (true) {
+    if (mbar_test_wait(bar, parity)) return true;
+    if ((++spins & 255u) == 0) {
       if (*abort_flag) return false;
       if (global_timer_ns() - t0 > limit_ns) {
         *abort_flag = where;
