@@ -381,12 +381,22 @@ kt_status kt_quant4_error(kt_ctx* ctx, kt_mat X, const float* R, double* mse);
  *   Q(y) = clamp(round_half_even((y - b) / s), lo, hi) * s + b;  s == 0 -> Q(y) = b.
  * `clip` in (0, 1] shrinks the range towards zero before the step is formed
  * ("Setup" clips activations; 1 = no clipping, the definition of Section 2).
- * All decisions in IEEE float32.  {4, 0, 1.0} is kt_quant4_error. */
+ * "Setup" words the clipping of activations as "a quantile of 0.98", which can
+ * be read two ways; both are here.  clip_mode 0: `clip` is a ratio, as above.
+ * clip_mode 1 (symmetric only): `clip` is a quantile level and the range is the
+ * clip-quantile of the row's |y| -- with the d magnitudes sorted,
+ * a[0] <= ... <= a[d-1], and h = clip (d - 1) = k + t (k integer, 0 <= t < 1),
+ * range = a[k] + t (a[k+1] - a[k]); entries beyond it saturate.  The order
+ * statistic is exact (a selection on the float32 bit patterns), the
+ * interpolation is float32.  A quantile needs a whole row of Y at once, so
+ * this mode works on a given Y (kt_quant_codes, kt_quant_error_given), not
+ * inside the GEMM passes of kt_quant_error (KT_ERR_INVALID_ARG there).
+ * All decisions in IEEE float32.  {4, 0, 1.0, 0} is kt_quant4_error. */
 typedef struct {
   int32_t bits;       /* 2..8 */
   int32_t asymmetric; /* 0 or 1 */
   float clip;         /* (0, 1] */
-  int32_t reserved;
+  int32_t clip_mode;  /* 0 = ratio of the row's range, 1 = quantile level of |y| */
 } kt_quant_spec;
 
 /* *mse (host) = mean over all N*d entries of (Y - Q(Y))^2, Y = X R recomputed in
@@ -399,6 +409,14 @@ kt_status kt_quant_error(kt_ctx* ctx, kt_mat X, const float* R, const kt_quant_s
  * No workspace needed.  Stream ordered. */
 kt_status kt_quant_codes(kt_ctx* ctx, const float* Y, int64_t N, int64_t d, const kt_quant_spec* spec,
                          int16_t* codes, float* scales, float* shifts);
+
+/* *mse (host) = mean over all N*d entries of (Y - Q(Y))^2 for a given float32 Y
+ * (N x d dense, device; e.g. from kt_rotate), any `spec` including clip_mode 1
+ * (Section 2, Eq. 1 with the quantizer of "Setup").  One block per row, then a
+ * fixed-order sum; uses the first N*8 bytes of the workspace
+ * (KT_ERR_WORKSPACE if it is smaller).  Synchronises. */
+kt_status kt_quant_error_given(kt_ctx* ctx, const float* Y, int64_t N, int64_t d, const kt_quant_spec* spec,
+                               double* mse);
 
 /* Success rate of Section 3 (the comparison of per-token maxima): *rate (host) =
  * the fraction of tokens t with max_j |(X R_a)_tj| < max_j |(X R_b)_tj|.  R_b may

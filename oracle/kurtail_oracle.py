@@ -351,16 +351,37 @@ def quant4_error(Y32):
     return float((diff * diff).sum() / Y.size)
 
 
-def quant_codes(Y32, bits=4, asymmetric=False, clip=1.0):
+def row_abs_quantile(Y32, level):
+    """Per row, the `level`-quantile of |y| with linear interpolation between
+    order statistics: sort the n magnitudes, h = level*(n-1), lo = floor(h),
+    value = a[lo] + (h - lo)*(a[lo+1] - a[lo]).  The position is taken in
+    float64, the interpolation in float32.  (Section 4, "Setup": activations are
+    "clipped using a quantile of 0.98", read as a per-token quantile of the
+    magnitudes.)"""
+    A = np.sort(np.abs(np.asarray(Y32, dtype=np.float32)), axis=1)
+    n = A.shape[1]
+    h = float(level) * (n - 1)
+    lo = int(np.floor(h))
+    hi = min(lo + 1, n - 1)
+    t = np.float32(h - lo)
+    a0, a1 = A[:, lo], A[:, hi]
+    return (a0 + (t * (a1 - a0).astype(np.float32)).astype(np.float32)).astype(np.float32)
+
+
+def quant_codes(Y32, bits=4, asymmetric=False, clip=1.0, clip_quantile=False):
     """The k-bit quantizer of Section 2, "Uniform Quantization for k-bit
     Precision", per row, in float32 throughout:
       symmetric:  b = 0, s = clip*max|y| / (2^(k-1) - 1), codes in [-(2^(k-1)-1), 2^(k-1)-1];
       asymmetric: b = clip*min(y), s = (clip*max(y) - b) / (2^k - 1), codes in [0, 2^k - 1];
       code = clamp(rint((y - b) / s), lo, hi), ties to even; s == 0 gives code 0.
     `clip` in (0, 1] shrinks the range towards zero (Section 4, "Setup" clips
-    activations).  Returns (codes int16 N x n, s float32 N, b float32 N)."""
+    activations).  clip_quantile (symmetric only): the range is not clip*max|y|
+    but the clip-quantile of the row's |y| (row_abs_quantile); larger entries
+    saturate.  Returns (codes int16 N x n, s float32 N, b float32 N)."""
     Y = np.asarray(Y32, dtype=np.float32)
     c = np.float32(clip)
+    if clip_quantile and asymmetric:
+        raise ValueError("quantile clipping is defined for the symmetric quantizer only")
     if asymmetric:
         den = np.float32(2 ** bits - 1)
         lo, hi = np.float32(0.0), den
@@ -370,7 +391,7 @@ def quant_codes(Y32, bits=4, asymmetric=False, clip=1.0):
         den = np.float32(2 ** (bits - 1) - 1)
         lo, hi = -den, den
         b = np.zeros(Y.shape[0], dtype=np.float32)
-        rng = (c * np.abs(Y).max(axis=1)).astype(np.float32)
+        rng = row_abs_quantile(Y, clip) if clip_quantile else (c * np.abs(Y).max(axis=1)).astype(np.float32)
     s = (rng / den).astype(np.float32)
     safe = np.where(s == 0, np.float32(1.0), s).astype(np.float32)
     q = np.rint(((Y - b[:, None]).astype(np.float32) / safe[:, None]).astype(np.float32))
@@ -379,11 +400,11 @@ def quant_codes(Y32, bits=4, asymmetric=False, clip=1.0):
     return q.astype(np.int16), s, b
 
 
-def quant_error(Y32, bits=4, asymmetric=False, clip=1.0):
+def quant_error(Y32, bits=4, asymmetric=False, clip=1.0, clip_quantile=False):
     """Eq. 1 for quant_codes: mean (Y - Q(Y))^2 with Q(Y) = code*s + b formed in
     float32, the difference and the sum in float64."""
     Y = np.asarray(Y32, dtype=np.float32)
-    codes, s, b = quant_codes(Y, bits, asymmetric, clip)
+    codes, s, b = quant_codes(Y, bits, asymmetric, clip, clip_quantile)
     deq = ((codes.astype(np.float32) * s[:, None]).astype(np.float32) + b[:, None]).astype(np.float32)
     diff = Y.astype(np.float64) - deq.astype(np.float64)
     return float((diff * diff).sum() / Y.size)

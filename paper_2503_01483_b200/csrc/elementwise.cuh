@@ -1124,14 +1124,88 @@ __global__ void k_quant4_codes(const float* __restrict__ Y, int d, int8_t* __res
   }
 }
 
+// The `level`-quantile of the magnitudes of one row (d float32 values), by the whole block (256 threads), exactly:
+// with the magnitudes sorted, a[0] <= ... <= a[d-1], the result is a[k0] + t (a[k0 + 1] - a[k0]) in float32, where
+// k0 = floor(level (d - 1)) and t = level (d - 1) - k0 are given by the host (Section 4, "Setup": activations are
+// "clipped using a quantile of 0.98").  The order statistic is found by a radix select on the magnitudes' bit
+// patterns (which order like the values): four passes over the row, each fixing 8 (the last: 7) more bits of a[k0]
+// from a 256-bin histogram of the candidates left; a fifth pass counts the entries <= a[k0] and finds the smallest
+// larger one, which is a[k0 + 1] unless a[k0] occurs again.  `hist` (256 words) and `sel` (4 words) are shared
+// memory.  Every thread returns the same value.
+__device__ float row_abs_quantile(const float* __restrict__ y, int d, int k0, float t, unsigned int* hist,
+                                  unsigned int* sel) {
+  unsigned int prefix = 0u, mask = 0u, rank = static_cast<unsigned int>(k0);
+#pragma unroll 1
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 23 - 8 * pass < 0 ? 0 : 23 - 8 * pass;   // 23, 15, 7, 0
+    const unsigned int width = pass == 3 ? 0x7fu : 0xffu;
+    hist[threadIdx.x] = 0u;
+    __syncthreads();
+    for (int j = threadIdx.x; j < d; j += 256) {
+      const unsigned int key = __float_as_uint(y[j]) & 0x7fffffffu;
+      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & width], 1u);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      unsigned int cum = 0u, b = 0u;
+      for (; b < width; ++b) {           // (the last bin takes whatever is left)
+        if (cum + hist[b] > rank) break;
+        cum += hist[b];
+      }
+      sel[0] = b;
+      sel[1] = rank - cum;
+    }
+    __syncthreads();
+    prefix |= sel[0] << shift;
+    mask |= width << shift;
+    rank = sel[1];
+    __syncthreads();
+  }
+  // prefix = bits of a[k0]; a[k0 + 1]
+  unsigned int le = 0u, next = 0x7fffffffu;
+  for (int j = threadIdx.x; j < d; j += 256) {
+    const unsigned int key = __float_as_uint(y[j]) & 0x7fffffffu;
+    if (key <= prefix) ++le;
+    else next = key < next ? key : next;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    le += __shfl_xor_sync(0xffffffffu, le, o);
+    const unsigned int other = __shfl_xor_sync(0xffffffffu, next, o);
+    next = other < next ? other : next;
+  }
+  if ((threadIdx.x & 31) == 0) {
+    hist[threadIdx.x >> 5] = le;
+    hist[8 + (threadIdx.x >> 5)] = next;
+  }
+  __syncthreads();
+  le = 0u;
+  next = 0x7fffffffu;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    le += hist[i];
+    next = hist[8 + i] < next ? hist[8 + i] : next;
+  }
+  __syncthreads();
+  const float a0 = __uint_as_float(prefix);
+  const float a1 = (le >= static_cast<unsigned int>(k0) + 2u || k0 + 1 >= d) ? a0 : __uint_as_float(next);
+  return __fadd_rn(a0, __fmul_rn(t, __fsub_rn(a1, a0)));
+}
+
 // The general k-bit quantizer of Section 2 on a dense float32 Y (N x d), one block per row:
 //   symmetric:  s = clip * max|Y_t| / (2^(k-1) - 1), b = 0,            codes in [-(2^(k-1) - 1), 2^(k-1) - 1]
 //   asymmetric: b = clip * min Y_t, s = (clip * max Y_t - b) / (2^k - 1), codes in [0, 2^k - 1]
 //   code = clamp(rint((y - b) / s), lo, hi); s == 0 -> code 0.  All in IEEE float32, ties to even.
+// q_k0 >= 0: the symmetric quantizer's range is the quantile a[q_k0] + q_t (a[q_k0 + 1] - a[q_k0]) of the row's
+// magnitudes instead of clip * max|Y_t| (see row_abs_quantile); larger entries saturate.
+// err != null: instead of writing codes, the row's sum of (y - Q(y))^2 goes to err[row] (float64; Q(y) = code s + b
+// formed in float32).
 __global__ void k_quant_codes(const float* __restrict__ Y, int d, int asym, float clip, float den, float lo,
                               float hi, short* __restrict__ codes, float* __restrict__ scales,
-                              float* __restrict__ shifts) {
+                              float* __restrict__ shifts, int q_k0, float q_t, double* __restrict__ err) {
   __shared__ float shx[8], shn[8];
+  __shared__ unsigned int hist[256], sel[4];
+  __shared__ double she[8];
   const long long base = static_cast<long long>(blockIdx.x) * d;
   float mx = asym ? -INFINITY : 0.f, mn = INFINITY;
   for (int j = threadIdx.x; j < d; j += 256) {
@@ -1160,21 +1234,40 @@ __global__ void k_quant_codes(const float* __restrict__ Y, int d, int asym, floa
   if (asym) {
     b = __fmul_rn(clip, mn);
     range = __fsub_rn(__fmul_rn(clip, mx), b);
+  } else if (q_k0 >= 0) {
+    range = row_abs_quantile(Y + base, d, q_k0, q_t, hist, sel);
   } else {
     range = __fmul_rn(clip, mx);
   }
   const float s = __fdiv_rn(range, den);
-  if (threadIdx.x == 0) {
+  if (threadIdx.x == 0 && scales != nullptr) {
     scales[blockIdx.x] = s;
     shifts[blockIdx.x] = b;
   }
+  double e2 = 0.0;
   for (int j = threadIdx.x; j < d; j += 256) {
+    const float y = Y[base + j];
     float qv = 0.f;
     if (s > 0.f) {
-      qv = rintf(__fdiv_rn(__fsub_rn(Y[base + j], b), s));
+      qv = rintf(__fdiv_rn(__fsub_rn(y, b), s));
       qv = fminf(fmaxf(qv, lo), hi);
     }
-    codes[base + j] = static_cast<short>(qv);
+    if (err != nullptr) {
+      const double df = static_cast<double>(y) - static_cast<double>(__fadd_rn(__fmul_rn(qv, s), b));
+      e2 += df * df;
+    } else {
+      codes[base + j] = static_cast<short>(qv);
+    }
+  }
+  if (err != nullptr) {   // fixed order: lanes by shuffle tree, then the eight warps
+    e2 = warp_sum(e2);
+    if ((threadIdx.x & 31) == 0) she[threadIdx.x >> 5] = e2;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      double t = 0.0;
+      for (int i = 0; i < 8; ++i) t += she[i];
+      err[blockIdx.x] = t;
+    }
   }
 }
 

@@ -1565,7 +1565,8 @@ struct QuantLevels {
 static kt_status quant_levels(const kt_quant_spec* spec, QuantLevels* q) {
   if (!spec) return KT_ERR_INVALID_ARG;
   if (spec->bits < 2 || spec->bits > 8 || (spec->asymmetric != 0 && spec->asymmetric != 1) ||
-      !(spec->clip > 0.f && spec->clip <= 1.f))
+      !(spec->clip > 0.f && spec->clip <= 1.f) || (spec->clip_mode != 0 && spec->clip_mode != 1) ||
+      (spec->clip_mode == 1 && spec->asymmetric != 0))
     return KT_ERR_INVALID_ARG;
   if (spec->asymmetric) {
     q->den = static_cast<float>((1 << spec->bits) - 1);
@@ -1579,10 +1580,22 @@ static kt_status quant_levels(const kt_quant_spec* spec, QuantLevels* q) {
   return KT_OK;
 }
 
+// clip_mode 1: position of the clip-quantile among the d sorted magnitudes of a row, h = clip (d - 1) = k0 + t.
+static void quantile_position(const kt_quant_spec* spec, int64_t d, int* k0, float* t) {
+  *k0 = -1;
+  *t = 0.f;
+  if (spec->clip_mode != 1) return;
+  const double h = static_cast<double>(spec->clip) * static_cast<double>(d - 1);
+  const double fl = floor(h);
+  *k0 = static_cast<int>(fl);
+  *t = static_cast<float>(h - fl);
+}
+
 kt_status kt_quant_error(kt_ctx* ctx, kt_mat X, const float* R, const kt_quant_spec* spec, double* mse) {
   if (!ctx || !R || !mse) return KT_ERR_INVALID_ARG;
   QuantLevels q;
   KT_TRY(quant_levels(spec, &q));
+  if (spec->clip_mode != 0) return KT_ERR_INVALID_ARG;  // a quantile needs the whole row: kt_quant_error_given
   int64_t N64, d64;
   KT_TRY(check_x(X, &N64, &d64));
   if (!aligned16(R)) return KT_ERR_ALIGN;
@@ -1632,7 +1645,7 @@ kt_status kt_quant4_error(kt_ctx* ctx, kt_mat X, const float* R, double* mse) {
   spec.bits = 4;
   spec.asymmetric = 0;
   spec.clip = 1.0f;
-  spec.reserved = 0;
+  spec.clip_mode = 0;
   return kt_quant_error(ctx, X, R, &spec, mse);
 }
 
@@ -1642,11 +1655,38 @@ kt_status kt_quant_codes(kt_ctx* ctx, const float* Y, int64_t N, int64_t d, cons
   QuantLevels q;
   KT_TRY(quant_levels(spec, &q));
   if (N < 1 || d < 1 || N > 0x7fffffffll || d > 0x7fffffffll) return KT_ERR_SHAPE;
+  int k0;
+  float t;
+  quantile_position(spec, d, &k0, &t);
   k_quant_codes<<<static_cast<unsigned>(N), 256, 0, ctx->stream>>>(Y, static_cast<int>(d), spec->asymmetric,
                                                                    spec->clip, q.den, q.lo, q.hi, codes, scales,
-                                                                   shifts);
+                                                                   shifts, k0, t, nullptr);
   KT_LAUNCH_CHECK();
   return KT_OK;
+}
+
+kt_status kt_quant_error_given(kt_ctx* ctx, const float* Y, int64_t N, int64_t d, const kt_quant_spec* spec,
+                               double* mse) {
+  if (!ctx || !Y || !mse) return KT_ERR_INVALID_ARG;
+  QuantLevels q;
+  KT_TRY(quant_levels(spec, &q));
+  if (N < 1 || d < 1 || N > 0x7fffffffll || d > 0x7fffffffll) return KT_ERR_SHAPE;
+  // one double per row, then a fixed-order sum: the workspace must hold N doubles
+  if (ctx->ws == nullptr || ctx->ws_bytes < static_cast<size_t>(N) * 8) return KT_ERR_WORKSPACE;
+  double* row_err = reinterpret_cast<double*>(ctx->ws);
+  int k0;
+  float t;
+  quantile_position(spec, d, &k0, &t);
+  k_quant_codes<<<static_cast<unsigned>(N), 256, 0, ctx->stream>>>(Y, static_cast<int>(d), spec->asymmetric,
+                                                                   spec->clip, q.den, q.lo, q.hi, nullptr, nullptr,
+                                                                   nullptr, k0, t, row_err);
+  KT_LAUNCH_CHECK();
+  k_final_sum<<<1, 256, 0, ctx->stream>>>(row_err, static_cast<int>(N), 1.0 / (static_cast<double>(N) * d),
+                                          &ctx->d_blk->sc.qmse, nullptr, nullptr, nullptr);
+  KT_LAUNCH_CHECK();
+  KT_TRY(sync_scalars(ctx));
+  *mse = ctx->h_blk->sc.qmse;
+  return isfinite(*mse) ? KT_OK : KT_ERR_NONFINITE;
 }
 
 kt_status kt_rowmax_success(kt_ctx* ctx, kt_mat X, const float* R_a, const float* R_b, double* rate) {

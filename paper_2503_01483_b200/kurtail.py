@@ -43,7 +43,7 @@ class kt_config(C.Structure):
 
 
 class kt_quant_spec(C.Structure):
-    _fields_ = [("bits", C.c_int32), ("asymmetric", C.c_int32), ("clip", C.c_float), ("reserved", C.c_int32)]
+    _fields_ = [("bits", C.c_int32), ("asymmetric", C.c_int32), ("clip", C.c_float), ("clip_mode", C.c_int32)]
 
 
 class kt_adam_state(C.Structure):
@@ -66,7 +66,8 @@ EXPORTS = ["kt_default_config", "kt_create", "kt_destroy", "kt_status_string", "
            "kt_rotate", "kt_orth_step", "kt_adam_step", "kt_orth_error", "kt_fit", "kt_fit_layers",
            "kt_fit_shared_workspace_bytes", "kt_fit_shared", "kt_fit_host", "kt_fit_sharded", "kt_fit_shared_sharded",
            "kt_test_wait_timeout",
-           "kt_quant4_error", "kt_quant4_codes", "kt_quant_error", "kt_quant_codes", "kt_rowmax_success", "kt_profile_begin", "kt_profile_end",
+           "kt_quant4_error", "kt_quant4_codes", "kt_quant_error", "kt_quant_codes", "kt_quant_error_given",
+           "kt_rowmax_success", "kt_profile_begin", "kt_profile_end",
            "kt_kurtosis_loss_noalloc"]
 
 # int32 reduce(void* user, void* dev_ptr, int64 count, int32 dtype, void* cuda_stream)
@@ -117,6 +118,7 @@ def lib():
     L.kt_quant4_codes.argtypes = [vp, vp, i64, i64, vp, vp]
     L.kt_quant_error.argtypes = [vp, kt_mat, vp, C.POINTER(kt_quant_spec), dp]
     L.kt_quant_codes.argtypes = [vp, vp, i64, i64, C.POINTER(kt_quant_spec), vp, vp, vp]
+    L.kt_quant_error_given.argtypes = [vp, vp, i64, i64, C.POINTER(kt_quant_spec), dp]
     L.kt_rowmax_success.argtypes = [vp, kt_mat, vp, vp, dp]
     L.kt_kurtosis_loss_noalloc.argtypes = [kt_mat, vp, vp, vp]
     L.kt_profile_begin.argtypes = [vp]
@@ -366,22 +368,31 @@ class Context:
         _check(lib().kt_quant4_error(self._h, m, R.data_ptr(), C.byref(out)), "kt_quant4_error")
         return out.value
 
-    def quant_error(self, X, R, bits=4, asymmetric=False, clip=1.0):
+    def quant_error(self, X, R, bits=4, asymmetric=False, clip=1.0, clip_mode=0):
         m = self._prep(X)
-        spec = kt_quant_spec(bits, int(asymmetric), clip, 0)
+        spec = kt_quant_spec(bits, int(asymmetric), clip, clip_mode)
         out = C.c_double()
         _check(lib().kt_quant_error(self._h, m, R.data_ptr(), C.byref(spec), C.byref(out)), "kt_quant_error")
         return out.value
 
-    def quant_codes(self, Y, bits=4, asymmetric=False, clip=1.0):
+    def quant_codes(self, Y, bits=4, asymmetric=False, clip=1.0, clip_mode=0):
         N, d = Y.shape
-        spec = kt_quant_spec(bits, int(asymmetric), clip, 0)
+        spec = kt_quant_spec(bits, int(asymmetric), clip, clip_mode)
         codes = torch.empty((N, d), dtype=torch.int16, device=Y.device)
         scales = torch.empty((N,), dtype=torch.float32, device=Y.device)
         shifts = torch.empty((N,), dtype=torch.float32, device=Y.device)
         _check(lib().kt_quant_codes(self._h, Y.data_ptr(), N, d, C.byref(spec), codes.data_ptr(), scales.data_ptr(),
                                     shifts.data_ptr()), "kt_quant_codes")
         return codes, scales, shifts
+
+    def quant_error_given(self, Y, bits=4, asymmetric=False, clip=1.0, clip_mode=0):
+        N, d = Y.shape
+        self.ensure_workspace(N, max(128, (d + 127) // 128 * 128), KT_BF16)
+        spec = kt_quant_spec(bits, int(asymmetric), clip, clip_mode)
+        out = C.c_double()
+        _check(lib().kt_quant_error_given(self._h, Y.data_ptr(), N, d, C.byref(spec), C.byref(out)),
+               "kt_quant_error_given")
+        return out.value
 
     def rowmax_success(self, X, R_a, R_b=None):
         m = self._prep(X)

@@ -100,3 +100,78 @@ def test_rowmax_success(ctx):
     assert ctx.rowmax_success(X, H) > 0.95
     # identity against the un-rotated token: equal maxima, strict inequality, no success
     assert ctx.rowmax_success(X, ctx.init_rotation(d, "identity")) == 0.0
+
+
+# ------------------------------------------------- the range as a per-row quantile of the magnitudes
+def _f32(level):
+    """The level as the library sees it (kt_quant_spec.clip is a float32)."""
+    return float(np.float32(level))
+
+
+@pytest.mark.parametrize("bits,level", [(4, 0.98), (4, 0.5), (8, 0.999), (3, 0.25), (4, 1.0)])
+@pytest.mark.parametrize("N,d", [(300, 256), (64, 4096), (20, 14336), (9, 1000)])
+def test_quantile_clip_codes_bit_exact(ctx, N, d, bits, level):
+    # the order statistic is an exact selection on the float32 bit patterns and the interpolation is float32 on both
+    # sides: scales and codes must agree bit for bit, ties, repeated magnitudes and constant rows included
+    g = torch.Generator(device="cpu").manual_seed(N + d + bits)
+    Y = torch.distributions.StudentT(3.0).sample((N, d)).float()
+    Y = (Y * torch.rand((N, 1), generator=g) * 10).to(DEV)
+    Y[0] = 0.0                                               # an all-zero row
+    Y[1] = -2.5                                              # a constant row
+    Y[2, :] = (torch.arange(d, device=DEV) % 7 - 3.0)        # seven magnitudes, each many times
+    Y[3, : d // 2] = Y[3, 0]                                 # half of the row equal
+    Y[4, 0] = 1.0e30                                         # one huge entry
+    codes, s, b = ctx.quant_codes(Y, bits, False, level, clip_mode=1)
+    rc, rs, rb = ko.quant_codes(Y.cpu().numpy(), bits, False, _f32(level), clip_quantile=True)
+    assert np.array_equal(s.cpu().numpy(), rs)
+    assert float(b.abs().max()) == 0.0
+    assert np.array_equal(codes.cpu().numpy(), rc)
+    if level == 1.0:                                         # the plain quantizer
+        c0, s0, _ = ctx.quant_codes(Y, bits, False, 1.0)
+        assert torch.equal(c0, codes) and torch.equal(s0, s)
+
+
+@pytest.mark.parametrize("bits,asym,clip,mode", [(4, False, 0.98, 1), (4, False, 0.9, 1), (4, False, 1.0, 0),
+                                                 (8, True, 0.9, 0)])
+def test_quant_error_of_a_given_y(ctx, bits, asym, clip, mode):
+    # Eq. 1 on a given Y (here the library's own X R), for both readings of "Setup"'s clipping
+    N, d = 1000, 1024
+    X = synth.activations(N, d, dist="student_t", nu=3.0, n_outliers=4, outlier_scale=50.0, seed=303,
+                          dtype=torch.bfloat16, device=DEV)
+    R = synth.random_orthogonal(d, seed=32, device=DEV).contiguous()
+    Y = ctx.rotate(X, R)
+    got = ctx.quant_error_given(Y, bits, asym, clip, clip_mode=mode)
+    want = ko.quant_error(Y.cpu().numpy(), bits, asym, _f32(clip), clip_quantile=bool(mode))
+    assert got == pytest.approx(want, rel=1e-9)
+    assert ctx.quant_error_given(Y, bits, asym, clip, clip_mode=mode) == got      # fixed-order sums
+    if mode == 0:
+        # the same quantity from the two GEMM passes that never store Y
+        assert ctx.quant_error(X, R, bits, asym, clip) == pytest.approx(got, rel=1e-6)
+
+
+def test_quantile_clip_lowers_the_4bit_error_of_heavy_tailed_tokens(ctx):
+    # why "Setup" clips: on heavy-tailed rows the 0.98-quantile as range beats the maximum
+    N, d = 2048, 4096
+    X = synth.activations(N, d, dist="student_t", nu=3.0, n_outliers=16, outlier_scale=100.0, seed=304,
+                          dtype=torch.bfloat16, device=DEV)
+    R = ctx.init_rotation(d, "hadamard")
+    Y = ctx.rotate(X, R)
+    plain = ctx.quant_error_given(Y, 4, False, 1.0)
+    clipped = ctx.quant_error_given(Y, 4, False, 0.98, clip_mode=1)
+    assert clipped < plain
+    assert clipped == pytest.approx(ko.quant_error(Y.cpu().numpy(), 4, False, _f32(0.98), clip_quantile=True), rel=1e-9)
+
+
+def test_quantile_clip_argument_errors(ctx):
+    Y = torch.randn((8, 256), device=DEV)
+    X = Y.to(torch.bfloat16)
+    R = ctx.init_rotation(256, "identity")
+    with pytest.raises(kurtail.KtError) as e:       # a quantile is defined for the symmetric quantizer only
+        ctx.quant_codes(Y, 4, True, 0.98, clip_mode=1)
+    assert e.value.status == 1
+    with pytest.raises(kurtail.KtError) as e:       # the GEMM passes never hold a whole row
+        ctx.quant_error(X, R, 4, False, 0.98, clip_mode=1)
+    assert e.value.status == 1
+    with pytest.raises(kurtail.KtError) as e:
+        ctx.quant_codes(Y, 4, False, 0.98, clip_mode=2)
+    assert e.value.status == 1

@@ -621,3 +621,66 @@ def test_rowmax_success_rate():
     assert ko.rowmax_success(np.ones((4, d)), H) == 0.0
     # a mix: exactly the one-hot half succeeds
     assert ko.rowmax_success(np.vstack([X, np.ones((10, d))]), H) == 0.5
+
+
+# ---------------- quantile clipping of the symmetric quantizer ----------------
+def _golden_quantile_cases():
+    cases = []
+    with open(os.path.join(GOLD, "quant_quantile_cases.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            bits, level, vals, rng, codes = [p.strip() for p in line.split(";")]
+            cases.append((int(bits), float(level), np.array(vals.split(), dtype=np.float32)[None, :], float(rng),
+                          np.array(codes.split(), dtype=np.int16)))
+    return cases
+
+
+def test_quantile_clip_golden_rows():
+    cases = _golden_quantile_cases()
+    assert len(cases) == 5
+    for bits, level, Y, rng, want in cases:
+        assert float(ko.row_abs_quantile(Y, level)[0]) == pytest.approx(rng, rel=1e-6)
+        codes, s, b = ko.quant_codes(Y, bits, False, level, clip_quantile=True)
+        assert np.array_equal(codes[0], want), (level, codes[0], want)
+        assert s[0] == pytest.approx(rng / (2 ** (bits - 1) - 1), rel=1e-6) and b[0] == 0.0
+
+
+def test_row_abs_quantile_is_the_library_quantile_of_the_magnitudes():
+    # the written-out rule against numpy's routine (method "linear"), on ragged sizes, with ties and with signs
+    rng = np.random.default_rng(3)
+    for n in (2, 5, 128, 1000, 4097):
+        Y = rng.standard_t(3, size=(7, n)).astype(np.float32)
+        Y[1, : n // 2] = Y[1, 0]                        # many equal magnitudes
+        Y[2] = -np.abs(Y[2])
+        for level in (0.0, 0.25, 0.5, 0.9, 0.98, 0.999, 1.0):
+            got = ko.row_abs_quantile(Y, level)
+            want = np.quantile(np.abs(Y).astype(np.float64), level, axis=1, method="linear")
+            assert np.allclose(got, want, rtol=2e-6, atol=0.0), (n, level)
+    # level 1 is the maximum exactly, level 0 the smallest magnitude exactly; monotone in the level
+    Y = rng.standard_normal((4, 333)).astype(np.float32)
+    assert np.array_equal(ko.row_abs_quantile(Y, 1.0), np.abs(Y).max(axis=1))
+    assert np.array_equal(ko.row_abs_quantile(Y, 0.0), np.abs(Y).min(axis=1))
+    qs = np.stack([ko.row_abs_quantile(Y, q) for q in np.linspace(0, 1, 21)])
+    assert np.all(np.diff(qs, axis=0) >= 0)
+
+
+def test_quantile_clip_saturates_the_expected_share_and_reduces_to_no_clipping():
+    rng = np.random.default_rng(4)
+    Y = rng.standard_t(3, size=(64, 4096)).astype(np.float32)
+    # level 1: the plain quantizer, bit for bit
+    c1, s1, _ = ko.quant_codes(Y, 4, False, 1.0, clip_quantile=True)
+    c0, s0, _ = ko.quant_codes(Y, 4, False, 1.0)
+    assert np.array_equal(c1, c0) and np.array_equal(s1, s0)
+    assert ko.quant_error(Y, 4, False, 1.0, clip_quantile=True) == ko.quant_error(Y, 4, False, 1.0)
+    # level 0.98: about 2 % of every row lies beyond the range and saturates at the largest code
+    c, s, _ = ko.quant_codes(Y, 4, False, 0.98, clip_quantile=True)
+    beyond = (np.abs(Y) > (7.0 * s)[:, None]).mean()
+    assert beyond == pytest.approx(0.02, abs=5e-4)
+    assert np.all(np.abs(c[np.abs(Y) > (7.0 * s)[:, None]]) == 7)
+    # on heavy-tailed rows clipping at the quantile lowers the 4-bit error (the reason "Setup" gives for it)
+    assert ko.quant_error(Y, 4, False, 0.98, clip_quantile=True) < ko.quant_error(Y, 4, False, 1.0)
+    # not defined for the asymmetric quantizer
+    with pytest.raises(ValueError):
+        ko.quant_codes(Y, 4, True, 0.98, clip_quantile=True)
