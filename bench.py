@@ -586,24 +586,31 @@ def main():
     if world == 1 and not args.no_extras and args.workload == "llama2_7b_attn" and not args.rows:
         extras = {}
 
-        def short_fit(c, Xw, Rw, steps, lr_w, warm=3):
+        def short_fit(c, Xw, Rw, steps, lr_w, warm=3, tries=3):
+            """The fastest of `tries` fits of `steps` steps (these side figures follow minutes of power-capped work,
+            and the part's clock right after it varies from one short run to the next)."""
             c.fit(Xw, Rw, warm, lr_w)
-            torch.cuda.synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            c.profile_begin()
-            a.record()
-            r = c.fit(Xw, Rw, steps, lr_w)
-            b.record()
-            torch.cuda.synchronize()
-            pr = c.profile_end()
-            return a.elapsed_time(b) / steps, r, pr
+            best = None
+            for _ in range(tries):
+                torch.cuda.synchronize()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                c.profile_begin()
+                a.record()
+                r = c.fit(Xw, Rw, steps, lr_w)
+                b.record()
+                torch.cuda.synchronize()
+                pr = c.profile_end()
+                ms_t = a.elapsed_time(b) / steps
+                if best is None or ms_t < best[0]:
+                    best = (ms_t, r, pr)
+            return best
 
         for name, kwx in (("backward_recompute", dict(backward_mode=1)), ("backward_stored_f32", dict(backward_mode=2)),
                           ("optimizer_adam", dict(optimizer=1)),
                           ("lr_10_full_series", dict())):
             c2 = kurtail.Context(dev, **kwx)
             ms_x, r_x, _ = short_fit(c2, X, fresh_R(c2), 20, 10.0 if name == "lr_10_full_series" else lr)
-            extras[name] = {"ms_per_step": ms_x, "tokens_per_s": N / (ms_x * 1e-3), "steps": 20,
+            extras[name] = {"ms_per_step": ms_x, "tokens_per_s": N / (ms_x * 1e-3), "steps": 20, "best_of": 3,
                             "series_terms_last": r_x["series_terms_last"], "p0_terms_last": r_x["p0_terms_last"],
                             "guards_run": r_x["guards_run"], "orth_err": r_x["orth_err"]}
             c2.close()
@@ -627,7 +634,7 @@ def main():
                 Rw = fresh_R(c2, dw, wc["init"])
             ms_x, r_x, pr = short_fit(c2, Xw, Rw, steps_w, wc["lr"])
             gg = pr["gemm"]
-            ex = {"ms_per_step": ms_x, "tokens_per_s": Nw / (ms_x * 1e-3), "steps": steps_w, "N": Nw, "d": dw,
+            ex = {"ms_per_step": ms_x, "tokens_per_s": Nw / (ms_x * 1e-3), "steps": steps_w, "best_of": 3, "N": Nw, "d": dw,
                   "orth_err": r_x["orth_err"]}
             if gg["fused"]["launches"]:
                 t_f = gg["fused"]["ms"] / gg["fused"]["launches"] * 1e-3
