@@ -277,7 +277,8 @@ kt_status kt_orth_step(kt_ctx* ctx, float* R, const float* dR, int64_t d, float 
  * the first step) are updated in place; dR is read only.  *st (host) carries
  * v and the step count between calls: zero it before the first step; it is
  * read on entry and written on return.  beta1, beta2, adam_eps come from the
- * context's configuration.  Always runs the general tensor-core path.  Uses
+ * context's configuration.  d <= 512 takes the one-launch float32 step like
+ * kt_orth_step (kt_config.small_d_orth), larger d the tensor-core path.  Uses
  * the workspace (sized for any N >= 1 and this d).  Synchronises. */
 typedef struct {
   double v;        /* running mean of ||dR||_F^2 */

@@ -828,7 +828,8 @@ static bool use_small_orth(const kt_ctx* ctx, int d) { return d <= 512 && ctx->c
 // then polish already at a quarter of the threshold, as the general path does inside kt_fit).
 // parts != null (d == 128): dR is summed inside the launch from the single-pass kernel's partials.
 static kt_status small_orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, float lr, const WsLayout& L,
-                                       int run_guard, bool adaptive, const FusedPartials* parts = nullptr) {
+                                       int run_guard, bool adaptive, const FusedPartials* parts = nullptr,
+                                       float* adam_m = nullptr) {
   const kt_config& c = ctx->cfg;
   SmallOrthParams p;
   memset(&p, 0, sizeof(p));
@@ -856,7 +857,12 @@ static kt_status small_orth_step_async(kt_ctx* ctx, float* R, const float* dR, i
   p.P1 = sm + 4 * dd;
   p.Rs = sm + 5 * dd;
   p.norm_part = reinterpret_cast<double*>(sm + 6 * dd);
-  p.max_part = reinterpret_cast<float*>(p.norm_part + kSoGrid);
+  p.g2_part = p.norm_part + kSoGrid;
+  p.max_part = reinterpret_cast<float*>(p.g2_part + kSoGrid);
+  p.adam_m = adam_m;
+  p.beta1 = c.beta1;
+  p.beta2 = c.beta2;
+  p.adam_eps = c.adam_eps;
   p.sc = &ctx->d_blk->sc;
   p.r_hi = at<__nv_bfloat16>(ctx, L.r_hi);
   p.rt_hi = at<__nv_bfloat16>(ctx, L.rt_hi);
@@ -902,8 +908,9 @@ static kt_status small_orth_step_async(kt_ctx* ctx, float* R, const float* dR, i
 static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, float lr, const WsLayout& L,
                                  int guard_mode, bool forms_current, bool adaptive = false, float* adam_m = nullptr,
                                  bool dr_hi_ready = false) {
-  if (!adam_m && use_small_orth(ctx, d))
-    return small_orth_step_async(ctx, R, dR, d, lr, L, guard_mode == 1 ? 1 : (guard_mode == 2 ? 0 : 2), adaptive);
+  if (use_small_orth(ctx, d))
+    return small_orth_step_async(ctx, R, dR, d, lr, L, guard_mode == 1 ? 1 : (guard_mode == 2 ? 0 : 2), adaptive,
+                                 nullptr, adam_m);
   const kt_config& c = ctx->cfg;
   Scalars* sc = &ctx->d_blk->sc;
   const uint64_t ld = static_cast<uint64_t>(d);

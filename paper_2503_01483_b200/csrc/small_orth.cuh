@@ -241,6 +241,11 @@ struct SmallOrthParams {
   int d;
   int iters;           // s: series terms 0..s
   int gate_terms;      // 1: series terms that cannot change the float32 R are not evaluated
+  // Cayley Adam (adam_m != null): d x d float32 momentum, in/out; v and the step count live in the scalar block.
+  // The direction is then W = skew(M R^T) / r with M <- beta1 M + (1 - beta1) dR, and M <- r W R afterwards.
+  float* adam_m;
+  float beta1, beta2, adam_eps;
+  double* g2_part;     // [kSoGrid] per-CTA sums of dR^2
   int run_guard;       // 1: measure R^T R - I, 0: do not, 2: when the device's drift bound reaches thresh / 2
   float lr, q, eps, thresh;
   float polish_at;     // the polish runs when the measured error exceeds this (<= thresh)
@@ -335,6 +340,9 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
     p.Rs[static_cast<long long>(i0 + r) * d + j] = rcur[r];
   }
   const float drift_in = p.sc->drift;  // (written only by the end of an earlier launch)
+  const bool adam = p.adam_m != nullptr;
+  const unsigned int adam_k_in = p.sc->adam_k;   // (likewise; block 0 writes the new values after the first barrier)
+  const double adam_v_in = p.sc->adam_v;
   float dr_own = 0.f;
   if (ROWS == 1 && p.use_parts) {
     // this CTA's row of dR from the single-pass kernel's partials, and its term of the loss correction
@@ -345,16 +353,58 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
     const double row = row_sum_128(p.fp.correct ? first_order_term(raw, rc) : 0.0, sh4);
     if (threadIdx.x == 0) p.fp.rowdot[blockIdx.x] = row;
   }
+  // Cayley Adam: this CTA's rows of M <- beta1 M + (1 - beta1) dR, and its part of ||dR||_F^2
+  float mrow[ROWS];
+  if (adam) {
+    double g2 = 0.0;
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) {
+      const long long o = static_cast<long long>(i0 + r) * d + j;
+      const float g = (ROWS == 1 && p.use_parts) ? dr_own : p.dR[o];
+      mrow[r] = fmaf(p.beta1, p.adam_m[o], (1.f - p.beta1) * g);
+      g2 += static_cast<double>(g) * g;
+    }
+    g2 = warp_sum(g2);
+    if (lane == 0) shd[warp] = g2;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      double t = 0.0;
+      for (int w = 0; w < nwarps; ++w) t += shd[w];
+      p.g2_part[blockIdx.x] = t;
+    }
+    __syncthreads();
+  }
   grid.sync();
   if (ROWS == 1 && p.use_parts && blockIdx.x == 0) {
     __shared__ double shl[256], shr[128];
     __shared__ unsigned int shdg[256];
     finish_fused_loss(p.fp, p.sc, shl, shr, shdg);
   }
+  // r = (1 - beta1^k) sqrt(v / (1 - beta2^k) + eps), the same in every CTA
+  double adam_r = 1.0;
+  if (adam) {
+    double g2 = 0.0;
+    for (int c = 0; c < kSoGrid; ++c) g2 += __ldcg(p.g2_part + c);
+    const unsigned int k = adam_k_in + 1u;
+    const double b1 = static_cast<double>(p.beta1), b2 = static_cast<double>(p.beta2);
+    const double v = b2 * adam_v_in + (1.0 - b2) * g2;
+    const double vhat = v / (1.0 - pow(b2, static_cast<double>(k)));
+    adam_r = (1.0 - pow(b1, static_cast<double>(k))) * sqrt(vhat + static_cast<double>(p.adam_eps));
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+      p.sc->adam_k = k;
+      p.sc->adam_v = v;
+      p.sc->adam_r = adam_r;
+    }
+  }
 
-  // A = dR R^T:  A[i][j] = sum_k dR[i][k] Rt[k][j]
+  // A = dR R^T (Cayley Adam: M R^T):  A[i][j] = sum_k dR[i][k] Rt[k][j]
   float acc[ROWS];
-  if (ROWS == 1 && p.use_parts) {
+  if (adam) {
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) arow[r][j] = mrow[r];
+    __syncthreads();
+  } else if (ROWS == 1 && p.use_parts) {
     __syncthreads();
     arow[0][j] = dr_own;
     __syncthreads();
@@ -368,10 +418,12 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
 
   // W = (A - A^T)/2 and ||W||_F^2 (per-CTA partial, then every CTA sums the partials in the same order)
   {
+    // (Cayley Adam divides the skew part by r: the same float for (i, j) and (j, i), so W stays exactly skew)
+    const float half_scale = adam ? static_cast<float>(0.5 / adam_r) : 0.5f;
     double n2 = 0.0;
 #pragma unroll
     for (int r = 0; r < ROWS; ++r) {
-      const float w = 0.5f * (acc[r] - p.A[static_cast<long long>(j) * d + i0 + r]);
+      const float w = half_scale * (acc[r] - p.A[static_cast<long long>(j) * d + i0 + r]);
       p.W[static_cast<long long>(i0 + r) * d + j] = w;
       n2 += static_cast<double>(w) * w;
     }
@@ -440,6 +492,8 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
       for (int r = 0; r < ROWS; ++r) {
         rcur[r] = fmaf(ck, acc[r], rcur[r]);
         if (k + 1 < n_terms) dst[static_cast<long long>(i0 + r) * d + j] = acc[r];
+        // Cayley Adam: the momentum goes back onto the tangent space at R, M <- r W R
+        if (adam && k == 0) p.adam_m[static_cast<long long>(i0 + r) * d + j] = static_cast<float>(adam_r) * acc[r];
       }
       ck *= -0.5f * alpha;
       if (k + 1 < n_terms) {

@@ -109,3 +109,38 @@ def test_fit_adam_descends_and_stays_orthogonal():
     c.fit(X, R2, 100, 5e-2)
     assert torch.equal(R, R2)
     c.close()
+
+
+@pytest.mark.parametrize("d", [128, 384, 512])
+def test_adam_one_launch_step_is_float32_exact_and_agrees_with_the_tensor_core_path(d):
+    # d <= 512: the whole Cayley-Adam step is one cooperative launch with float32 products, so it follows the oracle
+    # far more closely than the bf16 tensor-core path, which stays available (small_d_orth = 0) and must agree
+    X = make_x(700, d, seed=93)
+    R0t = synth.random_orthogonal(d, seed=13, device=DEV).contiguous()
+    one = kurtail.Context(DEV)
+    gen = kurtail.Context(DEV, small_d_orth=0)
+    Ra, Rb = R0t.clone(), R0t.clone()
+    Ma = torch.zeros((d, d), dtype=torch.float32, device=DEV)
+    Mb = torch.zeros_like(Ma)
+    sa, sb = dict(v=0.0, step=0), dict(v=0.0, step=0)
+    for it in range(3):
+        _, dR = one.loss_grad(X, Ra)
+        ost = dict(M=f64(Ma), v=sa["v"], k=sa["step"])
+        ref = ko.cayley_adam_step(f64(Ra), f64(dR), ost, 1e-2, beta1=0.9, beta2=0.99, adam_eps=1e-8, iters=2, q=0.5,
+                                  eps=1e-8, polish_thresh=1e-5)
+        R_in = f64(Ra)
+        Rb.copy_(Ra)
+        Mb.copy_(Ma)
+        sb.update(sa)
+        one.adam_step(Ra, dR, Ma, sa, 1e-2)
+        gen.adam_step(Rb, dR, Mb, sb, 1e-2)
+        upd = np.abs(ref - R_in).max()
+        assert sa["step"] == sb["step"] == ost["k"] == it + 1
+        # (beta2 reaches the library as a float32: 1 - beta2 differs from the oracle's by 1e-6 of itself)
+        assert sa["v"] == pytest.approx(ost["v"], rel=2e-6) and sb["v"] == pytest.approx(ost["v"], rel=2e-6)
+        assert np.linalg.norm(f64(Ma) - ost["M"]) <= 2e-5 * np.linalg.norm(ost["M"])
+        assert np.abs(f64(Ra) - ref).max() <= 1e-3 * upd + 3e-7
+        assert np.abs(f64(Rb) - ref).max() <= 2e-2 * upd + 3e-7
+        assert ko.orthogonality_error(f64(Ra)) <= 2e-5
+    one.close()
+    gen.close()
