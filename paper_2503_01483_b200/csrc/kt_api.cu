@@ -1141,7 +1141,7 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
     }
     // from the second step on, the previous step left the bf16 forms of R in the workspace
     // d = 128 with the one-launch orthogonal step: that launch also sums the single-pass kernel's partials
-    const bool fold = fused && !adam && use_small_orth(ctx, d) && ctx->reduce_fn == nullptr;
+    const bool fold = fused && use_small_orth(ctx, d) && ctx->reduce_fn == nullptr;
     FusedPartials parts;
     // (that launch also leaves the bf16 forms of the new Rc^T; any other step leaves those of R^T, so the
     // single-pass kernel's operand is then made afresh)
@@ -1160,7 +1160,7 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
       guard_mode = (k == 0 || k + 1 == steps) ? 1 : 0;
     if (fold)
       KT_TRY(small_orth_step_async(ctx, R, dR, d, lr, L, guard_mode == 1 ? 1 : (guard_mode == 2 ? 0 : 2),
-                                   ctx->cfg.guard_every < 1, &parts));
+                                   ctx->cfg.guard_every < 1, &parts, adam_m));
     else
       // (the single-pass kernel has put the forms of Rc^T where the step expects those of R^T: not current then)
       KT_TRY(orth_step_async(ctx, R, dR, d, lr, L, guard_mode, k > 0 && !fused, ctx->cfg.guard_every < 1, adam_m,
