@@ -175,7 +175,20 @@ typedef struct {
   float rms_eps;        /* [1e-6] (0 is allowed: all-zero rows then get factor 0) */
   int32_t wait_limit_ms;/* [4000] bound of every device-side wait, in
                            milliseconds (<= 0: the default)                    */
-  int32_t reserved;
+  int32_t forward_bf16; /* [0]   operand type of the forward pass's token GEMMs
+                           when R enters as one term (forward_terms == 1, or
+                           automatic with d > 512).  0 = float16: the GEMMs
+                           read a copy of X whose rows are scaled by a power
+                           of two into float16's range (exact for bf16 data;
+                           made once per call, N*d*2 bytes of workspace) and R
+                           rounded to float16, and the epilogues undo the row
+                           factor: 2^-12 instead of 2^-9 relative rounding of
+                           R at the same tensor-core rate.  It matters once R
+                           is no longer bf16-exact: with bf16 the loss and the
+                           gradient are those at bf16(R), which after a few
+                           steps from a Hadamard start is 2e-2 of the gradient's
+                           norm away from the gradient at R (3e-3 with
+                           float16).  1 = bf16 operands, X read in place       */
 } kt_config;
 
 /* Filled by kt_fit / kt_fit_layers (host memory). */
@@ -467,7 +480,9 @@ kt_status kt_quant4_codes(kt_ctx* ctx, const float* Y, int64_t N, int64_t d, int
  * contents (the call clears the words that must start at zero itself).  Two
  * calls that overlap on the GPU -- different streams, or different host threads
  * without ordering between their streams -- race on it; order them yourself.
- * The default configuration (kappa_target 1.8, forward_terms auto) applies. */
+ * The default configuration (kappa_target 1.8, forward_terms auto) applies,
+ * with bf16 operands throughout (forward_bf16 = 1: the float16 copy of X that
+ * the regular entry points make would not fit the built-in array). */
 #define KT_NOALLOC_MAX_N 16384
 #define KT_NOALLOC_MAX_D 1024
 kt_status kt_kurtosis_loss_noalloc(kt_mat X, const float* R, double* loss_dev, void* cuda_stream);

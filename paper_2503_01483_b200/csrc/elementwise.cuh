@@ -5,6 +5,7 @@
 // repeated runs are bit-identical.
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdint.h>
@@ -104,6 +105,97 @@ __global__ void k_split_bf16(const float* __restrict__ src, long long ld, __nv_b
 
 __device__ __forceinline__ float to_f32(float x) { return x; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+// ------------------------------------------- float16 operands of the forward pass
+// With R rounded to bf16 the forward GEMM evaluates the loss and the gradient not at R but at bf16(R), 2^-9
+// away in every entry -- which, once R has moved off a bf16-exact start by less than that, is a different point
+// altogether: measured at d = 4096 after three steps from the Hadamard start, the gradient is then 2.5e-2 of its norm
+// away from the float64 one.  float16 keeps three more bits of R at the same tensor-core rate (3e-3 in that case),
+// but both operands of an MMA must have the same type, and X is bf16 data with bf16's exponent range.  So the
+// forward GEMMs read a copy of X in which every row is multiplied by the power of two that brings its largest
+// entry into [1, 2), as float16: exact for bf16 entries within 2^14 of the row's largest, smaller ones lose bits
+// worth < 2^-25 of the row's size.  The epilogues multiply the accumulator rows by the inverse factor again (an exact
+// operation), so everything after the product sees Y = X R as before.
+//
+// src: bf16 rows (N x d, leading dimension ld).  x16: N x d float16.  acc[t] = 2^e_t (the inverse of row t's
+// factor), times rms[t] when the RMSNorm factors are given: what the epilogues multiply row t by.
+// A row with a NaN or Inf becomes all NaN; an all-zero row stays zero with factor 1.  One block of 256 threads per
+// row; the row is read twice (the second time from cache).
+__global__ void k_encode_rows_f16(const __nv_bfloat16* __restrict__ src, long long ld, int d, __half* __restrict__ x16,
+                                  const float* __restrict__ rms, float* __restrict__ acc) {
+  __shared__ float shm[8];
+  __shared__ int shb[8];
+  const __nv_bfloat16* x = src + static_cast<long long>(blockIdx.x) * ld;
+  __half* o = x16 + static_cast<long long>(blockIdx.x) * d;
+  float amax = 0.f;
+  int bad = 0;
+  for (int j = threadIdx.x * 8; j < d; j += 256 * 8) {   // d is a multiple of 128: whole 16-byte pieces
+    const uint4 raw = *reinterpret_cast<const uint4*>(x + j);
+    const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float2 f = __bfloat1622float2(p2[e]);
+      amax = fmaxf(amax, fmaxf(fabsf(f.x), fabsf(f.y)));
+      bad |= (!(fabsf(f.x) <= 3.4e38f) || !(fabsf(f.y) <= 3.4e38f)) ? 1 : 0;
+    }
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
+    bad |= __shfl_xor_sync(0xffffffffu, bad, off);
+  }
+  if ((threadIdx.x & 31) == 0) {
+    shm[threadIdx.x >> 5] = amax;
+    shb[threadIdx.x >> 5] = bad;
+  }
+  __syncthreads();
+  amax = shm[0];
+  bad = shb[0];
+#pragma unroll
+  for (int i = 1; i < 8; ++i) {
+    amax = fmaxf(amax, shm[i]);
+    bad |= shb[i];
+  }
+  float scale = 1.0f, inv = 1.0f;
+  if (amax > 0.f) {
+    int e = static_cast<int>((__float_as_uint(amax) >> 23) & 0xffu) - 127;   // amax in [2^e, 2^(e+1)); subnormal: -127
+    e = e < -126 ? -126 : (e > 126 ? 126 : e);
+    scale = __uint_as_float(static_cast<uint32_t>(127 - e) << 23);           // 2^-e, e in [-126, 126]
+    inv = __uint_as_float(static_cast<uint32_t>(127 + e) << 23);             // 2^e
+  }
+  if (threadIdx.x == 0) acc[blockIdx.x] = (rms != nullptr ? rms[blockIdx.x] : 1.0f) * inv;
+  const float nanv = __uint_as_float(0x7fc00000u);
+  for (int j = threadIdx.x * 8; j < d; j += 256 * 8) {
+    const uint4 raw = *reinterpret_cast<const uint4*>(x + j);
+    const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+    uint4 outv;
+    __half2* po = reinterpret_cast<__half2*>(&outv);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float2 f = __bfloat1622float2(p2[e]);
+      po[e] = bad ? __floats2half2_rn(nanv, nanv) : __floats2half2_rn(f.x * scale, f.y * scale);
+    }
+    *reinterpret_cast<uint4*>(o + j) = outv;
+  }
+}
+
+// R (d x d float32) -> R^T as float16 (the second operand of those GEMMs).  grid (d/32, d/32), block (32, 8).
+__global__ void k_rt_f16(const float* __restrict__ R, int d, __half* __restrict__ rt16) {
+  __shared__ float tile[32][33];
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  float x[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) x[q] = R[static_cast<long long>(r0 + ty + 8 * q) * d + c0 + tx];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) tile[ty + 8 * q][tx] = x[q];
+  __syncthreads();
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int c = ty + 8 * q;
+    rt16[static_cast<long long>(c0 + c) * d + r0 + tx] = __float2half_rn(tile[tx][c]);
+  }
+}
 
 // X (N x d, leading dimension ld, T = float or bf16) -> Xt (d x ldt bf16, the
 // transpose, columns in [N, 64*ceil(N/64)) zero) and, when xb != null, a dense

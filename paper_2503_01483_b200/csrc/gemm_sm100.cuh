@@ -77,6 +77,8 @@ struct GemmParams {
   // row's mean and sum of squares so that no entry can exceed 2^14; e goes to out16_exp[2 * n_tile + half][row].
   __half* out16;
   unsigned char* out16_exp;
+  // != 0: the operands are float16, not bf16 (every term; see k_encode_rows_f16)
+  int f16_operands;
 };
 
 // Unsigned keys that order like the floats they encode (negative floats reversed, positive ones above them).
@@ -131,6 +133,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
   const int first_unit = blockIdx.x / CTAS, unit_step = gridDim.x / CTAS;
 
   if (p.gate != nullptr && *p.gate < p.gate_min) return;  // uniform over the grid
+  const uint32_t idesc = p.f16_operands ? umma_idesc_f16_f32(kTileM, BN) : kIdesc;
   int n_terms = p.terms;
   if (p.terms_dev != nullptr) {
     const int t = static_cast<int>(*p.terms_dev);
@@ -304,9 +307,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
           for (int kk = 0; kk < kBK / 16; ++kk) {
             // 16 k-elements = 32 bytes further along the swizzled row: +2 in address>>4 units
             if constexpr (CTAS == 2)
-              tc_mma_bf16_pair(d_tmem, a_desc + 2u * kk, b_desc + 2u * kk, kIdesc, (it > 0 || kk > 0) ? 1u : 0u);
+              tc_mma_bf16_pair(d_tmem, a_desc + 2u * kk, b_desc + 2u * kk, idesc, (it > 0 || kk > 0) ? 1u : 0u);
             else
-              tc_mma_bf16(d_tmem, a_desc + 2u * kk, b_desc + 2u * kk, kIdesc, (it > 0 || kk > 0) ? 1u : 0u);
+              tc_mma_bf16(d_tmem, a_desc + 2u * kk, b_desc + 2u * kk, idesc, (it > 0 || kk > 0) ? 1u : 0u);
           }
           // frees the stage (in both CTAs of a pair) once these MMAs have read it
           if constexpr (CTAS == 2) tc_commit_pair(empty_bar(stage), 3); else tc_commit(empty_bar(stage));

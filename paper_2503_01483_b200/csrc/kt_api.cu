@@ -97,10 +97,23 @@ struct WsLayout {
   size_t flat;          // flattened-kurtosis mode: the global coefficients, the global mean, 3 x [blocks] doubles
   size_t rowscale;      // [N] float: RMSNorm factor of every row (kt_config.rmsnorm), or, for the single-pass
                         // d = 128 kernel, the mean square of every row of X
+  // float16 operands of the forward GEMMs (see k_encode_rows_f16): the encoded X [N][d], the factor the epilogues
+  // multiply each accumulator row by [N], and R^T as float16 [d][d]
+  size_t x16, rowacc, rt16;
+  bool f16;             // those three exist
   size_t total;
   long long ldt;
   int P, bn, loss_blocks, norm_n;
 };
+
+// The token GEMMs of the forward pass take float16 operands whenever R would otherwise enter as a single bf16 term
+// (d > 512 by default), unless the configuration asks for bf16.
+static bool forward_is_f16(const kt_config* cfg, int64_t d, int gather_batch) {
+  (void)gather_batch;
+  const int terms = cfg == nullptr ? 0 : cfg->forward_terms;
+  const bool one_term = terms == 1 || (terms != 2 && d > 512);
+  return one_term && (cfg == nullptr || cfg->forward_bf16 == 0);
+}
 
 // cfg == null: the default configuration (no momentum buffer, no RMSNorm factors).
 // gather_batch > 0: the layout of kt_fit_shared (N = batch * rows per sample): the dense bf16 matrix is the gathered
@@ -171,6 +184,11 @@ static WsLayout make_layout(int64_t N, int64_t d, int32_t x_dtype, const kt_conf
   L.flat = take(static_cast<size_t>(L.loss_blocks) * 8 * 3 + 64);
   // (d = 128: the single-pass kernel's per-row mean square of X lives here too)
   L.rowscale = take(((cfg != nullptr && cfg->rmsnorm != 0) || d == kFsD) ? static_cast<size_t>(N) * 4 : 0);
+  const bool f16 = forward_is_f16(cfg, d, gather_batch);
+  L.f16 = f16;
+  L.x16 = take(f16 ? static_cast<size_t>(N) * d * 2 : 0);
+  L.rowacc = take(f16 ? static_cast<size_t>(N) * 4 : 0);
+  L.rt16 = take(f16 ? dd * 2 : 0);
   L.total = off;
   return L;
 }
@@ -413,7 +431,13 @@ struct XView {
   long long ldx;
   const float* row_scale;   // RMSNorm factor of every row (kt_config.rmsnorm), or null
   const float* row_ms;      // single-pass d = 128 kernel: mean square of every row of X
+  const __half* x16;        // the rows in the float16 encoding of the forward GEMMs (dense, N x d), or null
+  const float* acc_scale;   // what the forward GEMMs' epilogues multiply each accumulator row by, or null: the
+                            // RMSNorm factor, times the inverse of the float16 encoding's row factor
 };
+
+// Completes a view whose bf16 rows (and RMSNorm factors) are set: the float16 encoding when this problem uses it.
+static kt_status finish_view(kt_ctx* ctx, int64_t N, int64_t d, const WsLayout& L, XView* v);
 
 // The single-pass d = 128 kernel's own encoding of X (row-normalised float16, see k_encode_rows_128) and each encoded
 // row's mean square: one pass over X, needed once per X.
@@ -448,11 +472,15 @@ static kt_status row_scale_x(kt_ctx* ctx, const kt_mat& X, const WsLayout& L, XV
 static kt_status ingest_x_forward(kt_ctx* ctx, const kt_mat& X, const WsLayout& L, XView* v, bool want_scale = true) {
   const int64_t N = X.rows, d = X.cols;
   v->row_scale = nullptr;
-  if (ctx->cfg.rmsnorm != 0 && want_scale) return row_scale_x(ctx, X, L, v);
+  v->row_ms = nullptr;
+  if (ctx->cfg.rmsnorm != 0 && want_scale) {
+    KT_TRY(row_scale_x(ctx, X, L, v));
+    return finish_view(ctx, N, d, L, v);
+  }
   if (X.dtype == KT_BF16) {
     v->xb = static_cast<const __nv_bfloat16*>(X.data);
     v->ldx = X.ld;
-    return KT_OK;
+    return finish_view(ctx, N, d, L, v);
   }
   __nv_bfloat16* xb = at<__nv_bfloat16>(ctx, L.xb);
   const long long pairs = N * d / 2;
@@ -461,7 +489,7 @@ static kt_status ingest_x_forward(kt_ctx* ctx, const kt_mat& X, const WsLayout& 
   KT_LAUNCH_CHECK();
   v->xb = xb;
   v->ldx = d;
-  return KT_OK;
+  return finish_view(ctx, N, d, L, v);
 }
 
 // X^T of a bf16 X (no dense copy needed): the wide-load transpose.
@@ -478,6 +506,7 @@ static kt_status ingest_x_full(kt_ctx* ctx, const kt_mat& X, const WsLayout& L, 
   dim3 grid(d / 64, (N + 63) / 64), block(32, 8);
   __nv_bfloat16* xt = at<__nv_bfloat16>(ctx, L.xt);
   v->row_scale = nullptr;
+  v->row_ms = nullptr;
   if (ctx->cfg.rmsnorm != 0) {
     KT_TRY(row_scale_x(ctx, X, L, v));
     KT_TRY(transpose_x_bf16(ctx, v->xb, v->ldx, N, d, L));
@@ -492,6 +521,20 @@ static kt_status ingest_x_full(kt_ctx* ctx, const kt_mat& X, const WsLayout& L, 
     v->xb = xb;
     v->ldx = d;
   }
+  return finish_view(ctx, N, d, L, v);
+}
+
+static kt_status finish_view(kt_ctx* ctx, int64_t N, int64_t d, const WsLayout& L, XView* v) {
+  v->x16 = nullptr;
+  v->acc_scale = v->row_scale;
+  if (!L.f16) return KT_OK;
+  __half* x16 = at<__half>(ctx, L.x16);
+  float* acc = at<float>(ctx, L.rowacc);
+  k_encode_rows_f16<<<static_cast<unsigned>(N), 256, 0, ctx->stream>>>(v->xb, v->ldx, static_cast<int>(d), x16,
+                                                                       v->row_scale, acc);
+  KT_LAUNCH_CHECK();
+  v->x16 = x16;
+  v->acc_scale = acc;
   return KT_OK;
 }
 
@@ -507,22 +550,42 @@ static int forward_terms(const kt_ctx* ctx, int d, long long N) {
   return d <= 512 ? 2 : 1;
 }
 
+// R^T as float16 for the forward GEMMs of a problem that uses the float16 encoding (no kernel of the orthogonal
+// step keeps this form up to date: it is made afresh before every forward pass).
+static kt_status cast_rt16(kt_ctx* ctx, const float* R, int d, const WsLayout& L) {
+  if (!L.f16) return KT_OK;
+  dim3 grid(d / 32, d / 32), block(32, 8);
+  k_rt_f16<<<grid, block, 0, ctx->stream>>>(R, d, at<__half>(ctx, L.rt16));
+  KT_LAUNCH_CHECK();
+  return KT_OK;
+}
+
 static kt_status cast_rt(kt_ctx* ctx, const float* R, int d, long long N, const WsLayout& L) {
   dim3 grid(d / 32, d / 32), block(32, 8);
   k_split_bf16<true><<<grid, block, 0, ctx->stream>>>(
       R, d, at<__nv_bfloat16>(ctx, L.rt_hi), forward_terms(ctx, d, N) == 2 ? at<__nv_bfloat16>(ctx, L.rt_lo) : nullptr,
       d);
   KT_LAUNCH_CHECK();
+  KT_TRY(cast_rt16(ctx, R, d, L));
   return KT_OK;
 }
 
-// Operands of Y = X R for the token GEMMs: X against R^T hi (and lo).
+// Operands of Y = X R for the token GEMMs: X against R^T hi (and lo) in bf16, or the float16 encoding of X against
+// R^T as float16.  fwd_operands() also sets the parameters that go with the choice (operand type, row factors).
 struct FwdOperands {
   Operand A[2], B[2];
   int terms;
 };
-static FwdOperands fwd_operands(kt_ctx* ctx, const XView& xv, int d, long long N, const WsLayout& L) {
+static FwdOperands fwd_operands(kt_ctx* ctx, const XView& xv, int d, long long N, const WsLayout& L, GemmParams* p) {
   FwdOperands f;
+  p->row_scale = xv.acc_scale;
+  if (xv.x16 != nullptr) {
+    f.terms = 1;
+    f.A[0] = f.A[1] = Operand{xv.x16, static_cast<uint64_t>(d)};
+    f.B[0] = f.B[1] = Operand{at<__half>(ctx, L.rt16), static_cast<uint64_t>(d)};
+    p->f16_operands = 1;
+    return f;
+  }
   f.terms = forward_terms(ctx, d, N);
   f.A[0] = f.A[1] = Operand{xv.xb, static_cast<uint64_t>(xv.ldx)};
   f.B[0] = Operand{at<__nv_bfloat16>(ctx, L.rt_hi), static_cast<uint64_t>(d)};
@@ -548,9 +611,8 @@ static kt_status forward_loss(kt_ctx* ctx, const XView& xv, int N, int d, const 
     p.out16_exp = at<unsigned char>(ctx, L.yexp);
     p.ldo = d;
   }
-  p.row_scale = xv.row_scale;
   const double n_mean = mean_rows(ctx, N);
-  const FwdOperands f = fwd_operands(ctx, xv, d, N, L);
+  const FwdOperands f = fwd_operands(ctx, xv, d, N, L, &p);
   KT_TRY(run_gemm<kMoments>(ctx, N, d, d, f.terms, f.A, f.B, p, kCatForward));
   k_moments_finalize<<<L.loss_blocks, 256, 0, ctx->stream>>>(at<float4>(ctx, L.partial), L.P, N, d, L.bn,
                                                             ctx->cfg.kappa_target, at<float4>(ctx, L.moments),
@@ -630,8 +692,7 @@ static kt_status backward(kt_ctx* ctx, const XView& xv, int N, int d, const WsLa
     p.coef = at<float4>(ctx, L.coef);
     p.gt = at<__nv_bfloat16>(ctx, L.gt);
     p.ldg = L.ldt;
-    p.row_scale = xv.row_scale;
-    const FwdOperands f = fwd_operands(ctx, xv, d, N, L);
+    const FwdOperands f = fwd_operands(ctx, xv, d, N, L, &p);
     KT_TRY(run_gemm<kGrad>(ctx, N, d, d, f.terms, f.A, f.B, p, kCatBackwardA));
   }
   GemmParams p2 = blank_params();
@@ -656,6 +717,7 @@ static kt_status backward(kt_ctx* ctx, const XView& xv, int N, int d, const WsLa
 static kt_status loss_grad_async(kt_ctx* ctx, const XView& xv, int N, int d, const WsLayout& L, const float* R,
                                  float* dR, double* hist_slot, bool rt_current, __nv_bfloat16* dr_hi = nullptr) {
   if (!rt_current) KT_TRY(cast_rt(ctx, R, d, N, L));
+  else KT_TRY(cast_rt16(ctx, R, d, L));
   KT_TRY(forward_loss(ctx, xv, N, d, L, hist_slot, keep_y_for_backward(ctx)));
   KT_TRY(backward(ctx, xv, N, d, L, dR, dr_hi));
   KT_TRY(reduce_shards(ctx, dR, static_cast<int64_t>(d) * d, KT_F32));  // the gradient of the whole batch
@@ -1137,6 +1199,7 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
       xv.ldx = d;
       if (!fused) {  // the token GEMM of the backward pass reads the transpose
         KT_TRY(transpose_x_bf16(ctx, xb, d, N, d, L));
+        KT_TRY(finish_view(ctx, N, d, L, &xv));   // (and the forward pass, maybe, the float16 encoding)
       }
     }
     // from the second step on, the previous step left the bf16 forms of R in the workspace
@@ -1224,6 +1287,7 @@ void kt_default_config(kt_config* cfg) {
   cfg->adam_eps = 1e-8f;
   cfg->norm_iters = 2;
   cfg->backward_mode = 0;
+  cfg->forward_bf16 = 0;
   cfg->cta_pairs = 1;
   cfg->loss_mode = 0;
   cfg->rmsnorm = 0;
@@ -1379,8 +1443,7 @@ kt_status kt_rotate(kt_ctx* ctx, kt_mat X, const float* R, float* Y) {
   GemmParams p = blank_params();
   p.out = Y;
   p.ldo = d;
-  p.row_scale = xv.row_scale;
-  const FwdOperands f = fwd_operands(ctx, xv, static_cast<int>(d), N, L);
+  const FwdOperands f = fwd_operands(ctx, xv, static_cast<int>(d), N, L, &p);
   return run_gemm<kStoreF32>(ctx, static_cast<int>(N), static_cast<int>(d), static_cast<int>(d), f.terms, f.A, f.B, p,
                              kCatForward);
 }
@@ -1616,16 +1679,16 @@ kt_status kt_quant_error(kt_ctx* ctx, kt_mat X, const float* R, const kt_quant_s
   unsigned int* rowmin = spec->asymmetric ? at<unsigned int>(ctx, L.rowmin) : nullptr;
   KT_CUDA(cudaMemsetAsync(rowmax, 0, static_cast<size_t>(N) * 4, ctx->stream));
   if (rowmin) KT_CUDA(cudaMemsetAsync(rowmin, 0xff, static_cast<size_t>(N) * 4, ctx->stream));
-  const FwdOperands f = fwd_operands(ctx, xv, d, N, L);
   {
     GemmParams p = blank_params();
+    const FwdOperands f = fwd_operands(ctx, xv, d, N, L, &p);
     p.rowmax = rowmax;
     p.rowmin = rowmin;
-    p.row_scale = xv.row_scale;
     KT_TRY(run_gemm<kAbsMax>(ctx, N, d, d, f.terms, f.A, f.B, p, kCatQuant));
   }
   {
     GemmParams p = blank_params();
+    const FwdOperands f = fwd_operands(ctx, xv, d, N, L, &p);
     p.rowmax = rowmax;
     p.rowmin = rowmin;
     p.qerr = at<float>(ctx, L.qerr);
@@ -1633,7 +1696,6 @@ kt_status kt_quant_error(kt_ctx* ctx, kt_mat X, const float* R, const kt_quant_s
     p.q_den = q.den;
     p.q_lo = q.lo;
     p.q_hi = q.hi;
-    p.row_scale = xv.row_scale;
     KT_TRY(run_gemm<kQuantErr>(ctx, N, d, d, f.terms, f.A, f.B, p, kCatQuant));
   }
   const long long n = static_cast<long long>(L.P) * N;
@@ -1719,8 +1781,8 @@ kt_status kt_rowmax_success(kt_ctx* ctx, kt_mat X, const float* R_a, const float
     }
     KT_TRY(cast_rt(ctx, Rs[which], d, N, L));
     KT_CUDA(cudaMemsetAsync(outs[which], 0, static_cast<size_t>(N) * 4, ctx->stream));
-    const FwdOperands f = fwd_operands(ctx, xv, d, N, L);
     GemmParams p = blank_params();
+    const FwdOperands f = fwd_operands(ctx, xv, d, N, L, &p);
     p.rowmax = outs[which];
     KT_TRY(run_gemm<kAbsMax>(ctx, N, d, d, f.terms, f.A, f.B, p, kCatQuant));
   }
@@ -1886,9 +1948,9 @@ kt_status kt_kurtosis_loss_noalloc(kt_mat X, const float* R, double* loss_dev, v
   // (the time-out flag is only ever raised by atomicMax); everything else is written before it is read
   KT_CUDA(cudaMemsetAsync(&ctx->d_blk->sc, 0, sizeof(Scalars), ctx->stream));
   XView xv;
+  memset(&xv, 0, sizeof(xv));
   xv.xb = static_cast<const __nv_bfloat16*>(X.data);
   xv.ldx = X.ld;
-  xv.row_scale = nullptr;
   KT_TRY(cast_rt(ctx, R, static_cast<int>(d), N, L));
   // nobody reads the status word of this stream-ordered call on the host: a wait that ran out shows as a NaN loss
   return forward_loss(ctx, xv, static_cast<int>(N), static_cast<int>(d), L, loss_dev, false, true);

@@ -39,7 +39,7 @@ class kt_config(C.Structure):
                 ("forward_terms", C.c_int32), ("small_d_fused", C.c_int32), ("small_d_orth", C.c_int32),
                 ("optimizer", C.c_int32), ("beta1", C.c_float), ("beta2", C.c_float), ("adam_eps", C.c_float),
                 ("norm_iters", C.c_int32), ("backward_mode", C.c_int32), ("cta_pairs", C.c_int32), ("loss_mode", C.c_int32), ("rmsnorm", C.c_int32), ("rms_eps", C.c_float),
-                ("wait_limit_ms", C.c_int32), ("reserved", C.c_int32)]
+                ("wait_limit_ms", C.c_int32), ("forward_bf16", C.c_int32)]
 
 
 class kt_quant_spec(C.Structure):
