@@ -390,8 +390,17 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
         tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) release_acc(buf);
+        // With float16 operands the accumulator holds the product of rows scaled into [1, 2): the row factor is not
+        // applied to the entries but to the results (the mean by f, the k-th central sum by f^k) and to the stored
+        // copies on their way out (the float16 one takes it into its own factor), one multiplication per entry less.
+        // With bf16 operands the accumulator carries X's own scale, and the factor (RMSNorm's) has to come first, so
+        // that the fourth powers stay in range whatever that scale is.
+        const bool pre = scaled && p.f16_operands == 0;
+        if (pre) {
 #pragma unroll
-        for (int c = 0; c < kChunks; ++c) scale32(vv[c]);
+          for (int c = 0; c < kChunks; ++c) scale32(vv[c]);
+        }
+        const float post = (scaled && !pre) ? rs : 1.0f;
         // pass 1: mean of the kHalf columns; pass 2: central power sums about it
         float s1 = 0.f;
 #pragma unroll
@@ -406,14 +415,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
           }
           s1 += (a0 + a1) + (a2 + a3);
         }
-        const float mean = s1 * (1.0f / kHalf);
+        float mean = s1 * (1.0f / kHalf);
         float s2 = 0.f, s3 = 0.f, s4 = 0.f;
 #pragma unroll
         for (int c = 0; c < kChunks; ++c) {
-          // keep the float32 tile for the backward pass (the caller's choice; see kt_config.backward_mode)
-          if (p.out != nullptr && row_ok)
-            store_row32(p.out + static_cast<long long>(row) * p.ldo + n0 + cbeg + 32 * c, vv[c],
-                        p.out_sector_aligned != 0);
           float b2 = 0.f, b3 = 0.f, b4 = 0.f;
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
@@ -427,7 +432,25 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
           s3 += b3;
           s4 += b4;
         }
+        if (post != 1.0f) {   // (factor by factor: no power of f is formed that the result does not need)
+          mean *= post;
+          s2 = (s2 * post) * post;
+          s3 = ((s3 * post) * post) * post;
+          s4 = (((s4 * post) * post) * post) * post;
+        }
         if (row_ok) p.partial[static_cast<long long>(2 * n_tile + half) * p.M + row] = make_float4(mean, s2, s3, s4);
+        // keep the float32 tile for the backward pass (the caller's choice; see kt_config.backward_mode)
+        if (p.out != nullptr && row_ok) {
+#pragma unroll
+          for (int c = 0; c < kChunks; ++c) {
+            if (post != 1.0f) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) vv[c][j] = __float_as_uint(__uint_as_float(vv[c][j]) * post);
+            }
+            store_row32(p.out + static_cast<long long>(row) * p.ldo + n0 + cbeg + 32 * c, vv[c],
+                        p.out_sector_aligned != 0);
+          }
+        }
         if (p.out16 != nullptr && row_ok) {
           // float16 copy of the half row for the backward pass.  |y| <= |mean| + |c| and c^2 <= sum of c^2:
           // with e the biased exponent of that bound (< 2^(e - 126)), 2^(140 - e) brings every entry below 2^14.
@@ -435,7 +458,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_tn_kernel(const __grid_c
           const float bound = fabsf(mean) + sqrtf(s2);
           unsigned int e = (__float_as_uint(bound) >> 23) & 0xffu;
           e = e < 14u ? 14u : (e > 254u ? 254u : e);
-          const float mul = __uint_as_float((267u - e) << 23);
+          const float mul = __uint_as_float((267u - e) << 23) * post;   // (entries not yet scaled: post is their factor)
           p.out16_exp[static_cast<long long>(2 * n_tile + half) * p.M + row] = static_cast<unsigned char>(e);
           __half* dst = p.out16 + static_cast<long long>(row) * p.ldo + n0 + cbeg;
 #pragma unroll
