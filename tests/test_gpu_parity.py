@@ -249,6 +249,34 @@ def test_loss_grad_tiny_config_float32(ctx):
     assert np.linalg.norm(f64(dR) - dR_ref) / np.linalg.norm(dR_ref) <= 1e-2
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_float16_forward_operands_on_wide_rows(ctx, dtype):
+    # d > 512: the forward GEMMs read a float16 copy of X with one power-of-two factor per row and R rounded to
+    # float16.  Rows of very different scale, a row of zeros, a strided X and a float32 X all take that path; the
+    # results are held to the oracle (which sees X's own values), rerun bit for bit, and are the bf16-operand path's
+    # for an R that bf16 holds exactly.
+    N, d = 700, 1024
+    big = synth.activations(N, 2 * d, "student_t", 3.0, 8, 50.0, seed=48, dtype=torch.float32, device=DEV)
+    big *= torch.logspace(-8, 8, N, base=2.0, device=DEV)[:, None]
+    big[11] = 0.0
+    X = big.to(dtype)[:, :d]                     # leading dimension 2 d
+    R = rand_orth(d, seed=9)
+    loss, dR = ctx.loss_grad(X, R)
+    L_ref, dR_ref = ko.loss_grad(f64(X), f64(R))
+    assert abs(loss - L_ref) <= 1e-3 * abs(L_ref)
+    assert rel_fro(f64(dR), dR_ref) <= 1e-2
+    l2, d2 = ctx.loss_grad(X.contiguous(), R)
+    assert l2 == loss and torch.equal(d2, dR)
+    Y = ctx.rotate(X, R)
+    ref = f64(X.to(torch.bfloat16)) @ f64(R)
+    assert np.abs(f64(Y) - ref).max() <= 2e-3 * np.abs(ref).max()
+    Rb = R.to(torch.bfloat16).float()            # exact in bf16, and in float16 but for entries below 2^-17
+    b = kurtail.Context(DEV, forward_bf16=1)
+    Ya, Yb = ctx.rotate(X, Rb), b.rotate(X, Rb)
+    assert np.abs(f64(Ya) - f64(Yb)).max() <= 1e-5 * np.abs(f64(Yb)).max()
+    b.close()
+
+
 def test_loss_grad_is_deterministic(ctx):
     X = make_x(3000, 256, seed=41)
     R = rand_orth(256, seed=6)
