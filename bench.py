@@ -70,14 +70,14 @@ def kernel_source_hash(kernel):
     return h.hexdigest()[:16]
 
 
-def recorded_traffic(kernel, role):
+def recorded_traffic(kernel, role, d):
     """DRAM bytes (read + written) per token of one launch, from the ncu capture summarised under profiles/.
 
     profiles/dram_traffic.txt holds one line per captured launch:
         kernel role rows d bytes_read bytes_write fixed_bytes source_hash
     (fixed_bytes: the part that does not grow with the rows, e.g. the d x d operand).  Returns
-    (bytes per row, fixed bytes) or None when there is no line for this kernel and role, or when the kernel's
-    source has changed since the counters were taken."""
+    (bytes per row, fixed bytes) or None when there is no line for this kernel, role and width d, or when the
+    kernel's source has changed since the counters were taken."""
     path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
     if not os.path.exists(path):
         return None
@@ -87,8 +87,8 @@ def recorded_traffic(kernel, role):
             parts = line.split()
             if len(parts) != 8 or parts[0].startswith("#"):
                 continue
-            k, r, rows, _d, rd, wr, fixed, src = parts
-            if k == kernel and r == role and src == want:
+            k, r, rows, dd, rd, wr, fixed, src = parts
+            if k == kernel and r == role and int(dd) == int(d) and src == want:
                 return (float(rd) + float(wr) - float(fixed)) / float(rows), float(fixed)
     return None
 
@@ -489,7 +489,7 @@ def main():
         alg_bytes = 2.0 * N * d
         achieved = alg_bytes / t_f / 1e9
         peak = peaks["hbm_gbs"]
-        tr = recorded_traffic("fused_small_kernel", "terms%d" % fwd_terms)
+        tr = recorded_traffic("fused_small_kernel", "terms%d" % fwd_terms, d)
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "traffic": (tr[0] * N + tr[1]) if tr else None, "algorithmic_bytes": alg_bytes,
                     "kernel": "fused_small_kernel (loss + gradient in one pass over X): N*d*2 bytes per launch",
@@ -506,7 +506,7 @@ def main():
         # power cap, the sustained one for a region of a second or more or one whose clock record shows the cap
         use_burst = (not capped) and timed_s < 1.0
         peak = peaks["tflops_burst"] if use_burst else peaks["tflops_sustained"]
-        trs = [recorded_traffic("gemm_tn_kernel", r) for r in
+        trs = [recorded_traffic("gemm_tn_kernel", r, d) for r in
                ({"stored": "forward_stored", "stored_f32": "forward_stored_f32", "recompute": "forward"}[args.backward],
                 "backward_b")]
         traffic = None

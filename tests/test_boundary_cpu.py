@@ -133,7 +133,8 @@ def test_bench_quotes_dram_counters_only_for_the_kernel_they_were_taken_from(tmp
         "gemm_tn_kernel backward_b 1000 4096 5000000 1000000 2000000 %s\n"
         "gemm_tn_kernel forward 1000 4096 5000000 1000000 2000000 0123456789abcdef\n" % now)
     monkeypatch.setattr(bench, "ROOT", str(fake_root))
-    per_row, fixed = bench.recorded_traffic("gemm_tn_kernel", "backward_b")
+    per_row, fixed = bench.recorded_traffic("gemm_tn_kernel", "backward_b", 4096)
     assert per_row == pytest.approx(4000.0) and fixed == 2000000.0
-    assert bench.recorded_traffic("gemm_tn_kernel", "forward") is None        # stale fingerprint
-    assert bench.recorded_traffic("fused_small_kernel", "terms1") is None     # no line at all
+    assert bench.recorded_traffic("gemm_tn_kernel", "backward_b", 8192) is None     # counters of another width
+    assert bench.recorded_traffic("gemm_tn_kernel", "forward", 4096) is None        # stale fingerprint
+    assert bench.recorded_traffic("fused_small_kernel", "terms1", 128) is None      # no line at all
