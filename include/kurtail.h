@@ -97,16 +97,17 @@ typedef struct {
                            polish_thresh; in this mode the polish already runs
                            at a quarter of polish_thresh, so that measurements
                            stay rare.  kt_orth_step always measures           */
-  int32_t forward_terms;/* [0]   bf16 terms of R in the token GEMMs: 1 = R rounded
-                           to bf16; 2 = hi + lo (about 16 significant bits,
-                           twice the MMA work); 0 = automatic: 2 when d <= 512
-                           (with few channels the rounding error of R is
-                           systematic over tokens and one term can miss the
-                           1e-3 loss tolerance), else 1.  The single-pass
-                           d == 128 kernel of kt_loss_grad / kt_fit uses one
-                           term in the automatic mode too and corrects the loss
-                           to first order, L(R) = L(bf16 R) + <dR, R - bf16 R>,
-                           from the gradient the same pass yields                */
+  int32_t forward_terms;/* [0]   16-bit terms of R in the token GEMMs: 1 = R rounded
+                           once (to float16, or to bf16 with forward_bf16);
+                           2 = bf16 hi + lo (about 16 significant bits, twice
+                           the MMA work); 0 = automatic: 2 when d <= 512 (with
+                           few channels the rounding error of R is systematic
+                           over tokens and one term can miss the 1e-3 loss
+                           tolerance), else 1.  The single-pass d == 128 kernel
+                           of kt_loss_grad / kt_fit uses one float16 term in
+                           the automatic mode too and corrects the loss to
+                           first order, L(R) = L(f16 R) + <dR, R - f16 R>, from
+                           the gradient the same pass yields                    */
   int32_t small_d_fused;/* [1]   d == 128: kt_loss_grad / kt_fit use the single-pass
                            kernel (X read once per evaluation); 0 = the general
                            three-GEMM path                                      */
