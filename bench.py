@@ -19,6 +19,7 @@ from __future__ import annotations
 
 import argparse
 import hashlib
+import re
 import json
 import os
 import subprocess
@@ -62,11 +63,15 @@ def measured_peaks():
 
 
 def kernel_source_hash(kernel):
-    """Fingerprint of the files a kernel is compiled from: DRAM counters taken from an older kernel are not quoted."""
+    """Fingerprint of the code a kernel is compiled from (comments and white space left out): DRAM counters taken
+    from an older kernel are not quoted."""
     h = hashlib.sha256()
     for name in KERNEL_SOURCES[kernel]:
-        with open(os.path.join(ROOT, "paper_2503_01483_b200", "csrc", name), "rb") as f:
-            h.update(f.read())
+        with open(os.path.join(ROOT, "paper_2503_01483_b200", "csrc", name), "r") as f:
+            text = f.read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        text = re.sub(r"//[^\n]*", "", text)
+        h.update("".join(text.split()).encode())
     return h.hexdigest()[:16]
 
 

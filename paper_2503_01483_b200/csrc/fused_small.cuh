@@ -4,17 +4,23 @@
 // A whole row of Y = X R fits one 128-column tensor-memory tile, so one CTA can take a tile of 128
 // tokens through the complete chain without leaving the SM:
 //
-//   TMA:  X tile (128 tokens x 128 channels, bf16)                     -> shared memory
+//   TMA:  X tile (128 tokens x 128 channels, float16 encoding)        -> shared memory
 //   MMA1: C = X Rc (Rc = R with each row's mean taken off, so that C is Y = X R minus its row means;
 //             Rc^T resident in shared memory, hi [+ lo])               -> tensor memory
 //   epilogue (two groups of 4 warps that take alternate tiles, one row per thread): m2, m4 (Eq. 3),
 //             kappa, loss term, then
-//             G = a c^3 - ab c as bf16 (the gradient with respect to C) -> shared memory
+//             G = a c^3 - ab c as float16 (the gradient w.r.t. C)      -> shared memory
 //   MMA2: dRc += X^T G (both operands read token-major straight from the tiles above,
 //             "MN-major" shared-memory descriptors)                    -> one persistent accumulator
 //
 // X is read from HBM exactly once per evaluation; Y and G never leave the SM.  Each CTA ends by
 // writing its partial dR (128 x 128 float32) and partial loss; a fixed-order sum over CTAs follows.
+//
+// What bounds it.  Both products take both operands from shared memory, and such an MMA reads 4 KB + 4 KB per
+// 128 x 128 x 16 step of 64 cycles: the whole 128-byte-per-clock port.  Per 32 KB tile of X the kernel moves 192 KB
+// through that port (TMA write 32, MMA1 64, G stores 32, MMA2 64), so a tile cannot take fewer than about 1600
+// cycles however the stages, warps and buffers are arranged; it takes 1700.  HBM, the tensor pipe and the
+// float32 pipes all idle behind that.
 //
 // Operand encoding.  The kernel does not read the caller's bf16 X but a copy made once per X (k_encode_rows_128):
 // every row multiplied by the power of two that brings its largest entry into [1, 2), as float16.  A bf16 value
@@ -37,7 +43,7 @@ constexpr int kFsD = 128;          // channels = rows of a token tile
 constexpr int kFsThreads = 352;    // warp 0: TMA, warp 1: MMA1, warps 2..5 and 6..9: two epilogue groups, warp 10: MMA2
 constexpr int kFsMma2Warp = 10;
 constexpr int kFsHalf = 128 * 64 * 2;      // bytes of one 128-row x 64-element swizzled block
-constexpr int kFsTile = 2 * kFsHalf;       // one 128 x 128 bf16 tile
+constexpr int kFsTile = 2 * kFsHalf;       // one 128 x 128 tile of 16-bit elements
 // Shared memory: R^T (hi, and lo when TERMS == 2), four X stages, and the G tiles: one per epilogue group with
 // one term, a single one with two.  (Measured with one term: five X stages and a single G tile are 8 % slower
 // than four and two, because a group's G stores then wait for MMA2 of the other group's tile.)
@@ -64,7 +70,7 @@ struct FusedParams {
   const float* row_ms;      // [N] mean square of every encoded row of X (for the rule that skips rows without spread)
 };
 
-// Shared-memory descriptor for an "MN-major" bf16 operand stored as rows of 64 elements (128 bytes,
+// Shared-memory descriptor for an "MN-major" 16-bit operand stored as rows of 64 elements (128 bytes,
 // 128-byte swizzle) where the ROW index is the contraction index k and the 64 contiguous elements run
 // along M (or N): eight k-rows form a 1024-byte group (stride field), the next 64 elements of M/N live
 // `lead_bytes` further on (leading field).
