@@ -957,12 +957,13 @@ __global__ void k_force_guard(Scalars* sc) {
 // Y_k = R - alpha/2 W (R + Y_{k-1})).  This kernel adds term k in place, R += c_k P with
 // c_k = -alpha (-alpha/2)^k.  Terms k >= sc->n_terms do nothing.  A term that is not the last one evaluated writes
 // P^T as bf16 (pt_hi) for the next product; the last one writes the bf16 forms of the new R instead: r_hi (as is),
-// rt_hi/rt_lo (transposed hi/lo).  adam_m != null (given with k = 0 only): also M <- adam_r * P.
+// rt_hi/rt_lo (transposed hi/lo) and, when rt16 != null, the transpose as float16 (the forward pass's second operand
+// when it runs on float16 operands).  adam_m != null (given with k = 0 only): also M <- adam_r * P.
 // grid (d/32, min(d/32, 32)), block (32, 8); each block walks row tiles.
 __global__ void k_series_term(float* __restrict__ R, const float* __restrict__ P, const Scalars* __restrict__ sc,
                               int k, int d, __nv_bfloat16* __restrict__ pt_hi, __nv_bfloat16* __restrict__ r_hi,
                               __nv_bfloat16* __restrict__ rt_hi, __nv_bfloat16* __restrict__ rt_lo,
-                              float* __restrict__ adam_m) {
+                              float* __restrict__ adam_m, __half* __restrict__ rt16) {
   const unsigned int n_terms = sc->n_terms;
   if (static_cast<unsigned int>(k) >= n_terms) return;
   const bool last = (static_cast<unsigned int>(k) + 1u == n_terms);
@@ -1001,6 +1002,7 @@ __global__ void k_series_term(float* __restrict__ R, const float* __restrict__ P
         split_bf16(tile[tx][c], h, l);
         rt_hi[o] = h;
         rt_lo[o] = l;
+        if (rt16) rt16[o] = __float2half_rn(tile[tx][c]);
       } else {
         pt_hi[o] = __float2bfloat16_rn(tile[tx][c]);
       }
@@ -1147,12 +1149,12 @@ __global__ void k_guard_decide(Scalars* sc, float polish_at) {
 }
 
 // When the gate is open: R <- R - Q/2 (one Newton-Schulz step, Q = R E) and the bf16 forms of the
-// new R (r_hi, rt_hi, rt_lo) are rewritten.  grid (d/32, 16), block (32, 8): each block walks the row tiles
+// new R (r_hi, rt_hi, rt_lo, and rt16 when given) are rewritten.  grid (d/32, 16), block (32, 8): each block walks the row tiles
 // blockIdx.y, blockIdx.y + 16, ... (a small grid, because in most steps the gate is closed and the kernel only
 // has to find that out).
 __global__ void k_polish_apply(float* __restrict__ R, const float* __restrict__ Q, const Scalars* __restrict__ sc,
                                int d, __nv_bfloat16* __restrict__ r_hi, __nv_bfloat16* __restrict__ rt_hi,
-                               __nv_bfloat16* __restrict__ rt_lo) {
+                               __nv_bfloat16* __restrict__ rt_lo, __half* __restrict__ rt16) {
   if (sc->gate == 0u) return;
   __shared__ float tile[32][33];
   const int c0 = blockIdx.x * 32;
@@ -1183,6 +1185,7 @@ __global__ void k_polish_apply(float* __restrict__ R, const float* __restrict__ 
       const long long o = static_cast<long long>(c0 + c) * d + r0 + tx;
       rt_hi[o] = h;
       rt_lo[o] = l;
+      if (rt16) rt16[o] = __float2half_rn(tile[tx][c]);
     }
     __syncthreads();
   }

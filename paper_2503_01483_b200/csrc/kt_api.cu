@@ -550,8 +550,8 @@ static int forward_terms(const kt_ctx* ctx, int d, long long N) {
   return d <= 512 ? 2 : 1;
 }
 
-// R^T as float16 for the forward GEMMs of a problem that uses the float16 encoding (no kernel of the orthogonal
-// step keeps this form up to date: it is made afresh before every forward pass).
+// R^T as float16 for the forward GEMMs of a problem that uses the float16 encoding.  Inside a fit the orthogonal
+// step keeps it up to date together with the bf16 forms (k_series_term, k_polish_apply).
 static kt_status cast_rt16(kt_ctx* ctx, const float* R, int d, const WsLayout& L) {
   if (!L.f16) return KT_OK;
   dim3 grid(d / 32, d / 32), block(32, 8);
@@ -714,10 +714,12 @@ static kt_status backward(kt_ctx* ctx, const XView& xv, int N, int d, const WsLa
   return KT_OK;
 }
 
+static bool use_small_orth(const kt_ctx* ctx, int d);
+
 static kt_status loss_grad_async(kt_ctx* ctx, const XView& xv, int N, int d, const WsLayout& L, const float* R,
                                  float* dR, double* hist_slot, bool rt_current, __nv_bfloat16* dr_hi = nullptr) {
   if (!rt_current) KT_TRY(cast_rt(ctx, R, d, N, L));
-  else KT_TRY(cast_rt16(ctx, R, d, L));
+  else if (use_small_orth(ctx, d)) KT_TRY(cast_rt16(ctx, R, d, L));  // (the one-launch step leaves the bf16 forms only)
   KT_TRY(forward_loss(ctx, xv, N, d, L, hist_slot, keep_y_for_backward(ctx)));
   KT_TRY(backward(ctx, xv, N, d, L, dR, dr_hi));
   KT_TRY(reduce_shards(ctx, dR, static_cast<int64_t>(d) * d, KT_F32));  // the gradient of the whole batch
@@ -877,8 +879,8 @@ static kt_status guard(kt_ctx* ctx, const float* R_in, float* R, int d, const Ws
     Operand A{r_hi, ld}, B{e_hi, ld};  // (R E)[i][j] = sum_k R[i][k] E[j][k], E symmetric
     KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 1, &A, &B, p, kCatSquare));
   }
-  k_polish_apply<<<dim3(d / 32, d / 32 < 16 ? d / 32 : 16), tblock, 0, ctx->stream>>>(R, fbuf, sc, d, r_hi, rt_hi,
-                                                                                         rt_lo);
+  k_polish_apply<<<dim3(d / 32, d / 32 < 16 ? d / 32 : 16), tblock, 0, ctx->stream>>>(
+      R, fbuf, sc, d, r_hi, rt_hi, rt_lo, L.f16 ? at<__half>(ctx, L.rt16) : nullptr);
   KT_LAUNCH_CHECK();
   return KT_OK;
 }
@@ -1057,7 +1059,8 @@ static kt_status orth_step_async(kt_ctx* ctx, float* R, const float* dR, int d, 
       KT_TRY(run_gemm<kStoreF32>(ctx, d, d, d, 1, &A, &B, p, kCatSquare));
     }
     k_series_term<<<lgrid, tblock, 0, ctx->stream>>>(R, fbuf, sc, k, d, z_hi, r_hi, rt_hi, rt_lo,
-                                                     k == 0 ? adam_m : nullptr);
+                                                     k == 0 ? adam_m : nullptr,
+                                                     L.f16 ? at<__half>(ctx, L.rt16) : nullptr);
     KT_LAUNCH_CHECK();
   }
   if (guard_mode != 2) {

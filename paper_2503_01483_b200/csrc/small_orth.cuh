@@ -307,6 +307,28 @@ __device__ __forceinline__ void rows_times_staged_matrix(const float (*arow)[512
   }
 }
 
+// Sum (or maximum) of the kSoGrid per-CTA partials another phase of this launch left in global memory, the same
+// bits in every CTA: thread c < kSoGrid loads partial c (one round trip to L2 for the block, not one per partial),
+// the warps reduce with the fixed shuffle tree, and the four warp results are combined in order.  Every thread of
+// the block calls it (blockDim.x >= kSoGrid) and gets the result.
+__device__ __forceinline__ double sum_of_parts(const double* part, double* sh /*4*/) {
+  double v = (threadIdx.x < kSoGrid) ? __ldcg(part + threadIdx.x) : 0.0;
+  v = warp_sum(v);
+  __syncthreads();  // sh is free
+  if (threadIdx.x < kSoGrid && (threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+  __syncthreads();
+  return ((sh[0] + sh[1]) + sh[2]) + sh[3];
+}
+__device__ __forceinline__ float max_of_parts(const float* part, float* sh /*4*/) {
+  float v = (threadIdx.x < kSoGrid) ? __ldcg(part + threadIdx.x) : 0.f;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  __syncthreads();
+  if (threadIdx.x < kSoGrid && (threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+  __syncthreads();
+  return fmaxf(fmaxf(sh[0], sh[1]), fmaxf(sh[2], sh[3]));
+}
+
 // Dynamic shared memory: d * d floats when d == 128 (the staged products above), none otherwise.
 template <int ROWS>
 __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParams p) {
@@ -383,8 +405,7 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
   // r = (1 - beta1^k) sqrt(v / (1 - beta2^k) + eps), the same in every CTA
   double adam_r = 1.0;
   if (adam) {
-    double g2 = 0.0;
-    for (int c = 0; c < kSoGrid; ++c) g2 += __ldcg(p.g2_part + c);
+    const double g2 = sum_of_parts(p.g2_part, shd);
     const unsigned int k = adam_k_in + 1u;
     const double b1 = static_cast<double>(p.beta1), b2 = static_cast<double>(p.beta2);
     const double v = b2 * adam_v_in + (1.0 - b2) * g2;
@@ -442,8 +463,7 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
   float drift;     // bound on the orthogonality error accumulated since the last measurement
   int n_terms;     // series terms evaluated (the same in every CTA: the grid-wide barriers below depend on it)
   {
-    double s = 0.0;
-    for (int c = 0; c < kSoGrid; ++c) s += __ldcg(p.norm_part + c);
+    const double s = sum_of_parts(p.norm_part, shd);
     const double nrm = sqrt(s);
     const double cap = 2.0 * static_cast<double>(p.q) / (nrm + static_cast<double>(p.eps));
     const double a = (static_cast<double>(p.lr) < cap) ? static_cast<double>(p.lr) : cap;
@@ -533,7 +553,7 @@ __global__ void __launch_bounds__(512, 1) small_orth_kernel(const SmallOrthParam
       p.max_part[blockIdx.x] = mx;
     }
     grid.sync();
-    for (int c = 0; c < kSoGrid; ++c) max_e = fmaxf(max_e, __ldcg(p.max_part + c));
+    max_e = max_of_parts(p.max_part, shf);
     if (max_e > p.polish_at) {  // same value in every CTA: the branch is grid-uniform
       // R <- R - R E / 2; each CTA reads only its own rows of R and all of E
       load_rows(p.R);

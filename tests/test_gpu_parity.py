@@ -426,10 +426,16 @@ def test_fit_100_steps_stays_orthogonal_and_descends(ctx):
     assert rep["loss_first"] == pytest.approx(L0, rel=1e-12)
 
 
-@pytest.mark.parametrize("d", [256, 1024])
-def test_fit_equals_composed_calls(d):
-    # the identity holds when every step measures orthogonality (guard_every = 1), as kt_orth_step always does
-    ctx = kurtail.Context(DEV, guard_every=1)
+@pytest.mark.parametrize("d,extra", [(256, {}), (1024, {}),
+                                     # one float16 term of R with the one-launch step, which leaves no float16 form
+                                     (256, {"forward_terms": 1}),
+                                     # a threshold every step exceeds: the polish rewrites R and all its 16-bit forms
+                                     (1024, {"polish_thresh": 1e-9})])
+def test_fit_equals_composed_calls(d, extra):
+    # the identity holds when every step measures orthogonality (guard_every = 1), as kt_orth_step always does.
+    # Inside the fit the forward pass reads the 16-bit forms of R that the previous step left behind; the composed
+    # calls make them afresh from R every time.
+    ctx = kurtail.Context(DEV, guard_every=1, **extra)
     X = make_x(1500, d, seed=71)
     Ra = ctx.init_rotation(d, "hadamard")
     Rb = Ra.clone()
