@@ -234,8 +234,12 @@ __global__ void k_prepare_x(const T* __restrict__ X, long long ld, int N, int d,
 
 // The same transpose for a bf16 X with no dense copy asked for, in tiles of 64 tokens x 128 channels with 16-byte
 // loads (four in flight per thread).  d a multiple of 128.  grid (d/128, ceil(N/64)), block 256.
+// bases != null: row t is not X[t] but row t of the minibatch `ids` gathered from several buffers (see
+// k_gather_samples for the numbering), read where it lies.
 __global__ void k_transpose_x_bf16(const __nv_bfloat16* __restrict__ X, long long ld, int N, int d,
-                                   __nv_bfloat16* __restrict__ xt, long long ldt) {
+                                   __nv_bfloat16* __restrict__ xt, long long ldt,
+                                   const void* const* __restrict__ bases = nullptr, int samples_per_buf = 0,
+                                   int rps = 0, const int* __restrict__ ids = nullptr) {
   __shared__ __nv_bfloat16 tile[64][130];
   const int c0 = blockIdx.x * 128, r0 = blockIdx.y * 64;
   const int rr = threadIdx.x >> 4, cc = (threadIdx.x & 15) * 8;  // 16 rows per pass, 8 channels per thread
@@ -243,8 +247,14 @@ __global__ void k_transpose_x_bf16(const __nv_bfloat16* __restrict__ X, long lon
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
     const int row = r0 + rr + 16 * q;
-    v[q] = (row < N) ? *reinterpret_cast<const uint4*>(X + static_cast<long long>(row) * ld + c0 + cc)
-                     : make_uint4(0u, 0u, 0u, 0u);
+    const __nv_bfloat16* src = X + static_cast<long long>(row) * ld;
+    if (bases != nullptr && row < N) {
+      const int b = row / rps, r = row - b * rps;
+      const int id = ids[b];
+      const int buf = id / samples_per_buf, smp = id - buf * samples_per_buf;
+      src = static_cast<const __nv_bfloat16*>(bases[buf]) + (static_cast<long long>(smp) * rps + r) * ld;
+    }
+    v[q] = (row < N) ? *reinterpret_cast<const uint4*>(src + c0 + cc) : make_uint4(0u, 0u, 0u, 0u);
   }
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
@@ -633,6 +643,86 @@ __global__ void k_row_scale(const T* X, long long ld, int d, float eps, float* _
     const double ms = acc / d + static_cast<double>(eps);
     if (mean_square) rowscale[blockIdx.x] = static_cast<float>(acc / d);
     else rowscale[blockIdx.x] = ms > 0.0 ? static_cast<float>(1.0 / sqrt(ms)) : 0.f;
+  }
+}
+
+// A minibatch gathered from several bf16 buffers straight into the forward pass's float16 encoding: what
+// k_row_scale (gather + RMSNorm factor) followed by k_encode_rows_f16 compute, bit for bit, without the dense bf16
+// copy in between.  Row t is read where it lies (numbering as in k_gather_samples), twice (the second time from
+// cache).  rowscale != null: receives the RMSNorm factor of row t, and acc[t] includes it; null: no RMSNorm.
+// One block of 256 threads per row; d a multiple of 128.
+__global__ void k_gather_encode_rows_f16(const void* const* __restrict__ bases, long long ld, int samples_per_buf,
+                                         int rps, const int* __restrict__ ids, int d, float eps,
+                                         float* __restrict__ rowscale, __half* __restrict__ x16,
+                                         float* __restrict__ acc) {
+  __shared__ double sh[8];
+  __shared__ float shm[8];
+  __shared__ int shb[8];
+  __shared__ float sh_rms;
+  const int b = blockIdx.x / rps, r = blockIdx.x - b * rps;
+  const int id = ids[b];
+  const int buf = id / samples_per_buf, smp = id - buf * samples_per_buf;
+  const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(bases[buf]) + (static_cast<long long>(smp) * rps + r) * ld;
+  __half* o = x16 + static_cast<long long>(blockIdx.x) * d;
+  float part = 0.f, amax = 0.f;
+  int bad = 0;
+  for (int j = threadIdx.x * 8; j < d; j += 256 * 8) {
+    float v[8];
+    load8(x + j, v);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      part = fmaf(v[e], v[e], part);
+      amax = fmaxf(amax, fabsf(v[e]));
+      bad |= !(fabsf(v[e]) <= 3.4e38f) ? 1 : 0;
+    }
+  }
+  const double sumsq = block_sum_256(static_cast<double>(part), sh, threadIdx.x);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
+    bad |= __shfl_xor_sync(0xffffffffu, bad, off);
+  }
+  if ((threadIdx.x & 31) == 0) {
+    shm[threadIdx.x >> 5] = amax;
+    shb[threadIdx.x >> 5] = bad;
+  }
+  if (threadIdx.x == 0) {
+    float f = 1.0f;
+    if (rowscale != nullptr) {
+      const double ms = sumsq / d + static_cast<double>(eps);
+      f = ms > 0.0 ? static_cast<float>(1.0 / sqrt(ms)) : 0.f;
+      rowscale[blockIdx.x] = f;
+    }
+    sh_rms = f;
+  }
+  __syncthreads();
+  amax = shm[0];
+  bad = shb[0];
+#pragma unroll
+  for (int i = 1; i < 8; ++i) {
+    amax = fmaxf(amax, shm[i]);
+    bad |= shb[i];
+  }
+  float scale = 1.0f, inv = 1.0f;
+  if (amax > 0.f) {
+    int e = static_cast<int>((__float_as_uint(amax) >> 23) & 0xffu) - 127;   // amax in [2^e, 2^(e+1)); subnormal: -127
+    e = e < -126 ? -126 : (e > 126 ? 126 : e);
+    scale = __uint_as_float(static_cast<uint32_t>(127 - e) << 23);           // 2^-e, e in [-126, 126]
+    inv = __uint_as_float(static_cast<uint32_t>(127 + e) << 23);             // 2^e
+  }
+  if (threadIdx.x == 0) acc[blockIdx.x] = sh_rms * inv;
+  const float nanv = __uint_as_float(0x7fc00000u);
+  for (int j = threadIdx.x * 8; j < d; j += 256 * 8) {
+    const uint4 raw = *reinterpret_cast<const uint4*>(x + j);
+    const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+    uint4 outv;
+    __half2* po = reinterpret_cast<__half2*>(&outv);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float2 f = __bfloat1622float2(p2[e]);
+      po[e] = bad ? __floats2half2_rn(nanv, nanv) : __floats2half2_rn(f.x * scale, f.y * scale);
+    }
+    *reinterpret_cast<uint4*>(o + j) = outv;
   }
 }
 

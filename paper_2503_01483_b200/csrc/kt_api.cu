@@ -1182,6 +1182,13 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
         else
           k_encode_rows_128<float><<<eg, 256, 0, ctx->stream>>>(nullptr, X.ld, N, x16, ms, bases, spb, rps, ids);
         xv.row_ms = ms;
+      } else if (L.f16 && X.dtype == KT_BF16) {
+        // float16 forward operands: the samples' rows go straight into that encoding (with the RMSNorm factors when
+        // asked for) and, below, into the transpose; no dense bf16 copy of the minibatch is made
+        float* rsc = norm ? at<float>(ctx, L.rowscale) : nullptr;
+        k_gather_encode_rows_f16<<<N, 256, 0, ctx->stream>>>(bases, X.ld, spb, rps, ids, d, ctx->cfg.rms_eps, rsc,
+                                                             at<__half>(ctx, L.x16), at<float>(ctx, L.rowacc));
+        xv.row_scale = rsc;
       } else if (norm) {
         // gather and RMSNorm factors in one pass over the samples' rows
         float* rsc = at<float>(ctx, L.rowscale);
@@ -1200,7 +1207,15 @@ static kt_status fit_impl(kt_ctx* ctx, const kt_mat& X, float* R, int32_t steps,
       KT_LAUNCH_CHECK();
       xv.xb = xb;
       xv.ldx = d;
-      if (!fused) {  // the token GEMM of the backward pass reads the transpose
+      if (!fused && L.f16 && X.dtype == KT_BF16) {
+        dim3 tg(d / 128, (N + 63) / 64);
+        k_transpose_x_bf16<<<tg, 256, 0, ctx->stream>>>(nullptr, X.ld, N, d, at<__nv_bfloat16>(ctx, L.xt), L.ldt,
+                                                        bases, spb, rps, ids);
+        KT_LAUNCH_CHECK();
+        xv.xb = nullptr;   // (not made; the forward pass reads the encoding)
+        xv.x16 = at<__half>(ctx, L.x16);
+        xv.acc_scale = at<float>(ctx, L.rowacc);
+      } else if (!fused) {  // the token GEMM of the backward pass reads the transpose
         KT_TRY(transpose_x_bf16(ctx, xb, d, N, d, L));
         KT_TRY(finish_view(ctx, N, d, L, &xv));   // (and the forward pass, maybe, the float16 encoding)
       }
