@@ -201,3 +201,32 @@ def test_gradient_at_a_rotation_that_bf16_cannot_hold(workload, d, rows, steps):
     _, dRb = b.loss_grad(X, R)
     assert rel_fro(f64(dRb), dR_ref) > err
     b.close()
+
+
+def test_full_batch_loss_and_gradient_against_the_oracle_on_every_row():
+    # The benchmark's own configuration, nothing sampled: N = 65536 rows at d = 4096, R a few steps away from the
+    # Hadamard start (so no longer exact in any 16-bit format), in the launch configuration bench.py times.  The
+    # oracle takes the rows in blocks (its loss and gradient are means over tokens: the blocks combine with their
+    # row counts as weights) -- about 9 TFLOP in float64 on the host cores.
+    cfg = synth.config("llama2_7b_attn", device=DEV)
+    X = cfg["X"]
+    N, d = X.shape
+    assert (N, d) == (65536, 4096)
+    c = kurtail.Context(DEV)
+    R = c.init_rotation(d, "hadamard")
+    c.fit(X, R, 3, 1e-2)
+    loss, dR = c.loss_grad(X, R)
+    R64 = f64(R)
+    L_ref, G_ref = 0.0, np.zeros((d, d))
+    for r0 in range(0, N, 8192):
+        Xb = f64(X[r0:r0 + 8192])
+        l, g = ko.loss_grad(Xb, R64)
+        L_ref += l * Xb.shape[0]
+        G_ref += g * Xb.shape[0]
+    L_ref /= N
+    G_ref /= N
+    assert abs(loss - L_ref) <= 1e-3 * abs(L_ref)
+    err = rel_fro(f64(dR), G_ref)
+    assert err <= 1e-2, err
+    assert ko.orthogonality_error(R64) <= 1e-4
+    c.close()
