@@ -247,14 +247,19 @@ __global__ void k_transpose_x_bf16(const __nv_bfloat16* __restrict__ X, long lon
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
     const int row = r0 + rr + 16 * q;
-    const __nv_bfloat16* src = X + static_cast<long long>(row) * ld;
-    if (bases != nullptr && row < N) {
-      const int b = row / rps, r = row - b * rps;
-      const int id = ids[b];
-      const int buf = id / samples_per_buf, smp = id - buf * samples_per_buf;
-      src = static_cast<const __nv_bfloat16*>(bases[buf]) + (static_cast<long long>(smp) * rps + r) * ld;
+    v[q] = make_uint4(0u, 0u, 0u, 0u);
+    if (row < N) {
+      const __nv_bfloat16* src;
+      if (bases != nullptr) {
+        const int b = row / rps, r = row - b * rps;
+        const int id = ids[b];
+        const int buf = id / samples_per_buf, smp = id - buf * samples_per_buf;
+        src = static_cast<const __nv_bfloat16*>(bases[buf]) + (static_cast<long long>(smp) * rps + r) * ld;
+      } else {
+        src = X + static_cast<long long>(row) * ld;
+      }
+      v[q] = *reinterpret_cast<const uint4*>(src + c0 + cc);
     }
-    v[q] = (row < N) ? *reinterpret_cast<const uint4*>(src + c0 + cc) : make_uint4(0u, 0u, 0u, 0u);
   }
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
