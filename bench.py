@@ -648,6 +648,10 @@ def main():
                 t_f = gg["fused"]["ms"] / gg["fused"]["launches"] * 1e-3
                 ex["single_pass_kernel_us"] = t_f * 1e6
                 ex["hbm_frac_of_measured"] = 2.0 * Nw * dw / t_f / 1e9 / peaks["hbm_gbs"]
+                # (what the kernel saturates is not HBM: per 32 KB tile of X it moves 192 KB through the SM's
+                # 128-byte-per-clock shared-memory port -- TMA write, two products with both operands there, the
+                # stores of G -- 1603 wavefronts counted against the 1700-1750 cycles a tile takes)
+                ex["limiter"] = "shared-memory data path of the SM (6 bytes per byte of HBM)"
             else:
                 tk = [gg[k] for k in ("forward", "backward_b")]
                 t_l = sum(x["ms"] for x in tk) / max(sum(x["launches"] for x in tk), 1) * 1e-3
