@@ -15,9 +15,10 @@
  *   16 (the tiles are fetched by TMA).  R and dR are dense d x d float32,
  *   16-byte aligned.
  * Precision.  X is used as bfloat16 (float32 X is rounded once on entry), R is
- *   kept in float32 and rounded to bfloat16 for the token GEMMs (see
- *   kt_config.forward_terms); all products accumulate in float32 on the
- *   tensor cores.
+ *   kept in float32 and enters the token GEMMs in a 16-bit form: float16
+ *   against an exact float16 re-encoding of X's rows, or bfloat16 terms (see
+ *   kt_config.forward_terms and forward_bf16); all products accumulate in
+ *   float32 on the tensor cores.
  * Stream.  All work is issued on the stream given to kt_create().  Calls that
  *   return a host scalar synchronise that stream; the others are stream
  *   ordered and return after enqueueing.
@@ -350,10 +351,11 @@ kt_status kt_fit_layers(kt_ctx* ctx, const kt_mat* X_layers, float* const* R_lay
  * "sample" is a run of rows_per_sample consecutive rows (rows must be a
  * multiple of it), numbered id = buffer * (rows / rows_per_sample) + index
  * within the buffer.  Step k fits on the minibatch of the `batch` samples
- * order[k*batch .. (k+1)*batch): their rows are gathered (in that order) into
- * a dense bf16 matrix of batch*rows_per_sample rows in the workspace, and the
- * step is the one kt_fit takes on that matrix (loss_mode, rmsnorm, optimizer
- * as configured).  The shuffle is the caller's: `order` (host, steps*batch
+ * order[k*batch .. (k+1)*batch): their rows, in that order, form a matrix of
+ * batch*rows_per_sample rows (gathered in the workspace into the operand
+ * forms of the token GEMMs; never more than one minibatch at a time), and the
+ * step is the one kt_fit takes on that matrix, bit for bit (loss_mode,
+ * rmsnorm, optimizer as configured).  The shuffle is the caller's: `order` (host, steps*batch
  * entries) is an input, so that a run can be reproduced exactly.  Needs a
  * workspace of kt_fit_shared_workspace_bytes().  KT_ERR_INVALID_ARG if an id
  * is out of range (checked before any work).  Synchronises at the end. */
